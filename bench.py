@@ -1,0 +1,399 @@
+#!/usr/bin/env python
+"""Benchmark of the blockwise-quantization hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Workload: the 1 GiB bf16 block-size sweep ([16, 4096, 8192], Laplace(0, 0.5) with 8 outlier
+channels x60, seed 4).  One step is one pass of the whole hot path over that tensor: for
+each block size in {64, 256, 1024, 4096}: bq_quantize, bq_dequantize and the fused
+bq_roundtrip (12 kernel launches).  The metric is GB/s of input activation processed
+(n * 2 bytes per call, 12 calls per step).  The tensor is larger than L2, so every launch
+streams from HBM.  One JSON line is printed by rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2407_19775_b200 import workloads
+
+WORKLOAD = "sweep1g"
+BLOCKS = (64, 256, 1024, 4096)
+OPS = ("quantize", "dequantize", "roundtrip")
+METRIC = "quantize+dequantize GB/s of activations and fraction of HBM roofline, 1xB200"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def algorithmic_bytes(op: str, n: int, block: int, s_in: int = 2, s_out: int = 2) -> float:
+    """Bytes one launch must move: input read once, outputs written once."""
+    nb = (n + block - 1) // block
+    if op == "quantize":
+        return n * s_in + n + 4 * nb
+    if op == "dequantize":
+        return n + 4 * nb + n * s_out
+    return n * s_in + n * s_out
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------------------------------ distributed plumbing
+
+def dist_setup(n_gpus: int, backend: str):
+    """Returns (rank, world).  One process per GPU; torchrun sets the environment."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29511")
+        if not dist.is_initialized():
+            dist.init_process_group(backend=backend, rank=rank, world_size=world)
+    return rank, world
+
+
+def barrier(world: int, device=None):
+    if world > 1:
+        import torch.distributed as dist
+        if device is not None and device.type == "cuda":
+            dist.barrier(device_ids=[device.index])
+        else:
+            dist.barrier()
+
+
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    if world == 1:
+        return value
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank: float, world: int, max_seconds: float) -> float:
+    """Weak scaling: every rank processes the same number of units; the job's rate is all
+    ranks' units over the slowest rank's time."""
+    return units_per_rank * world / max_seconds
+
+
+# ------------------------------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = f"/tmp/bq_clocks_{os.getpid()}.csv"
+
+    def start(self):
+        try:
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100"], stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, smax, power, reasons = [], [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        try:
+            for line in open(self.path):
+                f = [c.strip() for c in line.split(",")]
+                if len(f) < 9:
+                    continue
+                sm.append(float(f[1])); smax.append(float(f[2])); power.append(float(f[3]))
+                for name, v in zip(names, f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.remove(self.path)
+        except Exception:
+            pass
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(smax)), "power_w_max": float(max(power)),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------ the CUDA arm
+
+def run_ours(args):
+    import paper_2407_19775_b200 as bq
+    from paper_2407_19775_b200 import binding
+    binding.lib()                                   # fail now if the CUDA library is missing
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the hot path has no CPU fallback")
+    rank, world = dist_setup(args.gpus, "nccl")
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+
+    w = workloads.WORKLOADS[WORKLOAD]
+    x_host = workloads.make(WORKLOAD).view(-1)
+    n = x_host.numel()
+    x_pin = x_host.pin_memory()
+    del x_host
+    cb = bq.Codebook(device=dev)
+    x = x_pin.to(dev, non_blocking=True)
+    codes = torch.empty(n, dtype=torch.uint8, device=dev)
+    absmax = {b: torch.empty(n // b, dtype=torch.float32, device=dev) for b in BLOCKS}
+    y = torch.empty(n, dtype=w.dtype, device=dev)
+    torch.cuda.synchronize()
+
+    def launch(op, b):
+        if op == "quantize":
+            bq.bq_quantize(x, b, cb, codes, absmax[b])
+        elif op == "dequantize":
+            bq.bq_dequantize(codes, absmax[b], b, cb, w.dtype, y)
+        else:
+            bq.bq_roundtrip(x, b, cb, y_out=y)
+
+    def step(events=None):
+        for b in BLOCKS:
+            for op in OPS:
+                if events is not None:
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    launch(op, b)
+                    e1.record()
+                    events.append((op, b, e0, e1))
+                else:
+                    launch(op, b)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    events = []
+    barrier(world, dev)
+    torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.steps):
+        step(events)
+    t1.record()
+    torch.cuda.synchronize()
+    barrier(world, dev)
+    local_s = t0.elapsed_time(t1) / 1e3
+    clocks = sampler.stop() if rank == 0 else None
+    max_s = max_over_ranks(local_s, world, dev)
+
+    bytes_per_step = n * 2 * len(BLOCKS) * len(OPS)
+    value = whole_job_value(bytes_per_step * args.steps, world, max_s) / 1e9
+
+    # per-kernel durations from the events recorded inside the timed region
+    peak, peak_kind = measured_peak()
+    per = {}
+    for op, b, e0, e1 in events:
+        per.setdefault((op, b), []).append(e0.elapsed_time(e1))
+    kernels = {}
+    for (op, b), ms in per.items():
+        avg = float(np.mean(ms))
+        ab = algorithmic_bytes(op, n, b)
+        kernels[f"{op}_b{b}"] = {
+            "ms": round(avg, 4), "ms_min": round(float(np.min(ms)), 4),
+            "input_gbs": round(n * (1 if op == "dequantize" else 2) / avg / 1e6, 1),
+            "total_gbs": round(ab / avg / 1e6, 1),
+            "frac_of_measured": round(ab / avg / 1e6 / peak, 4),
+            "frac_of_nominal_8tbs": round(ab / avg / 1e6 / NOMINAL_HBM_GBS, 4),
+        }
+    totals = {k: v["ms"] for k, v in kernels.items()}
+    dominant = max(totals, key=totals.get)
+    dop, db = dominant.split("_b")
+    dab = algorithmic_bytes(dop, n, int(db))
+    achieved = dab / kernels[dominant]["ms"] / 1e6
+    roofline = {"bound": "hbm", "kernel": dominant, "achieved": round(achieved, 1), "peak": peak, "peak_kind": peak_kind,
+                "unit": "GB/s", "frac": round(achieved / peak, 4), "traffic": TRAFFIC_BYTES.get(dominant)}
+
+    # end to end: host buffers in, host buffers out, copies inside the timed region
+    e2e = run_e2e(bq, cb, x_pin, dev, w.dtype, n, args, world)
+
+    # compression and reconstruction error (block 4096 outputs are still resident: recompute per block cheaply)
+    quality = {}
+    for b in BLOCKS:
+        bq.bq_roundtrip(x, b, cb, y_out=y)
+        num = torch.zeros((), dtype=torch.float64, device=dev)
+        den = torch.zeros((), dtype=torch.float64, device=dev)
+        for s in range(0, n, 1 << 27):
+            xs, ys = x[s:s + (1 << 27)].float(), y[s:s + (1 << 27)].float()
+            num += ((xs - ys) ** 2).sum(dtype=torch.float64)
+            den += (xs ** 2).sum(dtype=torch.float64)
+        quality[f"b{b}"] = {"compression_ratio": round(2 * b / (b + 4), 3), "rel_rms_error": round(float((num / den).sqrt().item()), 5)}
+
+    cpu = cpu_baseline(x_pin, rank) if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": round(value, 1), "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": round(max_s * 1e3 / args.steps, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "sweep1g: [16,4096,8192] bf16, Laplace(0,0.5), 8 outlier channels x60, seed 4; blocks 64/256/1024/4096; "
+                                   "quantize+dequantize+roundtrip per block", "elements": n, "l2": "input (1 GiB) larger than L2, no flush needed",
+                       "parallelism": f"replicated x{world}, no collective"},
+            "e2e": e2e, "gpu_launches": len(events), "clocks": clocks, "roofline": roofline, "kernels": kernels,
+            "quality": quality, "cpu_baseline": cpu,
+            "paper_context": "the paper reports no throughput for this path; it states only that hidden-state quantization halves the bandwidth",
+        }
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+# DRAM bytes per launch from ncu captures (profiles/); filled in once a capture exists and
+# cleared when the kernel changes.
+TRAFFIC_BYTES = {}
+
+
+def run_e2e(bq, cb, x_pin, dev, dtype, n, args, world):
+    """One end-to-end step per block size, everything starting and ending in pinned host
+    memory: sender (H2D x, quantize, D2H codes+absmax), receiver (H2D codes+absmax,
+    dequantize, D2H y) and the fused loop (H2D x, roundtrip, D2H y)."""
+    steps = max(1, min(args.steps, args.e2e_steps))
+    xd = torch.empty(n, dtype=dtype, device=dev)
+    cd = torch.empty(n, dtype=torch.uint8, device=dev)
+    yd = torch.empty(n, dtype=dtype, device=dev)
+    c_pin = torch.empty(n, dtype=torch.uint8).pin_memory()
+    y_pin = torch.empty(n, dtype=dtype).pin_memory()
+    a_pin = {b: torch.empty(n // b, dtype=torch.float32).pin_memory() for b in BLOCKS}
+    ad = {b: torch.empty(n // b, dtype=torch.float32, device=dev) for b in BLOCKS}
+    h2d = d2h = 0
+
+    def one_step(count=False):
+        nonlocal h2d, d2h
+        for b in BLOCKS:
+            xd.copy_(x_pin, non_blocking=True)
+            bq.bq_quantize(xd, b, cb, cd, ad[b])
+            c_pin.copy_(cd, non_blocking=True); a_pin[b].copy_(ad[b], non_blocking=True)
+            cd.copy_(c_pin, non_blocking=True); ad[b].copy_(a_pin[b], non_blocking=True)
+            bq.bq_dequantize(cd, ad[b], b, cb, dtype, yd)
+            y_pin.copy_(yd, non_blocking=True)
+            xd.copy_(x_pin, non_blocking=True)
+            bq.bq_roundtrip(xd, b, cb, y_out=yd)
+            y_pin.copy_(yd, non_blocking=True)
+            if count:
+                h2d += 2 * n * 2 + n + 4 * (n // b)
+                d2h += n + 4 * (n // b) + 2 * n * 2
+
+    one_step()
+    torch.cuda.synchronize()
+    barrier(world, dev)
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for i in range(steps):
+        one_step(count=(i == 0))
+    t1.record()
+    torch.cuda.synchronize()
+    barrier(world, dev)
+    sec = max_over_ranks(t0.elapsed_time(t1) / 1e3, world, dev)
+    bytes_per_step = n * 2 * len(BLOCKS) * len(OPS)
+    return {"value": round(whole_job_value(bytes_per_step * steps, world, sec) / 1e9, 2), "unit": "GB/s", "steps": steps,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+
+# ------------------------------------------------------------------------------------------ the CPU oracle arm
+
+def oracle_step(oracle, xb, cb, threads):
+    for b in BLOCKS:
+        c, a = oracle.quantize_sharded(xb, oracle.BF16, b, cb, threads)
+        oracle.dequantize_sharded(c, a, b, cb, oracle.BF16, threads)
+        oracle.roundtrip_sharded(xb, oracle.BF16, b, cb, oracle.BF16, threads)
+
+
+def cpu_baseline(x_pin, rank, rows=512):
+    """The CPU oracle, as it stands, on a bounded sample (the first `rows` rows) of the same
+    tensor, one thread."""
+    import oracle
+    xb = workloads.as_numpy_bits(x_pin[: rows * 8192])
+    cb = oracle.make_codebook()
+    oracle_step(oracle, xb[:8192 * 8], cb, 1)        # touch the library once
+    t = time.perf_counter()
+    oracle_step(oracle, xb, cb, 1)
+    sec = time.perf_counter() - t
+    return {"value": round(xb.size * 2 * len(BLOCKS) * len(OPS) / sec / 1e9, 5), "unit": "GB/s", "cores": 1, "kind": "oracle",
+            "host_cores_total": os.cpu_count(), "seconds": round(sec, 2),
+            "sample": f"first {rows} rows ({xb.size} elements) of sweep1g, all 4 block sizes x 3 ops, single thread"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    threads = os.cpu_count() or 1
+    # size the sample so that the whole run stays within about two minutes
+    per_elem_s = 3.3e-6 / max(1, threads) * 1.5
+    rows = int(120.0 / ((args.steps + args.warmup) * per_elem_s) // 8192)
+    rows = max(8, min(rows, 4096))
+    x = workloads.make(WORKLOAD, rows=rows).view(-1)
+    xb = workloads.as_numpy_bits(x)
+    cb = oracle.make_codebook()
+    for _ in range(args.warmup):
+        oracle_step(oracle, xb, cb, threads)
+    t = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(oracle, xb, cb, threads)
+    sec = time.perf_counter() - t
+    value = xb.size * 2 * len(BLOCKS) * len(OPS) * args.steps / sec / 1e9
+    sample = f"first {rows} rows ({xb.size} elements) of sweep1g per step, all 4 block sizes x 3 ops, {threads} threads over whole blocks"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": round(value, 5), "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(sec * 1e3 / args.steps, 3), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "sweep1g: [16,4096,8192] bf16, Laplace(0,0.5), 8 outlier channels x60, seed 4; blocks 64/256/1024/4096; "
+                               "quantize+dequantize+roundtrip per block", "sample": sample},
+        "cpu_baseline": {"value": round(value, 5), "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": round(value, 5), "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

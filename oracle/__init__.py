@@ -127,30 +127,75 @@ def roundtrip(x: np.ndarray, xdt: int, block: int, cb: np.ndarray, ydt: int, sid
     return (y, codes, absmax) if side else y
 
 
-def roundtrip_sharded(x: np.ndarray, xdt: int, block: int, cb: np.ndarray, ydt: int, threads: int):
-    """Run the unchanged single-threaded oracle on contiguous ranges of whole blocks, one
-    range per host thread (blocks are independent, so the result is the same bytes).
-    Returns (y, codes, absmax).  The threading is here, outside the oracle's functions."""
+def _shard_ranges(n: int, block: int, threads: int):
+    nb = (n + block - 1) // block
+    threads = max(1, min(threads, nb))
+    per = (nb + threads - 1) // threads
+    out = []
+    for t in range(threads):
+        b0, b1 = t * per, min(nb, (t + 1) * per)
+        if b0 < b1:
+            out.append((b0, b1, b0 * block, min(n, b1 * block)))
+    return nb, out
+
+
+def _run_sharded(work, ranges, threads: int, what: str) -> None:
+    with ThreadPoolExecutor(max(1, threads)) as ex:
+        rcs = list(ex.map(work, ranges))
+    if any(rcs):
+        raise ValueError(f"{what}: bad argument")
+
+
+# The three *_sharded helpers run the unchanged single-threaded oracle on contiguous ranges
+# of whole blocks, one range per host thread.  Blocks are independent, so the bytes are the
+# same as one call over everything; the threading is here, outside the oracle's functions.
+
+def quantize_sharded(x: np.ndarray, xdt: int, block: int, cb: np.ndarray, threads: int):
     x = _check_in(x, xdt)
     n = x.size
-    nb = (n + block - 1) // block
+    nb, ranges = _shard_ranges(n, block, threads)
+    codes = np.empty(n, np.uint8)
+    absmax = np.empty(nb, np.float32)
+    L = lib()
+
+    def work(r):
+        b0, b1, e0, e1 = r
+        return L.bq_oracle_quantize(_ptr(x[e0:e1]), xdt, e1 - e0, block, _ptr(cb), _ptr(codes[e0:e1]), _ptr(absmax[b0:b1]))
+
+    _run_sharded(work, ranges, threads, "bq_oracle_quantize")
+    return codes, absmax
+
+
+def dequantize_sharded(codes: np.ndarray, absmax: np.ndarray, block: int, cb: np.ndarray, ydt: int, threads: int):
+    codes = np.ascontiguousarray(codes, np.uint8).reshape(-1)
+    absmax = np.ascontiguousarray(absmax, np.float32).reshape(-1)
+    n = codes.size
+    _, ranges = _shard_ranges(n, block, threads)
+    y = np.empty(n, _np_dtype(ydt))
+    L = lib()
+
+    def work(r):
+        b0, b1, e0, e1 = r
+        return L.bq_oracle_dequantize(_ptr(codes[e0:e1]), _ptr(absmax[b0:b1]), e1 - e0, block, _ptr(cb), _ptr(y[e0:e1]), ydt)
+
+    _run_sharded(work, ranges, threads, "bq_oracle_dequantize")
+    return y
+
+
+def roundtrip_sharded(x: np.ndarray, xdt: int, block: int, cb: np.ndarray, ydt: int, threads: int):
+    """Returns (y, codes, absmax)."""
+    x = _check_in(x, xdt)
+    n = x.size
+    nb, ranges = _shard_ranges(n, block, threads)
     y = np.empty(n, _np_dtype(ydt))
     codes = np.empty(n, np.uint8)
     absmax = np.empty(nb, np.float32)
-    threads = max(1, min(threads, nb))
-    per = (nb + threads - 1) // threads
     L = lib()
 
-    def work(t: int) -> int:
-        b0, b1 = t * per, min(nb, (t + 1) * per)
-        if b0 >= b1:
-            return 0
-        e0, e1 = b0 * block, min(n, b1 * block)
+    def work(r):
+        b0, b1, e0, e1 = r
         return L.bq_oracle_roundtrip(_ptr(x[e0:e1]), xdt, e1 - e0, block, _ptr(cb), _ptr(y[e0:e1]), ydt,
                                      _ptr(codes[e0:e1]), _ptr(absmax[b0:b1]))
 
-    with ThreadPoolExecutor(threads) as ex:
-        rcs = list(ex.map(work, range(threads)))
-    if any(rcs):
-        raise ValueError("bq_oracle_roundtrip: bad argument")
+    _run_sharded(work, ranges, threads, "bq_oracle_roundtrip")
     return y, codes, absmax

@@ -3,4 +3,9 @@
 ``workloads`` (seeded input generators) imports without the CUDA library; the binding
 loads ``libbq.so`` on first use and raises if it has not been built.
 """
-__all__ = ["workloads"]
+from . import workloads
+from .binding import (BF16, DYNAMIC_TREE, F16, F32, USER, BqError, Codebook, bq_dequantize, bq_quantize, bq_roundtrip,
+                      n_blocks)
+
+__all__ = ["workloads", "Codebook", "BqError", "bq_quantize", "bq_dequantize", "bq_roundtrip", "n_blocks",
+           "F32", "F16", "BF16", "DYNAMIC_TREE", "USER"]

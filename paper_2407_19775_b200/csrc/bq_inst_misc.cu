@@ -1,0 +1,78 @@
+// General (any block / alignment / codebook) kernels and the tuned dequantize kernel.
+#include "bq_launch.h"
+
+namespace bql {
+namespace {
+
+template <int XDT, int YDT>
+cudaError_t fwd_general_mode(bool wy, bool wq, const void* x, void* y, uint8_t* codes, float* absmax, size_t n, size_t block,
+                             size_t first_block, const bqk::DeviceTables& tab, unsigned grid, cudaStream_t stream) {
+    if (wy && wq) bqk::fwd_general<XDT, YDT, true, true><<<grid, 256, 0, stream>>>(x, y, codes, absmax, n, block, first_block, tab);
+    else if (wy) bqk::fwd_general<XDT, YDT, true, false><<<grid, 256, 0, stream>>>(x, y, codes, absmax, n, block, first_block, tab);
+    else bqk::fwd_general<XDT, YDT, false, true><<<grid, 256, 0, stream>>>(x, y, codes, absmax, n, block, first_block, tab);
+    return cudaGetLastError();
+}
+
+template <int XDT>
+cudaError_t fwd_general_y(int ydt, bool wy, bool wq, const void* x, void* y, uint8_t* codes, float* absmax, size_t n, size_t block,
+                          size_t first_block, const bqk::DeviceTables& tab, unsigned grid, cudaStream_t stream) {
+    switch (ydt) {
+        case BQ_F32: return fwd_general_mode<XDT, bqk::kF32>(wy, wq, x, y, codes, absmax, n, block, first_block, tab, grid, stream);
+        case BQ_F16: return fwd_general_mode<XDT, bqk::kF16>(wy, wq, x, y, codes, absmax, n, block, first_block, tab, grid, stream);
+        default: return fwd_general_mode<XDT, bqk::kBF16>(wy, wq, x, y, codes, absmax, n, block, first_block, tab, grid, stream);
+    }
+}
+
+constexpr int kDeqNT = 512;
+
+template <int YDT>
+cudaError_t deq_fast_go(const uint8_t* codes, const float* absmax, void* y, size_t n16, int log2_block, const bqk::DeviceTables& tab,
+                        int sm_count, cudaStream_t stream) {
+    size_t grid = (n16 + kDeqNT - 1) / kDeqNT;
+    const size_t cap = size_t(sm_count) * 4;
+    if (grid > cap) grid = cap;
+    bqk::deq_fast<YDT, kDeqNT><<<unsigned(grid), kDeqNT, bqk::kDeqSmemBytes, stream>>>(codes, absmax, y, n16, log2_block, tab);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_fwd_general(int xdt, int ydt, bool write_y, bool write_q, const void* x, void* y, uint8_t* codes, float* absmax,
+                               size_t n, size_t block, size_t first_block, const bqk::DeviceTables& tab, int sm_count,
+                               cudaStream_t stream) {
+    const size_t nb = (n + block - 1) / block - first_block;
+    size_t grid = (nb + 7) / 8;
+    const size_t cap = size_t(sm_count) * 8;
+    if (grid > cap) grid = cap;
+    if (grid < 1) grid = 1;
+    switch (xdt) {
+        case BQ_F32: return fwd_general_y<bqk::kF32>(ydt, write_y, write_q, x, y, codes, absmax, n, block, first_block, tab, unsigned(grid), stream);
+        case BQ_F16: return fwd_general_y<bqk::kF16>(ydt, write_y, write_q, x, y, codes, absmax, n, block, first_block, tab, unsigned(grid), stream);
+        default: return fwd_general_y<bqk::kBF16>(ydt, write_y, write_q, x, y, codes, absmax, n, block, first_block, tab, unsigned(grid), stream);
+    }
+}
+
+cudaError_t launch_deq_fast(int ydt, const uint8_t* codes, const float* absmax, void* y, size_t n16, int log2_block,
+                            const bqk::DeviceTables& tab, int sm_count, int /*device*/, cudaStream_t stream) {
+    switch (ydt) {
+        case BQ_F32: return deq_fast_go<bqk::kF32>(codes, absmax, y, n16, log2_block, tab, sm_count, stream);
+        case BQ_F16: return deq_fast_go<bqk::kF16>(codes, absmax, y, n16, log2_block, tab, sm_count, stream);
+        default: return deq_fast_go<bqk::kBF16>(codes, absmax, y, n16, log2_block, tab, sm_count, stream);
+    }
+}
+
+cudaError_t launch_deq_general(int ydt, const uint8_t* codes, const float* absmax, void* y, size_t n, size_t block, size_t first_elem,
+                               const bqk::DeviceTables& tab, int sm_count, cudaStream_t stream) {
+    size_t grid = (n - first_elem + 255) / 256;
+    const size_t cap = size_t(sm_count) * 8;
+    if (grid > cap) grid = cap;
+    if (grid < 1) grid = 1;
+    switch (ydt) {
+        case BQ_F32: bqk::deq_general<bqk::kF32><<<unsigned(grid), 256, 0, stream>>>(codes, absmax, y, n, block, first_elem, tab); break;
+        case BQ_F16: bqk::deq_general<bqk::kF16><<<unsigned(grid), 256, 0, stream>>>(codes, absmax, y, n, block, first_elem, tab); break;
+        default: bqk::deq_general<bqk::kBF16><<<unsigned(grid), 256, 0, stream>>>(codes, absmax, y, n, block, first_elem, tab); break;
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace bql

@@ -1,0 +1,446 @@
+// bq_kernels.cuh -- device code of libbq (sm_100a).
+//
+// Three kernels:
+//   fwd_fast     : quantize, or the fused quantize->dequantize roundtrip, for power-of-two
+//                  blocks on 16-byte aligned tensors.  One pass over HBM: a tile of the
+//                  input sits in registers between the absmax reduction and the search.
+//   deq_fast     : dequantize, 16 codes per thread.
+//   *_general    : any block size, any alignment, any codebook; one warp per block.
+//
+// Arithmetic contract shared by all of them (it is what makes the results bit-identical
+// to the plain definition): absmax is an exact fp32 max; xhat is the correctly rounded
+// fp32 quotient x / absmax; the code is #{ j : t_j < xhat } over the exact midpoints; the
+// inverse is one fp32 multiply followed by a round-to-nearest-even conversion.  No fused
+// contraction, fast division or flush-to-zero is allowed to change any of these.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace bqk {
+
+enum { kF32 = 0, kF16 = 1, kBF16 = 2 };
+
+constexpr int kCells = 897;
+constexpr uint32_t kCellBase = 0x38800000u >> 17;
+constexpr float kCellBias = 6.103515625e-05f;          // 2^-14
+
+// Shared-memory image of the folded search tables.  Every entry is replicated 32 times,
+// one copy per lane in that lane's own bank (entry e, lane l at byte e*128 + l*4), so a
+// data-dependent lookup by 32 lanes never has a bank conflict.
+constexpr uint32_t kTkOff = 0;                          // 128 threshold keys
+constexpr uint32_t kCmOff = kTkOff + 128u * 128u;       // 129 magnitudes (132 rows reserved)
+constexpr uint32_t kGuessOff = kCmOff + 132u * 128u;    // kCells first guesses
+constexpr uint32_t kRedOff = kGuessOff + uint32_t(kCells) * 128u;   // cross-warp partial maxima
+constexpr uint32_t kFwdSmemBytes = kRedOff + 2u * 32u * 4u;
+
+constexpr uint32_t kDeqSmemBytes = 256u * 128u;         // signed code values, replicated per lane
+
+struct DeviceTables {
+    const float* values;        // [256]
+    const float* thr_down;      // [256], last = +inf
+    const uint32_t* tk;         // [128]
+    const float* cmag;          // [132]
+    const uint32_t* guess;      // [kCells]
+    float neg_limit;
+};
+
+// ------------------------------------------------------------------------------------------
+// small helpers
+
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
+    uint32_t v;
+    asm("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts_u32(uint32_t addr, uint32_t v) {
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint4 ldg_stream_16(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void stg_stream_16(void* p, uint4 v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void stg_stream_8(void* p, uint2 v) {
+    asm volatile("st.global.cs.v2.u32 [%0], {%1,%2};" ::"l"(p), "r"(v.x), "r"(v.y) : "memory");
+}
+__device__ __forceinline__ void stg_stream_4(void* p, uint32_t v) {
+    asm volatile("st.global.cs.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+template <int DT> struct Elem;
+template <> struct Elem<kF32> { static constexpr int kBytes = 4; static constexpr int kPerChunk = 4; };
+template <> struct Elem<kF16> { static constexpr int kBytes = 2; static constexpr int kPerChunk = 8; };
+template <> struct Elem<kBF16> { static constexpr int kBytes = 2; static constexpr int kPerChunk = 8; };
+
+// Widen the elements of one 16-byte chunk to fp32 (exact).
+template <int DT, int N>
+__device__ __forceinline__ void widen_chunk(const uint4& w, float (&f)[N]) {
+    const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+    if constexpr (DT == kF32) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) f[i] = __uint_as_float(u[i]);
+    } else if constexpr (DT == kBF16) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            f[2 * i] = __uint_as_float(u[i] << 16);
+            f[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 p = __half22float2(*reinterpret_cast<const __half2*>(&u[i]));
+            f[2 * i] = p.x;
+            f[2 * i + 1] = p.y;
+        }
+    }
+}
+
+// Round-to-nearest-even narrowing of one chunk's worth of fp32 values.
+template <int DT, int N>
+__device__ __forceinline__ uint4 narrow_chunk(const float (&v)[N]) {
+    uint32_t u[4];
+    if constexpr (DT == kF32) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) u[i] = __float_as_uint(v[i]);
+    } else if constexpr (DT == kBF16) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const __nv_bfloat162 p = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+            u[i] = *reinterpret_cast<const uint32_t*>(&p);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const __half2 p = __floats2half2_rn(v[2 * i], v[2 * i + 1]);
+            u[i] = *reinterpret_cast<const uint32_t*>(&p);
+        }
+    }
+    return make_uint4(u[0], u[1], u[2], u[3]);
+}
+
+template <int DT>
+__device__ __forceinline__ float load_elem(const void* x, size_t i) {
+    if constexpr (DT == kF32) return static_cast<const float*>(x)[i];
+    else if constexpr (DT == kBF16) return __uint_as_float(uint32_t(static_cast<const uint16_t*>(x)[i]) << 16);
+    else return __half2float(static_cast<const __half*>(x)[i]);
+}
+
+template <int DT>
+__device__ __forceinline__ void store_elem(void* y, size_t i, float v) {
+    if constexpr (DT == kF32) static_cast<float*>(y)[i] = v;
+    else if constexpr (DT == kBF16) static_cast<__nv_bfloat16*>(y)[i] = __float2bfloat16_rn(v);
+    else static_cast<__half*>(y)[i] = __float2half_rn(v);
+}
+
+// ------------------------------------------------------------------------------------------
+// Normalisation.  The contract is the correctly rounded quotient x / d.
+//
+// For 16-bit inputs (significands of at most 11 bits) and d within [2^-64, 2^64] the
+// quotient is obtained from a per-block correctly rounded reciprocal r = RN(1/d):
+//     q0 = RN(x r);  e = x - d q0 (one exact fma);  q = RN(q0 + e r).
+// That this equals RN(x / d) for every pair of significands and every exponent gap that
+// can reach a non-zero code is checked exhaustively on the host by the test-suite; outside
+// the exponent window, and for fp32 inputs, the IEEE division is used.
+
+template <int DT>
+struct Normaliser {
+    float d, r;
+    bool fast;
+    __device__ __forceinline__ explicit Normaliser(float absmax) {
+        d = (absmax != 0.0f) ? absmax : 1.0f;
+        if constexpr (DT == kF32) {
+            fast = false;
+            r = 0.0f;
+        } else {
+            fast = (d >= 5.421010862427522e-20f) && (d <= 1.8446744073709552e19f);    // 2^-64 .. 2^64
+            r = __frcp_rn(d);
+        }
+    }
+    __device__ __forceinline__ float quick(float x) const {
+        const float q0 = __fmul_rn(x, r);
+        const float e = __fmaf_rn(-d, q0, x);
+        return __fmaf_rn(e, r, q0);
+    }
+    __device__ __forceinline__ float exact(float x) const { return __fdiv_rn(x, d); }
+};
+
+// ------------------------------------------------------------------------------------------
+// Folded search: first guess from the cell table, one key compare, optional value lookup.
+
+struct Found {
+    uint32_t guess128;     // first guess * 128
+    bool bump;             // true: one more threshold lies below the key
+    uint32_t bits;         // bit pattern of the clamped xhat
+};
+
+__device__ __forceinline__ Found search_folded(float xhat, float neg_limit, uint32_t sm_lane) {
+    Found f;
+    xhat = fmaxf(xhat, neg_limit);
+    f.bits = __float_as_uint(xhat);
+    const uint32_t key = __funnelshift_l(f.bits, f.bits, 1);
+    const float mb = fabsf(xhat) + kCellBias;
+    const uint32_t cell128 = (__float_as_uint(mb) >> 10) & 0xffffff80u;
+    f.guess128 = lds_u32(sm_lane + cell128 + (kGuessOff - kCellBase * 128u));
+    const uint32_t tk = lds_u32(sm_lane + f.guess128 + kTkOff);
+    f.bump = tk < key;
+    return f;
+}
+
+__device__ __forceinline__ uint32_t code_of(const Found& f) {
+    const uint32_t p = (f.guess128 >> 7) + (f.bump ? 1u : 0u);
+    const uint32_t sm = uint32_t(int32_t(f.bits) >> 31);           // all ones for a negative xhat
+    return 127u + ((p ^ sm) - sm);
+}
+
+// c[code] * absmax as one rounding: the magnitude times the signed absmax, plus +0.0 so
+// that a zero magnitude gives +0.0 whatever the sign.
+__device__ __forceinline__ float value_of(const Found& f, float absmax, uint32_t sm_lane) {
+    const uint32_t va = sm_lane + f.guess128 + (f.bump ? (kCmOff + 128u) : kCmOff);
+    const float cm = __uint_as_float(lds_u32(va));
+    const float as = __uint_as_float(__float_as_uint(absmax) | (f.bits & 0x80000000u));
+    return __fmaf_rn(cm, as, 0.0f);
+}
+
+__device__ __forceinline__ void fill_fwd_tables(const DeviceTables& t, uint32_t sm_base, int nthreads) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = nthreads >> 5;
+    const uint32_t sm_lane = sm_base + uint32_t(lane) * 4u;
+    for (int e = warp; e < 128; e += nwarps) sts_u32(sm_lane + kTkOff + uint32_t(e) * 128u, __ldg(t.tk + e));
+    for (int e = warp; e < 132; e += nwarps) sts_u32(sm_lane + kCmOff + uint32_t(e) * 128u, __float_as_uint(__ldg(t.cmag + e)));
+#pragma unroll 4
+    for (int e = warp; e < kCells; e += nwarps) sts_u32(sm_lane + kGuessOff + uint32_t(e) * 128u, __ldg(t.guess + e));
+}
+
+// ------------------------------------------------------------------------------------------
+// fwd_fast
+//
+//   XDT          element type of x (and of y: the fused kernel keeps the type)
+//   B            block size, a power of two, >= 64
+//   R            16-byte chunks ("rows") each thread keeps in registers per tile
+//   TW           warps that share one block (1 unless B > R * 32 * elements-per-chunk)
+//   WRITE_Y      store the dequantised tensor
+//   WRITE_Q      store codes and absmax
+//
+// A row is 32 consecutive chunks, one per lane (512 contiguous bytes).  Blocks no longer
+// than a row occupy B / kPerChunk consecutive lanes of one row and are reduced with
+// segmented shuffles; longer blocks take R rows of TW warps.
+template <int XDT, int B, int R, int TW, bool WRITE_Y, bool WRITE_Q, int NT>
+__global__ void __launch_bounds__(NT, 1)
+fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__ codes, float* __restrict__ absmax_out,
+         size_t n_full, DeviceTables tab) {
+    constexpr int EPC = Elem<XDT>::kPerChunk;
+    constexpr int EB = Elem<XDT>::kBytes;
+    constexpr int ROW = 32 * EPC;
+    constexpr bool IN_ROW = (B <= ROW);
+    constexpr int LPB = IN_ROW ? B / EPC : 32;                 // lanes per block inside a row
+    static_assert(IN_ROW ? (TW == 1) : (TW * R * ROW == B), "tile must be one block when blocks span rows");
+    constexpr int WARPS = NT / 32;
+
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const uint32_t sm_base = uint32_t(__cvta_generic_to_shared(smem_raw));
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t sm_lane = sm_base + uint32_t(lane) * 4u;
+
+    fill_fwd_tables(tab, sm_base, NT);
+    __syncthreads();
+
+    const float neg_limit = tab.neg_limit;
+    const char* xb = static_cast<const char*>(x);
+    char* yb = static_cast<char*>(y);
+
+    constexpr size_t TILE = size_t(TW) * R * ROW;
+    const size_t ntiles = (n_full + TILE - 1) / TILE;
+    const size_t team = size_t(blockIdx.x) * (WARPS / TW) + size_t(warp / TW);
+    const size_t nteams = size_t(gridDim.x) * (WARPS / TW);
+    const int wt = warp % TW;
+    int parity = 0;
+
+    for (size_t t = team; t < ntiles; t += nteams) {
+        const size_t base = t * TILE + size_t(wt) * R * ROW + size_t(lane) * EPC;
+        uint4 w[R];
+        bool valid[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const size_t off = base + size_t(r) * ROW;
+            valid[r] = IN_ROW ? (off < n_full) : true;
+            w[r] = valid[r] ? ldg_stream_16(xb + off * EB) : make_uint4(0, 0, 0, 0);
+        }
+        float f[R][EPC];
+        float amax[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            widen_chunk<XDT>(w[r], f[r]);
+            float a = 0.0f;
+#pragma unroll
+            for (int i = 0; i < EPC; ++i) a = fmaxf(a, fabsf(f[r][i]));
+            amax[r] = a;
+        }
+        if constexpr (IN_ROW) {
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+#pragma unroll
+                for (int s = 1; s < LPB; s <<= 1) amax[r] = fmaxf(amax[r], __shfl_xor_sync(0xffffffffu, amax[r], s));
+        } else {
+            float a = amax[0];
+#pragma unroll
+            for (int r = 1; r < R; ++r) a = fmaxf(a, amax[r]);
+#pragma unroll
+            for (int s = 1; s < 32; s <<= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, s));
+            if constexpr (TW > 1) {
+                // partial maxima of the team's warps meet in shared memory; two slots alternate so
+                // that one barrier per tile is enough
+                const uint32_t slot = sm_base + kRedOff + uint32_t(parity) * 128u + uint32_t(warp / TW) * TW * 4u;
+                if (lane == 0) sts_u32(slot + uint32_t(wt) * 4u, __float_as_uint(a));
+                asm volatile("bar.sync %0, %1;" ::"r"(1 + warp / TW), "r"(TW * 32) : "memory");
+#pragma unroll
+                for (int k = 0; k < TW; ++k) a = fmaxf(a, __uint_as_float(lds_u32(slot + uint32_t(k) * 4u)));
+                parity ^= 1;
+            }
+#pragma unroll
+            for (int r = 0; r < R; ++r) amax[r] = a;
+        }
+
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const Normaliser<XDT> nrm(amax[r]);
+            bool quick = false;
+            if constexpr (XDT != kF32) quick = __all_sync(0xffffffffu, nrm.fast);
+            float out[EPC];
+            uint32_t q[EPC];
+#pragma unroll
+            for (int i = 0; i < EPC; ++i) {
+                const float xhat = quick ? nrm.quick(f[r][i]) : nrm.exact(f[r][i]);
+                const Found fd = search_folded(xhat, neg_limit, sm_lane);
+                if constexpr (WRITE_Q) q[i] = code_of(fd);
+                if constexpr (WRITE_Y) out[i] = value_of(fd, amax[r], sm_lane);
+            }
+            if (valid[r]) {
+                const size_t off = base + size_t(r) * ROW;
+                if constexpr (WRITE_Y) stg_stream_16(yb + off * EB, narrow_chunk<XDT>(out));
+                if constexpr (WRITE_Q) {
+                    if constexpr (EPC == 8) {
+                        const uint32_t lo = q[0] | (q[1] << 8) | (q[2] << 16) | (q[3] << 24);
+                        const uint32_t hi = q[4] | (q[5] << 8) | (q[6] << 16) | (q[7] << 24);
+                        stg_stream_8(codes + off, make_uint2(lo, hi));
+                    } else {
+                        stg_stream_4(codes + off, q[0] | (q[1] << 8) | (q[2] << 16) | (q[3] << 24));
+                    }
+                    if constexpr (IN_ROW) {
+                        if ((lane % LPB) == 0) absmax_out[off / B] = amax[r];
+                    }
+                }
+            }
+        }
+        if constexpr (WRITE_Q && !IN_ROW) {
+            if (lane == 0 && wt == 0) absmax_out[t] = amax[0];
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// deq_fast: 16 codes per thread, signed code values replicated per lane in shared memory.
+template <int YDT, int NT>
+__global__ void __launch_bounds__(NT)
+deq_fast(const uint8_t* __restrict__ codes, const float* __restrict__ absmax, void* __restrict__ y, size_t n16 /* n / 16 */,
+         int log2_block, DeviceTables tab) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const uint32_t sm_base = uint32_t(__cvta_generic_to_shared(smem_raw));
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t sm_lane = sm_base + uint32_t(lane) * 4u;
+    for (int e = warp; e < 256; e += NT / 32) sts_u32(sm_lane + uint32_t(e) * 128u, __float_as_uint(__ldg(tab.values + e)));
+    __syncthreads();
+
+    char* yb = static_cast<char*>(y);
+    constexpr int EB = Elem<YDT>::kBytes;
+    const size_t stride = size_t(gridDim.x) * NT;
+    for (size_t c = size_t(blockIdx.x) * NT + threadIdx.x; c < n16; c += stride) {
+        const uint4 w = ldg_stream_16(codes + c * 16);
+        const float a = __ldg(absmax + ((c * 16) >> log2_block));
+        const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+        float v[16];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            v[4 * k + 0] = __fmul_rn(__uint_as_float(lds_u32(sm_lane + ((u[k] << 7) & 0x7f80u))), a);
+            v[4 * k + 1] = __fmul_rn(__uint_as_float(lds_u32(sm_lane + ((u[k] >> 1) & 0x7f80u))), a);
+            v[4 * k + 2] = __fmul_rn(__uint_as_float(lds_u32(sm_lane + ((u[k] >> 9) & 0x7f80u))), a);
+            v[4 * k + 3] = __fmul_rn(__uint_as_float(lds_u32(sm_lane + ((u[k] >> 17) & 0x7f80u))), a);
+        }
+        char* out = yb + c * 16 * EB;
+        if constexpr (YDT == kF32) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float t[4] = {v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]};
+                stg_stream_16(out + 16 * k, narrow_chunk<kF32>(t));
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const float t[8] = {v[8 * k], v[8 * k + 1], v[8 * k + 2], v[8 * k + 3], v[8 * k + 4], v[8 * k + 5], v[8 * k + 6], v[8 * k + 7]};
+                stg_stream_16(out + 16 * k, narrow_chunk<YDT>(t));
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// General kernels: any block, any alignment, any valid codebook.  One warp per block, two
+// passes over the block (the second pass hits L1/L2), 8-step branch-free binary search over
+// the 255 round-down midpoints in shared memory.
+
+__device__ __forceinline__ int search_general(const float* thr /* shared, 256 entries */, float xhat) {
+    int q = 0;
+#pragma unroll
+    for (int s = 128; s >= 1; s >>= 1) q += (thr[q + s - 1] < xhat) ? s : 0;
+    return q;
+}
+
+template <int XDT, int YDT, bool WRITE_Y, bool WRITE_Q>
+__global__ void __launch_bounds__(256)
+fwd_general(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__ codes, float* __restrict__ absmax_out,
+            size_t n, size_t block, size_t first_block, DeviceTables tab) {
+    __shared__ float thr[256];
+    __shared__ float val[256];
+    thr[threadIdx.x] = tab.thr_down[threadIdx.x];
+    val[threadIdx.x] = tab.values[threadIdx.x];
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const size_t nb = (n + block - 1) / block;
+    const size_t wstride = size_t(gridDim.x) * 8;
+    for (size_t b = first_block + size_t(blockIdx.x) * 8 + (threadIdx.x >> 5); b < nb; b += wstride) {
+        const size_t lo = b * block;
+        const size_t hi = (lo + block < n) ? lo + block : n;
+        float a = 0.0f;
+        for (size_t i = lo + lane; i < hi; i += 32) a = fmaxf(a, fabsf(load_elem<XDT>(x, i)));
+#pragma unroll
+        for (int s = 1; s < 32; s <<= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, s));
+        const float d = (a != 0.0f) ? a : 1.0f;
+        for (size_t i = lo + lane; i < hi; i += 32) {
+            const float xhat = __fdiv_rn(load_elem<XDT>(x, i), d);
+            const int q = search_general(thr, xhat);
+            if constexpr (WRITE_Q) codes[i] = uint8_t(q);
+            if constexpr (WRITE_Y) store_elem<YDT>(y, i, __fmul_rn(val[q], a));
+        }
+        if constexpr (WRITE_Q) {
+            if (lane == 0) absmax_out[b] = a;
+        }
+    }
+}
+
+template <int YDT>
+__global__ void __launch_bounds__(256)
+deq_general(const uint8_t* __restrict__ codes, const float* __restrict__ absmax, void* __restrict__ y, size_t n, size_t block,
+            size_t first_elem, DeviceTables tab) {
+    __shared__ float val[256];
+    val[threadIdx.x] = tab.values[threadIdx.x];
+    __syncthreads();
+    const size_t stride = size_t(gridDim.x) * 256;
+    for (size_t i = first_elem + size_t(blockIdx.x) * 256 + threadIdx.x; i < n; i += stride)
+        store_elem<YDT>(y, i, __fmul_rn(val[codes[i]], absmax[i / block]));
+}
+
+}  // namespace bqk

@@ -1,0 +1,48 @@
+// bq_launch.h -- launchers of the kernel instantiations (internal to libbq).
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include "../../include/bq.h"
+#include "bq_kernels.cuh"
+#include "bq_tables.h"
+
+namespace bql {
+
+// Tuned forward kernels, one translation unit per element type.
+cudaError_t launch_fwd_fast_f32(int block, bool write_y, bool write_q, const void* x, void* y, uint8_t* codes, float* absmax,
+                                size_t n_full, const bqk::DeviceTables& tab, int sm_count, int device, cudaStream_t stream);
+cudaError_t launch_fwd_fast_f16(int block, bool write_y, bool write_q, const void* x, void* y, uint8_t* codes, float* absmax,
+                                size_t n_full, const bqk::DeviceTables& tab, int sm_count, int device, cudaStream_t stream);
+cudaError_t launch_fwd_fast_bf16(int block, bool write_y, bool write_q, const void* x, void* y, uint8_t* codes, float* absmax,
+                                 size_t n_full, const bqk::DeviceTables& tab, int sm_count, int device, cudaStream_t stream);
+
+inline cudaError_t launch_fwd_fast(int xdt, int block, bool write_y, bool write_q, const void* x, void* y, uint8_t* codes,
+                                   float* absmax, size_t n_full, const bqk::DeviceTables& tab, int sm_count, int device,
+                                   cudaStream_t stream) {
+    switch (xdt) {
+        case BQ_F32: return launch_fwd_fast_f32(block, write_y, write_q, x, y, codes, absmax, n_full, tab, sm_count, device, stream);
+        case BQ_F16: return launch_fwd_fast_f16(block, write_y, write_q, x, y, codes, absmax, n_full, tab, sm_count, device, stream);
+        default: return launch_fwd_fast_bf16(block, write_y, write_q, x, y, codes, absmax, n_full, tab, sm_count, device, stream);
+    }
+}
+
+cudaError_t launch_fwd_general(int xdt, int ydt, bool write_y, bool write_q, const void* x, void* y, uint8_t* codes, float* absmax,
+                               size_t n, size_t block, size_t first_block, const bqk::DeviceTables& tab, int sm_count,
+                               cudaStream_t stream);
+cudaError_t launch_deq_fast(int ydt, const uint8_t* codes, const float* absmax, void* y, size_t n16, int log2_block,
+                            const bqk::DeviceTables& tab, int sm_count, int device, cudaStream_t stream);
+cudaError_t launch_deq_general(int ydt, const uint8_t* codes, const float* absmax, void* y, size_t n, size_t block, size_t first_elem,
+                               const bqk::DeviceTables& tab, int sm_count, cudaStream_t stream);
+
+// Kernels that need more than 48 KB of dynamic shared memory must opt in once per device.
+template <auto Kernel>
+inline cudaError_t allow_smem(int bytes, int device) {
+    static bool done[64] = {};
+    if (device >= 0 && device < 64 && done[device]) return cudaSuccess;
+    const cudaError_t e = cudaFuncSetAttribute(Kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess && device >= 0 && device < 64) done[device] = true;
+    return e;
+}
+
+}  // namespace bql

@@ -1,0 +1,61 @@
+"""The C-ABI library loads and exports every function include/bq.h declares; argument
+errors come back as status codes before anything touches a device (CPU only)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "bq.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(bq_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(bq):
+    from paper_2407_19775_b200 import binding
+    L = binding.lib()
+    names = _declared()
+    assert {"bq_make_codebook", "bq_free_codebook", "bq_quantize", "bq_dequantize", "bq_roundtrip"} <= set(names)
+    for name in names:
+        assert hasattr(L, name), name
+    assert set(binding.SYMBOLS) == set(names)
+
+
+def test_status_strings(bq):
+    from paper_2407_19775_b200 import binding
+    L = binding.lib()
+    seen = {L.bq_status_string(i).decode() for i in range(7)}
+    assert len(seen) == 7 and L.bq_status_string(0) == b"ok"
+    assert L.bq_status_string(99) == b"unknown status"
+
+
+def test_argument_errors_need_no_device(bq):
+    from paper_2407_19775_b200 import binding
+    L = binding.lib()
+    one = ctypes.c_void_p(16)        # never dereferenced: every call below fails a check first
+    assert L.bq_quantize(one, 9, 4, 64, one, one, one, None) == 2          # dtype
+    assert L.bq_quantize(one, 0, 4, 0, one, one, one, None) == 3           # block
+    assert L.bq_quantize(one, 0, 1 << 41, 64, one, one, one, None) == 4    # size
+    assert L.bq_quantize(one, 0, 4, 64, None, one, one, None) == 5         # codebook handle
+    assert L.bq_quantize(None, 0, 0, 64, one, None, None, None) == 0       # n == 0: nothing to do
+    assert L.bq_quantize(None, 0, 4, 64, one, one, one, None) == 1         # null x
+    assert L.bq_dequantize(one, one, 4, 64, one, None, 0, None) == 1
+    assert L.bq_dequantize(one, one, 4, 64, one, one, 5, None) == 2
+    assert L.bq_roundtrip(one, 0, 4, 64, one, one, 0, one, None, None) == 1   # one side output without the other
+    assert L.bq_roundtrip(one, 0, 4, -1, one, one, 0, None, None, None) == 3
+    out = ctypes.c_void_p()
+    assert L.bq_make_codebook(7, None, None, ctypes.byref(out)) == 5
+    assert L.bq_make_codebook(0, None, None, None) == 1
+    assert L.bq_free_codebook(None) == 0
+
+
+def test_missing_library_is_an_error(monkeypatch):
+    from paper_2407_19775_b200 import binding
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libbq.so")
+    with pytest.raises(binding.BqError):
+        binding.lib()

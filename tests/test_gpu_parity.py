@@ -1,0 +1,288 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the
+same seeded bytes.  Codes, absmax and dequantised output must be bit-identical."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import midpoints, round_down32
+from paper_2407_19775_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+ODT = {torch.float32: oracle.F32, torch.float16: oracle.F16, torch.bfloat16: oracle.BF16}
+THREADS = max(1, (os.cpu_count() or 2))
+CANARY = 0xA5
+
+
+@pytest.fixture(scope="module")
+def gcb(bq):
+    return bq.Codebook(device="cuda:0")
+
+
+def _bits(t):
+    return workloads.as_numpy_bits(t)
+
+
+def _padded(n, dtype, dev, pad=64):
+    """An output buffer with canary bytes after its n elements."""
+    esz = torch.empty(0, dtype=dtype).element_size()
+    raw = torch.full((n * esz + pad,), CANARY, dtype=torch.uint8, device=dev)
+    return raw, raw[: n * esz].view(dtype)
+
+
+def _canary_ok(raw, nbytes):
+    return bool((raw[nbytes:] == CANARY).all().item())
+
+
+def check_all_ops(bq, gcb, cb, x_cpu: torch.Tensor, block: int, ydtypes=None, offset_elems: int = 0):
+    """quantize, dequantize, roundtrip (with and without side outputs) against the oracle."""
+    dev = torch.device("cuda:0")
+    x_cpu = x_cpu.contiguous().view(-1)
+    n = x_cpu.numel()
+    nb = (n + block - 1) // block
+    xdt = x_cpu.dtype
+    if offset_elems:
+        holder = torch.empty(n + offset_elems, dtype=xdt, device=dev)
+        xd = holder[offset_elems:]
+        xd.copy_(x_cpu)
+    else:
+        xd = x_cpu.to(dev)
+    craw, codes = _padded(n, torch.uint8, dev)
+    araw, absmax = _padded(nb, torch.float32, dev)
+    bq.bq_quantize(xd, block, gcb, codes, absmax)
+    ref_y, ref_c, ref_a = {}, None, None
+    for ydt in (ydtypes or [xdt]):
+        y, c, a = oracle.roundtrip_sharded(_bits(x_cpu), ODT[xdt], block, cb, ODT[ydt], THREADS)
+        ref_y[ydt], ref_c, ref_a = y, c, a
+    torch.cuda.synchronize()
+    assert np.array_equal(codes.cpu().numpy(), ref_c), "codes"
+    assert np.array_equal(absmax.cpu().numpy().view(np.uint32), ref_a.view(np.uint32)), "absmax"
+    assert _canary_ok(craw, n) and _canary_ok(araw, nb * 4)
+    for ydt, yref in ref_y.items():
+        esz = torch.empty(0, dtype=ydt).element_size()
+        yraw, y = _padded(n, ydt, dev)
+        bq.bq_dequantize(codes, absmax, block, gcb, ydt, y)
+        y2raw, y2 = _padded(n, ydt, dev)
+        bq.bq_roundtrip(xd, block, gcb, y_out=y2)
+        y3raw, y3 = _padded(n, ydt, dev)
+        c3raw, c3 = _padded(n, torch.uint8, dev)
+        a3raw, a3 = _padded(nb, torch.float32, dev)
+        bq.bq_roundtrip(xd, block, gcb, y_out=y3, codes_out=c3, absmax_out=a3)
+        torch.cuda.synchronize()
+        assert np.array_equal(_bits(y.cpu()), yref), f"dequantize {ydt}"
+        assert np.array_equal(_bits(y2.cpu()), yref), f"roundtrip {ydt}"
+        assert np.array_equal(_bits(y3.cpu()), yref), f"roundtrip+side {ydt}"
+        assert np.array_equal(c3.cpu().numpy(), ref_c) and np.array_equal(a3.cpu().numpy().view(np.uint32), ref_a.view(np.uint32))
+        for raw, nbytes in ((yraw, n * esz), (y2raw, n * esz), (y3raw, n * esz), (c3raw, n), (a3raw, nb * 4)):
+            assert _canary_ok(raw, nbytes)
+
+
+# ------------------------------------------------------------------------------- the configs
+
+def test_codebook_matches_oracle(bq, gcb, cb):
+    assert np.array_equal(gcb.values.view(np.uint32), cb.view(np.uint32))
+    assert gcb.folded
+
+
+def test_config_tiny(bq, gcb, cb):
+    check_all_ops(bq, gcb, cb, workloads.make("tiny"), 64, ydtypes=[torch.float32, torch.bfloat16, torch.float16])
+
+
+def test_config_prefill7b(bq, gcb, cb):
+    check_all_ops(bq, gcb, cb, workloads.make("prefill7b"), 256)
+
+
+def test_config_decode70b(bq, gcb, cb):
+    check_all_ops(bq, gcb, cb, workloads.make("decode70b"), 64)
+
+
+def _sampled_full_size(bq, gcb, cb, name, blocks, nsample=1536):
+    """Full-size run in the launch configuration the benchmark times; the oracle checks a
+    sample of whole blocks (first, last and random ones) bit for bit, and device-side
+    properties cover every element."""
+    dev = torch.device("cuda:0")
+    x_cpu = workloads.make(name).view(-1)
+    n = x_cpu.numel()
+    xd = x_cpu.to(dev)
+    xb = _bits(x_cpu)
+    odt = ODT[x_cpu.dtype]
+    rng = np.random.default_rng(123)
+    for block in blocks:
+        nb = n // block
+        codes, absmax = bq.bq_quantize(xd, block, gcb)
+        y = bq.bq_dequantize(codes, absmax, block, gcb, x_cpu.dtype)
+        y2 = bq.bq_roundtrip(xd, block, gcb)
+        torch.cuda.synchronize()
+        # every element: fused == separate; absmax == max|x| per block; error bound
+        assert torch.equal(y.view(torch.int16), y2.view(-1).view(torch.int16))
+        ref_absmax = xd.view(nb, block).abs().amax(dim=1).float()
+        assert torch.equal(absmax.view(torch.int32), ref_absmax.view(torch.int32))
+        step = 1 << 26
+        for s in range(0, n, step):
+            e = min(n, s + step)
+            a_el = absmax[s // block:(e + block - 1) // block].repeat_interleave(block)[: e - s]
+            err = (xd[s:e].float() - y[s:e].float()).abs()
+            bound = a_el * (0.00703125 + 2.0 ** -22) + (y[s:e].float().abs() * 2.0 ** -8)    # code gap + bf16 rounding of y
+            assert bool((err <= bound).all().item())
+        # sampled blocks, bit for bit
+        pick = np.unique(np.concatenate([[0, 1, nb - 2, nb - 1], rng.integers(0, nb, max(8, nsample * 64 // block))]))
+        idx = (pick[:, None] * block + np.arange(block)[None, :]).reshape(-1)
+        xs = np.ascontiguousarray(xb[idx])
+        ys, cs, as_ = oracle.roundtrip_sharded(xs, odt, block, cb, odt, THREADS)
+        tidx = torch.from_numpy(idx).to(dev)
+        assert np.array_equal(codes[tidx].cpu().numpy(), cs)
+        assert np.array_equal(absmax[torch.from_numpy(pick).to(dev)].cpu().numpy().view(np.uint32), as_.view(np.uint32))
+        assert np.array_equal(_bits(y[tidx].cpu()), ys)
+        del codes, absmax, y, y2
+
+
+def test_config_moe_prefill_full_size(bq, gcb, cb):
+    _sampled_full_size(bq, gcb, cb, "moe_prefill", [2048])
+
+
+def test_config_sweep1g_full_size(bq, gcb, cb):
+    _sampled_full_size(bq, gcb, cb, "sweep1g", [64, 256, 1024, 4096])
+
+
+# ------------------------------------------------------------------------------- shapes, tails, alignment
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("block", [64, 128, 256, 512, 1024, 2048, 4096])
+def test_tuned_blocks_many_tiles_and_ragged_tail(bq, gcb, cb, dtype, block):
+    g = torch.Generator().manual_seed(block + 17)
+    n = 148 * 16 * 1024 + 5 * block + 37             # more than one tile per warp of a full grid, then a short block
+    n = min(n, 3_000_000)
+    n = (n // block) * block + 37
+    x = (torch.randn(n, generator=g) * (1.0 + 30.0 * (torch.rand(n, generator=g) < 0.002))).to(dtype)
+    check_all_ops(bq, gcb, cb, x, block)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("n,block", [(1, 64), (63, 64), (64, 64), (65, 64), (1000, 7), (257, 1), (4096, 100), (5000, 4096),
+                                       (300, 3000), (2048 * 3 + 1, 2048)])
+def test_small_and_odd_shapes(bq, gcb, cb, dtype, n, block):
+    g = torch.Generator().manual_seed(n * 31 + block)
+    x = torch.randn(n, generator=g).to(dtype)
+    check_all_ops(bq, gcb, cb, x, block)
+
+
+@pytest.mark.parametrize("dtype,offset", [(torch.bfloat16, 1), (torch.bfloat16, 4), (torch.float32, 1), (torch.float16, 3)])
+def test_unaligned_input_pointer(bq, gcb, cb, dtype, offset):
+    g = torch.Generator().manual_seed(5)
+    x = torch.randn(64 * 300 + 11, generator=g).to(dtype)
+    check_all_ops(bq, gcb, cb, x, 64, offset_elems=offset)
+
+
+def test_mixed_output_types(bq, gcb, cb):
+    g = torch.Generator().manual_seed(8)
+    x = (torch.randn(256 * 100 + 3, generator=g) * 200.0).to(torch.bfloat16)
+    check_all_ops(bq, gcb, cb, x, 256, ydtypes=[torch.float32, torch.float16, torch.bfloat16])
+    x = (torch.randn(64 * 100, generator=g) * 1e5).float()            # overflows fp16 on the way out
+    check_all_ops(bq, gcb, cb, x, 64, ydtypes=[torch.float16, torch.bfloat16])
+
+
+def test_in_place_roundtrip(bq, gcb, cb):
+    x = workloads.make("prefill7b", rows=32).view(-1)
+    xd = x.to("cuda:0")
+    bq.bq_roundtrip(xd, 256, gcb, y_out=xd)
+    torch.cuda.synchronize()
+    yref = oracle.roundtrip(_bits(x), oracle.BF16, 256, cb, oracle.BF16)
+    assert np.array_equal(_bits(xd.cpu()), yref)
+
+
+def test_non_default_stream(bq, gcb, cb):
+    x = workloads.make("decode70b", rows=8).view(-1)
+    s = torch.cuda.Stream(device="cuda:0")
+    with torch.cuda.stream(s):
+        xd = x.to("cuda:0", non_blocking=False)
+        y = bq.bq_roundtrip(xd, 64, gcb)
+    s.synchronize()
+    assert np.array_equal(_bits(y.cpu()), oracle.roundtrip(_bits(x), oracle.F16, 64, cb, oracle.F16))
+
+
+# ------------------------------------------------------------------------------- degenerate values
+
+def test_zero_blocks_negative_zero_and_sign_of_absmax(bq, gcb, cb):
+    x = torch.zeros(64 * 8)
+    x[5] = -0.0
+    x[64] = -3.0                                      # absmax element negative -> xhat = -1 -> code 0
+    x[65:128] = torch.linspace(-3.0, 3.0, 63)
+    x[128:192] = 2.5                                  # all equal
+    x[192:256] = -2.5
+    x[256] = 1e-30; x[257] = -1e-38; x[258] = 1e-45   # tiny absmax, subnormals inside
+    x[320] = 3e38; x[321] = -1e30                     # huge absmax
+    x[384] = 1.0; x[385] = 2.7e-7; x[386] = -2.7e-7; x[387] = 2.8e-7; x[388] = -2.8e-7
+    x[448] = -1.0; x[449] = -0.9965; x[450] = -0.99649; x[451] = -0.997; x[452] = 0.997; x[453] = 0.9964
+    for dtype in (torch.float32, torch.bfloat16):
+        check_all_ops(bq, gcb, cb, x.to(dtype), 64)
+
+
+def test_every_breakpoint_exactly(bq, gcb, cb):
+    """Blocks whose absmax is a power of two, so xhat is exactly the chosen pattern: the
+    round-down midpoint of every code pair, its neighbours, and every code value."""
+    pats = []
+    for t in midpoints(cb):
+        lo = round_down32(t)
+        pats += [np.nextafter(lo, np.float32(-np.inf)), lo, np.nextafter(lo, np.float32(np.inf))]
+    pats += list(cb)
+    pats = np.array(pats, np.float32)
+    for scale in (1.0, 2.0 ** -40, 2.0 ** 70):       # inside and outside the reciprocal window (irrelevant for fp32)
+        rows = []
+        for i in range(0, pats.size, 63):
+            chunk = pats[i:i + 63]
+            rows.append(np.concatenate([[1.0], chunk, np.zeros(63 - chunk.size, np.float32)]))
+        x = torch.from_numpy((np.concatenate(rows) * np.float32(scale)).astype(np.float32))
+        check_all_ops(bq, gcb, cb, x, 64)
+
+
+@pytest.mark.parametrize("dtype,sig", [(torch.bfloat16, 8), (torch.float16, 11)])
+def test_all_significand_pairs_of_16bit_inputs(bq, gcb, cb, dtype, sig):
+    """Every (absmax significand, element significand) pair at a few exponent gaps: the
+    tuned kernels' reciprocal-based quotient must land on the same code as the division."""
+    half = 1 << (sig - 1)
+    sigs = (half + np.arange(half)).astype(np.float64)
+    gaps = (0, 1, 2, 3, 6, 10) if sig == 8 else (0, 1, 4)
+    blocks = []
+    for md in range(0, half, 1 if sig == 8 else 5):
+        d = sigs[md]
+        for gap in gaps:
+            xs = sigs * 2.0 ** (-gap)
+            xs = xs[xs <= d]
+            xs = np.concatenate([xs, -xs])
+            for i in range(0, xs.size, 63):
+                chunk = xs[i:i + 63]
+                blocks.append(np.concatenate([[d], chunk, np.zeros(63 - chunk.size)]))
+    x = np.concatenate(blocks) * 2.0 ** (-(sig - 1) - 3)
+    check_all_ops(bq, gcb, cb, torch.from_numpy(x.astype(np.float32)).to(dtype), 64)
+
+
+def test_fp16_subnormals_and_extremes(bq, gcb, cb):
+    bits = np.arange(65536, dtype=np.uint16)
+    t = workloads.from_numpy_bits(bits, torch.float16)
+    t = t[torch.isfinite(t.float())]
+    t = t[: (t.numel() // 64) * 64]
+    check_all_ops(bq, gcb, cb, t, 64)
+    b = workloads.from_numpy_bits(bits, torch.bfloat16)
+    b = b[torch.isfinite(b.float())]
+    b = b[: (b.numel() // 256) * 256]
+    check_all_ops(bq, gcb, cb, b, 256)                # blocks spanning 2^-133 .. 2^127: outside the reciprocal window
+
+
+# ------------------------------------------------------------------------------- user codebooks
+
+def test_user_codebook_general_path(bq, cb):
+    import ctypes
+    lin = np.concatenate([np.linspace(-1, 0, 128), np.linspace(0, 1, 129)[1:]]).astype(np.float32)
+    ucb = bq.Codebook(kind=bq.USER, user_values=lin, device="cuda:0")
+    assert not ucb.folded and np.array_equal(ucb.values, lin)
+    g = torch.Generator().manual_seed(4)
+    x = torch.randn(64 * 500 + 9, generator=g).to(torch.bfloat16)
+    check_all_ops(bq, ucb, lin, x, 64)
+    with pytest.raises(bq.BqError):
+        bq.Codebook(kind=bq.USER, user_values=np.linspace(-1, 1, 256).astype(np.float32), device="cuda:0")
+    mirrored = bq.Codebook(kind=bq.USER, user_values=cb.copy(), device="cuda:0")
+    assert mirrored.folded
+    check_all_ops(bq, mirrored, cb, x, 64)
