@@ -1,0 +1,53 @@
+"""Runs a few launches of one library call on a prefix of a workload, for profilers.
+
+    python -m paper_2407_19775_b200.profile_case --op roundtrip --block 4096 --rows 8192 --launches 3
+
+`--rows 8192` of `sweep1g` is 64 Mi bf16 elements (128 MiB in, larger than L2) and keeps the
+device footprint well under 1 GB, which is what a counter-collecting profiler wants.  Prints
+the CUDA-event time of each launch.
+"""
+from __future__ import annotations
+
+import argparse
+
+import torch
+
+from . import Codebook, bq_dequantize, bq_quantize, bq_roundtrip, workloads
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", default="sweep1g")
+    ap.add_argument("--op", default="roundtrip", choices=["quantize", "dequantize", "roundtrip", "roundtrip_side"])
+    ap.add_argument("--block", type=int, default=4096)
+    ap.add_argument("--rows", type=int, default=8192)
+    ap.add_argument("--launches", type=int, default=3)
+    args = ap.parse_args()
+    dev = torch.device("cuda:0")
+    x = workloads.make(args.workload, rows=args.rows).view(-1).to(dev)
+    n = x.numel()
+    cb = Codebook(device=dev)
+    codes = torch.empty(n, dtype=torch.uint8, device=dev)
+    absmax = torch.empty((n + args.block - 1) // args.block, dtype=torch.float32, device=dev)
+    y = torch.empty_like(x)
+    if args.op == "dequantize":
+        bq_quantize(x, args.block, cb, codes, absmax)
+    torch.cuda.synchronize()
+    for i in range(args.launches):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        if args.op == "quantize":
+            bq_quantize(x, args.block, cb, codes, absmax)
+        elif args.op == "dequantize":
+            bq_dequantize(codes, absmax, args.block, cb, x.dtype, y)
+        elif args.op == "roundtrip":
+            bq_roundtrip(x, args.block, cb, y_out=y)
+        else:
+            bq_roundtrip(x, args.block, cb, y_out=y, codes_out=codes, absmax_out=absmax)
+        e1.record()
+        torch.cuda.synchronize()
+        print(f"{args.op} block={args.block} n={n} launch {i}: {e0.elapsed_time(e1):.4f} ms")
+
+
+if __name__ == "__main__":
+    main()
