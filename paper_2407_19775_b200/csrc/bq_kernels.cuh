@@ -34,7 +34,7 @@ constexpr uint32_t kTkOff = 0;                          // 128 threshold keys
 constexpr uint32_t kCmOff = kTkOff + 128u * 128u;       // 129 magnitudes (132 rows reserved)
 constexpr uint32_t kGuessOff = kCmOff + 132u * 128u;    // kCells first guesses
 constexpr uint32_t kRedOff = kGuessOff + uint32_t(kCells) * 128u;   // cross-warp partial maxima
-constexpr uint32_t kFwdSmemBytes = kRedOff + 2u * 32u * 4u;
+constexpr uint32_t kFwdSmemBytes = kRedOff + 2u * 32u * 4u + 128u;    // + slack to align the base to 128 bytes
 
 constexpr uint32_t kDeqSmemBytes = 256u * 128u;         // signed code values, replicated per lane
 
@@ -139,70 +139,59 @@ __device__ __forceinline__ void store_elem(void* y, size_t i, float v) {
 }
 
 // ------------------------------------------------------------------------------------------
-// Normalisation.  The contract is the correctly rounded quotient x / d.
-//
-// For 16-bit inputs (significands of at most 11 bits) and d within [2^-64, 2^64] the
-// quotient is obtained from a per-block correctly rounded reciprocal r = RN(1/d):
-//     q0 = RN(x r);  e = x - d q0 (one exact fma);  q = RN(q0 + e r).
-// That this equals RN(x / d) for every pair of significands and every exponent gap that
-// can reach a non-zero code is checked exhaustively on the host by the test-suite; outside
-// the exponent window, and for fp32 inputs, the IEEE division is used.
-
-template <int DT>
-struct Normaliser {
-    float d, r;
-    bool fast;
-    __device__ __forceinline__ explicit Normaliser(float absmax) {
-        d = (absmax != 0.0f) ? absmax : 1.0f;
-        if constexpr (DT == kF32) {
-            fast = false;
-            r = 0.0f;
-        } else {
-            fast = (d >= 5.421010862427522e-20f) && (d <= 1.8446744073709552e19f);    // 2^-64 .. 2^64
-            r = __frcp_rn(d);
-        }
-    }
-    __device__ __forceinline__ float quick(float x) const {
-        const float q0 = __fmul_rn(x, r);
-        const float e = __fmaf_rn(-d, q0, x);
-        return __fmaf_rn(e, r, q0);
-    }
-    __device__ __forceinline__ float exact(float x) const { return __fdiv_rn(x, d); }
-};
-
-// ------------------------------------------------------------------------------------------
 // Folded search: first guess from the cell table, one key compare, optional value lookup.
+//
+// Shared-memory contents (all per lane, see the layout above): the guess table holds, for
+// each cell, the ADDRESS of this lane's copy of TK[guess]; the magnitude row of the same
+// index sits kCmOff - kTkOff bytes further, the next magnitude 128 bytes after that.
 
 struct Found {
-    uint32_t guess128;     // first guess * 128
-    bool bump;             // true: one more threshold lies below the key
+    uint32_t tk_addr;      // shared address of this lane's TK[guess]
+    uint32_t key;          // rotate-left-by-one of the clamped xhat's bits
     uint32_t bits;         // bit pattern of the clamped xhat
 };
 
-__device__ __forceinline__ Found search_folded(float xhat, float neg_limit, uint32_t sm_lane) {
+__device__ __forceinline__ Found search_folded(float xhat, float neg_limit, uint32_t guess_lane) {
     Found f;
     xhat = fmaxf(xhat, neg_limit);
     f.bits = __float_as_uint(xhat);
-    const uint32_t key = __funnelshift_l(f.bits, f.bits, 1);
+    f.key = __funnelshift_l(f.bits, f.bits, 1);
     const float mb = fabsf(xhat) + kCellBias;
-    const uint32_t cell128 = (__float_as_uint(mb) >> 10) & 0xffffff80u;
-    f.guess128 = lds_u32(sm_lane + cell128 + (kGuessOff - kCellBase * 128u));
-    const uint32_t tk = lds_u32(sm_lane + f.guess128 + kTkOff);
-    f.bump = tk < key;
+    uint32_t ga;
+    // cell * 128 + base as one multiply-add keeps this off the (busier) integer ALU
+    asm("mad.lo.u32 %0, %1, 128, %2;" : "=r"(ga) : "r"(__float_as_uint(mb) >> 17), "r"(guess_lane));
+    f.tk_addr = lds_u32(ga);
     return f;
 }
 
-__device__ __forceinline__ uint32_t code_of(const Found& f) {
-    const uint32_t p = (f.guess128 >> 7) + (f.bump ? 1u : 0u);
+// guess_lane for the call above: this lane's column of the guess table, rebased so that
+// the cell index can be used without subtracting the index of the first cell.
+__device__ __forceinline__ uint32_t guess_lane_of(uint32_t sm_lane) { return sm_lane + kGuessOff - kCellBase * 128u; }
+
+__device__ __forceinline__ uint32_t code_of(const Found& f, uint32_t tk_lane) {
+    const uint32_t tk = lds_u32(f.tk_addr);
+    const uint32_t p = ((f.tk_addr - tk_lane) >> 7) + (tk < f.key ? 1u : 0u);
     const uint32_t sm = uint32_t(int32_t(f.bits) >> 31);           // all ones for a negative xhat
     return 127u + ((p ^ sm) - sm);
 }
 
+// Magnitude of the chosen code: TK[guess] < key picks the upper of two neighbouring rows.
+__device__ __forceinline__ float magnitude_of(const Found& f) {
+    uint32_t cm;
+    asm("{\n\t.reg .pred p;\n\t.reg .u32 t;\n\t"
+        "ld.shared.u32 t, [%1];\n\t"
+        "setp.lt.u32 p, t, %2;\n\t"
+        "@p ld.shared.u32 %0, [%1+%3];\n\t"
+        "@!p ld.shared.u32 %0, [%1+%4];\n\t}"
+        : "=r"(cm)
+        : "r"(f.tk_addr), "r"(f.key), "n"(kCmOff - kTkOff + 128u), "n"(kCmOff - kTkOff));
+    return __uint_as_float(cm);
+}
+
 // c[code] * absmax as one rounding: the magnitude times the signed absmax, plus +0.0 so
 // that a zero magnitude gives +0.0 whatever the sign.
-__device__ __forceinline__ float value_of(const Found& f, float absmax, uint32_t sm_lane) {
-    const uint32_t va = sm_lane + f.guess128 + (f.bump ? (kCmOff + 128u) : kCmOff);
-    const float cm = __uint_as_float(lds_u32(va));
+__device__ __forceinline__ float value_of(const Found& f, float absmax) {
+    const float cm = magnitude_of(f);
     const float as = __uint_as_float(__float_as_uint(absmax) | (f.bits & 0x80000000u));
     return __fmaf_rn(cm, as, 0.0f);
 }
@@ -213,7 +202,36 @@ __device__ __forceinline__ void fill_fwd_tables(const DeviceTables& t, uint32_t 
     for (int e = warp; e < 128; e += nwarps) sts_u32(sm_lane + kTkOff + uint32_t(e) * 128u, __ldg(t.tk + e));
     for (int e = warp; e < 132; e += nwarps) sts_u32(sm_lane + kCmOff + uint32_t(e) * 128u, __float_as_uint(__ldg(t.cmag + e)));
 #pragma unroll 4
-    for (int e = warp; e < kCells; e += nwarps) sts_u32(sm_lane + kGuessOff + uint32_t(e) * 128u, __ldg(t.guess + e));
+    for (int e = warp; e < kCells; e += nwarps)
+        sts_u32(sm_lane + kGuessOff + uint32_t(e) * 128u, __ldg(t.guess + e) + sm_lane + kTkOff);
+}
+
+// Two fp32 lanes per instruction (sm_100 packed fp32 arithmetic).
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+    uint64_t v;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(a), "f"(b));
+    return v;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ float max3_abs(float a, float b, float c) {      // max(|a|, |b|, |c|)
+    float d;
+    asm("max.abs.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float rcp_approx(float d) {
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(d));
+    return r;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -228,7 +246,18 @@ __device__ __forceinline__ void fill_fwd_tables(const DeviceTables& t, uint32_t 
 //
 // A row is 32 consecutive chunks, one per lane (512 contiguous bytes).  Blocks no longer
 // than a row occupy B / kPerChunk consecutive lanes of one row and are reduced with
-// segmented shuffles; longer blocks take R rows of TW warps.
+// segmented shuffles; longer blocks take R rows of TW warps.  The loads of the next tile
+// are issued as soon as the current one has been widened, so they fly during the search.
+//
+// Normalisation.  The contract is the correctly rounded quotient x / d.  For 16-bit inputs
+// (significands of at most 11 bits) and d within [2^-64, 2^64] it is computed as
+//     q0 = RN(x r);  e = x - d q0 (exact in one fma);  q = RN(q0 + e r)
+// from any r within 2^-22 (relative) of 1/d, here the hardware's approximate reciprocal:
+// q0 + e r differs from x/d by a relative 2^-44 at most, while a quotient of two 11-bit
+// significands that is not itself an fp32 stays at least a relative 2^-36 away from every
+// rounding boundary, and never sits on one.  The CPU tests check every significand pair
+// with r perturbed by +-2 ulp.  Outside that window, and for fp32 inputs, the IEEE division
+// is used.
 template <int XDT, int B, int R, int TW, bool WRITE_Y, bool WRITE_Q, int NT>
 __global__ void __launch_bounds__(NT, 1)
 fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__ codes, float* __restrict__ absmax_out,
@@ -241,10 +270,12 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
     static_assert(IN_ROW ? (TW == 1) : (TW * R * ROW == B), "tile must be one block when blocks span rows");
     constexpr int WARPS = NT / 32;
 
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    const uint32_t sm_base = uint32_t(__cvta_generic_to_shared(smem_raw));
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const uint32_t sm_base = (uint32_t(__cvta_generic_to_shared(smem_raw)) + 127u) & ~127u;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t sm_lane = sm_base + uint32_t(lane) * 4u;
+    const uint32_t guess_lane = guess_lane_of(sm_lane);
+    const uint32_t tk_lane = sm_lane + kTkOff;
 
     fill_fwd_tables(tab, sm_base, NT);
     __syncthreads();
@@ -258,18 +289,22 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
     const size_t team = size_t(blockIdx.x) * (WARPS / TW) + size_t(warp / TW);
     const size_t nteams = size_t(gridDim.x) * (WARPS / TW);
     const int wt = warp % TW;
+    const size_t lane_off = size_t(wt) * R * ROW + size_t(lane) * EPC;
     int parity = 0;
 
-    for (size_t t = team; t < ntiles; t += nteams) {
-        const size_t base = t * TILE + size_t(wt) * R * ROW + size_t(lane) * EPC;
-        uint4 w[R];
-        bool valid[R];
+    uint4 w[R];
+    auto load_tile = [&](size_t t) {
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            const size_t off = base + size_t(r) * ROW;
-            valid[r] = IN_ROW ? (off < n_full) : true;
-            w[r] = valid[r] ? ldg_stream_16(xb + off * EB) : make_uint4(0, 0, 0, 0);
+            const size_t off = t * TILE + lane_off + size_t(r) * ROW;
+            const bool ok = IN_ROW ? (off < n_full) : true;
+            w[r] = ok ? ldg_stream_16(xb + off * EB) : make_uint4(0, 0, 0, 0);
         }
+    };
+    if (team < ntiles) load_tile(team);
+
+    for (size_t t = team; t < ntiles; t += nteams) {
+        const size_t base = t * TILE + lane_off;
         float f[R][EPC];
         float amax[R];
 #pragma unroll
@@ -277,20 +312,26 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
             widen_chunk<XDT>(w[r], f[r]);
             float a = 0.0f;
 #pragma unroll
-            for (int i = 0; i < EPC; ++i) a = fmaxf(a, fabsf(f[r][i]));
+            for (int i = 0; i < EPC; i += 2) a = max3_abs(a, f[r][i], f[r][i + 1]);
             amax[r] = a;
         }
+        if (t + nteams < ntiles) load_tile(t + nteams);          // in flight during everything below
+
         if constexpr (IN_ROW) {
 #pragma unroll
-            for (int r = 0; r < R; ++r)
+            for (int r = 0; r < R; ++r) {
+                if constexpr (LPB == 32) {
+                    amax[r] = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(amax[r])));
+                } else {
 #pragma unroll
-                for (int s = 1; s < LPB; s <<= 1) amax[r] = fmaxf(amax[r], __shfl_xor_sync(0xffffffffu, amax[r], s));
+                    for (int s = 1; s < LPB; s <<= 1) amax[r] = fmaxf(amax[r], __shfl_xor_sync(0xffffffffu, amax[r], s));
+                }
+            }
         } else {
             float a = amax[0];
 #pragma unroll
             for (int r = 1; r < R; ++r) a = fmaxf(a, amax[r]);
-#pragma unroll
-            for (int s = 1; s < 32; s <<= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, s));
+            a = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(a)));
             if constexpr (TW > 1) {
                 // partial maxima of the team's warps meet in shared memory; two slots alternate so
                 // that one barrier per tile is enough
@@ -298,29 +339,62 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
                 if (lane == 0) sts_u32(slot + uint32_t(wt) * 4u, __float_as_uint(a));
                 asm volatile("bar.sync %0, %1;" ::"r"(1 + warp / TW), "r"(TW * 32) : "memory");
 #pragma unroll
-                for (int k = 0; k < TW; ++k) a = fmaxf(a, __uint_as_float(lds_u32(slot + uint32_t(k) * 4u)));
+                for (int k = 0; k < TW; ++k) {
+                    uint32_t v;
+                    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(slot + uint32_t(k) * 4u) : "memory");
+                    a = fmaxf(a, __uint_as_float(v));
+                }
                 parity ^= 1;
             }
 #pragma unroll
             for (int r = 0; r < R; ++r) amax[r] = a;
         }
 
+        // normalise the whole tile in place; one warp-uniform choice between the reciprocal
+        // route and the IEEE division keeps the per-element code free of branches
+        {
+            bool ok = (XDT != kF32);
+            float d[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                d[r] = (amax[r] != 0.0f) ? amax[r] : 1.0f;
+                ok = ok && (d[r] >= 5.421010862427522e-20f) && (d[r] <= 1.8446744073709552e19f);      // 2^-64 .. 2^64
+            }
+            bool quick = false;
+            if constexpr (XDT != kF32) quick = __all_sync(0xffffffffu, ok);
+            if (quick) {
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    const float rc = rcp_approx(d[r]);
+                    const uint64_t r2 = pack2(rc, rc), nd2 = pack2(-d[r], -d[r]);
+#pragma unroll
+                    for (int i = 0; i < EPC; i += 2) {
+                        const uint64_t x2 = pack2(f[r][i], f[r][i + 1]);
+                        const uint64_t q0 = mul2(x2, r2);
+                        const uint64_t e = fma2(nd2, q0, x2);
+                        unpack2(fma2(e, r2, q0), f[r][i], f[r][i + 1]);
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+#pragma unroll
+                    for (int i = 0; i < EPC; ++i) f[r][i] = __fdiv_rn(f[r][i], d[r]);
+            }
+        }
+
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            const Normaliser<XDT> nrm(amax[r]);
-            bool quick = false;
-            if constexpr (XDT != kF32) quick = __all_sync(0xffffffffu, nrm.fast);
             float out[EPC];
             uint32_t q[EPC];
 #pragma unroll
             for (int i = 0; i < EPC; ++i) {
-                const float xhat = quick ? nrm.quick(f[r][i]) : nrm.exact(f[r][i]);
-                const Found fd = search_folded(xhat, neg_limit, sm_lane);
-                if constexpr (WRITE_Q) q[i] = code_of(fd);
-                if constexpr (WRITE_Y) out[i] = value_of(fd, amax[r], sm_lane);
+                const Found fd = search_folded(f[r][i], neg_limit, guess_lane);
+                if constexpr (WRITE_Q) q[i] = code_of(fd, tk_lane);
+                if constexpr (WRITE_Y) out[i] = value_of(fd, amax[r]);
             }
-            if (valid[r]) {
-                const size_t off = base + size_t(r) * ROW;
+            const size_t off = base + size_t(r) * ROW;
+            if (IN_ROW ? (off < n_full) : true) {
                 if constexpr (WRITE_Y) stg_stream_16(yb + off * EB, narrow_chunk<XDT>(out));
                 if constexpr (WRITE_Q) {
                     if constexpr (EPC == 8) {

@@ -89,7 +89,7 @@ void hc_codes_of_bits(uint32_t lo, uint32_t count, uint8_t* out_folded, uint8_t*
     }
 }
 
-// Exhaustive check of the reciprocal-based quotient for inputs with `sig_bits`-bit
+// Exhaustive check of the reciprocal-based quotient (reciprocal perturbed by -2..+2 ulp) for inputs with `sig_bits`-bit
 // significands: d = (2^(sig_bits-1) + md) * 2^ed and x = (2^(sig_bits-1) + mx) * 2^(ed - gap ...)
 // for every pair of significands and every exponent gap 0..max_gap with |x| <= d.
 // Returns the number of pairs whose quotient differs from x / d; *code_mismatch counts
@@ -100,7 +100,10 @@ long hc_check_quick_division(int sig_bits, int max_gap, int d_exp, long* code_mi
     long bad = 0, bad_code = 0, cnt = 0;
     for (int md = 0; md < half; ++md) {
         const float d = std::ldexp(float(half + md), d_exp - (sig_bits - 1));
-        const float r = 1.0f / d;
+        for (int dr = -2; dr <= 2; ++dr) {
+        // any reciprocal within 2 ulp of the correctly rounded one (the kernel uses the
+        // hardware's approximate reciprocal, whose last bits are not specified)
+        const float r = bqt::u2f(bqt::f2u(1.0f / d) + uint32_t(dr));
         for (int gap = 0; gap <= max_gap; ++gap) {
             for (int mx = 0; mx < half; ++mx) {
                 const float x = std::ldexp(float(half + mx), d_exp - gap - (sig_bits - 1));
@@ -118,6 +121,7 @@ long hc_check_quick_division(int sig_bits, int max_gap, int d_exp, long* code_mi
                     }
                 }
             }
+        }
         }
     }
     *code_mismatch = bad_code;
