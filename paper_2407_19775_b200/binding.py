@@ -14,7 +14,7 @@ F32, F16, BF16 = 0, 1, 2
 DYNAMIC_TREE, USER = 0, 1
 _DT = {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libbq.so")
+LIB_PATH = os.environ.get("BQ_LIB", os.path.join(_HERE, "libbq.so"))    # BQ_LIB: load another build of the library
 _lib = None
 
 SYMBOLS = ("bq_make_codebook", "bq_free_codebook", "bq_quantize", "bq_dequantize", "bq_roundtrip",

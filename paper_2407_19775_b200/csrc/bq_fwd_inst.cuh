@@ -5,14 +5,20 @@
 namespace bql {
 namespace {
 
-constexpr int kNT = 512;
+#ifndef BQ_NT
+#define BQ_NT 512
+#endif
+#ifndef BQ_RMAX
+#define BQ_RMAX 4
+#endif
+constexpr int kNT = BQ_NT;
 
 // Tile shape per block size: R chunks per thread, TW warps per block.
 template <int XDT, int B> struct Shape {
     static constexpr int ROW = 32 * bqk::Elem<XDT>::kPerChunk;
     static constexpr bool IN_ROW = B <= ROW;
-    static constexpr int ROWS = IN_ROW ? 4 : B / ROW;          // rows one tile must cover
-    static constexpr int R = ROWS <= 4 ? ROWS : 4;
+    static constexpr int ROWS = IN_ROW ? BQ_RMAX : B / ROW;    // rows one tile must cover
+    static constexpr int R = ROWS <= BQ_RMAX ? ROWS : BQ_RMAX;
     static constexpr int TW = IN_ROW ? 1 : ROWS / R;
 };
 

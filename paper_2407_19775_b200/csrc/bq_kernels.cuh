@@ -23,16 +23,15 @@ namespace bqk {
 
 enum { kF32 = 0, kF16 = 1, kBF16 = 2 };
 
-constexpr int kCells = 897;
-constexpr uint32_t kCellBase = 0x38800000u >> 17;
-constexpr float kCellBias = 6.103515625e-05f;          // 2^-14
+constexpr uint32_t kKeyLow = 0x69000000u;              // key of +2^-22: keys are clamped to it from below
+constexpr uint32_t kCellBase = kKeyLow >> 18;
+constexpr int kCells = int((0x7F000001u >> 18) - kCellBase) + 1;      // 1409
 
 // Shared-memory image of the folded search tables.  Every entry is replicated 32 times,
 // one copy per lane in that lane's own bank (entry e, lane l at byte e*128 + l*4), so a
 // data-dependent lookup by 32 lanes never has a bank conflict.
-constexpr uint32_t kTkOff = 0;                          // 128 threshold keys
-constexpr uint32_t kCmOff = kTkOff + 128u * 128u;       // 129 magnitudes (132 rows reserved)
-constexpr uint32_t kGuessOff = kCmOff + 132u * 128u;    // kCells first guesses
+constexpr uint32_t kCmOff = 0;                          // 129 magnitudes (132 rows reserved)
+constexpr uint32_t kGuessOff = kCmOff + 132u * 128u;    // kCells count entries
 constexpr uint32_t kRedOff = kGuessOff + uint32_t(kCells) * 128u;   // cross-warp partial maxima
 constexpr uint32_t kFwdSmemBytes = kRedOff + 2u * 32u * 4u + 128u;    // + slack to align the base to 128 bytes
 
@@ -139,59 +138,41 @@ __device__ __forceinline__ void store_elem(void* y, size_t i, float v) {
 }
 
 // ------------------------------------------------------------------------------------------
-// Folded search: first guess from the cell table, one key compare, optional value lookup.
-//
-// Shared-memory contents (all per lane, see the layout above): the guess table holds, for
-// each cell, the ADDRESS of this lane's copy of TK[guess]; the magnitude row of the same
-// index sits kCmOff - kTkOff bytes further, the next magnitude 128 bytes after that.
+// Folded search (see bq_tables.h): one lookup of the cell's entry, one addition, and the
+// count of thresholds below the key sits in the top byte.
 
 struct Found {
-    uint32_t tk_addr;      // shared address of this lane's TK[guess]
-    uint32_t key;          // rotate-left-by-one of the clamped xhat's bits
+    uint32_t count;        // P = #{ thresholds below the key }, 0..128
     uint32_t bits;         // bit pattern of the clamped xhat
 };
+
+// guess_lane: this lane's column of the entry table, rebased by the index of the first cell.
+__device__ __forceinline__ uint32_t guess_lane_of(uint32_t sm_lane) { return sm_lane + kGuessOff - kCellBase * 128u; }
 
 __device__ __forceinline__ Found search_folded(float xhat, float neg_limit, uint32_t guess_lane) {
     Found f;
     xhat = fmaxf(xhat, neg_limit);
     f.bits = __float_as_uint(xhat);
-    f.key = __funnelshift_l(f.bits, f.bits, 1);
-    const float mb = fabsf(xhat) + kCellBias;
+    const uint32_t key = max(__funnelshift_l(f.bits, f.bits, 1), kKeyLow);
     uint32_t ga;
-    // cell * 128 + base as one multiply-add keeps this off the (busier) integer ALU
-    asm("mad.lo.u32 %0, %1, 128, %2;" : "=r"(ga) : "r"(__float_as_uint(mb) >> 17), "r"(guess_lane));
-    f.tk_addr = lds_u32(ga);
+    // cell * 128 + base as one multiply-add (the fp32 multiplier pipe has room; the integer
+    // ALU is the busiest unit of this kernel)
+    asm("mad.lo.u32 %0, %1, 128, %2;" : "=r"(ga) : "r"(key >> 18), "r"(guess_lane));
+    f.count = (lds_u32(ga) + key) >> 24;
     return f;
 }
 
-// guess_lane for the call above: this lane's column of the guess table, rebased so that
-// the cell index can be used without subtracting the index of the first cell.
-__device__ __forceinline__ uint32_t guess_lane_of(uint32_t sm_lane) { return sm_lane + kGuessOff - kCellBase * 128u; }
-
-__device__ __forceinline__ uint32_t code_of(const Found& f, uint32_t tk_lane) {
-    const uint32_t tk = lds_u32(f.tk_addr);
-    const uint32_t p = ((f.tk_addr - tk_lane) >> 7) + (tk < f.key ? 1u : 0u);
+__device__ __forceinline__ uint32_t code_of(const Found& f) {
     const uint32_t sm = uint32_t(int32_t(f.bits) >> 31);           // all ones for a negative xhat
-    return 127u + ((p ^ sm) - sm);
-}
-
-// Magnitude of the chosen code: TK[guess] < key picks the upper of two neighbouring rows.
-__device__ __forceinline__ float magnitude_of(const Found& f) {
-    uint32_t cm;
-    asm("{\n\t.reg .pred p;\n\t.reg .u32 t;\n\t"
-        "ld.shared.u32 t, [%1];\n\t"
-        "setp.lt.u32 p, t, %2;\n\t"
-        "@p ld.shared.u32 %0, [%1+%3];\n\t"
-        "@!p ld.shared.u32 %0, [%1+%4];\n\t}"
-        : "=r"(cm)
-        : "r"(f.tk_addr), "r"(f.key), "n"(kCmOff - kTkOff + 128u), "n"(kCmOff - kTkOff));
-    return __uint_as_float(cm);
+    return 127u + ((f.count ^ sm) - sm);
 }
 
 // c[code] * absmax as one rounding: the magnitude times the signed absmax, plus +0.0 so
 // that a zero magnitude gives +0.0 whatever the sign.
-__device__ __forceinline__ float value_of(const Found& f, float absmax) {
-    const float cm = magnitude_of(f);
+__device__ __forceinline__ float value_of(const Found& f, float absmax, uint32_t cm_lane) {
+    uint32_t va;
+    asm("mad.lo.u32 %0, %1, 128, %2;" : "=r"(va) : "r"(f.count), "r"(cm_lane));
+    const float cm = __uint_as_float(lds_u32(va));
     const float as = __uint_as_float(__float_as_uint(absmax) | (f.bits & 0x80000000u));
     return __fmaf_rn(cm, as, 0.0f);
 }
@@ -199,11 +180,9 @@ __device__ __forceinline__ float value_of(const Found& f, float absmax) {
 __device__ __forceinline__ void fill_fwd_tables(const DeviceTables& t, uint32_t sm_base, int nthreads) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = nthreads >> 5;
     const uint32_t sm_lane = sm_base + uint32_t(lane) * 4u;
-    for (int e = warp; e < 128; e += nwarps) sts_u32(sm_lane + kTkOff + uint32_t(e) * 128u, __ldg(t.tk + e));
     for (int e = warp; e < 132; e += nwarps) sts_u32(sm_lane + kCmOff + uint32_t(e) * 128u, __float_as_uint(__ldg(t.cmag + e)));
 #pragma unroll 4
-    for (int e = warp; e < kCells; e += nwarps)
-        sts_u32(sm_lane + kGuessOff + uint32_t(e) * 128u, __ldg(t.guess + e) + sm_lane + kTkOff);
+    for (int e = warp; e < kCells; e += nwarps) sts_u32(sm_lane + kGuessOff + uint32_t(e) * 128u, __ldg(t.guess + e));
 }
 
 // Two fp32 lanes per instruction (sm_100 packed fp32 arithmetic).
@@ -269,13 +248,14 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
     constexpr int LPB = IN_ROW ? B / EPC : 32;                 // lanes per block inside a row
     static_assert(IN_ROW ? (TW == 1) : (TW * R * ROW == B), "tile must be one block when blocks span rows");
     constexpr int WARPS = NT / 32;
+    static_assert(WARPS % TW == 0 && TW <= 15, "teams must tile the CTA, one named barrier each");
 
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const uint32_t sm_base = (uint32_t(__cvta_generic_to_shared(smem_raw)) + 127u) & ~127u;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t sm_lane = sm_base + uint32_t(lane) * 4u;
     const uint32_t guess_lane = guess_lane_of(sm_lane);
-    const uint32_t tk_lane = sm_lane + kTkOff;
+    const uint32_t cm_lane = sm_lane + kCmOff;
 
     fill_fwd_tables(tab, sm_base, NT);
     __syncthreads();
@@ -390,8 +370,8 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
 #pragma unroll
             for (int i = 0; i < EPC; ++i) {
                 const Found fd = search_folded(f[r][i], neg_limit, guess_lane);
-                if constexpr (WRITE_Q) q[i] = code_of(fd, tk_lane);
-                if constexpr (WRITE_Y) out[i] = value_of(fd, amax[r]);
+                if constexpr (WRITE_Q) q[i] = code_of(fd);
+                if constexpr (WRITE_Y) out[i] = value_of(fd, amax[r], cm_lane);
             }
             const size_t off = base + size_t(r) * ROW;
             if (IN_ROW ? (off < n_full) : true) {

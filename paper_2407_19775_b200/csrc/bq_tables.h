@@ -13,9 +13,16 @@
 // the count P = #{ p : TK[p] < key } equals #{theta_p < m} for xhat >= 0 and
 // #{theta_p <= m} for xhat < 0, which is what the tie rule needs on each side:
 //     code = 127 + P (xhat >= 0),  127 - min(P, 127) (xhat < 0).
-// A first-guess table over coarse cells of m (cell = bits(m + bias) >> 17) stores, per
-// cell, how many thresholds lie wholly below the cell; the cells are fine enough that at
-// most one more threshold can lie inside, so one compare against TK[guess] finishes.
+//
+// P comes from ONE table lookup and one addition.  Keys are clamped from below to
+// kKeyLow (the key of 2^-22, below the smallest threshold) and cut into cells of 2^18
+// consecutive keys (exponent plus 6 fraction bits of m); no cell holds more than one
+// threshold.  For the cell that starts at key S, with P0 thresholds below S and (at most)
+// one threshold TK inside it, the entry is
+//     E = (P0 << 24 | 0xFC0000 | (0x3FFFF - (TK - S))) - S        (mod 2^32)
+// so that E + key = P0 << 24 | 0xFC0000 | ... plus a carry out of bit 17 exactly when
+// key > TK; the six set bits pass that carry on into the count, and (E + key) >> 24 = P.
+// A cell without a threshold uses TK - S = 0x3FFFF, which never carries.
 #pragma once
 
 #include <cmath>
@@ -25,10 +32,10 @@
 
 namespace bqt {
 
-constexpr int kCells = 897;                 // cells of |xhat| + 2^-14 over [2^-14, 1 + 2^-14]
-constexpr float kCellBias = 6.103515625e-05f;   // 2^-14
-constexpr uint32_t kCellBase = 0x38800000u >> 17;   // cell index of the bias itself
-constexpr int kCellShift = 17;
+constexpr uint32_t kKeyLow = 0x69000000u;               // key of +2^-22
+constexpr int kCellShift = 18;
+constexpr uint32_t kCellBase = kKeyLow >> kCellShift;    // index of the first cell
+constexpr int kCells = int((0x7F000001u >> kCellShift) - kCellBase) + 1;    // up to the key of -1.0: 1409 cells
 
 inline uint32_t f2u(float f) { uint32_t u; std::memcpy(&u, &f, 4); return u; }
 inline float u2f(uint32_t u) { float f; std::memcpy(&f, &u, 4); return f; }
@@ -39,7 +46,7 @@ struct Tables {
     bool folded;              // true when the magnitude-folded tables below are valid
     uint32_t tk[128];         // folded threshold keys
     float cmag[132];          // cmag[p] = values[127 + p], p = 0..128 (padded)
-    uint32_t guess[kCells];   // per cell: (number of thresholds below the cell) * 128
+    uint32_t guess[kCells];   // per cell: the entry E described above
     float neg_limit;          // xhat is clamped from below to this before the folded search
 };
 
@@ -82,11 +89,6 @@ inline float round_down_to_float(double t) {
     return g;
 }
 
-inline uint32_t cell_of(float m) {              // m >= 0
-    const float mb = m + kCellBias;             // one fp32 add, as the kernel does it
-    return (f2u(mb) >> kCellShift) - kCellBase;
-}
-
 inline void build(Tables& T) {
     for (int j = 0; j < 255; ++j) {
         const double t = (double(T.values[j]) + double(T.values[j + 1])) * 0.5;   // exact (see header)
@@ -108,27 +110,20 @@ inline void build(Tables& T) {
     // negative side: P must not count theta_127 (there is no code below -c_254)
     T.neg_limit = -u2f((T.tk[127] - 1u) >> 1);
 
-    // first-guess cells: smallest m of each cell by bisection over the bit pattern of m
-    auto count_below = [&](uint32_t key) { int c = 0; for (int p = 0; p < 128; ++p) c += (T.tk[p] < key); return c; };
-    const uint32_t one = f2u(1.0f);
-    std::vector<uint32_t> first(kCells + 1);
-    for (int c = 0; c <= kCells; ++c) {
-        uint32_t lo = 0, hi = one + 1;              // smallest bits(m) in [0, one] with cell_of >= c; one+1 if none
-        while (lo < hi) {
-            const uint32_t mid = lo + (hi - lo) / 2;
-            if (cell_of(u2f(mid)) >= uint32_t(c)) hi = mid; else lo = mid + 1;
-        }
-        first[size_t(c)] = lo;
-    }
-    if (cell_of(1.0f) != uint32_t(kCells - 1)) { T.folded = false; return; }
+    if (T.tk[0] <= kKeyLow) { T.folded = false; return; }          // clamped keys must sit below every threshold
+    int p = 0;                                                       // thresholds below the current cell
     for (int c = 0; c < kCells; ++c) {
-        const uint32_t m_min = first[size_t(c)], m_next = first[size_t(c) + 1];
-        if (m_min >= m_next) { T.guess[c] = (c ? T.guess[c - 1] : 0u); continue; }    // empty cell
-        const int below = count_below(2u * m_min);                    // smallest key in the cell (positive sign)
-        const int upto = count_below(2u * (m_next - 1u) + 1u);        // largest key in the cell (negative sign)
-        if (upto - below > 1) { T.folded = false; return; }
-        // a cell above every threshold keeps guess 127: TK[127] < key holds throughout it
-        T.guess[c] = uint32_t(below > 127 ? 127 : below) * 128u;
+        const uint32_t start = (kCellBase + uint32_t(c)) << kCellShift;
+        const uint64_t end = uint64_t(start) + (1u << kCellShift);
+        uint32_t inside = 0x3FFFFu;
+        int count = 0;
+        while (p + count < 128 && uint64_t(T.tk[p + count]) < end) {
+            inside = T.tk[p + count] - start;
+            ++count;
+        }
+        if (count > 1) { T.folded = false; return; }
+        T.guess[c] = ((uint32_t(p) << 24) | 0xFC0000u | (0x3FFFFu - inside)) - start;
+        p += count;
     }
 }
 

@@ -21,17 +21,16 @@ void ensure() {
     g_ready = true;
 }
 
-struct Found { uint32_t guess128; bool bump; uint32_t bits; };
+struct Found { uint32_t count; uint32_t bits; };
 
 Found search_folded(float xhat) {
     Found f;
     xhat = std::fmax(xhat, g_tab.neg_limit);
     f.bits = bqt::f2u(xhat);
-    const uint32_t key = (f.bits << 1) | (f.bits >> 31);
-    const float mb = std::fabs(xhat) + bqt::kCellBias;
-    const uint32_t cell = (bqt::f2u(mb) >> 17) - bqt::kCellBase;
-    f.guess128 = g_tab.guess[cell];
-    f.bump = g_tab.tk[f.guess128 >> 7] < key;
+    uint32_t key = (f.bits << 1) | (f.bits >> 31);
+    if (key < bqt::kKeyLow) key = bqt::kKeyLow;
+    const uint32_t cell = (key >> 18) - bqt::kCellBase;
+    f.count = (g_tab.guess[cell] + key) >> 24;
     return f;
 }
 }  // namespace
@@ -60,15 +59,14 @@ int hc_user_tables_folded(const float* values) {
 int hc_code_folded(float xhat) {
     ensure();
     const Found f = search_folded(xhat);
-    const uint32_t p = (f.guess128 >> 7) + (f.bump ? 1u : 0u);
     const uint32_t sm = uint32_t(int32_t(f.bits) >> 31);
-    return int(127u + ((p ^ sm) - sm));
+    return int(127u + ((f.count ^ sm) - sm));
 }
 
 float hc_value_folded(float xhat, float absmax) {
     ensure();
     const Found f = search_folded(xhat);
-    const float cm = g_tab.cmag[(f.guess128 >> 7) + (f.bump ? 1u : 0u)];
+    const float cm = g_tab.cmag[f.count];
     const float as = bqt::u2f(bqt::f2u(absmax) | (f.bits & 0x80000000u));
     return std::fmaf(cm, as, 0.0f);
 }
