@@ -23,15 +23,26 @@ cudaError_t fwd_general_y(int ydt, bool wy, bool wq, const void* x, void* y, uin
     }
 }
 
-constexpr int kDeqNT = 512;
+#ifndef BQ_DEQ_NT
+#define BQ_DEQ_NT 512
+#endif
+#ifndef BQ_DEQ_U
+#define BQ_DEQ_U 2
+#endif
+#ifndef BQ_DEQ_CTAS
+#define BQ_DEQ_CTAS 2
+#endif
+constexpr int kDeqNT = BQ_DEQ_NT;
+constexpr int kDeqU = BQ_DEQ_U;
 
 template <int YDT>
 cudaError_t deq_fast_go(const uint8_t* codes, const float* absmax, void* y, size_t n16, int log2_block, const bqk::DeviceTables& tab,
                         int sm_count, cudaStream_t stream) {
-    size_t grid = (n16 + kDeqNT - 1) / kDeqNT;
-    const size_t cap = size_t(sm_count) * 4;
+    const size_t tile = size_t(kDeqNT) * kDeqU;
+    size_t grid = (n16 + tile - 1) / tile;
+    const size_t cap = size_t(sm_count) * BQ_DEQ_CTAS;
     if (grid > cap) grid = cap;
-    bqk::deq_fast<YDT, kDeqNT><<<unsigned(grid), kDeqNT, bqk::kDeqSmemBytes, stream>>>(codes, absmax, y, n16, log2_block, tab);
+    bqk::deq_fast<YDT, kDeqNT, kDeqU><<<unsigned(grid), kDeqNT, bqk::kDeqSmemBytes, stream>>>(codes, absmax, y, n16, log2_block, tab);
     return cudaGetLastError();
 }
 

@@ -142,7 +142,7 @@ __device__ __forceinline__ void store_elem(void* y, size_t i, float v) {
 // count of thresholds below the key sits in the top byte.
 
 struct Found {
-    uint32_t count;        // P = #{ thresholds below the key }, 0..128
+    uint32_t sum;          // entry + key: its top byte is 127 + P, the code of a non-negative xhat
     uint32_t bits;         // bit pattern of the clamped xhat
 };
 
@@ -158,20 +158,31 @@ __device__ __forceinline__ Found search_folded(float xhat, float neg_limit, uint
     // cell * 128 + base as one multiply-add (the fp32 multiplier pipe has room; the integer
     // ALU is the busiest unit of this kernel)
     asm("mad.lo.u32 %0, %1, 128, %2;" : "=r"(ga) : "r"(key >> 18), "r"(guess_lane));
-    f.count = (lds_u32(ga) + key) >> 24;
+    f.sum = lds_u32(ga) + key;
     return f;
 }
 
-__device__ __forceinline__ uint32_t code_of(const Found& f) {
-    const uint32_t sm = uint32_t(int32_t(f.bits) >> 31);           // all ones for a negative xhat
-    return 127u + ((f.count ^ sm) - sm);
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+// Four codes as one word.  The top bytes of the four sums are the codes for non-negative
+// values, c = 127 + P; a negative value takes 127 - P = (c ^ 0xFF) - 1.  Both byte gathers
+// are single byte-permutes (the second one replicates each sign bit over its byte), and the
+// subtraction cannot borrow between bytes because c ^ 0xFF >= 1 wherever 1 is subtracted.
+__device__ __forceinline__ uint32_t pack_codes(const Found& f0, const Found& f1, const Found& f2, const Found& f3) {
+    const uint32_t c = prmt(prmt(f0.sum, f1.sum, 0x0073u), prmt(f2.sum, f3.sum, 0x0073u), 0x5410u);
+    const uint32_t m = prmt(prmt(f0.bits, f1.bits, 0x00FBu), prmt(f2.bits, f3.bits, 0x00FBu), 0x5410u);     // 0x8 in a selector: replicate the sign
+    return (c ^ m) - (m & 0x01010101u);
 }
 
 // c[code] * absmax as one rounding: the magnitude times the signed absmax, plus +0.0 so
-// that a zero magnitude gives +0.0 whatever the sign.
+// that a zero magnitude gives +0.0 whatever the sign.  cm_lane is rebased by -127 rows.
 __device__ __forceinline__ float value_of(const Found& f, float absmax, uint32_t cm_lane) {
     uint32_t va;
-    asm("mad.lo.u32 %0, %1, 128, %2;" : "=r"(va) : "r"(f.count), "r"(cm_lane));
+    asm("mad.lo.u32 %0, %1, 128, %2;" : "=r"(va) : "r"(f.sum >> 24), "r"(cm_lane));
     const float cm = __uint_as_float(lds_u32(va));
     const float as = __uint_as_float(__float_as_uint(absmax) | (f.bits & 0x80000000u));
     return __fmaf_rn(cm, as, 0.0f);
@@ -255,7 +266,7 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t sm_lane = sm_base + uint32_t(lane) * 4u;
     const uint32_t guess_lane = guess_lane_of(sm_lane);
-    const uint32_t cm_lane = sm_lane + kCmOff;
+    const uint32_t cm_lane = sm_lane + kCmOff - 127u * 128u;
 
     fill_fwd_tables(tab, sm_base, NT);
     __syncthreads();
@@ -366,23 +377,20 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
 #pragma unroll
         for (int r = 0; r < R; ++r) {
             float out[EPC];
-            uint32_t q[EPC];
+            Found fd[EPC];
 #pragma unroll
             for (int i = 0; i < EPC; ++i) {
-                const Found fd = search_folded(f[r][i], neg_limit, guess_lane);
-                if constexpr (WRITE_Q) q[i] = code_of(fd);
-                if constexpr (WRITE_Y) out[i] = value_of(fd, amax[r], cm_lane);
+                fd[i] = search_folded(f[r][i], neg_limit, guess_lane);
+                if constexpr (WRITE_Y) out[i] = value_of(fd[i], amax[r], cm_lane);
             }
             const size_t off = base + size_t(r) * ROW;
             if (IN_ROW ? (off < n_full) : true) {
                 if constexpr (WRITE_Y) stg_stream_16(yb + off * EB, narrow_chunk<XDT>(out));
                 if constexpr (WRITE_Q) {
                     if constexpr (EPC == 8) {
-                        const uint32_t lo = q[0] | (q[1] << 8) | (q[2] << 16) | (q[3] << 24);
-                        const uint32_t hi = q[4] | (q[5] << 8) | (q[6] << 16) | (q[7] << 24);
-                        stg_stream_8(codes + off, make_uint2(lo, hi));
+                        stg_stream_8(codes + off, make_uint2(pack_codes(fd[0], fd[1], fd[2], fd[3]), pack_codes(fd[4], fd[5], fd[6], fd[7])));
                     } else {
-                        stg_stream_4(codes + off, q[0] | (q[1] << 8) | (q[2] << 16) | (q[3] << 24));
+                        stg_stream_4(codes + off, pack_codes(fd[0], fd[1], fd[2], fd[3]));
                     }
                     if constexpr (IN_ROW) {
                         if ((lane % LPB) == 0) absmax_out[off / B] = amax[r];
@@ -397,8 +405,10 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
 }
 
 // ------------------------------------------------------------------------------------------
-// deq_fast: 16 codes per thread, signed code values replicated per lane in shared memory.
-template <int YDT, int NT>
+// deq_fast: 16 codes per 128-bit load, U loads per thread per tile, signed code values
+// replicated per lane in shared memory.  The loads of the next tile (codes and the blocks'
+// absmax) are issued before the current tile is expanded.
+template <int YDT, int NT, int U>
 __global__ void __launch_bounds__(NT)
 deq_fast(const uint8_t* __restrict__ codes, const float* __restrict__ absmax, void* __restrict__ y, size_t n16 /* n / 16 */,
          int log2_block, DeviceTables tab) {
@@ -411,31 +421,54 @@ deq_fast(const uint8_t* __restrict__ codes, const float* __restrict__ absmax, vo
 
     char* yb = static_cast<char*>(y);
     constexpr int EB = Elem<YDT>::kBytes;
-    const size_t stride = size_t(gridDim.x) * NT;
-    for (size_t c = size_t(blockIdx.x) * NT + threadIdx.x; c < n16; c += stride) {
-        const uint4 w = ldg_stream_16(codes + c * 16);
-        const float a = __ldg(absmax + ((c * 16) >> log2_block));
-        const uint32_t u[4] = {w.x, w.y, w.z, w.w};
-        float v[16];
+    constexpr size_t TILE = size_t(NT) * U;                      // chunks per tile
+    const size_t ntiles = (n16 + TILE - 1) / TILE;
+    const int log2_chunks = log2_block - 4;                      // chunks per block
+
+    uint4 w[U];
+    float a[U];
+    auto load_tile = [&](size_t t) {
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            v[4 * k + 0] = __fmul_rn(__uint_as_float(lds_u32(sm_lane + ((u[k] << 7) & 0x7f80u))), a);
-            v[4 * k + 1] = __fmul_rn(__uint_as_float(lds_u32(sm_lane + ((u[k] >> 1) & 0x7f80u))), a);
-            v[4 * k + 2] = __fmul_rn(__uint_as_float(lds_u32(sm_lane + ((u[k] >> 9) & 0x7f80u))), a);
-            v[4 * k + 3] = __fmul_rn(__uint_as_float(lds_u32(sm_lane + ((u[k] >> 17) & 0x7f80u))), a);
+        for (int u = 0; u < U; ++u) {
+            const size_t c = t * TILE + size_t(u) * NT + threadIdx.x;
+            const bool ok = c < n16;
+            w[u] = ok ? ldg_stream_16(codes + c * 16) : make_uint4(0, 0, 0, 0);
+            a[u] = ok ? __ldg(absmax + (c >> log2_chunks)) : 0.0f;
         }
-        char* out = yb + c * 16 * EB;
-        if constexpr (YDT == kF32) {
+    };
+    if (blockIdx.x < ntiles) load_tile(blockIdx.x);
+    for (size_t t = blockIdx.x; t < ntiles; t += gridDim.x) {
+        uint4 cw[U];
+        float ca[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) { cw[u] = w[u]; ca[u] = a[u]; }
+        if (t + gridDim.x < ntiles) load_tile(t + gridDim.x);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t c = t * TILE + size_t(u) * NT + threadIdx.x;
+            if (c >= n16) continue;
+            const uint32_t q[4] = {cw[u].x, cw[u].y, cw[u].z, cw[u].w};
+            float v[16];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const float t[4] = {v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]};
-                stg_stream_16(out + 16 * k, narrow_chunk<kF32>(t));
+                v[4 * k + 0] = __fmul_rn(__uint_as_float(lds_u32(sm_lane + ((q[k] << 7) & 0x7f80u))), ca[u]);
+                v[4 * k + 1] = __fmul_rn(__uint_as_float(lds_u32(sm_lane + ((q[k] >> 1) & 0x7f80u))), ca[u]);
+                v[4 * k + 2] = __fmul_rn(__uint_as_float(lds_u32(sm_lane + ((q[k] >> 9) & 0x7f80u))), ca[u]);
+                v[4 * k + 3] = __fmul_rn(__uint_as_float(lds_u32(sm_lane + ((q[k] >> 17) & 0x7f80u))), ca[u]);
             }
-        } else {
+            char* out = yb + c * 16 * EB;
+            if constexpr (YDT == kF32) {
 #pragma unroll
-            for (int k = 0; k < 2; ++k) {
-                const float t[8] = {v[8 * k], v[8 * k + 1], v[8 * k + 2], v[8 * k + 3], v[8 * k + 4], v[8 * k + 5], v[8 * k + 6], v[8 * k + 7]};
-                stg_stream_16(out + 16 * k, narrow_chunk<YDT>(t));
+                for (int k = 0; k < 4; ++k) {
+                    const float tt[4] = {v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]};
+                    stg_stream_16(out + 16 * k, narrow_chunk<kF32>(tt));
+                }
+            } else {
+#pragma unroll
+                for (int k = 0; k < 2; ++k) {
+                    const float tt[8] = {v[8 * k], v[8 * k + 1], v[8 * k + 2], v[8 * k + 3], v[8 * k + 4], v[8 * k + 5], v[8 * k + 6], v[8 * k + 7]};
+                    stg_stream_16(out + 16 * k, narrow_chunk<YDT>(tt));
+                }
             }
         }
     }

@@ -19,9 +19,10 @@
 // consecutive keys (exponent plus 6 fraction bits of m); no cell holds more than one
 // threshold.  For the cell that starts at key S, with P0 thresholds below S and (at most)
 // one threshold TK inside it, the entry is
-//     E = (P0 << 24 | 0xFC0000 | (0x3FFFF - (TK - S))) - S        (mod 2^32)
-// so that E + key = P0 << 24 | 0xFC0000 | ... plus a carry out of bit 17 exactly when
-// key > TK; the six set bits pass that carry on into the count, and (E + key) >> 24 = P.
+//     E = ((127 + P0) << 24 | 0xFC0000 | (0x3FFFF - (TK - S))) - S        (mod 2^32)
+// so that E + key = (127 + P0) << 24 | 0xFC0000 | ... plus a carry out of bit 17 exactly when
+// key > TK; the six set bits pass that carry on into the top byte: (E + key) >> 24 = 127 + P,
+// which is the code itself for xhat >= 0.
 // A cell without a threshold uses TK - S = 0x3FFFF, which never carries.
 #pragma once
 
@@ -122,7 +123,7 @@ inline void build(Tables& T) {
             ++count;
         }
         if (count > 1) { T.folded = false; return; }
-        T.guess[c] = ((uint32_t(p) << 24) | 0xFC0000u | (0x3FFFFu - inside)) - start;
+        T.guess[c] = ((uint32_t(127 + p) << 24) | 0xFC0000u | (0x3FFFFu - inside)) - start;
         p += count;
     }
 }

@@ -30,7 +30,7 @@ Found search_folded(float xhat) {
     uint32_t key = (f.bits << 1) | (f.bits >> 31);
     if (key < bqt::kKeyLow) key = bqt::kKeyLow;
     const uint32_t cell = (key >> 18) - bqt::kCellBase;
-    f.count = (g_tab.guess[cell] + key) >> 24;
+    f.count = ((g_tab.guess[cell] + key) >> 24) - 127u;
     return f;
 }
 }  // namespace
