@@ -80,7 +80,7 @@ int bq_make_codebook(int kind, const float* user_values256, float* host_values_o
     bqt::build(cb->host);
     if (host_values_out256) std::memcpy(host_values_out256, cb->host.values, 256 * sizeof(float));
 
-    // one device allocation: values | thr_down | tk | cmag | guess
+    // one device allocation: values | thr_down | tk | cmag | guess  (the kernels rely on guess following cmag directly)
     const size_t words = 256 + 256 + 128 + 132 + bqt::kCells;
     cudaError_t e = cudaGetDevice(&cb->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&cb->sm_count, cudaDevAttrMultiProcessorCount, cb->device);
@@ -130,9 +130,9 @@ int forward(const void* x, int xdt, size_t n, int block, const bq_codebook* cb, 
                           (!write_q || (aligned(codes, 8) && aligned(absmax, 4)));
     if (can_tune && n >= B) {
         const size_t n_full = (n / B) * B;
-        cudaError_t e = bql::launch_fwd_fast(xdt, block, write_y, write_q, x, y, codes, absmax, n_full, cb->dev, cb->sm_count, cb->device, stream);
+        cudaError_t e = bql::launch_fwd_fast(xdt, block, write_y, write_q, x, y, codes, absmax, n_full, cb->dev, cb->sm_count, cb->device, stream,
+                                             &done);
         if (e != cudaSuccess) return cuda_fail(e);
-        done = n_full;
     }
     if (done < n) {
         cudaError_t e = bql::launch_fwd_general(xdt, ydt, write_y, write_q, x, y, codes, absmax, n, B, done / B, cb->dev, cb->sm_count, stream);

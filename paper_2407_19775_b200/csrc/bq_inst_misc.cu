@@ -23,6 +23,9 @@ cudaError_t fwd_general_y(int ydt, bool wy, bool wq, const void* x, void* y, uin
     }
 }
 
+#ifndef BQ_LITE_MAX_LOG2
+#define BQ_LITE_MAX_LOG2 21
+#endif
 #ifndef BQ_DEQ_NT
 #define BQ_DEQ_NT 512
 #endif
@@ -38,11 +41,16 @@ constexpr int kDeqU = BQ_DEQ_U;
 template <int YDT>
 cudaError_t deq_fast_go(const uint8_t* codes, const float* absmax, void* y, size_t n16, int log2_block, const bqk::DeviceTables& tab,
                         int sm_count, cudaStream_t stream) {
+    if (n16 <= (size_t(1) << (BQ_LITE_MAX_LOG2 + 2 - 4))) {      // up to 8 Mi elements: no shared-memory table, one chunk per thread
+        const size_t grid = (n16 + 255) / 256;
+        bqk::deq_fast<YDT, 256, 1, true><<<unsigned(grid), 256, 0, stream>>>(codes, absmax, y, n16, log2_block, tab);
+        return cudaGetLastError();
+    }
     const size_t tile = size_t(kDeqNT) * kDeqU;
     size_t grid = (n16 + tile - 1) / tile;
     const size_t cap = size_t(sm_count) * BQ_DEQ_CTAS;
     if (grid > cap) grid = cap;
-    bqk::deq_fast<YDT, kDeqNT, kDeqU><<<unsigned(grid), kDeqNT, bqk::kDeqSmemBytes, stream>>>(codes, absmax, y, n16, log2_block, tab);
+    bqk::deq_fast<YDT, kDeqNT, kDeqU, false><<<unsigned(grid), kDeqNT, bqk::kDeqSmemBytes, stream>>>(codes, absmax, y, n16, log2_block, tab);
     return cudaGetLastError();
 }
 

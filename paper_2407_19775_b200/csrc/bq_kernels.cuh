@@ -34,6 +34,7 @@ constexpr uint32_t kCmOff = 0;                          // 129 magnitudes (132 r
 constexpr uint32_t kGuessOff = kCmOff + 132u * 128u;    // kCells count entries
 constexpr uint32_t kRedOff = kGuessOff + uint32_t(kCells) * 128u;   // cross-warp partial maxima
 constexpr uint32_t kFwdSmemBytes = kRedOff + 2u * 32u * 4u + 128u;    // + slack to align the base to 128 bytes
+constexpr uint32_t kFwdLiteSmemBytes = 2u * 32u * 4u + 128u;
 
 constexpr uint32_t kDeqSmemBytes = 256u * 128u;         // signed code values, replicated per lane
 
@@ -146,19 +147,44 @@ struct Found {
     uint32_t bits;         // bit pattern of the clamped xhat
 };
 
-// guess_lane: this lane's column of the entry table, rebased by the index of the first cell.
-__device__ __forceinline__ uint32_t guess_lane_of(uint32_t sm_lane) { return sm_lane + kGuessOff - kCellBase * 128u; }
+// Where the two tables are read from.  The tuned kernels keep them in shared memory, one
+// copy per lane (built once per CTA: worth it when the CTA then streams megabytes); the
+// LITE kernels, used for small tensors where that set-up would dominate, read the 6 KB of
+// tables straight from global memory through L1.
+template <bool LITE> struct TabRef;
+template <> struct TabRef<false> {
+    uint32_t guess_lane;   // this lane's column of the entry table, rebased by the index of the first cell
+    uint32_t cm_lane;      // this lane's column of the magnitude table, rebased by -127 rows
+    __device__ __forceinline__ TabRef(const DeviceTables&, uint32_t sm_lane)
+        : guess_lane(sm_lane + kGuessOff - kCellBase * 128u), cm_lane(sm_lane + kCmOff - 127u * 128u) {}
+    // index * 128 + base as one multiply-add (the fp32 multiplier pipe has room; the integer
+    // ALU is the busiest unit of these kernels)
+    __device__ __forceinline__ uint32_t entry(uint32_t key) const {
+        uint32_t ga;
+        asm("mad.lo.u32 %0, %1, 128, %2;" : "=r"(ga) : "r"(key >> 18), "r"(guess_lane));
+        return lds_u32(ga);
+    }
+    __device__ __forceinline__ float magnitude(uint32_t sum) const {
+        uint32_t va;
+        asm("mad.lo.u32 %0, %1, 128, %2;" : "=r"(va) : "r"(sum >> 24), "r"(cm_lane));
+        return __uint_as_float(lds_u32(va));
+    }
+};
+template <> struct TabRef<true> {
+    const uint32_t* guess;
+    const float* cmag;
+    __device__ __forceinline__ TabRef(const DeviceTables& t, uint32_t) : guess(t.guess - kCellBase), cmag(t.cmag - 127) {}
+    __device__ __forceinline__ uint32_t entry(uint32_t key) const { return __ldg(guess + (key >> 18)); }
+    __device__ __forceinline__ float magnitude(uint32_t sum) const { return __ldg(cmag + (sum >> 24)); }
+};
 
-__device__ __forceinline__ Found search_folded(float xhat, float neg_limit, uint32_t guess_lane) {
+template <bool LITE>
+__device__ __forceinline__ Found search_folded(float xhat, float neg_limit, const TabRef<LITE>& tab) {
     Found f;
     xhat = fmaxf(xhat, neg_limit);
     f.bits = __float_as_uint(xhat);
     const uint32_t key = max(__funnelshift_l(f.bits, f.bits, 1), kKeyLow);
-    uint32_t ga;
-    // cell * 128 + base as one multiply-add (the fp32 multiplier pipe has room; the integer
-    // ALU is the busiest unit of this kernel)
-    asm("mad.lo.u32 %0, %1, 128, %2;" : "=r"(ga) : "r"(key >> 18), "r"(guess_lane));
-    f.sum = lds_u32(ga) + key;
+    f.sum = tab.entry(key) + key;
     return f;
 }
 
@@ -179,21 +205,41 @@ __device__ __forceinline__ uint32_t pack_codes(const Found& f0, const Found& f1,
 }
 
 // c[code] * absmax as one rounding: the magnitude times the signed absmax, plus +0.0 so
-// that a zero magnitude gives +0.0 whatever the sign.  cm_lane is rebased by -127 rows.
-__device__ __forceinline__ float value_of(const Found& f, float absmax, uint32_t cm_lane) {
-    uint32_t va;
-    asm("mad.lo.u32 %0, %1, 128, %2;" : "=r"(va) : "r"(f.sum >> 24), "r"(cm_lane));
-    const float cm = __uint_as_float(lds_u32(va));
+// that a zero magnitude gives +0.0 whatever the sign.
+template <bool LITE>
+__device__ __forceinline__ float value_of(const Found& f, float absmax, const TabRef<LITE>& tab) {
+    const float cm = tab.magnitude(f.sum);
     const float as = __uint_as_float(__float_as_uint(absmax) | (f.bits & 0x80000000u));
     return __fmaf_rn(cm, as, 0.0f);
 }
 
-__device__ __forceinline__ void fill_fwd_tables(const DeviceTables& t, uint32_t sm_base, int nthreads) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = nthreads >> 5;
-    const uint32_t sm_lane = sm_base + uint32_t(lane) * 4u;
-    for (int e = warp; e < 132; e += nwarps) sts_u32(sm_lane + kCmOff + uint32_t(e) * 128u, __float_as_uint(__ldg(t.cmag + e)));
-#pragma unroll 4
-    for (int e = warp; e < kCells; e += nwarps) sts_u32(sm_lane + kGuessOff + uint32_t(e) * 128u, __ldg(t.guess + e));
+// Builds the per-lane copies.  The magnitude rows and the entry rows are consecutive both in
+// the device blob (cmag | guess) and in shared memory, so row i is word i of one array.  Each
+// warp first loads its rows coalesced (one word per lane, all loads in flight together), then
+// hands every word round with a shuffle so that all 32 lanes store it into their own column.
+template <int NT>
+__device__ __forceinline__ void fill_fwd_tables(const DeviceTables& t, uint32_t sm_base) {
+    constexpr int NROWS = 132 + kCells;
+    constexpr int NWARPS = NT / 32;
+    constexpr int ITERS = (NROWS + NWARPS * 32 - 1) / (NWARPS * 32);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t sm_lane = sm_base + uint32_t(lane) * 4u + kCmOff;
+    const uint32_t* src = reinterpret_cast<const uint32_t*>(t.cmag);
+    uint32_t v[ITERS];
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) {
+        const int row = (it * NWARPS + warp) * 32 + lane;
+        v[it] = row < NROWS ? __ldg(src + row) : 0u;
+    }
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) {
+        const int row0 = (it * NWARPS + warp) * 32;
+#pragma unroll
+        for (int k = 0; k < 32; ++k) {
+            const uint32_t word = __shfl_sync(0xffffffffu, v[it], k);
+            if (row0 + k < NROWS) sts_u32(sm_lane + uint32_t(row0 + k) * 128u, word);
+        }
+    }
 }
 
 // Two fp32 lanes per instruction (sm_100 packed fp32 arithmetic).
@@ -236,7 +282,8 @@ __device__ __forceinline__ float rcp_approx(float d) {
 //
 // A row is 32 consecutive chunks, one per lane (512 contiguous bytes).  Blocks no longer
 // than a row occupy B / kPerChunk consecutive lanes of one row and are reduced with
-// segmented shuffles; longer blocks take R rows of TW warps.  The loads of the next tile
+// segmented shuffles; longer blocks take R rows of TW warps.  Only whole tiles are handled
+// (the host sends the remainder to the general kernel).  The loads of the next tile
 // are issued as soon as the current one has been widened, so they fly during the search.
 //
 // Normalisation.  The contract is the correctly rounded quotient x / d.  For 16-bit inputs
@@ -248,10 +295,10 @@ __device__ __forceinline__ float rcp_approx(float d) {
 // rounding boundary, and never sits on one.  The CPU tests check every significand pair
 // with r perturbed by +-2 ulp.  Outside that window, and for fp32 inputs, the IEEE division
 // is used.
-template <int XDT, int B, int R, int TW, bool WRITE_Y, bool WRITE_Q, int NT>
+template <int XDT, int B, int R, int TW, bool WRITE_Y, bool WRITE_Q, int NT, bool LITE>
 __global__ void __launch_bounds__(NT, 1)
 fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__ codes, float* __restrict__ absmax_out,
-         size_t n_full, DeviceTables tab) {
+         size_t ntiles, DeviceTables tab) {
     constexpr int EPC = Elem<XDT>::kPerChunk;
     constexpr int EB = Elem<XDT>::kBytes;
     constexpr int ROW = 32 * EPC;
@@ -265,18 +312,19 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
     const uint32_t sm_base = (uint32_t(__cvta_generic_to_shared(smem_raw)) + 127u) & ~127u;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t sm_lane = sm_base + uint32_t(lane) * 4u;
-    const uint32_t guess_lane = guess_lane_of(sm_lane);
-    const uint32_t cm_lane = sm_lane + kCmOff - 127u * 128u;
+    const TabRef<LITE> tref(tab, sm_lane);
+    constexpr uint32_t RED = LITE ? 0u : kRedOff;
 
-    fill_fwd_tables(tab, sm_base, NT);
-    __syncthreads();
+    if constexpr (!LITE) {
+        fill_fwd_tables<NT>(tab, sm_base);
+        __syncthreads();
+    }
 
     const float neg_limit = tab.neg_limit;
     const char* xb = static_cast<const char*>(x);
     char* yb = static_cast<char*>(y);
 
     constexpr size_t TILE = size_t(TW) * R * ROW;
-    const size_t ntiles = (n_full + TILE - 1) / TILE;
     const size_t team = size_t(blockIdx.x) * (WARPS / TW) + size_t(warp / TW);
     const size_t nteams = size_t(gridDim.x) * (WARPS / TW);
     const int wt = warp % TW;
@@ -287,9 +335,7 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
     auto load_tile = [&](size_t t) {
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            const size_t off = t * TILE + lane_off + size_t(r) * ROW;
-            const bool ok = IN_ROW ? (off < n_full) : true;
-            w[r] = ok ? ldg_stream_16(xb + off * EB) : make_uint4(0, 0, 0, 0);
+            w[r] = ldg_stream_16(xb + (t * TILE + lane_off + size_t(r) * ROW) * EB);
         }
     };
     if (team < ntiles) load_tile(team);
@@ -326,7 +372,7 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
             if constexpr (TW > 1) {
                 // partial maxima of the team's warps meet in shared memory; two slots alternate so
                 // that one barrier per tile is enough
-                const uint32_t slot = sm_base + kRedOff + uint32_t(parity) * 128u + uint32_t(warp / TW) * TW * 4u;
+                const uint32_t slot = sm_base + RED + uint32_t(parity) * 128u + uint32_t(warp / TW) * TW * 4u;
                 if (lane == 0) sts_u32(slot + uint32_t(wt) * 4u, __float_as_uint(a));
                 asm volatile("bar.sync %0, %1;" ::"r"(1 + warp / TW), "r"(TW * 32) : "memory");
 #pragma unroll
@@ -380,11 +426,11 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
             Found fd[EPC];
 #pragma unroll
             for (int i = 0; i < EPC; ++i) {
-                fd[i] = search_folded(f[r][i], neg_limit, guess_lane);
-                if constexpr (WRITE_Y) out[i] = value_of(fd[i], amax[r], cm_lane);
+                fd[i] = search_folded(f[r][i], neg_limit, tref);
+                if constexpr (WRITE_Y) out[i] = value_of(fd[i], amax[r], tref);
             }
             const size_t off = base + size_t(r) * ROW;
-            if (IN_ROW ? (off < n_full) : true) {
+            {
                 if constexpr (WRITE_Y) stg_stream_16(yb + off * EB, narrow_chunk<XDT>(out));
                 if constexpr (WRITE_Q) {
                     if constexpr (EPC == 8) {
@@ -408,7 +454,7 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
 // deq_fast: 16 codes per 128-bit load, U loads per thread per tile, signed code values
 // replicated per lane in shared memory.  The loads of the next tile (codes and the blocks'
 // absmax) are issued before the current tile is expanded.
-template <int YDT, int NT, int U>
+template <int YDT, int NT, int U, bool LITE>
 __global__ void __launch_bounds__(NT)
 deq_fast(const uint8_t* __restrict__ codes, const float* __restrict__ absmax, void* __restrict__ y, size_t n16 /* n / 16 */,
          int log2_block, DeviceTables tab) {
@@ -416,8 +462,24 @@ deq_fast(const uint8_t* __restrict__ codes, const float* __restrict__ absmax, vo
     const uint32_t sm_base = uint32_t(__cvta_generic_to_shared(smem_raw));
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t sm_lane = sm_base + uint32_t(lane) * 4u;
-    for (int e = warp; e < 256; e += NT / 32) sts_u32(sm_lane + uint32_t(e) * 128u, __float_as_uint(__ldg(tab.values + e)));
-    __syncthreads();
+    if constexpr (!LITE) {
+        // one coalesced load of 32 values per warp, then a shuffle hands each value to all lanes
+        for (int row0 = warp * 32; row0 < 256; row0 += NT) {
+            const uint32_t mine = __float_as_uint(__ldg(tab.values + row0 + lane));
+#pragma unroll
+            for (int k = 0; k < 32; ++k) sts_u32(sm_lane + uint32_t(row0 + k) * 128u, __shfl_sync(0xffffffffu, mine, k));
+        }
+        __syncthreads();
+    }
+    // value of one code byte sitting at bit `shift` of a packed word
+    auto value = [&](uint32_t word, int shift) -> float {
+        if constexpr (LITE) {
+            return __ldg(tab.values + ((word >> shift) & 0xffu));
+        } else {
+            const uint32_t row = (shift >= 7 ? (word >> (shift - 7)) : (word << (7 - shift))) & 0x7f80u;
+            return __uint_as_float(lds_u32(sm_lane + row));
+        }
+    };
 
     char* yb = static_cast<char*>(y);
     constexpr int EB = Elem<YDT>::kBytes;
@@ -451,10 +513,10 @@ deq_fast(const uint8_t* __restrict__ codes, const float* __restrict__ absmax, vo
             float v[16];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                v[4 * k + 0] = __fmul_rn(__uint_as_float(lds_u32(sm_lane + ((q[k] << 7) & 0x7f80u))), ca[u]);
-                v[4 * k + 1] = __fmul_rn(__uint_as_float(lds_u32(sm_lane + ((q[k] >> 1) & 0x7f80u))), ca[u]);
-                v[4 * k + 2] = __fmul_rn(__uint_as_float(lds_u32(sm_lane + ((q[k] >> 9) & 0x7f80u))), ca[u]);
-                v[4 * k + 3] = __fmul_rn(__uint_as_float(lds_u32(sm_lane + ((q[k] >> 17) & 0x7f80u))), ca[u]);
+                v[4 * k + 0] = __fmul_rn(value(q[k], 0), ca[u]);
+                v[4 * k + 1] = __fmul_rn(value(q[k], 8), ca[u]);
+                v[4 * k + 2] = __fmul_rn(value(q[k], 16), ca[u]);
+                v[4 * k + 3] = __fmul_rn(value(q[k], 24), ca[u]);
             }
             char* out = yb + c * 16 * EB;
             if constexpr (YDT == kF32) {

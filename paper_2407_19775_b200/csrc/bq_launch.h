@@ -9,21 +9,22 @@
 
 namespace bql {
 
-// Tuned forward kernels, one translation unit per element type.
+// Tuned forward kernels, one translation unit per element type.  n_full is a whole number of
+// blocks; *done receives how many leading elements were handled (whole tiles only).
 cudaError_t launch_fwd_fast_f32(int block, bool write_y, bool write_q, const void* x, void* y, uint8_t* codes, float* absmax,
-                                size_t n_full, const bqk::DeviceTables& tab, int sm_count, int device, cudaStream_t stream);
+                                size_t n_full, const bqk::DeviceTables& tab, int sm_count, int device, cudaStream_t stream, size_t* done);
 cudaError_t launch_fwd_fast_f16(int block, bool write_y, bool write_q, const void* x, void* y, uint8_t* codes, float* absmax,
-                                size_t n_full, const bqk::DeviceTables& tab, int sm_count, int device, cudaStream_t stream);
+                                size_t n_full, const bqk::DeviceTables& tab, int sm_count, int device, cudaStream_t stream, size_t* done);
 cudaError_t launch_fwd_fast_bf16(int block, bool write_y, bool write_q, const void* x, void* y, uint8_t* codes, float* absmax,
-                                 size_t n_full, const bqk::DeviceTables& tab, int sm_count, int device, cudaStream_t stream);
+                                 size_t n_full, const bqk::DeviceTables& tab, int sm_count, int device, cudaStream_t stream, size_t* done);
 
 inline cudaError_t launch_fwd_fast(int xdt, int block, bool write_y, bool write_q, const void* x, void* y, uint8_t* codes,
                                    float* absmax, size_t n_full, const bqk::DeviceTables& tab, int sm_count, int device,
-                                   cudaStream_t stream) {
+                                   cudaStream_t stream, size_t* done) {
     switch (xdt) {
-        case BQ_F32: return launch_fwd_fast_f32(block, write_y, write_q, x, y, codes, absmax, n_full, tab, sm_count, device, stream);
-        case BQ_F16: return launch_fwd_fast_f16(block, write_y, write_q, x, y, codes, absmax, n_full, tab, sm_count, device, stream);
-        default: return launch_fwd_fast_bf16(block, write_y, write_q, x, y, codes, absmax, n_full, tab, sm_count, device, stream);
+        case BQ_F32: return launch_fwd_fast_f32(block, write_y, write_q, x, y, codes, absmax, n_full, tab, sm_count, device, stream, done);
+        case BQ_F16: return launch_fwd_fast_f16(block, write_y, write_q, x, y, codes, absmax, n_full, tab, sm_count, device, stream, done);
+        default: return launch_fwd_fast_bf16(block, write_y, write_q, x, y, codes, absmax, n_full, tab, sm_count, device, stream, done);
     }
 }
 
