@@ -33,7 +33,7 @@ cudaError_t fwd_general_y(int ydt, bool wy, bool wq, const void* x, void* y, uin
 #define BQ_DEQ_U 2
 #endif
 #ifndef BQ_DEQ_CTAS
-#define BQ_DEQ_CTAS 2
+#define BQ_DEQ_CTAS 3
 #endif
 constexpr int kDeqNT = BQ_DEQ_NT;
 constexpr int kDeqU = BQ_DEQ_U;

@@ -195,13 +195,20 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
 }
 
 // Four codes as one word.  The top bytes of the four sums are the codes for non-negative
-// values, c = 127 + P; a negative value takes 127 - P = (c ^ 0xFF) - 1.  Both byte gathers
-// are single byte-permutes (the second one replicates each sign bit over its byte), and the
-// subtraction cannot borrow between bytes because c ^ 0xFF >= 1 wherever 1 is subtracted.
-__device__ __forceinline__ uint32_t pack_codes(const Found& f0, const Found& f1, const Found& f2, const Found& f3) {
+// values, c = 127 + P; a negative value takes 127 - P = (c ^ 0xFF) - 1.  `neg` holds 0xFF in
+// the bytes of negative elements (sign_mask_* below: byte-permutes that replicate a sign bit
+// over its byte; taken from the inputs, whose signs the quotients share); the subtraction
+// cannot borrow between bytes because c ^ 0xFF >= 1 wherever 1 is subtracted (the clamp in
+// search_folded keeps c <= 254 on the negative side).
+__device__ __forceinline__ uint32_t pack_codes(const Found& f0, const Found& f1, const Found& f2, const Found& f3, uint32_t neg) {
     const uint32_t c = prmt(prmt(f0.sum, f1.sum, 0x0073u), prmt(f2.sum, f3.sum, 0x0073u), 0x5410u);
-    const uint32_t m = prmt(prmt(f0.bits, f1.bits, 0x00FBu), prmt(f2.bits, f3.bits, 0x00FBu), 0x5410u);     // 0x8 in a selector: replicate the sign
-    return (c ^ m) - (m & 0x01010101u);
+    return (c ^ neg) - (neg & 0x01010101u);
+}
+// sign bytes of four 16-bit elements held in two words (element sign bits sit in bytes 1, 3, 5, 7)
+__device__ __forceinline__ uint32_t sign_mask_16(uint32_t w0, uint32_t w1) { return prmt(w0, w1, 0xFDB9u); }
+// sign bytes of four fp32 elements
+__device__ __forceinline__ uint32_t sign_mask_32(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    return prmt(prmt(a, b, 0x00FBu), prmt(c, d, 0x00FBu), 0x5410u);
 }
 
 // c[code] * absmax as one rounding: the magnitude times the signed absmax, plus +0.0 so
@@ -344,8 +351,17 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
         const size_t base = t * TILE + lane_off;
         float f[R][EPC];
         float amax[R];
+        uint32_t neg[R][2];                                        // sign bytes, taken before w is reused
 #pragma unroll
         for (int r = 0; r < R; ++r) {
+            if constexpr (WRITE_Q) {
+                if constexpr (EPC == 8) {
+                    neg[r][0] = sign_mask_16(w[r].x, w[r].y);
+                    neg[r][1] = sign_mask_16(w[r].z, w[r].w);
+                } else {
+                    neg[r][0] = sign_mask_32(w[r].x, w[r].y, w[r].z, w[r].w);
+                }
+            }
             widen_chunk<XDT>(w[r], f[r]);
             float a = 0.0f;
 #pragma unroll
@@ -434,9 +450,9 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
                 if constexpr (WRITE_Y) stg_stream_16(yb + off * EB, narrow_chunk<XDT>(out));
                 if constexpr (WRITE_Q) {
                     if constexpr (EPC == 8) {
-                        stg_stream_8(codes + off, make_uint2(pack_codes(fd[0], fd[1], fd[2], fd[3]), pack_codes(fd[4], fd[5], fd[6], fd[7])));
+                        stg_stream_8(codes + off, make_uint2(pack_codes(fd[0], fd[1], fd[2], fd[3], neg[r][0]), pack_codes(fd[4], fd[5], fd[6], fd[7], neg[r][1])));
                     } else {
-                        stg_stream_4(codes + off, pack_codes(fd[0], fd[1], fd[2], fd[3]));
+                        stg_stream_4(codes + off, pack_codes(fd[0], fd[1], fd[2], fd[3], neg[r][0]));
                     }
                     if constexpr (IN_ROW) {
                         if ((lane % LPB) == 0) absmax_out[off / B] = amax[r];
@@ -454,8 +470,11 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
 // deq_fast: 16 codes per 128-bit load, U loads per thread per tile, signed code values
 // replicated per lane in shared memory.  The loads of the next tile (codes and the blocks'
 // absmax) are issued before the current tile is expanded.
+#ifndef BQ_DEQ_MINB
+#define BQ_DEQ_MINB 3
+#endif
 template <int YDT, int NT, int U, bool LITE>
-__global__ void __launch_bounds__(NT)
+__global__ void __launch_bounds__(NT, LITE ? 1 : BQ_DEQ_MINB)
 deq_fast(const uint8_t* __restrict__ codes, const float* __restrict__ absmax, void* __restrict__ y, size_t n16 /* n / 16 */,
          int log2_block, DeviceTables tab) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
