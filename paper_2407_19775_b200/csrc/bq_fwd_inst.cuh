@@ -6,20 +6,20 @@ namespace bql {
 namespace {
 
 #ifndef BQ_NT
-#define BQ_NT 512
+#define BQ_NT 384
 #endif
 #ifndef BQ_RMAX
-#define BQ_RMAX 4
+#define BQ_RMAX 8
 #endif
 constexpr int kNT = BQ_NT;
 
 // Tile shape per block size: R chunks per thread, TW warps per block.
-template <int XDT, int B> struct Shape {
+template <int XDT, int B, int RMAX> struct Shape {
     static constexpr int ROW = 32 * bqk::Elem<XDT>::kPerChunk;
     static constexpr bool IN_ROW = B <= ROW;
-    static constexpr int ROWS = IN_ROW ? BQ_RMAX : B / ROW;    // rows one tile must cover
-    static constexpr int R = ROWS <= BQ_RMAX ? ROWS : BQ_RMAX;
-    static constexpr int TW = IN_ROW ? 1 : ROWS / R;
+    static constexpr int ROWS = IN_ROW ? RMAX : B / ROW;       // rows of one block (any number when blocks fit in a row)
+    static constexpr int R = RMAX;                             // a warp holds RMAX rows: several blocks, one, or a share of one
+    static constexpr int TW = (IN_ROW || ROWS <= RMAX) ? 1 : ROWS / RMAX;
 };
 
 constexpr int kLiteNT = 256;
@@ -34,18 +34,23 @@ constexpr size_t kLiteMaxElems = size_t(1) << BQ_LITE_MAX_LOG2;
 template <int XDT, int B, bool WY, bool WQ>
 cudaError_t go(const void* x, void* y, uint8_t* codes, float* absmax, size_t n_full, const bqk::DeviceTables& tab, int sm_count,
                int device, cudaStream_t stream, size_t* done) {
-    using S = Shape<XDT, B>;
-    const size_t tile = size_t(S::TW) * S::R * S::ROW;
-    const size_t ntiles = n_full / tile;
-    *done = ntiles * tile;
-    if (ntiles == 0) return cudaSuccess;
     if (n_full <= kLiteMaxElems) {
+        using S = Shape<XDT, B, 4>;              // smaller tiles: more CTAs for a small tensor
+        const size_t tile = size_t(S::TW) * S::R * S::ROW;
+        const size_t ntiles = n_full / tile;
+        *done = ntiles * tile;
+        if (ntiles == 0) return cudaSuccess;
         constexpr auto kernel = bqk::fwd_fast<XDT, B, S::R, S::TW, WY, WQ, kLiteNT, true>;
         const size_t teams = (kLiteNT / 32) / S::TW;
         const size_t grid = (ntiles + teams - 1) / teams;
         kernel<<<unsigned(grid), kLiteNT, bqk::kFwdLiteSmemBytes, stream>>>(x, y, codes, absmax, ntiles, tab);
         return cudaGetLastError();
     }
+    using S = Shape<XDT, B, BQ_RMAX>;
+    const size_t tile = size_t(S::TW) * S::R * S::ROW;
+    const size_t ntiles = n_full / tile;
+    *done = ntiles * tile;
+    if (ntiles == 0) return cudaSuccess;
     constexpr auto kernel = bqk::fwd_fast<XDT, B, S::R, S::TW, WY, WQ, kNT, false>;
     cudaError_t e = allow_smem<kernel>(int(bqk::kFwdSmemBytes), device);
     if (e != cudaSuccess) return e;

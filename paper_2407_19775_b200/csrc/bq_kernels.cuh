@@ -311,7 +311,9 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
     constexpr int ROW = 32 * EPC;
     constexpr bool IN_ROW = (B <= ROW);
     constexpr int LPB = IN_ROW ? B / EPC : 32;                 // lanes per block inside a row
-    static_assert(IN_ROW ? (TW == 1) : (TW * R * ROW == B), "tile must be one block when blocks span rows");
+    constexpr int RPB = IN_ROW ? 1 : (B / ROW) / TW;           // rows of one warp that belong to one block
+    constexpr int NBLK = R / RPB;                              // blocks per tile when blocks span rows
+    static_assert(IN_ROW ? (TW == 1) : (RPB >= 1 && R % RPB == 0 && (TW == 1 || NBLK == 1)), "a tile holds whole blocks");
     constexpr int WARPS = NT / 32;
     static_assert(WARPS % TW == 0 && TW <= 15, "teams must tile the CTA, one named barrier each");
 
@@ -380,25 +382,34 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
                     for (int s = 1; s < LPB; s <<= 1) amax[r] = fmaxf(amax[r], __shfl_xor_sync(0xffffffffu, amax[r], s));
                 }
             }
+        } else if constexpr (TW == 1) {
+            // NBLK whole blocks of RPB rows each inside this warp
+#pragma unroll
+            for (int k = 0; k < NBLK; ++k) {
+                float a = amax[k * RPB];
+#pragma unroll
+                for (int r = 1; r < RPB; ++r) a = fmaxf(a, amax[k * RPB + r]);
+                a = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(a)));
+#pragma unroll
+                for (int r = 0; r < RPB; ++r) amax[k * RPB + r] = a;
+            }
         } else {
             float a = amax[0];
 #pragma unroll
             for (int r = 1; r < R; ++r) a = fmaxf(a, amax[r]);
             a = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(a)));
-            if constexpr (TW > 1) {
-                // partial maxima of the team's warps meet in shared memory; two slots alternate so
-                // that one barrier per tile is enough
-                const uint32_t slot = sm_base + RED + uint32_t(parity) * 128u + uint32_t(warp / TW) * TW * 4u;
-                if (lane == 0) sts_u32(slot + uint32_t(wt) * 4u, __float_as_uint(a));
-                asm volatile("bar.sync %0, %1;" ::"r"(1 + warp / TW), "r"(TW * 32) : "memory");
+            // partial maxima of the team's warps meet in shared memory; two slots alternate so
+            // that one barrier per tile is enough
+            const uint32_t slot = sm_base + RED + uint32_t(parity) * 128u + uint32_t(warp / TW) * TW * 4u;
+            if (lane == 0) sts_u32(slot + uint32_t(wt) * 4u, __float_as_uint(a));
+            asm volatile("bar.sync %0, %1;" ::"r"(1 + warp / TW), "r"(TW * 32) : "memory");
 #pragma unroll
-                for (int k = 0; k < TW; ++k) {
-                    uint32_t v;
-                    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(slot + uint32_t(k) * 4u) : "memory");
-                    a = fmaxf(a, __uint_as_float(v));
-                }
-                parity ^= 1;
+            for (int k = 0; k < TW; ++k) {
+                uint32_t v;
+                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(slot + uint32_t(k) * 4u) : "memory");
+                a = fmaxf(a, __uint_as_float(v));
             }
+            parity ^= 1;
 #pragma unroll
             for (int r = 0; r < R; ++r) amax[r] = a;
         }
@@ -461,7 +472,10 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
             }
         }
         if constexpr (WRITE_Q && !IN_ROW) {
-            if (lane == 0 && wt == 0) absmax_out[t] = amax[0];
+            if (lane == 0 && wt == 0) {
+#pragma unroll
+                for (int k = 0; k < NBLK; ++k) absmax_out[t * NBLK + k] = amax[k * RPB];
+            }
         }
     }
 }
