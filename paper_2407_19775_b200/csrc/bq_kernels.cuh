@@ -58,13 +58,35 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
 __device__ __forceinline__ void sts_u32(uint32_t addr, uint32_t v) {
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
+#ifndef BQ_LD
+#define BQ_LD 3
+#endif
+#ifndef BQ_ST
+#define BQ_ST 0
+#endif
 __device__ __forceinline__ uint4 ldg_stream_16(const void* p) {
     uint4 v;
+#if BQ_LD == 0
     asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+#elif BQ_LD == 1
+    asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+#elif BQ_LD == 2
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+#else
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+#endif
     return v;
 }
 __device__ __forceinline__ void stg_stream_16(void* p, uint4 v) {
+#if BQ_ST == 0
     asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+#else
+    asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+#endif
+}
+// 32 contiguous bytes per thread as one 256-bit store: a warp then writes whole 128-byte lines
+__device__ __forceinline__ void stg_stream_32(void* p, uint4 a, uint4 b) {
+    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w) : "memory");
 }
 __device__ __forceinline__ void stg_stream_8(void* p, uint2 v) {
     asm volatile("st.global.cs.v2.u32 [%0], {%1,%2};" ::"l"(p), "r"(v.x), "r"(v.y) : "memory");
@@ -554,16 +576,15 @@ deq_fast(const uint8_t* __restrict__ codes, const float* __restrict__ absmax, vo
             char* out = yb + c * 16 * EB;
             if constexpr (YDT == kF32) {
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const float tt[4] = {v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]};
-                    stg_stream_16(out + 16 * k, narrow_chunk<kF32>(tt));
+                for (int k = 0; k < 2; ++k) {
+                    const float t0[4] = {v[8 * k], v[8 * k + 1], v[8 * k + 2], v[8 * k + 3]};
+                    const float t1[4] = {v[8 * k + 4], v[8 * k + 5], v[8 * k + 6], v[8 * k + 7]};
+                    stg_stream_32(out + 32 * k, narrow_chunk<kF32>(t0), narrow_chunk<kF32>(t1));
                 }
             } else {
-#pragma unroll
-                for (int k = 0; k < 2; ++k) {
-                    const float tt[8] = {v[8 * k], v[8 * k + 1], v[8 * k + 2], v[8 * k + 3], v[8 * k + 4], v[8 * k + 5], v[8 * k + 6], v[8 * k + 7]};
-                    stg_stream_16(out + 16 * k, narrow_chunk<YDT>(tt));
-                }
+                const float t0[8] = {v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]};
+                const float t1[8] = {v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15]};
+                stg_stream_32(out, narrow_chunk<YDT>(t0), narrow_chunk<YDT>(t1));
             }
         }
     }
