@@ -22,9 +22,12 @@ def main() -> None:
     ap.add_argument("--block", type=int, default=4096)
     ap.add_argument("--rows", type=int, default=8192)
     ap.add_argument("--launches", type=int, default=3)
+    ap.add_argument("--dtype", default=None, choices=[None, "bf16", "fp16", "fp32"], help="cast the workload to this type first")
     args = ap.parse_args()
     dev = torch.device("cuda:0")
     x = workloads.make(args.workload, rows=args.rows).view(-1).to(dev)
+    if args.dtype is not None:
+        x = x.to({"bf16": torch.bfloat16, "fp16": torch.float16, "fp32": torch.float32}[args.dtype])
     n = x.numel()
     cb = Codebook(device=dev)
     codes = torch.empty(n, dtype=torch.uint8, device=dev)
@@ -46,7 +49,7 @@ def main() -> None:
             bq_roundtrip(x, args.block, cb, y_out=y, codes_out=codes, absmax_out=absmax)
         e1.record()
         torch.cuda.synchronize()
-        print(f"{args.op} block={args.block} n={n} launch {i}: {e0.elapsed_time(e1):.4f} ms")
+        print(f"{args.op} {str(x.dtype)[6:]} block={args.block} n={n} launch {i}: {e0.elapsed_time(e1):.4f} ms")
 
 
 if __name__ == "__main__":
