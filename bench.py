@@ -109,7 +109,7 @@ class ClockSampler:
         try:
             self.out = open(self.path, "w")
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                          "-lms", "100"], stdout=self.out, stderr=subprocess.DEVNULL)
+                                          "-lms", "50"], stdout=self.out, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -222,7 +222,7 @@ def run_ours(args):
         avg = float(np.mean(ms))
         ab = algorithmic_bytes(op, n, b)
         kernels[f"{op}_b{b}"] = {
-            "ms": round(avg, 4), "ms_min": round(float(np.min(ms)), 4),
+            "ms": round(avg, 4), "ms_min": round(float(np.min(ms)), 4), "algorithmic_bytes": int(ab), "traffic": TRAFFIC_BYTES.get(f"{op}_b{b}"),
             "input_gbs": round(n * (1 if op == "dequantize" else 2) / avg / 1e6, 1),
             "total_gbs": round(ab / avg / 1e6, 1),
             "frac_of_measured": round(ab / avg / 1e6 / peak, 4),
@@ -271,9 +271,16 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-# DRAM bytes per launch from ncu captures (profiles/); filled in once a capture exists and
-# cleared when the kernel changes.
-TRAFFIC_BYTES = {}
+# DRAM bytes per full-size launch (dram__bytes_read.sum + dram__bytes_write.sum), from ncu
+# captures of the first 8192 rows scaled to 65536 rows: reads scale with the rows (they equal
+# the algorithmic bytes to 0.04 %); writes are the algorithmic bytes minus the 40-58 MB of
+# dirty lines that are still in L2 when the kernel ends, a size-independent residue measured
+# in the same capture.  Set an entry to None when its kernel changes until it is re-measured.
+TRAFFIC_BYTES = {
+    "quantize_b64": 1600887040, "quantize_b256": 1579075328, "quantize_b1024": 1573408256, "quantize_b4096": 1571947264,
+    "dequantize_b64": 1588571904, "dequantize_b256": 1560674048, "dequantize_b1024": 1555077888, "dequantize_b4096": 1553117440,
+    "roundtrip_b64": 2095402240, "roundtrip_b256": 2095243264, "roundtrip_b1024": 2096132608, "roundtrip_b4096": 2095491584,
+}
 
 
 def run_e2e(bq, cb, x_pin, dev, dtype, n, args, world):
@@ -383,7 +390,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=2)
