@@ -284,31 +284,24 @@ TRAFFIC_BYTES = {
 
 
 def run_e2e(bq, cb, x_pin, dev, dtype, n, args, world):
-    """One end-to-end step per block size, everything starting and ending in pinned host
-    memory: sender (H2D x, quantize, D2H codes+absmax), receiver (H2D codes+absmax,
-    dequantize, D2H y) and the fused loop (H2D x, roundtrip, D2H y)."""
+    """One end-to-end step per block size through the host-to-host API, everything starting
+    and ending in pinned host memory: sender (x up, quantize, codes+absmax down), receiver
+    (codes+absmax up, dequantize, y down) and the fused loop (x up, roundtrip, y down).  The
+    three legs of each call overlap chunk by chunk on three streams."""
+    from paper_2407_19775_b200.pipeline import HostBoundary
     steps = max(1, min(args.steps, args.e2e_steps))
-    xd = torch.empty(n, dtype=dtype, device=dev)
-    cd = torch.empty(n, dtype=torch.uint8, device=dev)
-    yd = torch.empty(n, dtype=dtype, device=dev)
+    hb = HostBoundary(cb, dtype, chunk=1 << 25, slots=3, max_blocks_per_chunk=(1 << 25) // min(BLOCKS))
     c_pin = torch.empty(n, dtype=torch.uint8).pin_memory()
     y_pin = torch.empty(n, dtype=dtype).pin_memory()
     a_pin = {b: torch.empty(n // b, dtype=torch.float32).pin_memory() for b in BLOCKS}
-    ad = {b: torch.empty(n // b, dtype=torch.float32, device=dev) for b in BLOCKS}
     h2d = d2h = 0
 
     def one_step(count=False):
         nonlocal h2d, d2h
         for b in BLOCKS:
-            xd.copy_(x_pin, non_blocking=True)
-            bq.bq_quantize(xd, b, cb, cd, ad[b])
-            c_pin.copy_(cd, non_blocking=True); a_pin[b].copy_(ad[b], non_blocking=True)
-            cd.copy_(c_pin, non_blocking=True); ad[b].copy_(a_pin[b], non_blocking=True)
-            bq.bq_dequantize(cd, ad[b], b, cb, dtype, yd)
-            y_pin.copy_(yd, non_blocking=True)
-            xd.copy_(x_pin, non_blocking=True)
-            bq.bq_roundtrip(xd, b, cb, y_out=yd)
-            y_pin.copy_(yd, non_blocking=True)
+            hb.quantize(x_pin, b, c_pin, a_pin[b])
+            hb.dequantize(c_pin, a_pin[b], b, y_pin)
+            hb.roundtrip(x_pin, b, y_pin)
             if count:
                 h2d += 2 * n * 2 + n + 4 * (n // b)
                 d2h += n + 4 * (n // b) + 2 * n * 2
@@ -326,7 +319,7 @@ def run_e2e(bq, cb, x_pin, dev, dtype, n, args, world):
     sec = max_over_ranks(t0.elapsed_time(t1) / 1e3, world, dev)
     bytes_per_step = n * 2 * len(BLOCKS) * len(OPS)
     return {"value": round(whole_job_value(bytes_per_step * steps, world, sec) / 1e9, 2), "unit": "GB/s", "steps": steps,
-            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "api": "HostBoundary (32 Mi-element chunks, 3 streams)"}
 
 
 # ------------------------------------------------------------------------------------------ the CPU oracle arm

@@ -206,6 +206,53 @@ def test_non_default_stream(bq, gcb, cb):
     assert np.array_equal(_bits(y.cpu()), oracle.roundtrip(_bits(x), oracle.F16, 64, cb, oracle.F16))
 
 
+def test_host_to_host_pipeline(bq, gcb, cb):
+    """The chunked three-stream path between pinned host tensors gives the same bytes; the
+    chunk is small here so that slots are reused several times and the last piece is short."""
+    x = workloads.make("prefill7b", rows=200).view(-1)[: 200 * 4096 - 256 * 3].contiguous()
+    n, block = x.numel(), 256
+    hb = bq.HostBoundary(gcb, torch.bfloat16, chunk=256 * 300, slots=3)
+    x_pin = x.pin_memory()
+    c_pin = torch.empty(n, dtype=torch.uint8).pin_memory()
+    a_pin = torch.empty(n // block, dtype=torch.float32).pin_memory()
+    y_pin = torch.empty(n, dtype=torch.bfloat16).pin_memory()
+    y2_pin = torch.empty(n, dtype=torch.bfloat16).pin_memory()
+    hb.quantize(x_pin, block, c_pin, a_pin)
+    torch.cuda.synchronize()
+    hb.dequantize(c_pin, a_pin, block, y_pin)
+    hb.roundtrip(x_pin, block, y2_pin)
+    torch.cuda.synchronize()
+    yr, cr, ar = oracle.roundtrip_sharded(_bits(x), oracle.BF16, block, cb, oracle.BF16, THREADS)
+    assert np.array_equal(c_pin.numpy(), cr) and np.array_equal(a_pin.numpy().view(np.uint32), ar.view(np.uint32))
+    assert np.array_equal(_bits(y_pin), yr) and np.array_equal(_bits(y2_pin), yr)
+
+
+def test_non_finite_inputs_stay_in_bounds(bq, gcb, cb):
+    """NaN / Inf are outside the contract, but every code must be a byte written in bounds
+    (canaries intact) and blocks without such values must still match the oracle."""
+    g = torch.Generator().manual_seed(2)
+    for dtype, block in ((torch.bfloat16, 64), (torch.float32, 256), (torch.float16, 4096)):
+        n = block * 40
+        x = torch.randn(n, generator=g).to(dtype)
+        bad = [3 * block + 5, 3 * block + 6, 17 * block, 29 * block + block - 1]
+        x[bad[0]] = float("nan"); x[bad[1]] = float("inf"); x[bad[2]] = float("-inf"); x[bad[3]] = float("nan")
+        xd = x.to("cuda:0")
+        craw, codes = _padded(n, torch.uint8, xd.device)
+        araw, absmax = _padded(n // block, torch.float32, xd.device)
+        yraw, y = _padded(n, dtype, xd.device)
+        bq.bq_quantize(xd, block, gcb, codes, absmax)
+        bq.bq_roundtrip(xd, block, gcb, y_out=y)
+        torch.cuda.synchronize()
+        esz = x.element_size()
+        assert _canary_ok(craw, n) and _canary_ok(araw, (n // block) * 4) and _canary_ok(yraw, n * esz)
+        clean = np.ones(n // block, bool)
+        clean[[3, 17, 29]] = False
+        yr, cr, ar = oracle.roundtrip(_bits(x), ODT[dtype], block, cb, ODT[dtype], side=True)
+        keep = np.repeat(clean, block)
+        assert np.array_equal(codes.cpu().numpy()[keep], cr[keep])
+        assert np.array_equal(_bits(y.cpu())[keep], yr[keep])
+
+
 # ------------------------------------------------------------------------------- degenerate values
 
 def test_zero_blocks_negative_zero_and_sign_of_absmax(bq, gcb, cb):
