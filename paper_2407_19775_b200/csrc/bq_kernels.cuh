@@ -394,15 +394,54 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
         }
         if (t + nteams < ntiles) load_tile(t + nteams);          // in flight during everything below
 
+        float d[R], rcv[R];                                        // divisor and its reciprocal, per row
+        bool quick = false;                                        // warp-uniform: reciprocal route for the whole tile
+        constexpr bool QUICK_OK = (XDT != kF32);
         if constexpr (IN_ROW) {
+            // The tile holds R x (32 / LPB) blocks, at most one per lane.  A butterfly that hands
+            // half of the rows to the partner lane at each of its first log2(R) steps leaves every
+            // lane with the maximum of ONE row of its group (row rho below); the per-block scalars
+            // (divisor, window test, reciprocal) are then computed once, by that lane, and handed
+            // back with one shuffle per row, instead of by every lane for every row.
+            constexpr int LOGR = (R == 8) ? 3 : (R == 4) ? 2 : (R == 2) ? 1 : 0;
+            static_assert((1 << LOGR) == R && LPB >= R, "row-halving butterfly needs R a power of two and LPB >= R");
+            float v[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) v[r] = amax[r];
+#pragma unroll
+            for (int s = 0; s < LOGR; ++s) {
+                const bool up = (lane >> s) & 1;
+                const int half = R >> (s + 1);
+#pragma unroll
+                for (int i = 0; i < half; ++i) {
+                    const float keep = up ? v[i + half] : v[i];
+                    const float send = up ? v[i] : v[i + half];
+                    v[i] = fmaxf(keep, __shfl_xor_sync(0xffffffffu, send, 1 << s));
+                }
+            }
+            float m = v[0];
+#pragma unroll
+            for (int s = R; s < LPB; s <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, s));
+            // this lane's block: row rho = sum_s bit_s(lane) * (R >> (s+1)), group lane / LPB
+            const float dm = (m != 0.0f) ? m : 1.0f;
+            const float rm = QUICK_OK ? rcp_approx(dm) : 0.0f;
+            if constexpr (QUICK_OK)
+                quick = __all_sync(0xffffffffu, (dm >= 5.421010862427522e-20f) && (dm <= 1.8446744073709552e19f));    // 2^-64 .. 2^64
+            if constexpr (WRITE_Q) {
+                int rho = 0;
+#pragma unroll
+                for (int s = 0; s < LOGR; ++s) rho += ((lane >> s) & 1) * (R >> (s + 1));
+                if ((lane % LPB) < R) absmax_out[(base + size_t(rho) * ROW) / B] = m;
+            }
+            const int group_base = lane & ~(LPB - 1);
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                if constexpr (LPB == 32) {
-                    amax[r] = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(amax[r])));
-                } else {
+                int src = 0;                                        // the lane of the group that holds row r
 #pragma unroll
-                    for (int s = 1; s < LPB; s <<= 1) amax[r] = fmaxf(amax[r], __shfl_xor_sync(0xffffffffu, amax[r], s));
-                }
+                for (int s = 0; s < LOGR; ++s) src |= ((r >> (LOGR - 1 - s)) & 1) << s;
+                amax[r] = __shfl_sync(0xffffffffu, m, group_base + src);
+                d[r] = __shfl_sync(0xffffffffu, dm, group_base + src);
+                if constexpr (QUICK_OK) rcv[r] = __shfl_sync(0xffffffffu, rm, group_base + src);
             }
         } else if constexpr (TW == 1) {
             // NBLK whole blocks of RPB rows each inside this warp
@@ -438,35 +477,33 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
 
         // normalise the whole tile in place; one warp-uniform choice between the reciprocal
         // route and the IEEE division keeps the per-element code free of branches
-        {
-            bool ok = (XDT != kF32);
-            float d[R];
+        if constexpr (!IN_ROW) {
+            bool ok = QUICK_OK;
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 d[r] = (amax[r] != 0.0f) ? amax[r] : 1.0f;
                 ok = ok && (d[r] >= 5.421010862427522e-20f) && (d[r] <= 1.8446744073709552e19f);      // 2^-64 .. 2^64
+                rcv[r] = QUICK_OK ? rcp_approx(d[r]) : 0.0f;
             }
-            bool quick = false;
-            if constexpr (XDT != kF32) quick = __all_sync(0xffffffffu, ok);
-            if (quick) {
+            if constexpr (QUICK_OK) quick = __all_sync(0xffffffffu, ok);
+        }
+        if (quick) {
 #pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    const float rc = rcp_approx(d[r]);
-                    const uint64_t r2 = pack2(rc, rc), nd2 = pack2(-d[r], -d[r]);
+            for (int r = 0; r < R; ++r) {
+                const uint64_t r2 = pack2(rcv[r], rcv[r]), nd2 = pack2(-d[r], -d[r]);
 #pragma unroll
-                    for (int i = 0; i < EPC; i += 2) {
-                        const uint64_t x2 = pack2(f[r][i], f[r][i + 1]);
-                        const uint64_t q0 = mul2(x2, r2);
-                        const uint64_t e = fma2(nd2, q0, x2);
-                        unpack2(fma2(e, r2, q0), f[r][i], f[r][i + 1]);
-                    }
+                for (int i = 0; i < EPC; i += 2) {
+                    const uint64_t x2 = pack2(f[r][i], f[r][i + 1]);
+                    const uint64_t q0 = mul2(x2, r2);
+                    const uint64_t e = fma2(nd2, q0, x2);
+                    unpack2(fma2(e, r2, q0), f[r][i], f[r][i + 1]);
                 }
-            } else {
-#pragma unroll
-                for (int r = 0; r < R; ++r)
-#pragma unroll
-                    for (int i = 0; i < EPC; ++i) f[r][i] = __fdiv_rn(f[r][i], d[r]);
             }
+        } else {
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+#pragma unroll
+                for (int i = 0; i < EPC; ++i) f[r][i] = __fdiv_rn(f[r][i], d[r]);
         }
 
 #pragma unroll
@@ -486,9 +523,6 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
                         stg_stream_8(codes + off, make_uint2(pack_codes(fd[0], fd[1], fd[2], fd[3], neg[r][0]), pack_codes(fd[4], fd[5], fd[6], fd[7], neg[r][1])));
                     } else {
                         stg_stream_4(codes + off, pack_codes(fd[0], fd[1], fd[2], fd[3], neg[r][0]));
-                    }
-                    if constexpr (IN_ROW) {
-                        if ((lane % LPB) == 0) absmax_out[off / B] = amax[r];
                     }
                 }
             }
