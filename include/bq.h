@@ -15,6 +15,8 @@
  *     `block` elements; the last block may be short and uses only its real elements.
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t; NULL = legacy default stream) and
  *     the call returns without synchronising.
+ *   - The codebook handle belongs to the device that was current when it was made; data calls
+ *     must be made with that device current (BQ_ERR_CODEBOOK otherwise).
  *   - Return value: a bq_status.  Argument errors are found on the host before anything is
  *     launched; nothing throws, aborts or exits.  n == 0 returns BQ_OK without a launch.
  *   - Any block >= 1 and any pointer alignment is accepted.  Blocks of 64, 128, 256, 512,
@@ -42,7 +44,7 @@ typedef enum {
     BQ_ERR_DTYPE = 2,     /* element type is not one of bq_dtype                */
     BQ_ERR_BLOCK = 3,     /* block < 1                                          */
     BQ_ERR_SIZE = 4,      /* n does not fit the launch limits (n >= 2^40)       */
-    BQ_ERR_CODEBOOK = 5,  /* unknown kind, or user values break the rules below */
+    BQ_ERR_CODEBOOK = 5,  /* unknown kind, bad user values, NULL handle or wrong device */
     BQ_ERR_CUDA = 6       /* a CUDA runtime call or a launch failed             */
 } bq_status;
 

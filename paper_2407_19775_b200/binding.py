@@ -118,8 +118,9 @@ def bq_quantize(x: torch.Tensor, block: int, cb: Codebook, codes_out: torch.Tens
         codes_out = torch.empty(n, dtype=torch.uint8, device=x.device)
     if absmax_out is None:
         absmax_out = torch.empty(n_blocks(n, max(block, 1)), dtype=torch.float32, device=x.device)
-    rc = lib().bq_quantize(x.data_ptr(), _DT[x.dtype], n, block, cb.handle, _dev(codes_out, "codes_out").data_ptr(),
-                           _dev(absmax_out, "absmax_out").data_ptr(), _stream(x))
+    with torch.cuda.device(x.device):
+        rc = lib().bq_quantize(x.data_ptr(), _DT[x.dtype], n, block, cb.handle, _dev(codes_out, "codes_out").data_ptr(),
+                               _dev(absmax_out, "absmax_out").data_ptr(), _stream(x))
     _check(rc, "bq_quantize")
     return codes_out, absmax_out
 
@@ -132,8 +133,9 @@ def bq_dequantize(codes: torch.Tensor, absmax: torch.Tensor, block: int, cb: Cod
     n = codes.numel()
     if y_out is None:
         y_out = torch.empty(n, dtype=dtype, device=codes.device)
-    rc = lib().bq_dequantize(codes.data_ptr(), absmax.data_ptr(), n, block, cb.handle, _dev(y_out, "y_out").data_ptr(),
-                             _DT[y_out.dtype], _stream(codes))
+    with torch.cuda.device(codes.device):
+        rc = lib().bq_dequantize(codes.data_ptr(), absmax.data_ptr(), n, block, cb.handle, _dev(y_out, "y_out").data_ptr(),
+                                 _DT[y_out.dtype], _stream(codes))
     _check(rc, "bq_dequantize")
     return y_out
 
@@ -147,7 +149,8 @@ def bq_roundtrip(x: torch.Tensor, block: int, cb: Codebook, dtype: torch.dtype |
         y_out = torch.empty(x.shape, dtype=dtype or x.dtype, device=x.device)
     c = None if codes_out is None else _dev(codes_out, "codes_out").data_ptr()
     a = None if absmax_out is None else _dev(absmax_out, "absmax_out").data_ptr()
-    rc = lib().bq_roundtrip(x.data_ptr(), _DT[x.dtype], n, block, cb.handle, _dev(y_out, "y_out").data_ptr(), _DT[y_out.dtype], c, a,
-                            _stream(x))
+    with torch.cuda.device(x.device):
+        rc = lib().bq_roundtrip(x.data_ptr(), _DT[x.dtype], n, block, cb.handle, _dev(y_out, "y_out").data_ptr(), _DT[y_out.dtype], c, a,
+                                _stream(x))
     _check(rc, "bq_roundtrip")
     return y_out

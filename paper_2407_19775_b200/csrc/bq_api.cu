@@ -121,6 +121,13 @@ int bq_codebook_is_folded(const bq_codebook* cb) { return (cb && cb->host.folded
 
 namespace {
 
+// The handle's tables live on the device that was current when it was made; a call from
+// another current device would hand the kernels pointers they cannot reach.
+bool on_codebook_device(const bq_codebook* cb) {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == cb->device;
+}
+
 // Shared body of bq_quantize and bq_roundtrip.
 int forward(const void* x, int xdt, size_t n, int block, const bq_codebook* cb, void* y, int ydt, bool write_y,
             uint8_t* codes, float* absmax, bool write_q, cudaStream_t stream) {
@@ -153,6 +160,7 @@ int bq_quantize(const void* x, bq_dtype xdt, size_t n, int block, const bq_codeb
     if (!cb) return BQ_ERR_CODEBOOK;
     if (n == 0) return BQ_OK;
     if (!x || !codes_out || !absmax_out) return BQ_ERR_NULL;
+    if (!on_codebook_device(cb)) return BQ_ERR_CODEBOOK;
     return forward(x, xdt, n, block, cb, nullptr, xdt, false, codes_out, absmax_out, true, static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -165,6 +173,7 @@ int bq_roundtrip(const void* x, bq_dtype xdt, size_t n, int block, const bq_code
     if (n == 0) return BQ_OK;
     if (!x || !y_out) return BQ_ERR_NULL;
     if ((codes_out == nullptr) != (absmax_out == nullptr)) return BQ_ERR_NULL;
+    if (!on_codebook_device(cb)) return BQ_ERR_CODEBOOK;
     return forward(x, xdt, n, block, cb, y_out, ydt, true, codes_out, absmax_out, codes_out != nullptr,
                    static_cast<cudaStream_t>(cuda_stream));
 }
@@ -177,6 +186,7 @@ int bq_dequantize(const uint8_t* codes, const float* absmax, size_t n, int block
     if (!cb) return BQ_ERR_CODEBOOK;
     if (n == 0) return BQ_OK;
     if (!codes || !absmax || !y_out) return BQ_ERR_NULL;
+    if (!on_codebook_device(cb)) return BQ_ERR_CODEBOOK;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const size_t B = size_t(block);
     size_t done = 0;
