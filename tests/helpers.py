@@ -83,3 +83,26 @@ def codes_by_thresholds(xhat: np.ndarray, cb: np.ndarray) -> np.ndarray:
     midpoints are exact in float64 for this codebook (checked by the caller's test)."""
     t = (cb[:-1].astype(np.float64) + cb[1:].astype(np.float64)) / 2.0
     return np.searchsorted(t, xhat.astype(np.float64), side="left").astype(np.uint8)
+
+
+def reciprocal_sensitive_pairs(cb: np.ndarray, per_threshold: int = 3, seed: int = 0):
+    """(x, a) pairs, |x| <= a, whose correctly rounded quotient x / a sits exactly on a
+    round-down midpoint (so the code is j) while the product x * RN(1/a) lands one float
+    higher (code j + 1), or the other way round.  A normalisation that multiplies by a
+    rounded reciprocal gets these wrong; a true division gets them right."""
+    rng = np.random.default_rng(seed)
+    out = []
+    for t in midpoints(cb):
+        lo = round_down32(t)
+        if abs(float(lo)) < 1e-6:
+            continue
+        a = (1.0 + rng.random(4000)).astype(np.float32) * np.float32(2.0) ** rng.integers(-3, 4, 4000).astype(np.float32)
+        for target in (lo, np.nextafter(lo, np.float32(np.inf))):
+            x = (target * a).astype(np.float32)
+            q_div = (x / a).astype(np.float32)
+            q_rcp = (x * (np.float32(1.0) / a)).astype(np.float32)
+            lo_hi = (lo, np.nextafter(lo, np.float32(np.inf)))
+            hit = (q_div != q_rcp) & np.isin(q_div, lo_hi) & np.isin(q_rcp, lo_hi) & (np.abs(x) <= a)
+            for i in np.flatnonzero(hit)[:per_threshold]:
+                out.append((np.float32(x[i]), np.float32(a[i])))
+    return out

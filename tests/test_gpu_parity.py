@@ -7,7 +7,7 @@ import pytest
 import torch
 
 import oracle
-from helpers import midpoints, round_down32
+from helpers import midpoints, reciprocal_sensitive_pairs, round_down32
 from paper_2407_19775_b200 import workloads
 
 pytestmark = pytest.mark.gpu
@@ -286,6 +286,35 @@ def test_every_breakpoint_exactly(bq, gcb, cb):
             rows.append(np.concatenate([[1.0], chunk, np.zeros(63 - chunk.size, np.float32)]))
         x = torch.from_numpy((np.concatenate(rows) * np.float32(scale)).astype(np.float32))
         check_all_ops(bq, gcb, cb, x, 64)
+
+
+def test_quotients_that_a_rounded_reciprocal_gets_wrong(bq, gcb, cb):
+    """fp32 pairs where x / a lands exactly on a breakpoint but x * RN(1/a) lands one float
+    off (or the reverse): blocks [a, x, 0, ...] through the tuned and the general kernels."""
+    pairs = reciprocal_sensitive_pairs(cb)
+    rows = np.zeros((len(pairs), 64), np.float32)
+    rows[:, 0] = [p[1] for p in pairs]
+    rows[:, 1] = [p[0] for p in pairs]
+    check_all_ops(bq, gcb, cb, torch.from_numpy(rows.reshape(-1)), 64)
+    check_all_ops(bq, gcb, cb, torch.from_numpy(rows[:, :2].reshape(-1).copy()), 2)
+
+
+def test_random_shapes_types_and_offsets(bq, gcb, cb):
+    """Seeded fuzz: random length, block (powers of two and not), input type, pointer offset,
+    value scale; every call against the oracle."""
+    rng = np.random.default_rng(2024)
+    g = torch.Generator().manual_seed(2024)
+    dtypes = [torch.float32, torch.float16, torch.bfloat16]
+    for case in range(40):
+        block = int(rng.choice([1, 3, 16, 48, 64, 100, 128, 256, 512, 1000, 1024, 2048, 4096, 5000]))
+        n = int(rng.integers(1, 60_000))
+        dtype = dtypes[int(rng.integers(0, 3))]
+        scale = float(10.0 ** rng.uniform(-3, 3)) if dtype != torch.float16 else float(10.0 ** rng.uniform(-2, 2))
+        x = (torch.randn(n, generator=g) * scale).to(dtype)
+        if rng.random() < 0.3:
+            x[:: max(1, n // 7)] = 0.0
+        offset = int(rng.choice([0, 0, 0, 1, 2, 8]))
+        check_all_ops(bq, gcb, cb, x, block, offset_elems=offset)
 
 
 @pytest.mark.parametrize("dtype,sig", [(torch.bfloat16, 8), (torch.float16, 11)])

@@ -93,6 +93,19 @@ def test_quantize_tiny_exact_rational(cb):
             assert codes[4 * b + i] == nearest_exact(xhat, cb)
 
 
+def test_normalisation_is_a_true_division(cb):
+    """Pairs built so that x / a rounds onto a midpoint's round-down value while x * RN(1/a)
+    rounds to its neighbour (or the reverse): the code differs between the two."""
+    from helpers import reciprocal_sensitive_pairs, rn32
+    pairs = reciprocal_sensitive_pairs(cb)
+    assert len(pairs) > 200
+    x = np.array([v for pair in pairs for v in (pair[1], pair[0])], np.float32)      # blocks of 2: [a, x]
+    codes, absmax = oracle.quantize(x, F32, 2, cb)
+    for k, (xv, av) in enumerate(pairs):
+        assert absmax[k] == av
+        assert codes[2 * k + 1] == nearest_exact(rn32(frac_of(xv) / frac_of(av)), cb), (float(xv), float(av))
+
+
 def test_zero_block_negative_zero_and_flush(cb):
     x = np.zeros(64, np.float32)
     x[5] = -0.0
