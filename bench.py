@@ -277,9 +277,9 @@ def run_ours(args):
 # dirty lines that are still in L2 when the kernel ends, a size-independent residue measured
 # in the same capture.  Set an entry to None when its kernel changes until it is re-measured.
 TRAFFIC_BYTES = {
-    "quantize_b64": 1600887040, "quantize_b256": 1579075328, "quantize_b1024": 1573408256, "quantize_b4096": 1571947264,
-    "dequantize_b64": 1588571904, "dequantize_b256": 1560674048, "dequantize_b1024": 1555077888, "dequantize_b4096": 1553117440,
-    "roundtrip_b64": 2095402240, "roundtrip_b256": 2095243264, "roundtrip_b1024": 2096132608, "roundtrip_b4096": 2095491584,
+    "quantize_b64": 1599487744, "quantize_b256": 1578846464, "quantize_b1024": 1573560576, "quantize_b4096": 1572869632,
+    "dequantize_b64": 1586586368, "dequantize_b256": 1560828416, "dequantize_b1024": 1555288832, "dequantize_b4096": 1553292032,
+    "roundtrip_b64": 2095262976, "roundtrip_b256": 2095527936, "roundtrip_b1024": 2095371776, "roundtrip_b4096": 2095418624,
 }
 
 
