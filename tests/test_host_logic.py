@@ -85,7 +85,7 @@ def test_searches_agree_on_random_and_cell_edges(hc, cb):
     lo = np.uint32(0)
     out_f = np.empty(1 << 20, np.uint8); out_g = np.empty(1 << 20, np.uint8)
     bad = 0
-    # dense sweeps: the smallest decades, around 2^-22 (where keys are clamped), and the top of the range
+    # dense sweeps: the smallest decades, near 2^-22 (where keys are clamped), and the top of the range
     for start in (0x33000000, 0x34700000, 0x3F700000, 0xB3000000, 0xB4700000, 0xBF700000):
         hc.hc_codes_of_bits(ctypes.c_uint32(start), ctypes.c_uint32(1 << 20), _p(out_f), _p(out_g))
         bad += int((out_f != out_g).sum())

@@ -1,7 +1,7 @@
 """Pins for the oracle's dynamic-tree codebook (CPU only).
 
-What fixes the codebook (north-star reading of the paper's "dynamic blockwise
-quantization", section "Compression techniques" item 1): an 8-bit map over [-1, 1] made of a
+What fixes the codebook (the reading taken of the paper's "dynamic blockwise
+quantization", section "Compression techniques" item 1, which does not define the map): an 8-bit map over [-1, 1] made of a
 sign bit, a variable-length exponent field and a linear fraction.  The checks below rebuild
 it three independent ways (exact rationals, the bit-field decoding, structural invariants)."""
 import hashlib
