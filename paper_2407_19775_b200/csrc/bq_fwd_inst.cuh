@@ -22,7 +22,6 @@ template <int XDT, int B, int RMAX> struct Shape {
     static constexpr int TW = (IN_ROW || ROWS <= RMAX) ? 1 : ROWS / RMAX;
 };
 
-constexpr int kLiteNT = 256;
 // Below this many elements the per-CTA table set-up of the tuned kernel (193 KB of shared
 // memory to fill) costs more than it saves; the LITE kernels read the tables through L1.
 #ifndef BQ_LITE_MAX_LOG2
@@ -35,7 +34,9 @@ template <int XDT, int B, bool WY, bool WQ>
 cudaError_t go(const void* x, void* y, uint8_t* codes, float* absmax, size_t n_full, const bqk::DeviceTables& tab, int sm_count,
                int device, cudaStream_t stream, size_t* done) {
     if (n_full <= kLiteMaxElems) {
-        using S = Shape<XDT, B, 4>;              // smaller tiles: more CTAs for a small tensor
+        // small tiles and small CTAs, so that even a decode-step tensor spreads over all SMs
+        using S = Shape<XDT, B, (B <= 32 * bqk::Elem<XDT>::kPerChunk) ? 2 : 4>;
+        constexpr int kLiteNT = 32 * (S::TW > 4 ? S::TW : 4);
         const size_t tile = size_t(S::TW) * S::R * S::ROW;
         const size_t ntiles = n_full / tile;
         *done = ntiles * tile;
