@@ -4,7 +4,11 @@
 //   fwd_fast     : quantize, or the fused quantize->dequantize roundtrip, for power-of-two
 //                  blocks on 16-byte aligned tensors.  One pass over HBM: a tile of the
 //                  input sits in registers between the absmax reduction and the search.
-//   deq_fast     : dequantize, 16 codes per thread.
+//                  Built in two flavours: persistent CTAs with the search tables replicated
+//                  per lane in shared memory (large tensors), and LITE, which reads the
+//                  tables through L1 and has no set-up (small tensors).
+//   deq_fast     : dequantize, 16 codes per 128-bit load, one 256-bit store per 16 outputs;
+//                  the same two flavours.
 //   *_general    : any block size, any alignment, any codebook; one warp per block.
 //
 // Arithmetic contract shared by all of them (it is what makes the results bit-identical
@@ -42,9 +46,9 @@ struct DeviceTables {
     const float* values;        // [256]
     const float* thr_down;      // [256], last = +inf
     const uint32_t* tk;         // [128]
-    const float* cmag;          // [132]
+    const float* cmag;          // [132]; guess follows it directly in memory
     const uint32_t* guess;      // [kCells]
-    float neg_limit;
+    float neg_limit;            // -(largest |xhat| whose negative key does not pass the last threshold)
 };
 
 // ------------------------------------------------------------------------------------------
@@ -58,31 +62,16 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
 __device__ __forceinline__ void sts_u32(uint32_t addr, uint32_t v) {
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
-#ifndef BQ_LD
-#define BQ_LD 3
-#endif
-#ifndef BQ_ST
-#define BQ_ST 0
-#endif
+// Streaming accesses.  Loads skip L1 allocation (every byte is used once) but are not
+// marked read-only, so bq_roundtrip may run in place; stores are evict-first.  Of the
+// cache-operator combinations tried on a 1 GiB tensor this one was the fastest by 1-3 %.
 __device__ __forceinline__ uint4 ldg_stream_16(const void* p) {
     uint4 v;
-#if BQ_LD == 0
-    asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-#elif BQ_LD == 1
-    asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-#elif BQ_LD == 2
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-#else
     asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-#endif
     return v;
 }
 __device__ __forceinline__ void stg_stream_16(void* p, uint4 v) {
-#if BQ_ST == 0
     asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-#else
-    asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-#endif
 }
 // 32 contiguous bytes per thread as one 256-bit store: a warp then writes whole 128-byte lines
 __device__ __forceinline__ void stg_stream_32(void* p, uint4 a, uint4 b) {
