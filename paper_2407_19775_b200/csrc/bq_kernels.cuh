@@ -222,13 +222,31 @@ __device__ __forceinline__ uint32_t sign_mask_32(uint32_t a, uint32_t b, uint32_
     return prmt(prmt(a, b, 0x00FBu), prmt(c, d, 0x00FBu), 0x5410u);
 }
 
+// Two fp32 lanes per instruction (sm_100 packed fp32 arithmetic).
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+    uint64_t v;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(a), "f"(b));
+    return v;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
 // c[code] * absmax as one rounding: the magnitude times the signed absmax, plus +0.0 so
 // that a zero magnitude gives +0.0 whatever the sign.
 template <bool LITE>
-__device__ __forceinline__ float value_of(const Found& f, float absmax, const TabRef<LITE>& tab) {
-    const float cm = tab.magnitude(f.sum);
-    const float as = __uint_as_float(__float_as_uint(absmax) | (f.bits & 0x80000000u));
-    return __fmaf_rn(cm, as, 0.0f);
+__device__ __forceinline__ void values_of(const Found& f0, const Found& f1, float absmax, const TabRef<LITE>& tab, float& v0, float& v1) {
+    const float c0 = tab.magnitude(f0.sum), c1 = tab.magnitude(f1.sum);
+    const float a0 = __uint_as_float(__float_as_uint(absmax) | (f0.bits & 0x80000000u));
+    const float a1 = __uint_as_float(__float_as_uint(absmax) | (f1.bits & 0x80000000u));
+    unpack2(fma2(pack2(c0, c1), pack2(a0, a1), 0ull), v0, v1);         // two products per instruction; +0.0 addend
 }
 
 // Builds the per-lane copies.  The magnitude rows and the entry rows are consecutive both in
@@ -260,23 +278,6 @@ __device__ __forceinline__ void fill_fwd_tables(const DeviceTables& t, uint32_t 
     }
 }
 
-// Two fp32 lanes per instruction (sm_100 packed fp32 arithmetic).
-__device__ __forceinline__ uint64_t pack2(float a, float b) {
-    uint64_t v;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(a), "f"(b));
-    return v;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
-__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
-    uint64_t d;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-    uint64_t d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
 __device__ __forceinline__ float max3_abs(float a, float b, float c) {      // max(|a|, |b|, |c|)
     float d;
     asm("max.abs.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -500,9 +501,10 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
             float out[EPC];
             Found fd[EPC];
 #pragma unroll
-            for (int i = 0; i < EPC; ++i) {
+            for (int i = 0; i < EPC; i += 2) {
                 fd[i] = search_folded(f[r][i], neg_limit, tref);
-                if constexpr (WRITE_Y) out[i] = value_of(fd[i], amax[r], tref);
+                fd[i + 1] = search_folded(f[r][i + 1], neg_limit, tref);
+                if constexpr (WRITE_Y) values_of(fd[i], fd[i + 1], amax[r], tref, out[i], out[i + 1]);
             }
             const size_t off = base + size_t(r) * ROW;
             {
