@@ -1,0 +1,33 @@
+"""bench.py end to end on a GPU: one short run, then the JSON line is checked against the
+measurement contract (keys, units, launch count, sane roofline fractions)."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+
+pytestmark = pytest.mark.gpu
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_bench_line_has_the_contract_keys(bq):
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--steps", "4", "--warmup", "3", "--e2e-steps", "1", "--no-cpu-baseline"],
+                       capture_output=True, text=True, timeout=600, cwd=ROOT)
+    assert r.returncode == 0, r.stderr[-2000:]
+    d = json.loads(r.stdout.strip().splitlines()[-1])
+    for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling", "vs_baseline",
+                "dtype", "data", "config", "e2e", "gpu_launches", "clocks", "roofline", "cpu_baseline"):
+        assert key in d, key
+    assert d["unit"] == "GB/s" and d["n_gpus"] == 1 and d["steps"] == 4 and d["higher_is_better"] is True
+    assert d["data"] == "synthetic" and "workload" in d["config"] and d["vs_baseline"] is None
+    assert d["gpu_launches"] == 4 * 12
+    rf = d["roofline"]
+    assert rf["bound"] == "hbm" and rf["unit"] == "GB/s" and 0.3 < rf["frac"] < 1.1 and abs(rf["frac"] - rf["achieved"] / rf["peak"]) < 1e-3
+    assert rf["traffic"] is None or 0.9 < rf["traffic"] / d["kernels"][rf["kernel"]]["algorithmic_bytes"] < 1.1
+    e = d["e2e"]
+    assert e["unit"] == "GB/s" and 0 < e["value"] < d["value"] and e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] > 0
+    assert len(d["kernels"]) == 12 and all(0.2 < k["frac_of_measured"] < 1.1 for k in d["kernels"].values())
+    assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
+    for q in d["quality"].values():
+        assert 1.8 < q["compression_ratio"] < 2.0 and 0.003 < q["rel_rms_error"] < 0.03
