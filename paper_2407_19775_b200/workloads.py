@@ -151,3 +151,70 @@ def from_numpy_bits(a: np.ndarray, dtype: torch.dtype) -> torch.Tensor:
     if dtype == torch.float32:
         return torch.from_numpy(np.ascontiguousarray(a, np.float32))
     return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).view(dtype)
+
+
+# ------------------------------------------------------------------------------------------
+# Linear layers for the mixed matrix decomposition: activations X [tokens, in_features] with
+# a few persistent outlier features, weights W [out_features, in_features], and the indices
+# of the planted outlier features (what a calibration pass would report as critical).
+
+@dataclass(frozen=True)
+class LinearWorkload:
+    name: str
+    tokens: int
+    in_features: int
+    out_features: int
+    dtype: torch.dtype
+    n_outlier_features: int
+    seed: int
+    recipe: str
+
+
+LINEAR_WORKLOADS = {
+    "mmd_tiny": LinearWorkload("mmd_tiny", 37, 320, 72, torch.bfloat16, 3, 10,
+                               "X = 0.5 N(0,1), 3 features x40; W = 0.05 N(0,1); ragged tokens and out_features"),
+    "mmd_decode70b": LinearWorkload("mmd_decode70b", 64, 8192, 8192, torch.float16, 8, 11,
+                                    "X = 0.3 Student-t(3), 8 features x30; W = 0.02 N(0,1)"),
+    "mmd_prefill_moe": LinearWorkload("mmd_prefill_moe", 4096, 6144, 16384, torch.bfloat16, 6, 12,
+                                      "X = 0.5 N(0,1), 6 features x40; W = 0.02 N(0,1) with 0.05% entries x8"),
+}
+
+
+def make_linear(name: str, tokens: int | None = None, out_features: int | None = None):
+    """Draws (X, W, outlier_features) of linear workload ``name`` on the CPU.  ``tokens`` /
+    ``out_features`` keep only the first rows of X / W (a prefix equals the same rows of the
+    full draw).  outlier_features is an ascending int32 numpy array."""
+    w = LINEAR_WORKLOADS[name]
+    g = _gen(w.seed)
+    K = w.in_features
+    feats = torch.sort(torch.randperm(K, generator=g)[:w.n_outlier_features]).values
+    M = w.tokens if tokens is None else min(tokens, w.tokens)
+    N = w.out_features if out_features is None else min(out_features, w.out_features)
+    gx = _gen(w.seed + 1000)
+    gw = _gen(w.seed + 2000)
+    X = torch.empty((M, K), dtype=w.dtype)
+    step = _rows_per_chunk(K)
+    for r0 in range(0, M, step):
+        r1 = min(M, r0 + step)
+        if name == "mmd_decode70b":
+            z = torch.randn((r1 - r0, K), generator=gx)
+            chi2 = sum(torch.randn((r1 - r0, K), generator=gx) ** 2 for _ in range(3))
+            x = z / torch.sqrt(chi2 / 3.0) * 0.3
+            x[:, feats] *= 30.0
+        else:
+            x = torch.randn((r1 - r0, K), generator=gx) * 0.5
+            x[:, feats] *= 40.0
+        X[r0:r1] = x.to(w.dtype)
+    W = torch.empty((N, K), dtype=w.dtype)
+    for r0 in range(0, N, step):
+        r1 = min(N, r0 + step)
+        v = torch.randn((r1 - r0, K), generator=gw) * (0.05 if name == "mmd_tiny" else 0.02)
+        if name == "mmd_prefill_moe":
+            v = torch.where(torch.rand((r1 - r0, K), generator=gw) < 0.0005, v * 8.0, v)
+        W[r0:r1] = v.to(w.dtype)
+    return X.contiguous(), W.contiguous(), feats.numpy().astype(np.int32)
+
+
+def bits_2d(x: torch.Tensor) -> np.ndarray:
+    """A 2-D fp16 / bf16 CPU tensor as a uint16 bit-pattern array of the same shape."""
+    return as_numpy_bits(x).reshape(x.shape)
