@@ -1,0 +1,129 @@
+/*
+ * mmd.h -- C ABI of the mixed matrix decomposition in libbq: 16-bit weight matrices stored as
+ * 8-bit integers plus a small 16-bit part, and the linear layer computed from that form on
+ * the sm_100a tensor cores.
+ *
+ * Source of the operation: the paper's section "Compression techniques", item 2 ("Mixed
+ * matrix decomposition"): weights go from 16-bit to 8-bit values while a small fraction of
+ * critical weights is kept at 16-bit precision.  The paper gives no arithmetic; the reading
+ * implemented here is the vector-wise int8 decomposition with a 16-bit side matrix over a
+ * fixed, ascending set O of critical input features (columns):
+ *
+ *   rowquant of a [R, K] 16-bit matrix v, row by row:
+ *       a_r      = max over k not in O of |v[r,k]|           (fp32, exact)
+ *       q[r,k]   = 0 for k in O, else rint(RN32(RN32(127 v[r,k]) / d_r)), d_r = a_r or 1 if a_r == 0
+ *       scale[r] = RN32(a_r / 127)
+ *       side[r,j] = v[r, O_j] for j < |O|, and 0 for the padding columns j up to mmd_side_columns(|O|)
+ *   linear layer Y = X W^T from rowquant(X) (per call) and rowquant(W) (once, mmd_decompose):
+ *       acc[m,n]  = sum_k qx[m,k] qw[n,k]                    (int32, exact)
+ *       part[m,n] = sum_j sidex[m,j] sidew[n,j]              (fp32 accumulation)
+ *       Y[m,n]    = narrow( fma( fp32(acc[m,n]), RN32(scalex[m] scalew[n]), part[m,n] ) )
+ *
+ * Conventions
+ *   - Pointers are DEVICE pointers to contiguous row-major memory owned by the caller unless
+ *     a comment says HOST.  Status codes and element types are those of bq.h.
+ *   - Element types: BQ_F16 or BQ_BF16 for v, X, W; Y is the same type or BQ_F32.
+ *   - K must be a multiple of 16 and at most 262144; |O| at most 1024; rows at most 2^31 - 1.
+ *     Inputs must be finite with magnitudes below 2^120 (127 v must not overflow).
+ *   - Work is enqueued on `cuda_stream` and the call returns without synchronising; nothing
+ *     is allocated per call (mmd_decompose allocates the handle's device memory once).
+ *   - A handle belongs to the device that was current when it was made.
+ */
+#ifndef MMD_H
+#define MMD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#include "bq.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Additional status codes (continuing bq_status). */
+enum {
+    MMD_ERR_WORKSPACE = 7, /* workspace missing, misaligned (256 bytes) or too small   */
+    MMD_ERR_FEATURES = 8,  /* feature list not ascending, out of range or too long      */
+    MMD_ERR_PATH = 9       /* the requested kernel path cannot take this shape          */
+};
+
+/* Kernel choice of mmd_linear. */
+enum {
+    MMD_PATH_AUTO = 0,     /* tensor-core kernel when the shape allows, else the general one */
+    MMD_PATH_GENERAL = 1,  /* integer dot-product kernel, any M and N                       */
+    MMD_PATH_TENSOR = 2    /* tcgen05 kernel; needs N % 8 == 0 and 16-byte aligned Y        */
+};
+
+/* Opaque: the decomposed weights of one linear layer (int8 rows, row scales, 16-bit side
+ * columns, the feature list) on the device that was current when it was made. */
+typedef struct mmd_weights mmd_weights;
+
+/* Width of the side matrices for n_features critical features: the next multiple of 64
+ * (0 for 0). */
+int mmd_side_columns(int n_features);
+
+/*
+ * mmd_select_features -- the critical input features of a layer: those whose calibration
+ * magnitude reaches tau.  Host only.
+ *   feature_absmax: HOST, K floats (largest |activation| seen per input feature).
+ *   idx_out: HOST, room for K ints; receives the ascending indices.  count_out: HOST.
+ */
+int mmd_select_features(const float* feature_absmax, int K, float tau, int32_t* idx_out, int* count_out);
+
+/*
+ * mmd_rowquant -- the row operation defined at the top of this file.
+ *   v: [R, K] of type dt.  idx: n_features ascending ints on the DEVICE (may be NULL when 0).
+ *   q_out: [R, K] int8.  scale_out: [R] floats.  side_out: [R, mmd_side_columns(n_features)]
+ *   of type dt (may be NULL when n_features == 0).  v and q_out need 16-byte alignment.
+ */
+int mmd_rowquant(const void* v, bq_dtype dt, int R, int K, const int32_t* idx, int n_features,
+                 int8_t* q_out, float* scale_out, void* side_out, void* cuda_stream);
+
+/*
+ * mmd_decompose -- rowquant of a weight matrix W [N, K] into a new handle (the offline step).
+ *   idx_host: HOST, n_features ascending ints in [0, K).  Allocates device memory, enqueues
+ *   the row kernel on cuda_stream; the handle may be used by later calls on the same stream
+ *   (or after synchronising).  W may be freed once that work has run.  Free with mmd_free.
+ */
+int mmd_decompose(const void* W, bq_dtype dt, int N, int K, const int32_t* idx_host, int n_features,
+                  void* cuda_stream, mmd_weights** out);
+
+/* Frees the handle and its device memory.  NULL is allowed. */
+int mmd_free(mmd_weights* w);
+
+/* Device pointers and sizes of a handle's parts, for inspection (any out pointer may be NULL). */
+int mmd_weights_view(const mmd_weights* w, const int8_t** q, const float** scale, const void** side,
+                     const int32_t** idx, int* N, int* K, int* n_features, int* dtype);
+
+/*
+ * mmd_workspace_layout -- the scratch memory mmd_linear needs for M rows of activations:
+ * byte offsets of qx [M, K] int8, scalex [M] floats and sidex [M, side columns] inside the
+ * workspace, and its total size.  Host only.  offsets3 may be NULL.
+ */
+int mmd_workspace_layout(const mmd_weights* w, int M, size_t* offsets3, size_t* total_bytes);
+
+/*
+ * mmd_linear -- Y = X W^T through the decomposition: one row kernel over X into the
+ * workspace, then one product kernel.
+ *   X: [M, K] of the handle's element type (16-byte aligned).  Y: [M, N] of type ydt.
+ *   workspace: at least mmd_workspace_layout's total, 256-byte aligned; its contents after
+ *   the call are the decomposition of X (tests read them back).  Calls that share a
+ *   workspace must not overlap on the device.
+ *   path: MMD_PATH_*.  The two kernels give identical integer sums; their fp32 side sums may
+ *   differ in the order of the additions.
+ */
+int mmd_linear(const mmd_weights* w, const void* X, int M, void* Y, bq_dtype ydt,
+               void* workspace, size_t workspace_bytes, int path, void* cuda_stream);
+
+/*
+ * mmd_kernel_status -- synchronises the device and returns, through status_out (HOST), 0 or
+ * the code a tensor-core kernel left when one of its bounded waits ran out (it then stores
+ * nothing more and returns; the context stays usable).  Clears the code.
+ */
+int mmd_kernel_status(const mmd_weights* w, int* status_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -7,7 +7,8 @@ from . import workloads
 from .binding import (BF16, DYNAMIC_TREE, F16, F32, USER, BqError, Codebook, bq_dequantize, bq_quantize, bq_roundtrip,
                       n_blocks)
 
+from .mmd import DecomposedLinear, mmd_rowquant, mmd_select_features, mmd_side_columns
 from .pipeline import HostBoundary
 
-__all__ = ["workloads", "HostBoundary", "Codebook", "BqError", "bq_quantize", "bq_dequantize", "bq_roundtrip", "n_blocks",
+__all__ = ["workloads", "HostBoundary", "DecomposedLinear", "mmd_rowquant", "mmd_select_features", "mmd_side_columns", "Codebook", "BqError", "bq_quantize", "bq_dequantize", "bq_roundtrip", "n_blocks",
            "F32", "F16", "BF16", "DYNAMIC_TREE", "USER"]

@@ -1,6 +1,8 @@
 // bq_api.cu -- the C ABI of libbq (see include/bq.h): argument checks, codebook handles and
 // the choice of kernel.  Kernel instantiations live in bq_inst_*.cu so that they compile in
 // parallel; this file only calls their launchers.
+#include "../../include/mmd.h"
+#include "bq_error.h"
 #include "bq_launch.h"
 
 #include <cstring>
@@ -11,7 +13,7 @@ namespace {
 thread_local char g_last_error[256] = "";
 
 int cuda_fail(cudaError_t e) {
-    std::strncpy(g_last_error, cudaGetErrorString(e), sizeof(g_last_error) - 1);
+    bql::set_last_cuda_error(cudaGetErrorString(e));
     return BQ_ERR_CUDA;
 }
 
@@ -36,6 +38,8 @@ constexpr size_t kMaxElems = size_t(1) << 40;
 
 }  // namespace
 
+void bql::set_last_cuda_error(const char* text) { std::strncpy(g_last_error, text, sizeof(g_last_error) - 1); }
+
 struct bq_codebook {
     bqt::Tables host;
     bqk::DeviceTables dev;
@@ -55,6 +59,9 @@ const char* bq_status_string(int status) {
         case BQ_ERR_SIZE: return "element count out of range";
         case BQ_ERR_CODEBOOK: return "invalid codebook kind, values or handle";
         case BQ_ERR_CUDA: return "CUDA runtime error (see bq_last_cuda_error)";
+        case MMD_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case MMD_ERR_FEATURES: return "feature list not ascending, out of range or too long";
+        case MMD_ERR_PATH: return "the requested kernel path cannot take this shape";
         default: return "unknown status";
     }
 }

@@ -1,0 +1,309 @@
+// mmd_api.cu -- the C ABI of the mixed matrix decomposition (see include/mmd.h): argument
+// checks, the weight handle, tensor maps and the choice of kernel.
+#include "../../include/mmd.h"
+#include "bq_error.h"
+#include "mmd_kernels.cuh"
+
+#include <cstring>
+#include <new>
+
+namespace {
+
+constexpr int kMaxK = 262144;
+constexpr int kMaxFeatures = 1024;
+constexpr size_t kWsAlign = 256;
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+bool is16(int dt) { return dt == BQ_F16 || dt == BQ_BF16; }
+
+// cuTensorMapEncodeTiled through the runtime's entry-point lookup (no link against the driver library)
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess && qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// Row-major [rows, cols] matrix of 1- or 2-byte elements, tiles of box_rows x 128 bytes, 128-byte swizzle.
+bool make_map(CUtensorMap* map, const void* base, int elem_bytes, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * uint64_t(elem_bytes)};
+    const cuuint32_t box[2] = {cuuint32_t(128 / elem_bytes), box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUtensorMapDataType dt = (elem_bytes == 1) ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_UINT16;
+    return fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int DT>
+cudaError_t launch_rowquant(const void* v, int R, int K, const int32_t* idx, int ko, int8_t* q, float* scale, void* side, int sm_count,
+                            cudaStream_t stream) {
+    const size_t smem = round_up(size_t(K) / 8, 4);
+    if (smem > 48 * 1024) return cudaErrorInvalidValue;          // K <= kMaxK keeps the mask within the default limit
+    int grid = R;
+    const int cap = sm_count * 16;
+    if (grid > cap) grid = cap;
+    mmdk::rowquant<DT><<<grid, 256, smem, stream>>>(v, R, K, idx, ko, mmd_side_columns(ko), q, scale, side);
+    return cudaGetLastError();
+}
+
+cudaError_t rowquant_any(int dt, const void* v, int R, int K, const int32_t* idx, int ko, int8_t* q, float* scale, void* side, int sm_count,
+                         cudaStream_t stream) {
+    return dt == BQ_BF16 ? launch_rowquant<mmdk::kBF16>(v, R, K, idx, ko, q, scale, side, sm_count, stream)
+                         : launch_rowquant<mmdk::kF16>(v, R, K, idx, ko, q, scale, side, sm_count, stream);
+}
+
+int check_features(const int32_t* idx_host, int ko, int K) {
+    if (ko < 0 || ko > kMaxFeatures || ko >= K) return MMD_ERR_FEATURES;
+    if (ko > 0 && !idx_host) return BQ_ERR_NULL;
+    for (int j = 0; j < ko; ++j) {
+        if (idx_host[j] < 0 || idx_host[j] >= K) return MMD_ERR_FEATURES;
+        if (j > 0 && idx_host[j] <= idx_host[j - 1]) return MMD_ERR_FEATURES;
+    }
+    return BQ_OK;
+}
+
+int cuda_fail(cudaError_t e) {
+    bql::set_last_cuda_error(cudaGetErrorString(e));
+    return BQ_ERR_CUDA;
+}
+
+}  // namespace
+
+struct mmd_weights {
+    int N, K, ko, side_cols, dtype, device, sm_count;
+    void* blob;                  // q | scale | side | idx | status
+    int8_t* q;
+    float* scale;
+    void* side;
+    int32_t* idx;
+    int* status;
+    bool have_maps;
+    CUtensorMap map_q[3], map_side[3];       // weight tiles of 256, 128 and 64 rows
+};
+
+namespace {
+
+struct WsLayout { size_t q, scale, side, total; };
+
+WsLayout ws_layout(const mmd_weights* w, int M) {
+    WsLayout L;
+    L.q = 0;
+    L.scale = round_up(size_t(M) * w->K, kWsAlign);
+    L.side = L.scale + round_up(size_t(M) * 4, kWsAlign);
+    L.total = L.side + round_up(size_t(M) * w->side_cols * 2, kWsAlign);
+    return L;
+}
+
+bool on_device(const mmd_weights* w) {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == w->device;
+}
+
+int bn_slot(int bn) { return bn == 256 ? 0 : (bn == 128 ? 1 : 2); }
+
+template <int XDT, int YDT, int BN>
+cudaError_t launch_tc(const mmd_weights* w, const CUtensorMap& mqx, const CUtensorMap& msx, const float* sx, void* y, int M,
+                      cudaStream_t stream) {
+    using Cfg = mmdk::TcCfg<BN>;
+    static bool opted[64] = {};
+    if (w->device < 0 || w->device >= 64 || !opted[w->device]) {
+        const cudaError_t e = cudaFuncSetAttribute(mmdk::gemm_tc<XDT, YDT, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::kSmemBytes));
+        if (e != cudaSuccess) return e;
+        if (w->device >= 0 && w->device < 64) opted[w->device] = true;
+    }
+    const dim3 grid(unsigned((M + 127) / 128), unsigned((w->N + BN - 1) / BN));
+    const int kblocks = (w->K + 127) / 128, sblocks = w->side_cols / 64;
+    const int slot = bn_slot(BN);
+    mmdk::gemm_tc<XDT, YDT, BN><<<grid, mmdk::kTcThreads, Cfg::kSmemBytes, stream>>>(
+        mqx, w->map_q[slot], sblocks ? msx : mqx, sblocks ? w->map_side[slot] : w->map_q[slot], sx, w->scale, y, M, w->N, kblocks, sblocks, w->status);
+    return cudaGetLastError();
+}
+
+template <int XDT, int YDT>
+cudaError_t launch_tc_bn(const mmd_weights* w, const CUtensorMap& mqx, const CUtensorMap& msx, const float* sx, void* y, int M,
+                         cudaStream_t stream) {
+    // The widest tile has the highest arithmetic intensity; when it would leave SMs without a
+    // tile (few rows, as in a decode step, where the weights are read once and the kernel is
+    // bound by that stream) narrower tiles put more CTAs on the weight stream.
+    const long mt = (M + 127) / 128;
+    if (w->N >= 256 && mt * ((w->N + 255) / 256) >= w->sm_count) return launch_tc<XDT, YDT, 256>(w, mqx, msx, sx, y, M, stream);
+    if (w->N >= 128 && mt * ((w->N + 127) / 128) >= w->sm_count) return launch_tc<XDT, YDT, 128>(w, mqx, msx, sx, y, M, stream);
+    return launch_tc<XDT, YDT, 64>(w, mqx, msx, sx, y, M, stream);
+}
+
+template <int XDT, int YDT>
+cudaError_t launch_general(const mmd_weights* w, const int8_t* qx, const float* sx, const void* sidex, void* y, int M, cudaStream_t stream) {
+    const dim3 grid(unsigned((w->N + 63) / 64), unsigned((M + 63) / 64));
+    mmdk::gemm_general<XDT, YDT><<<grid, 256, 0, stream>>>(qx, w->q, sx, w->scale, sidex, w->side, w->side_cols, y, M, w->N, w->K);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+extern "C" {
+
+int mmd_side_columns(int n_features) {
+    return n_features <= 0 ? 0 : (n_features + mmdk::kSidePad - 1) / mmdk::kSidePad * mmdk::kSidePad;
+}
+
+int mmd_select_features(const float* feature_absmax, int K, float tau, int32_t* idx_out, int* count_out) {
+    if (!feature_absmax || !idx_out || !count_out) return BQ_ERR_NULL;
+    if (K < 1) return BQ_ERR_SIZE;
+    int c = 0;
+    for (int k = 0; k < K; ++k)
+        if (feature_absmax[k] >= tau) idx_out[c++] = k;
+    *count_out = c;
+    return BQ_OK;
+}
+
+int mmd_rowquant(const void* v, bq_dtype dt, int R, int K, const int32_t* idx, int n_features, int8_t* q_out, float* scale_out,
+                 void* side_out, void* cuda_stream) {
+    if (!is16(dt)) return BQ_ERR_DTYPE;
+    if (R < 0 || K < 16 || K % 16 != 0 || K > kMaxK) return BQ_ERR_SIZE;
+    if (n_features < 0 || n_features > kMaxFeatures || n_features >= K) return MMD_ERR_FEATURES;
+    if (R == 0) return BQ_OK;
+    if (!v || !q_out || !scale_out || (n_features > 0 && (!idx || !side_out))) return BQ_ERR_NULL;
+    if (!aligned(v, 16) || !aligned(q_out, 16)) return BQ_ERR_SIZE;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = rowquant_any(dt, v, R, K, idx, n_features, q_out, scale_out, side_out, sms, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? BQ_OK : cuda_fail(e);
+}
+
+int mmd_decompose(const void* W, bq_dtype dt, int N, int K, const int32_t* idx_host, int n_features, void* cuda_stream, mmd_weights** out) {
+    if (!out) return BQ_ERR_NULL;
+    *out = nullptr;
+    if (!is16(dt)) return BQ_ERR_DTYPE;
+    if (N < 1 || K < 16 || K % 16 != 0 || K > kMaxK) return BQ_ERR_SIZE;
+    const int fc = check_features(idx_host, n_features, K);
+    if (fc != BQ_OK) return fc;
+    if (!W) return BQ_ERR_NULL;
+    if (!aligned(W, 16)) return BQ_ERR_SIZE;
+    mmd_weights* w = new (std::nothrow) mmd_weights();
+    if (!w) return BQ_ERR_CUDA;
+    w->N = N; w->K = K; w->ko = n_features; w->side_cols = mmd_side_columns(n_features); w->dtype = dt;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaGetDevice(&w->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&w->sm_count, cudaDevAttrMultiProcessorCount, w->device);
+    const size_t o_q = 0;
+    const size_t o_scale = round_up(size_t(N) * K, kWsAlign);
+    const size_t o_side = o_scale + round_up(size_t(N) * 4, kWsAlign);
+    const size_t o_idx = o_side + round_up(size_t(N) * w->side_cols * 2, kWsAlign);
+    const size_t o_status = o_idx + round_up(size_t(kMaxFeatures) * 4, kWsAlign);
+    const size_t total = o_status + kWsAlign;
+    if (e == cudaSuccess) e = cudaMalloc(&w->blob, total);
+    if (e != cudaSuccess) { delete w; return cuda_fail(e); }
+    char* base = static_cast<char*>(w->blob);
+    w->q = reinterpret_cast<int8_t*>(base + o_q);
+    w->scale = reinterpret_cast<float*>(base + o_scale);
+    w->side = base + o_side;
+    w->idx = reinterpret_cast<int32_t*>(base + o_idx);
+    w->status = reinterpret_cast<int*>(base + o_status);
+    e = cudaMemsetAsync(w->status, 0, sizeof(int), stream);
+    // the feature list is copied from pageable host memory: the copy has left the host buffer when the call returns
+    if (e == cudaSuccess && n_features > 0) e = cudaMemcpyAsync(w->idx, idx_host, size_t(n_features) * 4, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = rowquant_any(dt, W, N, K, w->idx, n_features, w->q, w->scale, w->side, w->sm_count, stream);
+    if (e != cudaSuccess) { cudaFree(w->blob); delete w; return cuda_fail(e); }
+    w->have_maps = true;
+    const uint32_t boxes[3] = {256, 128, 64};
+    for (int s = 0; s < 3; ++s) {
+        w->have_maps = w->have_maps && make_map(&w->map_q[s], w->q, 1, uint64_t(N), uint64_t(K), boxes[s]);
+        if (w->side_cols > 0) w->have_maps = w->have_maps && make_map(&w->map_side[s], w->side, 2, uint64_t(N), uint64_t(w->side_cols), boxes[s]);
+    }
+    *out = w;
+    return BQ_OK;
+}
+
+int mmd_free(mmd_weights* w) {
+    if (!w) return BQ_OK;
+    const cudaError_t e = cudaFree(w->blob);
+    delete w;
+    return e == cudaSuccess ? BQ_OK : cuda_fail(e);
+}
+
+int mmd_weights_view(const mmd_weights* w, const int8_t** q, const float** scale, const void** side, const int32_t** idx, int* N, int* K,
+                     int* n_features, int* dtype) {
+    if (!w) return BQ_ERR_NULL;
+    if (q) *q = w->q;
+    if (scale) *scale = w->scale;
+    if (side) *side = w->side;
+    if (idx) *idx = w->idx;
+    if (N) *N = w->N;
+    if (K) *K = w->K;
+    if (n_features) *n_features = w->ko;
+    if (dtype) *dtype = w->dtype;
+    return BQ_OK;
+}
+
+int mmd_workspace_layout(const mmd_weights* w, int M, size_t* offsets3, size_t* total_bytes) {
+    if (!w || !total_bytes) return BQ_ERR_NULL;
+    if (M < 0) return BQ_ERR_SIZE;
+    const WsLayout L = ws_layout(w, M);
+    if (offsets3) { offsets3[0] = L.q; offsets3[1] = L.scale; offsets3[2] = L.side; }
+    *total_bytes = L.total;
+    return BQ_OK;
+}
+
+int mmd_linear(const mmd_weights* w, const void* X, int M, void* Y, bq_dtype ydt, void* workspace, size_t workspace_bytes, int path,
+               void* cuda_stream) {
+    if (!w) return BQ_ERR_NULL;
+    if (ydt != BQ_F32 && int(ydt) != w->dtype) return BQ_ERR_DTYPE;
+    if (M < 0) return BQ_ERR_SIZE;
+    if (path != MMD_PATH_AUTO && path != MMD_PATH_GENERAL && path != MMD_PATH_TENSOR) return MMD_ERR_PATH;
+    if (M == 0) return BQ_OK;
+    if (!X || !Y) return BQ_ERR_NULL;
+    if (!aligned(X, 16)) return BQ_ERR_SIZE;
+    const WsLayout L = ws_layout(w, M);
+    if (!workspace || !aligned(workspace, kWsAlign) || workspace_bytes < L.total) return MMD_ERR_WORKSPACE;
+    if (!on_device(w)) return BQ_ERR_CUDA;
+    const bool tc_ok = w->have_maps && (w->N % 8 == 0) && aligned(Y, 16);
+    if (path == MMD_PATH_TENSOR && !tc_ok) return MMD_ERR_PATH;
+    const bool use_tc = (path == MMD_PATH_TENSOR) || (path == MMD_PATH_AUTO && tc_ok);
+
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    char* ws = static_cast<char*>(workspace);
+    int8_t* qx = reinterpret_cast<int8_t*>(ws + L.q);
+    float* sx = reinterpret_cast<float*>(ws + L.scale);
+    void* sidex = ws + L.side;
+    cudaError_t e = rowquant_any(w->dtype, X, M, w->K, w->idx, w->ko, qx, sx, sidex, w->sm_count, stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+
+    const bool bf = (w->dtype == BQ_BF16), f32out = (ydt == BQ_F32);
+    if (use_tc) {
+        CUtensorMap mqx, msx;
+        if (!make_map(&mqx, qx, 1, uint64_t(M), uint64_t(w->K), 128)) return MMD_ERR_PATH;
+        if (w->side_cols > 0 && !make_map(&msx, sidex, 2, uint64_t(M), uint64_t(w->side_cols), 128)) return MMD_ERR_PATH;
+        if (w->side_cols == 0) msx = mqx;
+        if (bf) e = f32out ? launch_tc_bn<mmdk::kBF16, mmdk::kF32>(w, mqx, msx, sx, Y, M, stream) : launch_tc_bn<mmdk::kBF16, mmdk::kBF16>(w, mqx, msx, sx, Y, M, stream);
+        else e = f32out ? launch_tc_bn<mmdk::kF16, mmdk::kF32>(w, mqx, msx, sx, Y, M, stream) : launch_tc_bn<mmdk::kF16, mmdk::kF16>(w, mqx, msx, sx, Y, M, stream);
+    } else {
+        if (bf) e = f32out ? launch_general<mmdk::kBF16, mmdk::kF32>(w, qx, sx, sidex, Y, M, stream) : launch_general<mmdk::kBF16, mmdk::kBF16>(w, qx, sx, sidex, Y, M, stream);
+        else e = f32out ? launch_general<mmdk::kF16, mmdk::kF32>(w, qx, sx, sidex, Y, M, stream) : launch_general<mmdk::kF16, mmdk::kF16>(w, qx, sx, sidex, Y, M, stream);
+    }
+    return e == cudaSuccess ? BQ_OK : cuda_fail(e);
+}
+
+int mmd_kernel_status(const mmd_weights* w, int* status_out) {
+    if (!w || !status_out) return BQ_ERR_NULL;
+    if (!on_device(w)) return BQ_ERR_CUDA;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(status_out, w->status, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess && *status_out != 0) e = cudaMemset(w->status, 0, sizeof(int));
+    return e == cudaSuccess ? BQ_OK : cuda_fail(e);
+}
+
+}  // extern "C"

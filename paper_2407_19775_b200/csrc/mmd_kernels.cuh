@@ -1,0 +1,456 @@
+// mmd_kernels.cuh -- device code of the mixed matrix decomposition (sm_100a).
+//
+//   rowquant      : per row absmax over the regular features, int8 codes, row scale and the
+//                   16-bit side columns of the critical features.  One CTA per row.
+//   gemm_general  : Y = fma(fp32(qx qw^T), sx sw, sidex sidew^T) with integer dot products
+//                   (dp4a) for any M and N; the correctness path and the fallback.
+//   gemm_tc       : the same on the 5th-generation tensor cores: TMA loads 128-byte-swizzled
+//                   tiles into a 4-stage shared-memory ring, one thread issues tcgen05.mma
+//                   (kind::i8 into an int32 accumulator in tensor memory, then kind::f16 for
+//                   the side columns into a second, fp32 accumulator), four warps read both
+//                   accumulators back with tcgen05.ld and apply the scales.
+//
+// Arithmetic contract (it is what makes the integer part bit-identical to the plain
+// definition): 127 v is exact in fp32 for 16-bit v; one IEEE division; cvt.rni (ties to
+// even); int32 sums are exact; the output is one fma and one round-to-nearest-even narrowing.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mmdk {
+
+enum { kF32 = 0, kF16 = 1, kBF16 = 2 };
+
+constexpr int kSidePad = 64;
+
+template <int DT>
+__device__ __forceinline__ float widen16(uint32_t bits16) {
+    if constexpr (DT == kBF16) return __uint_as_float(bits16 << 16);
+    else return __half2float(__ushort_as_half(static_cast<unsigned short>(bits16)));
+}
+
+template <int DT>
+__device__ __forceinline__ void widen8(const uint4& w, float (&f)[8]) {
+    const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        f[2 * i] = widen16<DT>(u[i] & 0xffffu);
+        f[2 * i + 1] = widen16<DT>(u[i] >> 16);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// rowquant: one CTA of 256 threads per row.  A bit mask of the critical features sits in
+// shared memory, one byte per 16-byte chunk of the row, so the regular path costs one byte
+// load per eight elements.  The row is read twice (the second pass hits L1 / L2).
+template <int DT>
+__global__ void __launch_bounds__(256)
+rowquant(const void* __restrict__ v, int R, int K, const int32_t* __restrict__ idx, int ko, int side_cols,
+         int8_t* __restrict__ q_out, float* __restrict__ scale_out, void* __restrict__ side_out) {
+    extern __shared__ __align__(16) unsigned char mask[];       // K / 8 bytes
+    __shared__ float red[8];
+    const int nchunks = K / 8;
+    for (int c = threadIdx.x; c < (nchunks + 3) / 4; c += 256) reinterpret_cast<uint32_t*>(mask)[c] = 0u;
+    __syncthreads();
+    for (int j = threadIdx.x; j < ko; j += 256) {
+        const int k = idx[j];
+        atomicOr(reinterpret_cast<uint32_t*>(mask) + (k >> 5), 1u << (k & 31));
+    }
+    __syncthreads();
+
+    for (int r = blockIdx.x; r < R; r += gridDim.x) {
+        const uint4* row = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(v) + size_t(r) * K);
+        float a = 0.0f;
+        for (int c = threadIdx.x; c < nchunks; c += 256) {
+            const uint4 w = row[c];
+            const uint32_t mk = mask[c];
+            float f[8];
+            widen8<DT>(w, f);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) a = fmaxf(a, ((mk >> i) & 1u) ? 0.0f : fabsf(f[i]));
+        }
+#pragma unroll
+        for (int s = 16; s >= 1; s >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, s));
+        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = a;
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < 8; ++i) a = fmaxf(a, red[i]);
+        const float d = (a != 0.0f) ? a : 1.0f;
+        if (threadIdx.x == 0) scale_out[r] = __fdiv_rn(a, 127.0f);
+
+        uint2* qrow = reinterpret_cast<uint2*>(q_out + size_t(r) * K);
+        for (int c = threadIdx.x; c < nchunks; c += 256) {
+            const uint4 w = row[c];
+            const uint32_t mk = mask[c];
+            float f[8];
+            widen8<DT>(w, f);
+            uint32_t b[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int qi = __float2int_rn(__fdiv_rn(__fmul_rn(f[i], 127.0f), d));
+                b[i] = ((mk >> i) & 1u) ? 0u : (uint32_t(qi) & 0xffu);
+            }
+            qrow[c] = make_uint2(b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24), b[4] | (b[5] << 8) | (b[6] << 16) | (b[7] << 24));
+        }
+        uint16_t* srow = static_cast<uint16_t*>(side_out) + size_t(r) * side_cols;
+        const uint16_t* vrow = static_cast<const uint16_t*>(v) + size_t(r) * K;
+        for (int j = threadIdx.x; j < side_cols; j += 256) srow[j] = (j < ko) ? vrow[idx[j]] : uint16_t(0);
+        __syncthreads();                                         // red[] is reused by the next row
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// output of one element: the single fma of the definition and the narrowing
+template <int YDT>
+__device__ __forceinline__ void store_y(void* y, size_t i, float v) {
+    if constexpr (YDT == kF32) static_cast<float*>(y)[i] = v;
+    else if constexpr (YDT == kBF16) static_cast<__nv_bfloat16*>(y)[i] = __float2bfloat16_rn(v);
+    else static_cast<__half*>(y)[i] = __float2half_rn(v);
+}
+
+// ------------------------------------------------------------------------------------------
+// gemm_general: 64 x 64 outputs per CTA of 256 threads, 4 x 4 per thread (rows ty + 16 i,
+// columns tx + 16 j), 64 features per step through shared memory, four int8 products per dp4a.
+template <int XDT, int YDT>
+__global__ void __launch_bounds__(256)
+gemm_general(const int8_t* __restrict__ qx, const int8_t* __restrict__ qw, const float* __restrict__ sx, const float* __restrict__ sw,
+             const void* __restrict__ sidex, const void* __restrict__ sidew, int side_cols, void* __restrict__ y, int M, int N, int K) {
+    __shared__ uint32_t xs[64][17];
+    __shared__ uint32_t ws[64][17];
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+    int acc[4][4];
+    float part[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { acc[i][j] = 0; part[i][j] = 0.0f; }
+
+    const int lr = threadIdx.x >> 2, lc = threadIdx.x & 3;       // this thread's 16-byte piece of the 64 x 64-byte tiles
+    for (int k0 = 0; k0 < K; k0 += 64) {
+        uint4 a = make_uint4(0, 0, 0, 0), b = make_uint4(0, 0, 0, 0);
+        const int kk = k0 + lc * 16;
+        if (kk < K) {
+            if (m0 + lr < M) a = *reinterpret_cast<const uint4*>(qx + size_t(m0 + lr) * K + kk);
+            if (n0 + lr < N) b = *reinterpret_cast<const uint4*>(qw + size_t(n0 + lr) * K + kk);
+        }
+        __syncthreads();
+        xs[lr][lc * 4 + 0] = a.x; xs[lr][lc * 4 + 1] = a.y; xs[lr][lc * 4 + 2] = a.z; xs[lr][lc * 4 + 3] = a.w;
+        ws[lr][lc * 4 + 0] = b.x; ws[lr][lc * 4 + 1] = b.y; ws[lr][lc * 4 + 2] = b.z; ws[lr][lc * 4 + 3] = b.w;
+        __syncthreads();
+#pragma unroll
+        for (int kw = 0; kw < 16; ++kw) {
+            int av[4], bv[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { av[i] = int(xs[ty + 16 * i][kw]); bv[i] = int(ws[tx + 16 * i][kw]); }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = __dp4a(av[i], bv[j], acc[i][j]);
+        }
+    }
+    // side columns: 16 per step, widened to fp32 in shared memory
+    float* xf = reinterpret_cast<float*>(&xs[0][0]);
+    float* wf = reinterpret_cast<float*>(&ws[0][0]);
+    for (int k0 = 0; k0 < side_cols; k0 += 16) {
+        __syncthreads();
+        {
+            const int row = threadIdx.x >> 2, c4 = (threadIdx.x & 3) * 4;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int col = k0 + c4 + e;
+                float xv = 0.0f, wv = 0.0f;
+                if (m0 + row < M) xv = mmdk::widen16<XDT>(static_cast<const uint16_t*>(sidex)[size_t(m0 + row) * side_cols + col]);
+                if (n0 + row < N) wv = mmdk::widen16<XDT>(static_cast<const uint16_t*>(sidew)[size_t(n0 + row) * side_cols + col]);
+                xf[row * 17 + c4 + e] = xv;
+                wf[row * 17 + c4 + e] = wv;
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            float av[4], bv[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { av[i] = xf[(ty + 16 * i) * 17 + k]; bv[i] = wf[(tx + 16 * i) * 17 + k]; }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) part[i][j] = __fmaf_rn(av[i], bv[j], part[i][j]);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int m = m0 + ty + 16 * i;
+        if (m >= M) continue;
+        const float sxm = sx[m];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int n = n0 + tx + 16 * j;
+            if (n >= N) continue;
+            const float s = __fmul_rn(sxm, sw[n]);
+            store_y<YDT>(y, size_t(m) * N + n, __fmaf_rn(float(acc[i][j]), s, part[i][j]));
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// gemm_tc: tensor-core kernel.
+//
+// One CTA computes a 128 x BN tile of Y.  192 threads: warp 0 issues the TMA loads, warp 1
+// allocates tensor memory and issues the MMAs, warps 2-5 are the epilogue (warp w reads the
+// 32 accumulator lanes of its quarter, w % 4).  A stage of the ring holds a 128-row tile of
+// the activations and a BN-row tile of the weights, each row 128 bytes (128 int8 features,
+// or 64 side columns of 16 bits), written by TMA with the 128-byte swizzle that the MMA's
+// shared-memory descriptors name.  The int8 steps accumulate into columns [0, BN) of tensor
+// memory as int32; the side steps into columns [BN, 2 BN) as fp32.
+//
+// Every wait is bounded: a wait that runs out records a code in *status, raises the CTA's
+// abort flag and the kernel winds down (no further stores, tensor memory freed).
+
+constexpr int kTcThreads = 192;
+constexpr int kTcBM = 128;
+constexpr int kTcRowBytes = 128;
+constexpr long long kWaitLimitCycles = 4000000000ll;            // about two seconds
+
+template <int BN> struct TcCfg {
+    static constexpr int kStages = (BN >= 256) ? 4 : (BN >= 128 ? 6 : 8);
+    static constexpr uint32_t kABytes = kTcBM * kTcRowBytes;
+    static constexpr uint32_t kBBytes = BN * kTcRowBytes;
+    static constexpr uint32_t kStageBytes = kABytes + kBBytes;
+    static constexpr uint32_t kTmemCols = (2 * BN <= 32) ? 32 : 2 * BN;          // a power of two >= 32
+    static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 2048 /* barriers, scales */;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return uint32_t(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the limit ran out or another thread of the CTA gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try(bar, parity)) return true;
+        if ((it & 255u) == 0u) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > kWaitLimitCycles) {
+                *abort_flag = 1;
+                atomicCAS(status, 0, code);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+// K-major operand tile with 128-byte rows and the 128-byte swizzle: 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t addr) {
+    return uint64_t((addr & 0x3FFFFu) >> 4) | (uint64_t(1) << 16) | (uint64_t(1024 >> 4) << 32) | (uint64_t(1) << 46) | (uint64_t(2) << 61);
+}
+// instruction descriptor: D format (1 = fp32, 2 = int32), A / B format, both K-major, N / 8, M / 16
+__host__ __device__ constexpr uint32_t umma_idesc(uint32_t dfmt, uint32_t abfmt, uint32_t M, uint32_t N) {
+    return (dfmt << 4) | (abfmt << 7) | (abfmt << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+
+template <int XDT, int YDT, int BN>
+__global__ void __launch_bounds__(kTcThreads, 1)
+gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUtensorMap map_qw,
+        const __grid_constant__ CUtensorMap map_sidex, const __grid_constant__ CUtensorMap map_sidew,
+        const float* __restrict__ sx, const float* __restrict__ sw, void* __restrict__ y,
+        int M, int N, int kblocks /* int8 steps of 128 features */, int sblocks /* side steps of 64 columns */, int* status) {
+    using Cfg = TcCfg<BN>;
+    constexpr int S = Cfg::kStages;
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;               // swizzled tiles need 1024-byte alignment
+    unsigned char* ctrl = smem_raw + (tiles - smem_u32(smem_raw)) + S * Cfg::kStageBytes;
+    const uint32_t full0 = smem_u32(ctrl);                                      // S barriers: tile landed
+    const uint32_t empty0 = full0 + 8u * S;                                     // S barriers: tile consumed
+    const uint32_t accbar = empty0 + 8u * S;                                    // accumulators complete
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl + 8 * (2 * S + 1));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 8 * (2 * S + 1) + 8);
+    float* sw_s = reinterpret_cast<float*>(ctrl + 256);                         // BN scales of this tile's columns
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.x * kTcBM, n0 = blockIdx.y * BN;
+    const int steps = kblocks + sblocks;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, 1); }
+        mbar_init(accbar, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(Cfg::kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int i = 0; i < steps; ++i) {
+                const int s = i % S;
+                const uint32_t round = uint32_t(i / S);
+                if (!mbar_wait(empty0 + 8u * s, (round & 1u) ^ 1u, abort_flag, status, 1)) break;
+                const uint32_t a_dst = tiles + uint32_t(s) * Cfg::kStageBytes, b_dst = a_dst + Cfg::kABytes;
+                mbar_expect_tx(full0 + 8u * s, Cfg::kStageBytes);
+                if (i < kblocks) {
+                    tma_load_2d(a_dst, &map_qx, i * 128, m0, full0 + 8u * s);
+                    tma_load_2d(b_dst, &map_qw, i * 128, n0, full0 + 8u * s);
+                } else {
+                    tma_load_2d(a_dst, &map_sidex, (i - kblocks) * 64, m0, full0 + 8u * s);
+                    tma_load_2d(b_dst, &map_sidew, (i - kblocks) * 64, n0, full0 + 8u * s);
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc_i8 = umma_idesc(2, 1, kTcBM, BN);                   // int32 <- int8 x int8
+            constexpr uint32_t idesc_16 = umma_idesc(1, XDT == kBF16 ? 1u : 0u, kTcBM, BN);     // fp32 <- 16-bit x 16-bit
+            bool ok = true;
+            for (int i = 0; i < steps && ok; ++i) {
+                const int s = i % S;
+                const uint32_t round = uint32_t(i / S);
+                ok = mbar_wait(full0 + 8u * s, round & 1u, abort_flag, status, 2);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t a_src = tiles + uint32_t(s) * Cfg::kStageBytes, b_src = a_src + Cfg::kABytes;
+                const uint64_t adesc = umma_smem_desc(a_src), bdesc = umma_smem_desc(b_src);
+                if (i < kblocks) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)                       // 32 int8 features = 32 bytes per MMA
+                        umma_i8(tmem, adesc + uint64_t(2 * k), bdesc + uint64_t(2 * k), idesc_i8, (i > 0 || k > 0) ? 1u : 0u);
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)                       // 16 side columns = 32 bytes per MMA
+                        umma_f16(tmem + uint32_t(BN), adesc + uint64_t(2 * k), bdesc + uint64_t(2 * k), idesc_16, (i > kblocks || k > 0) ? 1u : 0u);
+                }
+                umma_commit(empty0 + 8u * s);                         // the stage is free once these MMAs have read it
+            }
+            if (ok) umma_commit(accbar);
+        }
+        __syncwarp();
+    } else {
+        // epilogue: 128 threads, one accumulator row each
+        const int et = threadIdx.x - 64;
+        for (int c = et; c < BN; c += 128) sw_s[c] = (n0 + c < N) ? sw[n0 + c] : 0.0f;
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        const int quarter = warp & 3;
+        const int m = m0 + quarter * 32 + lane;
+        const float sxm = (m < M) ? sx[m] : 0.0f;
+        bool ok = true;
+        if (lane == 0) ok = mbar_wait(accbar, 0, abort_flag, status, 3);
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (ok) {
+            const uint32_t lane_base = tmem + (uint32_t(quarter * 32) << 16);
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t ai[32], af[32];
+                tmem_ld32(lane_base + uint32_t(c0), ai);
+                if (sblocks > 0) tmem_ld32(lane_base + uint32_t(BN + c0), af);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                float out[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const float s = __fmul_rn(sxm, sw_s[c0 + j]);
+                    const float p = (sblocks > 0) ? __uint_as_float(af[j]) : 0.0f;
+                    out[j] = __fmaf_rn(float(int(ai[j])), s, p);
+                }
+                if (m < M) {
+                    const int n = n0 + c0;
+                    if constexpr (YDT == kF32) {
+                        float* dst = static_cast<float*>(y) + size_t(m) * N + n;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            if (n + j < N) *reinterpret_cast<float4*>(dst + j) = make_float4(out[j], out[j + 1], out[j + 2], out[j + 3]);
+                    } else {
+                        uint16_t* dst = static_cast<uint16_t*>(y) + size_t(m) * N + n;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8) {
+                            uint32_t pk[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                if constexpr (YDT == kBF16) {
+                                    const __nv_bfloat162 h = __floats2bfloat162_rn(out[j + 2 * e], out[j + 2 * e + 1]);
+                                    pk[e] = *reinterpret_cast<const uint32_t*>(&h);
+                                } else {
+                                    const __half2 h = __floats2half2_rn(out[j + 2 * e], out[j + 2 * e + 1]);
+                                    pk[e] = *reinterpret_cast<const uint32_t*>(&h);
+                                }
+                            }
+                            if (n + j < N) *reinterpret_cast<uint4*>(dst + j) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        }
+                    }
+                }
+            }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    }
+
+    __syncthreads();
+    if (*abort_flag) {
+        // copies that were issued but never waited for may still be landing in this CTA's
+        // shared memory: give them time before the memory is handed to another CTA
+        for (int i = 0; i < 64; ++i) __nanosleep(2000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(Cfg::kTmemCols) : "memory");
+    }
+}
+
+}  // namespace mmdk

@@ -1,4 +1,4 @@
-"""The C-ABI library loads and exports every function include/bq.h declares; argument
+"""The C-ABI library loads and exports every function include/*.h declares; argument
 errors come back as status codes before anything touches a device (CPU only)."""
 import ctypes
 import os
@@ -9,10 +9,10 @@ import pytest
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
-def _declared():
-    text = open(os.path.join(ROOT, "include", "bq.h")).read()
+def _declared(header="bq.h", prefix="bq_"):
+    text = open(os.path.join(ROOT, "include", header)).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(bq_[a-z_0-9]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(" + prefix + r"[a-z_0-9]+)\s*\(", text)))
 
 
 def test_every_declared_symbol_is_exported(bq):
@@ -23,6 +23,46 @@ def test_every_declared_symbol_is_exported(bq):
     for name in names:
         assert hasattr(L, name), name
     assert set(binding.SYMBOLS) == set(names)
+
+
+def test_every_header_is_covered():
+    assert sorted(os.listdir(os.path.join(ROOT, "include"))) == ["bq.h", "mmd.h"]
+
+
+def test_every_declared_mmd_symbol_is_exported(bq):
+    from paper_2407_19775_b200 import binding, mmd
+    L = binding.lib()
+    names = _declared("mmd.h", "mmd_")
+    assert {"mmd_rowquant", "mmd_decompose", "mmd_linear", "mmd_free"} <= set(names)
+    for name in names:
+        assert hasattr(L, name), name
+    assert set(mmd.SYMBOLS) == set(names)
+
+
+def test_mmd_argument_errors_need_no_device(bq):
+    import numpy as np
+    from paper_2407_19775_b200 import mmd
+    L = mmd._lib()
+    one = ctypes.c_void_p(256)       # never dereferenced: every call below fails a check first
+    assert L.mmd_rowquant(one, 0, 4, 64, None, 0, one, one, None, None) == 2          # fp32 rows are not taken
+    assert L.mmd_rowquant(one, 2, 4, 40, None, 0, one, one, None, None) == 4          # K not a multiple of 16
+    assert L.mmd_rowquant(one, 2, 4, 64, None, 2000, one, one, None, None) == 8       # too many features
+    assert L.mmd_rowquant(one, 2, 0, 64, None, 0, None, None, None, None) == 0        # no rows: nothing to do
+    assert L.mmd_rowquant(None, 2, 4, 64, None, 0, one, one, None, None) == 1
+    assert L.mmd_rowquant(ctypes.c_void_p(8), 2, 4, 64, None, 0, one, one, None, None) == 4   # misaligned rows
+    out = ctypes.c_void_p()
+    bad = np.array([5, 3], np.int32)
+    assert L.mmd_decompose(one, 2, 8, 64, bad.ctypes.data, 2, None, ctypes.byref(out)) == 8   # not ascending
+    far = np.array([3, 64], np.int32)
+    assert L.mmd_decompose(one, 2, 8, 64, far.ctypes.data, 2, None, ctypes.byref(out)) == 8   # out of range
+    assert L.mmd_decompose(one, 2, 8, 64, None, 1, None, ctypes.byref(out)) == 1
+    assert L.mmd_decompose(one, 2, 0, 64, None, 0, None, ctypes.byref(out)) == 4
+    assert L.mmd_decompose(one, 2, 8, 64, None, 0, None, None) == 1
+    assert L.mmd_linear(None, one, 4, one, 0, one, 1 << 20, 0, None) == 1
+    assert L.mmd_free(None) == 0
+    assert [L.mmd_side_columns(k) for k in (0, 1, 64, 65)] == [0, 64, 64, 128]
+    for code in (7, 8, 9):
+        assert L.bq_status_string(code) not in (b"unknown status", b"ok")
 
 
 def test_status_strings(bq):

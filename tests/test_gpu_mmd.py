@@ -1,0 +1,188 @@
+"""GPU parity of the mixed matrix decomposition against the CPU oracle, through the C ABI.
+
+Bar: the int8 codes, row scales and side columns are bit-exact; the layer's output is
+bit-exact when there are no critical features (integer sums are exact and the output is one
+fp32 product); with critical features the fp32 side sum is accumulated on the GPU in an
+unspecified order, so the output is compared within
+    tol = 2^-23 |y| + (side columns + 2) 2^-22 sum_j |x_j w_j|
+(one rounding of the result plus one rounding per accumulated product, with a factor 4 for
+tensor-core accumulation that may truncate), and 16-bit outputs must lie between the
+narrowings of y - tol and y + tol.
+"""
+import zlib
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import mmd_oracle as mo
+from paper_2407_19775_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+F32, F16, BF16 = 0, 1, 2
+DT = {torch.float16: F16, torch.bfloat16: BF16}
+
+
+def bits(t: torch.Tensor) -> np.ndarray:
+    return workloads.bits_2d(t.cpu())
+
+
+def as_f32(a: np.ndarray, dt: int) -> np.ndarray:
+    return a if dt == F32 else mo.widen(a, dt)
+
+
+def y_bits(y: torch.Tensor) -> np.ndarray:
+    return y.cpu().numpy() if y.dtype == torch.float32 else bits(y)
+
+
+def check_output(y_gpu: torch.Tensor, X, W, idx, dt, exact_expected: bool):
+    qw, sw, wo = mo.rowquant(bits(W), dt, idx)
+    ydt = F32 if y_gpu.dtype == torch.float32 else dt
+    y_ref, acc, side, sabs = mo.linear(bits(X), dt, qw, sw, wo, idx, ydt, parts=True)
+    got = y_bits(y_gpu)
+    if exact_expected:
+        assert np.array_equal(got.view(np.uint32 if ydt == F32 else np.uint16), y_ref.view(np.uint32 if ydt == F32 else np.uint16))
+        return
+    y32 = mo.linear(bits(X), dt, qw, sw, wo, idx, F32).astype(np.float64)
+    tol = 2.0 ** -23 * np.abs(y32) + (wo.shape[1] + 2) * 2.0 ** -22 * sabs
+    if ydt == F32:
+        assert np.all(np.abs(got.astype(np.float64) - y32) <= tol)
+    else:
+        lo = as_f32(mo.narrow((y32 - tol).astype(np.float32), ydt), ydt)
+        hi = as_f32(mo.narrow((y32 + tol).astype(np.float32), ydt), ydt)
+        g = as_f32(got, ydt)
+        assert np.all((g >= lo) & (g <= hi))
+        assert np.mean(got == y_ref) > 0.99                      # and nearly all are the oracle's own bits
+
+
+@pytest.mark.parametrize("tdt", [torch.bfloat16, torch.float16])
+def test_rowquant_bit_exact(bq, tdt):
+    dt = DT[tdt]
+    g = torch.Generator().manual_seed(21)
+    R, K = 75, 1040                                               # ragged: 130 chunks over 256 threads
+    v = (torch.randn(R, K, generator=g) * 1.3).to(tdt)
+    idx = np.array([0, 7, 8, 500, 1039], np.int32)
+    v[:, idx.tolist()] *= 25
+    v[3] = 0                                                      # zero row
+    v[4, :] = 0; v[4, 7] = 3.0                                    # only a critical feature is non-zero
+    v[5, 11] = -v[5].abs().max() * 2                              # the absmax element is negative
+    v[6, :16] = torch.tensor([127.0 / 64] + [h / 64 for h in (0.5, 1.5, 2.5, -4.5, -5.5, 100.5, -126.5)] + [0.0] * 8).to(tdt)
+    v[6, 16:] = 0; v[6, idx.tolist()] = 9.0                       # exact ties in the regular part
+    if tdt == torch.float16:
+        v[7] = v[7] * 1e-6                                        # fp16 subnormals
+    q_ref, s_ref, side_ref = mo.rowquant(bits(v), dt, idx)
+    q, s, side = bq.mmd_rowquant(v.cuda(), torch.from_numpy(idx).cuda())
+    torch.cuda.synchronize()
+    assert np.array_equal(q.cpu().numpy(), q_ref)
+    assert np.array_equal(s.cpu().numpy().view(np.uint32), s_ref.view(np.uint32))
+    assert np.array_equal(bits(side), side_ref)
+    q0, s0, side0 = bq.mmd_rowquant(v.cuda(), None)
+    q0_ref, s0_ref, _ = mo.rowquant(bits(v), dt, np.zeros(0, np.int32))
+    assert np.array_equal(q0.cpu().numpy(), q0_ref) and np.array_equal(s0.cpu().numpy(), s0_ref) and side0.shape == (R, 0)
+
+
+def test_rowquant_division_cases(bq):
+    """Pairs on which a multiplication by the reciprocal would land on another integer."""
+    vals = (np.arange(0x3C00, 0x4300, dtype=np.uint32) << 16).view(np.float32)
+    rows = []
+    for d in vals[::5]:
+        scaled = vals * np.float32(127)
+        differ = (np.rint(scaled / d) != np.rint(scaled * (np.float32(1) / d))) & (vals <= d)
+        rows += [(float(x), float(d)) for x in vals[differ][:3]]
+    assert len(rows) > 40
+    v = torch.zeros(len(rows), 16)
+    for r, (x, d) in enumerate(rows):
+        v[r, 0], v[r, 1], v[r, 2] = d, x, -x
+    v = v.to(torch.bfloat16)
+    q_ref, _, _ = mo.rowquant(bits(v), BF16, np.zeros(0, np.int32))
+    q, _, _ = bq.mmd_rowquant(v.cuda(), None)
+    assert np.array_equal(q.cpu().numpy(), q_ref)
+
+
+def test_decompose_matches_oracle(bq):
+    X, W, idx = workloads.make_linear("mmd_tiny")
+    lin = bq.DecomposedLinear(W.cuda(), idx)
+    q, s, side, didx = lin.view()
+    torch.cuda.synchronize()
+    q_ref, s_ref, side_ref = mo.rowquant(bits(W), BF16, idx)
+    assert np.array_equal(q.cpu().numpy(), q_ref)
+    assert np.array_equal(s.cpu().numpy().view(np.uint32), s_ref.view(np.uint32))
+    assert np.array_equal(bits(side), side_ref)
+    assert np.array_equal(didx.cpu().numpy(), idx)
+    lin.close()
+
+
+@pytest.mark.parametrize("path", [1, 2])                           # general, tensor
+@pytest.mark.parametrize("out", ["f32", "same"])
+def test_linear_tiny(bq, path, out):
+    X, W, idx = workloads.make_linear("mmd_tiny")                 # M = 37, K = 320, N = 72: ragged in every direction
+    lin = bq.DecomposedLinear(W.cuda(), idx)
+    y = lin.linear(X.cuda(), torch.float32 if out == "f32" else None, path=path)
+    assert lin.kernel_status() == 0
+    check_output(y, X, W, idx, BF16, exact_expected=False)
+    qx, sx, sd = lin.workspace_parts(X.shape[0])
+    q_ref, s_ref, side_ref = mo.rowquant(bits(X), BF16, idx)
+    assert np.array_equal(qx.cpu().numpy(), q_ref) and np.array_equal(sx.cpu().numpy(), s_ref) and np.array_equal(bits(sd), side_ref)
+    # no critical features: bit-exact
+    lin0 = bq.DecomposedLinear(W.cuda(), np.zeros(0, np.int32))
+    y0 = lin0.linear(X.cuda(), torch.float32 if out == "f32" else None, path=path)
+    assert lin0.kernel_status() == 0
+    check_output(y0, X, W, np.zeros(0, np.int32), BF16, exact_expected=True)
+
+
+# shapes chosen so that each tile width of the tensor-core kernel is taken (the width is picked
+# from the number of tiles against the SM count), with ragged last tiles in M, N and K
+TC_SHAPES = [
+    ("bn64", 300, 400, 520, torch.bfloat16, 5),
+    ("bn64_fp16", 129, 144, 72, torch.float16, 2),
+    ("bn128", 1300, 272, 2056, torch.bfloat16, 70),              # 11 x 17 tiles of 128; two side steps
+    ("bn256", 1300, 400, 4104, torch.float16, 3),                # 11 x 17 tiles of 256
+    ("one_row", 1, 128, 8, torch.bfloat16, 1),
+]
+
+
+@pytest.mark.parametrize("name,M,K,N,tdt,ko", TC_SHAPES, ids=[s[0] for s in TC_SHAPES])
+def test_linear_tensor_path(bq, name, M, K, N, tdt, ko):
+    dt = DT[tdt]
+    g = torch.Generator().manual_seed(zlib.crc32(name.encode()) % 1000)
+    X = (torch.randn(M, K, generator=g) * 0.7).to(tdt)
+    W = (torch.randn(N, K, generator=g) * 0.05).to(tdt)
+    idx = np.sort(torch.randperm(K, generator=g)[:ko].numpy()).astype(np.int32)
+    X[:, idx.tolist()] *= 30
+    for features, exact in ((idx, False), (np.zeros(0, np.int32), True)):
+        lin = bq.DecomposedLinear(W.cuda(), features)
+        for out in (torch.float32, None):
+            y = lin.linear(X.cuda(), out, path=2)
+            assert lin.kernel_status() == 0
+            check_output(y, X, W, features, dt, exact_expected=exact)
+        yg = lin.linear(X.cuda(), torch.float32, path=1)
+        if exact:
+            assert torch.equal(yg, lin.linear(X.cuda(), torch.float32, path=2))
+        lin.close()
+
+
+def test_linear_integer_part_saturating_inputs(bq):
+    """Every code at +-127 over a long row: sums far above 2^24 must come back exactly."""
+    M, K, N = 130, 4096, 264
+    X = torch.full((M, K), 2.0).to(torch.bfloat16)
+    W = torch.full((N, K), -0.5).to(torch.bfloat16)
+    W[::2] *= -1
+    none = np.zeros(0, np.int32)
+    lin = bq.DecomposedLinear(W.cuda(), none)
+    for path in (1, 2):
+        y = lin.linear(X.cuda(), torch.float32, path=path)
+        assert lin.kernel_status() == 0
+        check_output(y, X, W, none, BF16, exact_expected=True)
+        assert torch.allclose(y.cpu(), torch.tensor([4096.0, -4096.0]).repeat(N // 2).expand(M, N), rtol=1e-6)
+
+
+def test_decode_workload_rows(bq):
+    """The decode workload (fp16, K = 8192, 8 critical features) on a slice of the weights."""
+    X, W, idx = workloads.make_linear("mmd_decode70b", out_features=1024)
+    lin = bq.DecomposedLinear(W.cuda(), idx)
+    for path in (1, 2):
+        y = lin.linear(X.cuda(), torch.float32, path=path)
+        assert lin.kernel_status() == 0
+        check_output(y, X, W, idx, F16, exact_expected=False)
+    y16 = lin.linear(X.cuda(), None)
+    check_output(y16, X, W, idx, F16, exact_expected=False)
