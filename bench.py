@@ -252,6 +252,9 @@ def run_ours(args):
         quality[f"b{b}"] = {"compression_ratio": round(2 * b / (b + 4), 3), "rel_rms_error": round(float((num / den).sqrt().item()), 5)}
 
     cpu = cpu_baseline(x_pin, rank) if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
+    del x, y, codes, absmax
+    torch.cuda.empty_cache()
+    mmd = run_mmd(bq, dev, args) if (rank == 0 and not args.no_mmd) else None
 
     if rank == 0:
         line = {
@@ -262,13 +265,114 @@ def run_ours(args):
                                    "quantize+dequantize+roundtrip per block", "elements": n, "l2": "input (1 GiB) larger than L2, no flush needed",
                        "parallelism": f"replicated x{world}, no collective"},
             "e2e": e2e, "gpu_launches": len(events), "clocks": clocks, "roofline": roofline, "kernels": kernels,
-            "quality": quality, "cpu_baseline": cpu,
+            "quality": quality, "cpu_baseline": cpu, "mmd": mmd,
             "paper_context": "the paper reports no throughput for this path; it states only that hidden-state quantization halves the bandwidth",
         }
         print(json.dumps(line))
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------ the decomposed linear layer
+
+MMD_WORKLOAD = "mmd_prefill_moe"
+NOMINAL_INT8_OVER_BF16 = 2.0          # dense int8 (4.5 POP/s) over dense bf16 (2.25 PFLOP/s)
+FALLBACK_BF16_TFLOPS = 1590.0
+MMD_TRAFFIC_BYTES = None              # dram bytes per full-size product launch; None until an ncu capture of this kernel is scaled
+
+
+def measured_tensor_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured"
+    except Exception:
+        return FALLBACK_BF16_TFLOPS, "fallback"
+
+
+def run_mmd(bq, dev, args):
+    """The paper's second compression technique on one layer of the MoE-class prefill shape:
+    weights decomposed once, then timed calls of the layer (row kernel over the activations +
+    tensor-core product).  Reported beside the main metric with its own roofline."""
+    import oracle.mmd_oracle as mo
+    wl = workloads.LINEAR_WORKLOADS[MMD_WORKLOAD]
+    X, W, idx = workloads.make_linear(MMD_WORKLOAD)
+    M, K, N = X.shape[0], X.shape[1], W.shape[0]
+    x_pin, Xd, Wd = X.pin_memory(), X.to(dev), W.to(dev)
+    lin = bq.DecomposedLinear(Wd, idx)
+    y = torch.empty((M, N), dtype=wl.dtype, device=dev)
+    ws = lin.workspace(M)
+    idx_d = torch.from_numpy(idx).to(dev)
+    reps = max(3, min(args.steps, 50))
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        ev = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            ev.append((e0, e1))
+        torch.cuda.synchronize()
+        return float(np.mean([a.elapsed_time(b) for a, b in ev]))
+
+    qx, sx, sd = lin.workspace_parts(M, ws)
+    ms_call = timed(lambda: lin.linear(Xd, y_out=y, workspace=ws))
+    status = lin.kernel_status()
+    ms_row = timed(lambda: bq.mmd.rowquant_into(Xd, idx_d, qx, sx, sd))
+    ms_prod = ms_call - ms_row
+    ops = 2.0 * M * N * K
+    bf16, kind = measured_tensor_peak()
+    peak = bf16 * NOMINAL_INT8_OVER_BF16
+    hbm, _ = measured_peak()
+    row_bytes = M * K * 3 + M * 4 + M * sd.shape[1] * 2
+
+    # end to end: activations from pinned host memory, the result back to pinned host memory
+    y_pin = torch.empty((M, N), dtype=wl.dtype).pin_memory()
+    x_dev = torch.empty_like(Xd)
+
+    def e2e_call():
+        x_dev.copy_(x_pin, non_blocking=True)
+        lin.linear(x_dev, y_out=y, workspace=ws)
+        y_pin.copy_(y, non_blocking=True)
+
+    ms_e2e = timed(e2e_call)
+
+    # parity at full size, in this launch configuration: sampled rows against the oracle
+    rows = np.array([0, 1, 127, 128, 2049, M - 1])
+    Wb = workloads.bits_2d(W)
+    qw, sw, wo = mo.rowquant(Wb, mo.BF16, idx)
+    y_ref = mo.linear(workloads.bits_2d(X[rows]), mo.BF16, qw, sw, wo, idx, mo.BF16)
+    got = workloads.bits_2d(y[torch.from_numpy(rows).to(dev)].cpu())
+    agree = float(np.mean(got == y_ref))
+    q_dev, _, _, _ = lin.view()
+    weights_exact = bool(np.array_equal(q_dev[:256].cpu().numpy(), qw[:256]))
+
+    # the oracle on a bounded sample of the same layer (weights already decomposed, as on the GPU)
+    t = time.perf_counter()
+    mo.linear(workloads.bits_2d(X[:256]), mo.BF16, qw, sw, wo, idx, mo.BF16)
+    cpu_s = time.perf_counter() - t
+    rec = mo.reconstruct(qw[:1024], sw[:1024], wo[:1024], mo.BF16, idx)
+    wf = W[:1024].double().numpy()
+    lin.close()
+    return {
+        "workload": f"{MMD_WORKLOAD}: X [{M},{K}] x W [{N},{K}]^T bf16, {idx.size} critical features; {wl.recipe}",
+        "ms_per_call": round(ms_call, 4), "tops": round(ops / ms_call / 1e9, 1), "kernel_status": status,
+        "rowquant": {"ms": round(ms_row, 4), "algorithmic_bytes": int(row_bytes), "gbs": round(row_bytes / ms_row / 1e6, 1),
+                     "frac_of_measured_hbm": round(row_bytes / ms_row / 1e6 / hbm, 4)},
+        "roofline": {"bound": "tensor", "kernel": "gemm_tc (int8 tcgen05, fp32 side accumulator)", "achieved": round(ops / ms_prod / 1e9, 1),
+                     "peak": round(peak, 1), "peak_kind": f"{kind} bf16 x {NOMINAL_INT8_OVER_BF16} (nominal int8 / bf16 ratio)", "unit": "TOP/s",
+                     "frac": round(ops / ms_prod / 1e9 / peak, 4), "ms": round(ms_prod, 4), "traffic": MMD_TRAFFIC_BYTES},
+        "e2e": {"ms_per_call": round(ms_e2e, 4), "tops": round(ops / ms_e2e / 1e9, 1), "h2d_bytes_per_call": int(M * K * 2),
+                "d2h_bytes_per_call": int(M * N * 2)},
+        "parity": {"sampled_rows": rows.tolist(), "outputs_equal_to_oracle_bits": round(agree, 5), "weight_codes_exact_first_256_rows": weights_exact},
+        "quality": {"weight_bytes_ratio": round(2.0 * N * K / (N * K + 4 * N + 2 * N * sd.shape[1]), 3),
+                    "weight_rel_rms_error": round(float(np.sqrt(((rec - wf) ** 2).sum() / (wf ** 2).sum())), 5)},
+        "cpu_baseline": {"value": round(2.0 * 256 * N * K / cpu_s / 1e12, 4), "unit": "TOP/s", "cores": os.cpu_count(), "kind": "oracle",
+                         "sample": "first 256 tokens through the whole layer (weights already decomposed); numpy/BLAS threads"},
+        "gpu_launches": 2 * reps,
+    }
 
 
 # DRAM bytes per full-size launch (dram__bytes_read.sum + dram__bytes_write.sum), from ncu
@@ -388,6 +492,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-mmd", action="store_true", help="skip the decomposed-linear-layer section")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

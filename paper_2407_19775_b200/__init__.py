@@ -3,7 +3,7 @@
 ``workloads`` (seeded input generators) imports without the CUDA library; the binding
 loads ``libbq.so`` on first use and raises if it has not been built.
 """
-from . import workloads
+from . import mmd, workloads
 from .binding import (BF16, DYNAMIC_TREE, F16, F32, USER, BqError, Codebook, bq_dequantize, bq_quantize, bq_roundtrip,
                       n_blocks)
 

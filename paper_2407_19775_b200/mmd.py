@@ -64,6 +64,16 @@ def mmd_rowquant(v: torch.Tensor, idx: torch.Tensor | None):
     return q, scale, side
 
 
+def rowquant_into(v: torch.Tensor, idx: torch.Tensor | None, q: torch.Tensor, scale: torch.Tensor, side: torch.Tensor) -> None:
+    """``mmd_rowquant`` into caller-provided outputs."""
+    R, K = v.shape
+    ko = 0 if idx is None else idx.numel()
+    with torch.cuda.device(v.device):
+        rc = _lib().mmd_rowquant(_dev(v, "v").data_ptr(), _DT[v.dtype], R, K, None if ko == 0 else idx.data_ptr(), ko, q.data_ptr(),
+                                 scale.data_ptr(), side.data_ptr() if ko else None, _stream(v))
+    _check(rc, "mmd_rowquant")
+
+
 class DecomposedLinear:
     """Handle of one decomposed weight matrix (``mmd_decompose``) and its linear layer."""
 
