@@ -45,8 +45,12 @@ extern "C" {
 enum {
     MMD_ERR_WORKSPACE = 7, /* workspace missing, misaligned (256 bytes) or too small   */
     MMD_ERR_FEATURES = 8,  /* feature list not ascending, out of range or too long      */
-    MMD_ERR_PATH = 9       /* the requested kernel path cannot take this shape          */
+    MMD_ERR_PATH = 9,      /* the requested kernel path cannot take this shape          */
+    MMD_ERR_STATIC_LIMIT = 10 /* mmd_linear_static: the call needs more scratch than MMD_STATIC_SCRATCH_BYTES */
 };
+
+/* Size of the scratch array built into the library for mmd_linear_static. */
+#define MMD_STATIC_SCRATCH_BYTES (4u << 20)
 
 /* Kernel choice of mmd_linear. */
 enum {
@@ -115,6 +119,27 @@ int mmd_workspace_layout(const mmd_weights* w, int M, size_t* offsets3, size_t* 
  */
 int mmd_linear(const mmd_weights* w, const void* X, int M, void* Y, bq_dtype ydt,
                void* workspace, size_t workspace_bytes, int path, void* cuda_stream);
+
+/*
+ * mmd_linear_static -- mmd_linear without a workspace argument, for callers that cannot get
+ * device memory at the moment of the call: a serving process whose own pool already holds all
+ * of the GPU's memory, or a loop that cannot afford the device-wide synchronisation an
+ * allocation may cause.  (The paper has no counterpart of this call; it is a convenience of
+ * this library.)  The scratch is an array of MMD_STATIC_SCRATCH_BYTES (4 MiB) that is part of
+ * the library: every GPU that loads the library holds it until the process exits.  The call
+ * allocates and frees nothing.
+ *   Limit: the sizes must satisfy mmd_workspace_layout(w, M) <= MMD_STATIC_SCRATCH_BYTES --
+ *   about M (K + 4 + 2 side columns) bytes, e.g. 64 rows of 8192 features, a decode step;
+ *   otherwise MMD_ERR_STATIC_LIMIT is returned before anything is launched and
+ *   bq_last_cuda_error() names both sizes.
+ *   The first call on a device looks up the array's device address (one runtime call, no
+ *   allocation); make that first call before any stream capture is begun.
+ *   All calls on a device share the one array and it keeps what the last call wrote; no call
+ *   depends on its previous contents.  Two calls that overlap on the device (different
+ *   streams, or this call and an mmd_linear given the same memory) race on it: order them.
+ *   Arguments, results and the other error codes are those of mmd_linear.
+ */
+int mmd_linear_static(const mmd_weights* w, const void* X, int M, void* Y, bq_dtype ydt, int path, void* cuda_stream);
 
 /*
  * mmd_kernel_status -- synchronises the device and returns, through status_out (HOST), 0 or

@@ -62,6 +62,7 @@ const char* bq_status_string(int status) {
         case MMD_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case MMD_ERR_FEATURES: return "feature list not ascending, out of range or too long";
         case MMD_ERR_PATH: return "the requested kernel path cannot take this shape";
+        case MMD_ERR_STATIC_LIMIT: return "the call needs more scratch than the library's static array holds (see bq_last_cuda_error)";
         default: return "unknown status";
     }
 }

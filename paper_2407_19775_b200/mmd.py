@@ -14,7 +14,8 @@ PATH_AUTO, PATH_GENERAL, PATH_TENSOR = 0, 1, 2
 _TORCH_OF = {0: torch.float32, 1: torch.float16, 2: torch.bfloat16}
 
 SYMBOLS = ("mmd_side_columns", "mmd_select_features", "mmd_rowquant", "mmd_decompose", "mmd_free", "mmd_weights_view",
-           "mmd_workspace_layout", "mmd_linear", "mmd_kernel_status")
+           "mmd_workspace_layout", "mmd_linear", "mmd_linear_static", "mmd_kernel_status")
+STATIC_SCRATCH_BYTES = 4 << 20
 _typed = False
 
 
@@ -31,6 +32,7 @@ def _lib() -> ctypes.CDLL:
         L.mmd_weights_view.argtypes = [vp] + [ctypes.POINTER(vp)] * 4 + [ctypes.POINTER(i32)] * 4
         L.mmd_workspace_layout.argtypes = [vp, i32, ctypes.POINTER(sz), ctypes.POINTER(sz)]
         L.mmd_linear.argtypes = [vp, vp, i32, vp, i32, vp, sz, i32, vp]
+        L.mmd_linear_static.argtypes = [vp, vp, i32, vp, i32, i32, vp]
         L.mmd_kernel_status.argtypes = [vp, ctypes.POINTER(i32)]
         _typed = True
     return L
@@ -142,6 +144,23 @@ class DecomposedLinear:
             rc = _lib().mmd_linear(self._h, X.data_ptr(), M, _dev(y_out, "y_out").data_ptr(), _DT[y_out.dtype], ws.data_ptr(), ws.numel(),
                                    path, _stream(X))
         _check(rc, "mmd_linear")
+        return y_out
+
+    def linear_static(self, X: torch.Tensor, out_dtype: torch.dtype | None = None, path: int = PATH_AUTO,
+                      y_out: torch.Tensor | None = None) -> torch.Tensor:
+        """``mmd_linear_static``: the same layer with the library's built-in scratch array (small M only); the call
+        itself allocates nothing when ``y_out`` is given."""
+        _dev(X, "X")
+        if X.dtype != self.dtype or X.dim() != 2 or X.shape[1] != self.K:
+            raise BqError("X must be [M, K] of the weights' element type")
+        M = X.shape[0]
+        if y_out is None:
+            y_out = torch.empty((M, self.N), dtype=out_dtype or X.dtype, device=X.device)
+        with torch.cuda.device(X.device):
+            rc = _lib().mmd_linear_static(self._h, X.data_ptr(), M, _dev(y_out, "y_out").data_ptr(), _DT[y_out.dtype], path, _stream(X))
+        if rc == 10:
+            raise BqError("mmd_linear_static failed with status 10: " + _lib().bq_last_cuda_error().decode())
+        _check(rc, "mmd_linear_static")
         return y_out
 
     def workspace_parts(self, M: int, workspace: torch.Tensor | None = None):
