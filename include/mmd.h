@@ -56,7 +56,9 @@ enum {
 enum {
     MMD_PATH_AUTO = 0,     /* tensor-core kernel when the shape allows, else the general one */
     MMD_PATH_GENERAL = 1,  /* integer dot-product kernel, any M and N                       */
-    MMD_PATH_TENSOR = 2    /* tcgen05 kernel; needs N % 8 == 0 and 16-byte aligned Y        */
+    MMD_PATH_TENSOR = 2,   /* a tcgen05 kernel; needs N % 8 == 0 and 16-byte aligned Y: the persistent kernel for
+                              large products with at most 16 critical features, else one tile per CTA */
+    MMD_PATH_TENSOR_TILE = 3 /* the one-tile-per-CTA tcgen05 kernel, whatever the size                */
 };
 
 /* Opaque: the decomposed weights of one linear layer (int8 rows, row scales, 16-bit side

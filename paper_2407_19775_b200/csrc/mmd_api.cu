@@ -132,6 +132,27 @@ cudaError_t launch_tc(const mmd_weights* w, const CUtensorMap& mqx, const CUtens
 }
 
 template <int XDT, int YDT>
+cudaError_t launch_tcp(const mmd_weights* w, const CUtensorMap& mqx, const float* sx, const void* sidex, void* y, int M, cudaStream_t stream) {
+    static bool opted[64] = {};
+    if (w->device < 0 || w->device >= 64 || !opted[w->device]) {
+        const cudaError_t e = cudaFuncSetAttribute(mmdk::gemm_tcp<XDT, YDT>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(mmdk::kTcpSmemBytes));
+        if (e != cudaSuccess) return e;
+        if (w->device >= 0 && w->device < 64) opted[w->device] = true;
+    }
+    const int mtiles = (M + 127) / 128, ntiles = (w->N + mmdk::kTcpBN - 1) / mmdk::kTcpBN;
+    const long total = long(mtiles) * ntiles;
+    const unsigned grid = unsigned(total < w->sm_count ? total : w->sm_count);
+    mmdk::gemm_tcp<XDT, YDT><<<grid, mmdk::kTcThreads, mmdk::kTcpSmemBytes, stream>>>(
+        mqx, w->map_q[0], sx, w->scale, sidex, w->side, w->side_cols, w->ko, y, M, w->N, (w->K + 127) / 128, mtiles, ntiles, w->status);
+    return cudaGetLastError();
+}
+
+// Large products with few critical features take the persistent kernel.
+bool wants_persistent(const mmd_weights* w, int M) {
+    return w->ko <= mmdk::kTcpSide && w->N >= 256 && long((M + 127) / 128) * ((w->N + 255) / 256) >= w->sm_count;
+}
+
+template <int XDT, int YDT>
 cudaError_t launch_tc_bn(const mmd_weights* w, const CUtensorMap& mqx, const CUtensorMap& msx, const float* sx, void* y, int M,
                          cudaStream_t stream) {
     // The widest tile has the highest arithmetic intensity; when it would leave SMs without a
@@ -263,7 +284,7 @@ int mmd_linear(const mmd_weights* w, const void* X, int M, void* Y, bq_dtype ydt
     if (!w) return BQ_ERR_NULL;
     if (ydt != BQ_F32 && int(ydt) != w->dtype) return BQ_ERR_DTYPE;
     if (M < 0) return BQ_ERR_SIZE;
-    if (path != MMD_PATH_AUTO && path != MMD_PATH_GENERAL && path != MMD_PATH_TENSOR) return MMD_ERR_PATH;
+    if (path != MMD_PATH_AUTO && path != MMD_PATH_GENERAL && path != MMD_PATH_TENSOR && path != MMD_PATH_TENSOR_TILE) return MMD_ERR_PATH;
     if (M == 0) return BQ_OK;
     if (!X || !Y) return BQ_ERR_NULL;
     if (!aligned(X, 16)) return BQ_ERR_SIZE;
@@ -271,8 +292,9 @@ int mmd_linear(const mmd_weights* w, const void* X, int M, void* Y, bq_dtype ydt
     if (!workspace || !aligned(workspace, kWsAlign) || workspace_bytes < L.total) return MMD_ERR_WORKSPACE;
     if (!on_device(w)) return BQ_ERR_CUDA;
     const bool tc_ok = w->have_maps && (w->N % 8 == 0) && aligned(Y, 16);
-    if (path == MMD_PATH_TENSOR && !tc_ok) return MMD_ERR_PATH;
-    const bool use_tc = (path == MMD_PATH_TENSOR) || (path == MMD_PATH_AUTO && tc_ok);
+    if ((path == MMD_PATH_TENSOR || path == MMD_PATH_TENSOR_TILE) && !tc_ok) return MMD_ERR_PATH;
+    const bool use_tc = (path == MMD_PATH_TENSOR) || (path == MMD_PATH_TENSOR_TILE) || (path == MMD_PATH_AUTO && tc_ok);
+    const bool persistent = use_tc && path != MMD_PATH_TENSOR_TILE && wants_persistent(w, M);
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     char* ws = static_cast<char*>(workspace);
@@ -283,7 +305,12 @@ int mmd_linear(const mmd_weights* w, const void* X, int M, void* Y, bq_dtype ydt
     if (e != cudaSuccess) return cuda_fail(e);
 
     const bool bf = (w->dtype == BQ_BF16), f32out = (ydt == BQ_F32);
-    if (use_tc) {
+    if (persistent) {
+        CUtensorMap mqx;
+        if (!make_map(&mqx, qx, 1, uint64_t(M), uint64_t(w->K), 128)) return MMD_ERR_PATH;
+        if (bf) e = f32out ? launch_tcp<mmdk::kBF16, mmdk::kF32>(w, mqx, sx, sidex, Y, M, stream) : launch_tcp<mmdk::kBF16, mmdk::kBF16>(w, mqx, sx, sidex, Y, M, stream);
+        else e = f32out ? launch_tcp<mmdk::kF16, mmdk::kF32>(w, mqx, sx, sidex, Y, M, stream) : launch_tcp<mmdk::kF16, mmdk::kF16>(w, mqx, sx, sidex, Y, M, stream);
+    } else if (use_tc) {
         CUtensorMap mqx, msx;
         if (!make_map(&mqx, qx, 1, uint64_t(M), uint64_t(w->K), 128)) return MMD_ERR_PATH;
         if (w->side_cols > 0 && !make_map(&msx, sidex, 2, uint64_t(M), uint64_t(w->side_cols), 128)) return MMD_ERR_PATH;

@@ -453,4 +453,244 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
     }
 }
 
+
+// ------------------------------------------------------------------------------------------
+// gemm_tcp: persistent tensor-core kernel for large products with at most kTcpSide critical
+// features.
+//
+// One CTA per SM walks over 128 x 256 tiles (M-tile index fastest, so CTAs that run together
+// share weight tiles in L2).  Tensor memory holds TWO int32 accumulators (2 x 256 columns):
+// while the epilogue warps drain the accumulator of tile i, the MMA thread is already
+// accumulating tile i + 1 into the other one, and the TMA thread runs ahead through the
+// 4-stage ring, so set-up, the first load round trip and the epilogue no longer stop the
+// tensor pipe between tiles.  With both accumulators taken by integer sums the side columns
+// cannot use the tensor cores here; they are few, so the epilogue adds them with fp32 FMAs
+// in ascending feature order (the same order as gemm_general), hidden under the next tile's
+// MMAs.  Waits are bounded as in gemm_tc.
+
+constexpr int kTcpBN = 256;
+constexpr int kTcpStages = 4;
+constexpr int kTcpSide = 16;                                   // most critical features this kernel takes
+constexpr uint32_t kTcpStageBytes = (kTcBM + kTcpBN) * kTcRowBytes;
+constexpr uint32_t kTcpCtrlBytes = 512;
+constexpr uint32_t kTcpSwBytes = 2 * kTcpBN * 4;               // column scales, one copy per accumulator
+constexpr uint32_t kTcpWoBytes = kTcpBN * kTcpSide * 4;        // side columns of the tile's weight rows, fp32
+constexpr uint32_t kTcpSmemBytes = kTcpStages * kTcpStageBytes + 1024 + kTcpCtrlBytes + kTcpSwBytes + kTcpWoBytes;
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+template <int XDT, int YDT>
+__global__ void __launch_bounds__(kTcThreads, 1)
+gemm_tcp(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUtensorMap map_qw,
+         const float* __restrict__ sx, const float* __restrict__ sw, const void* __restrict__ sidex, const void* __restrict__ sidew,
+         int side_cols /* row pitch of the side matrices */, int ko /* critical features, <= kTcpSide */,
+         void* __restrict__ y, int M, int N, int kblocks, int mtiles, int ntiles, int* status) {
+    constexpr int S = kTcpStages;
+    constexpr int BN = kTcpBN;
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t tiles_sm = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* ctrl = smem_raw + (tiles_sm - smem_u32(smem_raw)) + S * kTcpStageBytes;
+    const uint32_t full0 = smem_u32(ctrl);                                      // S: tile landed
+    const uint32_t empty0 = full0 + 8u * S;                                     // S: tile consumed
+    const uint32_t accf0 = empty0 + 8u * S;                                     // 2: accumulator complete
+    const uint32_t acce0 = accf0 + 16u;                                         // 2: accumulator drained
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl + 8 * (2 * S + 4));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 8 * (2 * S + 4) + 8);
+    volatile int* epi_ok = reinterpret_cast<volatile int*>(ctrl + 8 * (2 * S + 4) + 12);     // the epilogue's shared verdict of its wait
+    float* sw_s = reinterpret_cast<float*>(ctrl + kTcpCtrlBytes);               // [2][BN]
+    float* wo_s = sw_s + 2 * BN;                                                // [BN][kTcpSide]
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int total_tiles = mtiles * ntiles;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8u * b, 1); mbar_init(acce0 + 8u * b, 4); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(2 * BN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                const int m0 = (t % mtiles) * kTcBM, n0 = (t / mtiles) * BN;
+                for (int i = 0; i < kblocks; ++i, ++it) {
+                    const uint32_t s = it % S, round = it / S;
+                    ok = mbar_wait(empty0 + 8u * s, (round & 1u) ^ 1u, abort_flag, status, 1);
+                    if (!ok) break;
+                    const uint32_t a_dst = tiles_sm + s * kTcpStageBytes, b_dst = a_dst + kTcBM * kTcRowBytes;
+                    mbar_expect_tx(full0 + 8u * s, kTcpStageBytes);
+                    tma_load_2d(a_dst, &map_qx, i * 128, m0, full0 + 8u * s);
+                    tma_load_2d(b_dst, &map_qw, i * 128, n0, full0 + 8u * s);
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc_i8 = umma_idesc(2, 1, kTcBM, BN);
+            uint32_t it = 0, lt = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++lt) {
+                const uint32_t buf = lt & 1u;
+                ok = mbar_wait(acce0 + 8u * buf, ((lt >> 1) & 1u) ^ 1u, abort_flag, status, 4);    // the epilogue has drained this accumulator
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t d_tmem = tmem + buf * uint32_t(BN);
+                for (int i = 0; i < kblocks; ++i, ++it) {
+                    const uint32_t s = it % S, round = it / S;
+                    ok = mbar_wait(full0 + 8u * s, round & 1u, abort_flag, status, 2);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a_src = tiles_sm + s * kTcpStageBytes, b_src = a_src + kTcBM * kTcRowBytes;
+                    const uint64_t adesc = umma_smem_desc(a_src), bdesc = umma_smem_desc(b_src);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        umma_i8(d_tmem, adesc + uint64_t(2 * k), bdesc + uint64_t(2 * k), idesc_i8, (i > 0 || k > 0) ? 1u : 0u);
+                    umma_commit(empty0 + 8u * s);
+                }
+                if (ok) umma_commit(accf0 + 8u * buf);
+            }
+        }
+        __syncwarp();
+    } else {
+        const int et = threadIdx.x - 64;
+        const int quarter = warp & 3;
+        const uint16_t* sxo = static_cast<const uint16_t*>(sidex);
+        const uint16_t* swo = static_cast<const uint16_t*>(sidew);
+        uint32_t lt = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++lt) {
+            const uint32_t buf = lt & 1u;
+            const int m0 = (t % mtiles) * kTcBM, n0 = (t / mtiles) * BN;
+            const int m = m0 + quarter * 32 + lane;
+            // this tile's column scales and side columns; they are read while the MMAs of the tile still run
+            float* sws = sw_s + buf * BN;
+            for (int c = et; c < BN; c += 128) sws[c] = (n0 + c < N) ? sw[n0 + c] : 0.0f;
+            float xo[kTcpSide];
+#pragma unroll
+            for (int j = 0; j < kTcpSide; ++j) xo[j] = 0.0f;
+            if (ko > 0) {
+                // side rows are at least 64 columns wide (128 bytes), so the first 16 columns are two aligned 16-byte loads
+                for (int c = et; c < BN; c += 128) {
+                    const int n = n0 + c;
+                    float f[kTcpSide];
+                    if (n < N) {
+                        const uint4* src = reinterpret_cast<const uint4*>(swo + size_t(n) * side_cols);
+                        float lo[8], hi[8];
+                        widen8<XDT>(src[0], lo);
+                        widen8<XDT>(src[1], hi);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) { f[j] = lo[j]; f[8 + j] = hi[j]; }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < kTcpSide; ++j) f[j] = 0.0f;
+                    }
+#pragma unroll
+                    for (int j = 0; j < kTcpSide; j += 4)
+                        *reinterpret_cast<float4*>(wo_s + c * kTcpSide + j) = make_float4(f[j], f[j + 1], f[j + 2], f[j + 3]);
+                }
+                if (m < M) {
+                    const uint4* src = reinterpret_cast<const uint4*>(sxo + size_t(m) * side_cols);
+                    float lo[8], hi[8];
+                    widen8<XDT>(src[0], lo);
+                    widen8<XDT>(src[1], hi);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) { xo[j] = lo[j]; xo[8 + j] = hi[j]; }
+                }
+            }
+            const float sxm = (m < M) ? sx[m] : 0.0f;
+            // one thread waits for the accumulator, with the bound; its verdict reaches the other 127 through the
+            // barrier that also publishes the scales above, so the four warps always take the same way
+            if (et == 0) *epi_ok = mbar_wait(accf0 + 8u * buf, (lt >> 1) & 1u, abort_flag, status, 3) ? 1 : 0;
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            ok = (*epi_ok != 0);
+            if (ok) (void)mbar_try(accf0 + 8u * buf, (lt >> 1) & 1u);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (ok) {
+                const uint32_t lane_base = tmem + (uint32_t(quarter * 32) << 16) + buf * uint32_t(BN);
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    uint32_t ai[32];
+                    tmem_ld32(lane_base + uint32_t(c0), ai);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    float out[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        float p = 0.0f;
+                        if (ko > 0) {
+                            const float4* wrow = reinterpret_cast<const float4*>(wo_s + (c0 + j) * kTcpSide);
+#pragma unroll
+                            for (int q = 0; q < kTcpSide / 4; ++q) {
+                                if (q * 4 < ko) {
+                                    const float4 wv = wrow[q];
+                                    p = __fmaf_rn(xo[4 * q + 0], wv.x, p);
+                                    p = __fmaf_rn(xo[4 * q + 1], wv.y, p);
+                                    p = __fmaf_rn(xo[4 * q + 2], wv.z, p);
+                                    p = __fmaf_rn(xo[4 * q + 3], wv.w, p);
+                                }
+                            }
+                        }
+                        out[j] = __fmaf_rn(float(int(ai[j])), __fmul_rn(sxm, sws[c0 + j]), p);
+                    }
+                    if (m < M) {
+                        const int n = n0 + c0;
+                        if constexpr (YDT == kF32) {
+                            float* dst = static_cast<float*>(y) + size_t(m) * N + n;
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4)
+                                if (n + j < N) *reinterpret_cast<float4*>(dst + j) = make_float4(out[j], out[j + 1], out[j + 2], out[j + 3]);
+                        } else {
+                            uint16_t* dst = static_cast<uint16_t*>(y) + size_t(m) * N + n;
+#pragma unroll
+                            for (int j = 0; j < 32; j += 8) {
+                                uint32_t pk[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    if constexpr (YDT == kBF16) {
+                                        const __nv_bfloat162 h = __floats2bfloat162_rn(out[j + 2 * e], out[j + 2 * e + 1]);
+                                        pk[e] = *reinterpret_cast<const uint32_t*>(&h);
+                                    } else {
+                                        const __half2 h = __floats2half2_rn(out[j + 2 * e], out[j + 2 * e + 1]);
+                                        pk[e] = *reinterpret_cast<const uint32_t*>(&h);
+                                    }
+                                }
+                                if (n + j < N) *reinterpret_cast<uint4*>(dst + j) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                            }
+                        }
+                    }
+                }
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(acce0 + 8u * buf);         // this warp's quarter of the accumulator is free again
+            }
+            asm volatile("bar.sync 2, 128;" ::: "memory");             // wo_s is rewritten for the next tile
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    }
+
+    __syncthreads();
+    if (*abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(2000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(2 * BN) : "memory");
+    }
+}
+
 }  // namespace mmdk

@@ -136,7 +136,9 @@ TC_SHAPES = [
     ("bn64", 300, 400, 520, torch.bfloat16, 5),
     ("bn64_fp16", 129, 144, 72, torch.float16, 2),
     ("bn128", 1300, 272, 2056, torch.bfloat16, 70),              # 11 x 17 tiles of 128; two side steps
-    ("bn256", 1300, 400, 4104, torch.float16, 3),                # 11 x 17 tiles of 256
+    ("bn256", 1300, 400, 4104, torch.float16, 3),                # 11 x 17 tiles of 256: persistent kernel, one or two tiles per CTA
+    ("bn256_many", 2560, 144, 6152, torch.bfloat16, 16),         # 20 x 25 tiles: three to four per CTA, fewer K steps than ring stages
+    ("bn256_side", 1300, 400, 4104, torch.bfloat16, 17),         # too many features for the persistent kernel
     ("one_row", 1, 128, 8, torch.bfloat16, 1),
 ]
 
@@ -151,13 +153,15 @@ def test_linear_tensor_path(bq, name, M, K, N, tdt, ko):
     X[:, idx.tolist()] *= 30
     for features, exact in ((idx, False), (np.zeros(0, np.int32), True)):
         lin = bq.DecomposedLinear(W.cuda(), features)
-        for out in (torch.float32, None):
-            y = lin.linear(X.cuda(), out, path=2)
-            assert lin.kernel_status() == 0
-            check_output(y, X, W, features, dt, exact_expected=exact)
+        for path in (2, 3):                                       # persistent where it applies / always one tile per CTA
+            for out in (torch.float32, None):
+                y = lin.linear(X.cuda(), out, path=path)
+                assert lin.kernel_status() == 0
+                check_output(y, X, W, features, dt, exact_expected=exact)
         yg = lin.linear(X.cuda(), torch.float32, path=1)
         if exact:
             assert torch.equal(yg, lin.linear(X.cuda(), torch.float32, path=2))
+            assert torch.equal(yg, lin.linear(X.cuda(), torch.float32, path=3))
         lin.close()
 
 
