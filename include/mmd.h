@@ -56,9 +56,11 @@ enum {
 enum {
     MMD_PATH_AUTO = 0,     /* tensor-core kernel when the shape allows, else the general one */
     MMD_PATH_GENERAL = 1,  /* integer dot-product kernel, any M and N                       */
-    MMD_PATH_TENSOR = 2,   /* a tcgen05 kernel; needs N % 8 == 0 and 16-byte aligned Y: the persistent kernel for
-                              large products with at most 16 critical features, else one tile per CTA */
-    MMD_PATH_TENSOR_TILE = 3 /* the one-tile-per-CTA tcgen05 kernel, whatever the size                */
+    MMD_PATH_TENSOR = 2,   /* a tcgen05 kernel; needs N % 8 == 0 and 16-byte aligned Y: the persistent CTA-pair
+                              kernel for large products with at most 16 critical features, else one tile per CTA */
+    MMD_PATH_TENSOR_TILE = 3, /* the one-tile-per-CTA tcgen05 kernel, whatever the size                */
+    MMD_PATH_TENSOR_SOLO = 4  /* the persistent kernel without CTA pairs (same limits as the pair kernel; MMD_ERR_PATH
+                                 when the product is too small or has more than 16 critical features) */
 };
 
 /* Opaque: the decomposed weights of one linear layer (int8 rows, row scales, 16-bit side

@@ -147,7 +147,35 @@ cudaError_t launch_tcp(const mmd_weights* w, const CUtensorMap& mqx, const float
     return cudaGetLastError();
 }
 
-// Large products with few critical features take the persistent kernel.
+template <int XDT, int YDT>
+cudaError_t launch_tc2(const mmd_weights* w, const CUtensorMap& mqx, const float* sx, const void* sidex, void* y, int M, cudaStream_t stream) {
+    static bool opted[64] = {};
+    static int max_pairs[64] = {};
+    const int d = (w->device >= 0 && w->device < 64) ? w->device : 0;
+    if (!opted[d]) {
+        cudaError_t e = cudaFuncSetAttribute(mmdk::gemm_tc2<XDT, YDT>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(mmdk::kPairSmemBytes));
+        if (e != cudaSuccess) return e;
+        // how many CTA pairs the device runs at once: the persistent grid must not exceed it
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(unsigned(w->sm_count & ~1), 1, 1);
+        cfg.blockDim = dim3(mmdk::kTcThreads, 1, 1);
+        cfg.dynamicSmemBytes = mmdk::kPairSmemBytes;
+        int n = 0;
+        e = cudaOccupancyMaxActiveClusters(&n, mmdk::gemm_tc2<XDT, YDT>, &cfg);
+        if (e != cudaSuccess) return e;
+        if (n < 1) return cudaErrorInvalidConfiguration;
+        max_pairs[d] = n;
+        opted[d] = true;
+    }
+    const int mpairs = (M + 255) / 256, ntiles = (w->N + mmdk::kTcpBN - 1) / mmdk::kTcpBN;
+    const long total = long(mpairs) * ntiles;
+    const unsigned pairs = unsigned(total < max_pairs[d] ? total : max_pairs[d]);
+    mmdk::gemm_tc2<XDT, YDT><<<2 * pairs, mmdk::kTcThreads, mmdk::kPairSmemBytes, stream>>>(
+        mqx, w->map_q[1], sx, w->scale, sidex, w->side, w->side_cols, w->ko, y, M, w->N, (w->K + 127) / 128, mpairs, ntiles, w->status);
+    return cudaGetLastError();
+}
+
+// Large products with few critical features take the persistent kernels.
 bool wants_persistent(const mmd_weights* w, int M) {
     return w->ko <= mmdk::kTcpSide && w->N >= 256 && long((M + 127) / 128) * ((w->N + 255) / 256) >= w->sm_count;
 }
@@ -284,7 +312,7 @@ int mmd_linear(const mmd_weights* w, const void* X, int M, void* Y, bq_dtype ydt
     if (!w) return BQ_ERR_NULL;
     if (ydt != BQ_F32 && int(ydt) != w->dtype) return BQ_ERR_DTYPE;
     if (M < 0) return BQ_ERR_SIZE;
-    if (path != MMD_PATH_AUTO && path != MMD_PATH_GENERAL && path != MMD_PATH_TENSOR && path != MMD_PATH_TENSOR_TILE) return MMD_ERR_PATH;
+    if (path < MMD_PATH_AUTO || path > MMD_PATH_TENSOR_SOLO) return MMD_ERR_PATH;
     if (M == 0) return BQ_OK;
     if (!X || !Y) return BQ_ERR_NULL;
     if (!aligned(X, 16)) return BQ_ERR_SIZE;
@@ -292,9 +320,11 @@ int mmd_linear(const mmd_weights* w, const void* X, int M, void* Y, bq_dtype ydt
     if (!workspace || !aligned(workspace, kWsAlign) || workspace_bytes < L.total) return MMD_ERR_WORKSPACE;
     if (!on_device(w)) return BQ_ERR_CUDA;
     const bool tc_ok = w->have_maps && (w->N % 8 == 0) && aligned(Y, 16);
-    if ((path == MMD_PATH_TENSOR || path == MMD_PATH_TENSOR_TILE) && !tc_ok) return MMD_ERR_PATH;
-    const bool use_tc = (path == MMD_PATH_TENSOR) || (path == MMD_PATH_TENSOR_TILE) || (path == MMD_PATH_AUTO && tc_ok);
+    if (path >= MMD_PATH_TENSOR && !tc_ok) return MMD_ERR_PATH;
+    if (path == MMD_PATH_TENSOR_SOLO && !wants_persistent(w, M)) return MMD_ERR_PATH;
+    const bool use_tc = (path >= MMD_PATH_TENSOR) || (path == MMD_PATH_AUTO && tc_ok);
     const bool persistent = use_tc && path != MMD_PATH_TENSOR_TILE && wants_persistent(w, M);
+    const bool pairs = persistent && path != MMD_PATH_TENSOR_SOLO;
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     char* ws = static_cast<char*>(workspace);
@@ -305,7 +335,12 @@ int mmd_linear(const mmd_weights* w, const void* X, int M, void* Y, bq_dtype ydt
     if (e != cudaSuccess) return cuda_fail(e);
 
     const bool bf = (w->dtype == BQ_BF16), f32out = (ydt == BQ_F32);
-    if (persistent) {
+    if (pairs) {
+        CUtensorMap mqx;
+        if (!make_map(&mqx, qx, 1, uint64_t(M), uint64_t(w->K), 128)) return MMD_ERR_PATH;
+        if (bf) e = f32out ? launch_tc2<mmdk::kBF16, mmdk::kF32>(w, mqx, sx, sidex, Y, M, stream) : launch_tc2<mmdk::kBF16, mmdk::kBF16>(w, mqx, sx, sidex, Y, M, stream);
+        else e = f32out ? launch_tc2<mmdk::kF16, mmdk::kF32>(w, mqx, sx, sidex, Y, M, stream) : launch_tc2<mmdk::kF16, mmdk::kF16>(w, mqx, sx, sidex, Y, M, stream);
+    } else if (persistent) {
         CUtensorMap mqx;
         if (!make_map(&mqx, qx, 1, uint64_t(M), uint64_t(w->K), 128)) return MMD_ERR_PATH;
         if (bf) e = f32out ? launch_tcp<mmdk::kBF16, mmdk::kF32>(w, mqx, sx, sidex, Y, M, stream) : launch_tcp<mmdk::kBF16, mmdk::kBF16>(w, mqx, sx, sidex, Y, M, stream);

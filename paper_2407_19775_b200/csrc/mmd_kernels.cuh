@@ -693,4 +693,287 @@ gemm_tcp(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUt
     }
 }
 
+
+// ------------------------------------------------------------------------------------------
+// gemm_tc2: persistent kernel on CTA pairs (clusters of two, tcgen05 cta_group::2).
+//
+// The two SMs of a TPC share a 256 x 256 tile: each CTA loads its own 128 activation rows and
+// only HALF of the weight rows (32 KB per K step of 128 features instead of 48 KB), and one
+// thread of the even CTA issues MMAs of shape 256 x 256 x 32 that read both halves from the
+// two shared memories and write each CTA's 128 rows into that CTA's own tensor memory.
+// Otherwise as gemm_tcp: a ring (6 stages here), two accumulators per CTA, epilogue under the
+// next tile's MMAs, side features by ordered fp32 FMAs.
+//
+// Barriers: "tile landed" lives in the even CTA and counts the bytes of both CTAs' loads (the
+// odd CTA's TMA loads name the even CTA's barrier); "stage free" and "accumulator complete"
+// are signalled in both CTAs by one multicast tcgen05.commit; "accumulator drained" lives in
+// the even CTA and takes one arrival per epilogue warp of both CTAs.  No load is multicast.
+
+constexpr int kPairStages = 6;
+constexpr uint32_t kPairHalfBytes = 128 * kTcRowBytes;                        // 128 rows of activations, or of weights
+constexpr uint32_t kPairStageBytes = 2 * kPairHalfBytes;
+constexpr uint32_t kPairSmemBytes = kPairStages * kPairStageBytes + 1024 + kTcpCtrlBytes + kTcpSwBytes + kTcpWoBytes;
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// the address, in the cluster's shared window, of this CTA's shared address `addr` in CTA `rank`
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar_cluster_addr) {
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ void umma_i8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// arrives on the barrier at this shared address in both CTAs of the pair once the MMAs issued so far are done
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(uint16_t(3)) : "memory");
+}
+
+// Scales and side columns of one tile's 256 weight rows into shared memory, and this thread's
+// own activation row's side values into registers (epilogue threads, et = 0..127).
+template <int XDT>
+__device__ __forceinline__ void stage_tile_side(int et, int n0, int N, int m, int M, int ko, int side_cols, const float* __restrict__ sw,
+                                                const uint16_t* __restrict__ sxo, const uint16_t* __restrict__ swo, float* sws, float* wo_s,
+                                                float (&xo)[kTcpSide]) {
+    for (int c = et; c < kTcpBN; c += 128) sws[c] = (n0 + c < N) ? sw[n0 + c] : 0.0f;
+#pragma unroll
+    for (int j = 0; j < kTcpSide; ++j) xo[j] = 0.0f;
+    if (ko > 0) {
+        for (int c = et; c < kTcpBN; c += 128) {
+            const int n = n0 + c;
+            float f[kTcpSide];
+            if (n < N) {
+                const uint4* src = reinterpret_cast<const uint4*>(swo + size_t(n) * side_cols);
+                float lo[8], hi[8];
+                widen8<XDT>(src[0], lo);
+                widen8<XDT>(src[1], hi);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) { f[j] = lo[j]; f[8 + j] = hi[j]; }
+            } else {
+#pragma unroll
+                for (int j = 0; j < kTcpSide; ++j) f[j] = 0.0f;
+            }
+#pragma unroll
+            for (int j = 0; j < kTcpSide; j += 4)
+                *reinterpret_cast<float4*>(wo_s + c * kTcpSide + j) = make_float4(f[j], f[j + 1], f[j + 2], f[j + 3]);
+        }
+        if (m < M) {
+            const uint4* src = reinterpret_cast<const uint4*>(sxo + size_t(m) * side_cols);
+            float lo[8], hi[8];
+            widen8<XDT>(src[0], lo);
+            widen8<XDT>(src[1], hi);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { xo[j] = lo[j]; xo[8 + j] = hi[j]; }
+        }
+    }
+}
+
+// One accumulator row of 256 int32 sums -> scaled, side part added, narrowed, stored.
+template <int YDT>
+__device__ __forceinline__ void drain_row(uint32_t lane_base, float sxm, const float* sws, const float* wo_s, const float (&xo)[kTcpSide], int ko,
+                                          void* __restrict__ y, int m, int M, int n0, int N) {
+#pragma unroll 1
+    for (int c0 = 0; c0 < kTcpBN; c0 += 32) {
+        uint32_t ai[32];
+        tmem_ld32(lane_base + uint32_t(c0), ai);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        float out[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            float p = 0.0f;
+            if (ko > 0) {
+                const float4* wrow = reinterpret_cast<const float4*>(wo_s + (c0 + j) * kTcpSide);
+#pragma unroll
+                for (int q = 0; q < kTcpSide / 4; ++q) {
+                    if (q * 4 < ko) {
+                        const float4 wv = wrow[q];
+                        p = __fmaf_rn(xo[4 * q + 0], wv.x, p);
+                        p = __fmaf_rn(xo[4 * q + 1], wv.y, p);
+                        p = __fmaf_rn(xo[4 * q + 2], wv.z, p);
+                        p = __fmaf_rn(xo[4 * q + 3], wv.w, p);
+                    }
+                }
+            }
+            out[j] = __fmaf_rn(float(int(ai[j])), __fmul_rn(sxm, sws[c0 + j]), p);
+        }
+        if (m < M) {
+            const int n = n0 + c0;
+            if constexpr (YDT == kF32) {
+                float* dst = static_cast<float*>(y) + size_t(m) * N + n;
+#pragma unroll
+                for (int j = 0; j < 32; j += 4)
+                    if (n + j < N) *reinterpret_cast<float4*>(dst + j) = make_float4(out[j], out[j + 1], out[j + 2], out[j + 3]);
+            } else {
+                uint16_t* dst = static_cast<uint16_t*>(y) + size_t(m) * N + n;
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) {
+                    uint32_t pk[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        if constexpr (YDT == kBF16) {
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(out[j + 2 * e], out[j + 2 * e + 1]);
+                            pk[e] = *reinterpret_cast<const uint32_t*>(&h);
+                        } else {
+                            const __half2 h = __floats2half2_rn(out[j + 2 * e], out[j + 2 * e + 1]);
+                            pk[e] = *reinterpret_cast<const uint32_t*>(&h);
+                        }
+                    }
+                    if (n + j < N) *reinterpret_cast<uint4*>(dst + j) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                }
+            }
+        }
+    }
+}
+
+template <int XDT, int YDT>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTcThreads, 1)
+gemm_tc2(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUtensorMap map_qw /* boxes of 128 weight rows */,
+         const float* __restrict__ sx, const float* __restrict__ sw, const void* __restrict__ sidex, const void* __restrict__ sidew,
+         int side_cols, int ko, void* __restrict__ y, int M, int N, int kblocks, int mpairs /* tiles of 256 rows */, int ntiles, int* status) {
+    constexpr int S = kPairStages;
+    constexpr int BN = kTcpBN;
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t tiles_sm = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* ctrl = smem_raw + (tiles_sm - smem_u32(smem_raw)) + S * kPairStageBytes;
+    const uint32_t full0 = smem_u32(ctrl);                                      // S: tile landed (used in the even CTA)
+    const uint32_t empty0 = full0 + 8u * S;                                     // S: stage free
+    const uint32_t accf0 = empty0 + 8u * S;                                     // 2: accumulator complete
+    const uint32_t acce0 = accf0 + 16u;                                         // 2: accumulator drained (used in the even CTA)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl + 8 * (2 * S + 4));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 8 * (2 * S + 4) + 8);
+    volatile int* epi_ok = reinterpret_cast<volatile int*>(ctrl + 8 * (2 * S + 4) + 12);
+    float* sw_s = reinterpret_cast<float*>(ctrl + kTcpCtrlBytes);               // [2][BN]
+    float* wo_s = sw_s + 2 * BN;                                                // [BN][kTcpSide]
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_rank();
+    const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+    const int total_tiles = mpairs * ntiles;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8u * b, 1); mbar_init(acce0 + 8u * b, 8); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(2 * BN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    cluster_sync_all();                                                          // both CTAs' barriers exist before either signals the other
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int t = pair; t < total_tiles && ok; t += npairs) {
+                const int m0 = (t % mpairs) * 256 + int(rank) * 128;             // this CTA's activation rows
+                const int nb0 = (t / mpairs) * BN + int(rank) * 128;             // this CTA's half of the weight rows
+                for (int i = 0; i < kblocks; ++i, ++it) {
+                    const uint32_t s = it % S, round = it / S;
+                    ok = mbar_wait(empty0 + 8u * s, (round & 1u) ^ 1u, abort_flag, status, 1);
+                    if (!ok) break;
+                    const uint32_t a_dst = tiles_sm + s * kPairStageBytes, b_dst = a_dst + kPairHalfBytes;
+                    const uint32_t full_even = map_to_cta(full0 + 8u * s, 0);
+                    if (rank == 0) mbar_expect_tx(full0 + 8u * s, 2 * kPairStageBytes);      // both CTAs' bytes
+                    tma_load_2d_pair(a_dst, &map_qx, i * 128, m0, full_even);
+                    tma_load_2d_pair(b_dst, &map_qw, i * 128, nb0, full_even);
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc_i8 = umma_idesc(2, 1, 256, BN);
+            uint32_t it = 0, lt = 0;
+            bool ok = true;
+            for (int t = pair; t < total_tiles && ok; t += npairs, ++lt) {
+                const uint32_t buf = lt & 1u;
+                ok = mbar_wait(acce0 + 8u * buf, ((lt >> 1) & 1u) ^ 1u, abort_flag, status, 4);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t d_tmem = tmem + buf * uint32_t(BN);
+                for (int i = 0; i < kblocks; ++i, ++it) {
+                    const uint32_t s = it % S, round = it / S;
+                    ok = mbar_wait(full0 + 8u * s, round & 1u, abort_flag, status, 2);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a_src = tiles_sm + s * kPairStageBytes, b_src = a_src + kPairHalfBytes;
+                    const uint64_t adesc = umma_smem_desc(a_src), bdesc = umma_smem_desc(b_src);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        umma_i8_pair(d_tmem, adesc + uint64_t(2 * k), bdesc + uint64_t(2 * k), idesc_i8, (i > 0 || k > 0) ? 1u : 0u);
+                    umma_commit_pair(empty0 + 8u * s);
+                }
+                if (ok) umma_commit_pair(accf0 + 8u * buf);
+            }
+        }
+        __syncwarp();
+    } else {
+        const int et = threadIdx.x - 64;
+        const int quarter = warp & 3;
+        const uint16_t* sxo = static_cast<const uint16_t*>(sidex);
+        const uint16_t* swo = static_cast<const uint16_t*>(sidew);
+        uint32_t lt = 0;
+        bool ok = true;
+        for (int t = pair; t < total_tiles && ok; t += npairs, ++lt) {
+            const uint32_t buf = lt & 1u;
+            const int m0 = (t % mpairs) * 256 + int(rank) * 128, n0 = (t / mpairs) * BN;
+            const int m = m0 + quarter * 32 + lane;
+            float* sws = sw_s + buf * BN;
+            float xo[kTcpSide];
+            stage_tile_side<XDT>(et, n0, N, m, M, ko, side_cols, sw, sxo, swo, sws, wo_s, xo);
+            const float sxm = (m < M) ? sx[m] : 0.0f;
+            if (et == 0) *epi_ok = mbar_wait(accf0 + 8u * buf, (lt >> 1) & 1u, abort_flag, status, 3) ? 1 : 0;
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            ok = (*epi_ok != 0);
+            if (ok) (void)mbar_try(accf0 + 8u * buf, (lt >> 1) & 1u);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (ok) {
+                drain_row<YDT>(tmem + (uint32_t(quarter * 32) << 16) + buf * uint32_t(BN), sxm, sws, wo_s, xo, ko, y, m, M, n0, N);
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(acce0 + 8u * buf, 0));
+            }
+            asm volatile("bar.sync 2, 128;" ::: "memory");
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    }
+
+    __syncthreads();
+    if (*abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(2000);
+        __syncthreads();
+    }
+    cluster_sync_all();                                                          // neither CTA leaves while the other may still signal it
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(2 * BN) : "memory");
+    }
+}
+
 }  // namespace mmdk

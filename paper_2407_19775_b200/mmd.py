@@ -10,7 +10,7 @@ import torch
 
 from .binding import _DT, BqError, _check, _dev, _stream, lib
 
-PATH_AUTO, PATH_GENERAL, PATH_TENSOR, PATH_TENSOR_TILE = 0, 1, 2, 3
+PATH_AUTO, PATH_GENERAL, PATH_TENSOR, PATH_TENSOR_TILE, PATH_TENSOR_SOLO = 0, 1, 2, 3, 4
 _TORCH_OF = {0: torch.float32, 1: torch.float16, 2: torch.bfloat16}
 
 SYMBOLS = ("mmd_side_columns", "mmd_select_features", "mmd_rowquant", "mmd_decompose", "mmd_free", "mmd_weights_view",
