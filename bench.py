@@ -293,7 +293,9 @@ def measured_tensor_peak():
 def run_mmd(bq, dev, args):
     """The paper's second compression technique on one layer of the MoE-class prefill shape:
     weights decomposed once, then timed calls of the layer (row kernel over the activations +
-    tensor-core product).  Reported beside the main metric with its own roofline."""
+    tensor-core product).  Reported beside the main metric with its own roofline: operations
+    2 M N K per call over the product kernel's time (the call's time minus the row kernel's,
+    each averaged over the same number of event-timed launches)."""
     import oracle.mmd_oracle as mo
     wl = workloads.LINEAR_WORKLOADS[MMD_WORKLOAD]
     X, W, idx = workloads.make_linear(MMD_WORKLOAD)
@@ -361,7 +363,7 @@ def run_mmd(bq, dev, args):
         "ms_per_call": round(ms_call, 4), "tops": round(ops / ms_call / 1e9, 1), "kernel_status": status,
         "rowquant": {"ms": round(ms_row, 4), "algorithmic_bytes": int(row_bytes), "gbs": round(row_bytes / ms_row / 1e6, 1),
                      "frac_of_measured_hbm": round(row_bytes / ms_row / 1e6 / hbm, 4)},
-        "roofline": {"bound": "tensor", "kernel": "gemm_tc (int8 tcgen05, fp32 side accumulator)", "achieved": round(ops / ms_prod / 1e9, 1),
+        "roofline": {"bound": "tensor", "kernel": "gemm_tc2 (persistent CTA pairs, int8 tcgen05 cta_group::2)", "achieved": round(ops / ms_prod / 1e9, 1),
                      "peak": round(peak, 1), "peak_kind": f"{kind} bf16 x {NOMINAL_INT8_OVER_BF16} (nominal int8 / bf16 ratio)", "unit": "TOP/s",
                      "frac": round(ops / ms_prod / 1e9 / peak, 4), "ms": round(ms_prod, 4), "traffic": MMD_TRAFFIC_BYTES},
         "e2e": {"ms_per_call": round(ms_e2e, 4), "tops": round(ops / ms_e2e / 1e9, 1), "h2d_bytes_per_call": int(M * K * 2),
