@@ -81,6 +81,25 @@ def test_rowquant_bit_exact(bq, tdt):
     assert np.array_equal(q0.cpu().numpy(), q0_ref) and np.array_equal(s0.cpu().numpy(), s0_ref) and side0.shape == (R, 0)
 
 
+@pytest.mark.parametrize("K", [16, 2064, 6144, 8192, 12288, 16384, 16400])
+def test_rowquant_row_lengths(bq, K):
+    """Rows from one chunk to more chunks than the CTA has threads (several trips of its loops), with ragged last trips;
+    rows scaled far down and far up (tiny and huge divisors) and a zero row."""
+    g = torch.Generator().manual_seed(K)
+    R = 9
+    v = torch.randn(R, K, generator=g)
+    v[1] *= 1e-25; v[2] *= 1e25; v[3] *= 2.0 ** -64; v[4] *= 2.0 ** 63; v[5] = 0
+    v = v.to(torch.bfloat16)
+    ko = min(5, K - 1)
+    idx = np.sort(torch.randperm(K, generator=g)[:ko].numpy()).astype(np.int32)
+    v[:, idx.tolist()] *= 8
+    q_ref, s_ref, side_ref = mo.rowquant(bits(v), BF16, idx)
+    q, s, side = bq.mmd_rowquant(v.cuda(), torch.from_numpy(idx).cuda())
+    assert np.array_equal(q.cpu().numpy(), q_ref)
+    assert np.array_equal(s.cpu().numpy().view(np.uint32), s_ref.view(np.uint32))
+    assert np.array_equal(bits(side), side_ref)
+
+
 def test_rowquant_division_cases(bq):
     """Pairs on which a multiplication by the reciprocal would land on another integer."""
     vals = (np.arange(0x3C00, 0x4300, dtype=np.uint32) << 16).view(np.float32)
