@@ -187,6 +187,31 @@ def test_linear_tensor_path(bq, name, M, K, N, tdt, ko):
         lin.close()
 
 
+def test_linear_seeded_fuzz(bq):
+    """Random small shapes, feature counts, element types and value scales through every kernel that takes them."""
+    rng = np.random.default_rng(2024)
+    for case in range(16):
+        M = int(rng.integers(1, 300)); K = 16 * int(rng.integers(1, 40)); N = 8 * int(rng.integers(1, 70))
+        ko = int(rng.integers(0, min(20, K - 1)))
+        tdt = torch.bfloat16 if case % 2 else torch.float16
+        dt = DT[tdt]
+        g = torch.Generator().manual_seed(1000 + case)
+        scale_x = float(10.0 ** rng.uniform(-2, 1)); scale_w = float(10.0 ** rng.uniform(-3, 0))
+        X = (torch.randn(M, K, generator=g) * scale_x).to(tdt)
+        W = (torch.randn(N, K, generator=g) * scale_w).to(tdt)
+        if case % 5 == 0:
+            X[int(rng.integers(0, M))] = 0                      # a zero activation row
+            W[int(rng.integers(0, N))] = 0
+        idx = np.sort(rng.choice(K, ko, replace=False)).astype(np.int32)
+        X[:, idx.tolist()] *= 20
+        lin = bq.DecomposedLinear(W.cuda(), idx)
+        for path in (1, 2, 3):
+            y = lin.linear(X.cuda(), torch.float32 if case % 3 else None, path=path)
+            assert lin.kernel_status() == 0
+            check_output(y, X, W, idx, dt, exact_expected=(ko == 0))
+        lin.close()
+
+
 def test_linear_integer_part_saturating_inputs(bq):
     """Every code at +-127 over a long row: sums far above 2^24 must come back exactly."""
     M, K, N = 130, 4096, 264
