@@ -304,7 +304,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUtensorMap map_qw,
         const __grid_constant__ CUtensorMap map_sidex, const __grid_constant__ CUtensorMap map_sidew,
         const float* __restrict__ sx, const float* __restrict__ sw, void* __restrict__ y,
-        int M, int N, int kblocks /* int8 steps of 128 features */, int sblocks /* side steps of 64 columns */, int* status) {
+        int M, int N, int kblocks /* int8 steps of 128 features */, int sblocks /* side steps of 64 columns */,
+        uint32_t stage_tx_bytes /* bytes the two loads of a stage bring: (activation rows in the map's box + BN) * 128 */, int* status) {
     using Cfg = TcCfg<BN>;
     constexpr int S = Cfg::kStages;
     extern __shared__ unsigned char smem_raw[];
@@ -344,7 +345,9 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
                 const uint32_t round = uint32_t(i / S);
                 if (!mbar_wait(empty0 + 8u * s, (round & 1u) ^ 1u, abort_flag, status, 1)) break;
                 const uint32_t a_dst = tiles + uint32_t(s) * Cfg::kStageBytes, b_dst = a_dst + Cfg::kABytes;
-                mbar_expect_tx(full0 + 8u * s, Cfg::kStageBytes);
+                // with at most 64 activation rows the host's maps load 64-row boxes: the MMA still reads 128 rows of
+                // shared memory, and what it makes of the stale upper half lands in accumulator rows that are never stored
+                mbar_expect_tx(full0 + 8u * s, stage_tx_bytes);
                 if (i < kblocks) {
                     tma_load_2d(a_dst, &map_qx, i * 128, m0, full0 + 8u * s);
                     tma_load_2d(b_dst, &map_qw, i * 128, n0, full0 + 8u * s);
