@@ -31,3 +31,10 @@ def test_bench_line_has_the_contract_keys(bq):
     assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
     for q in d["quality"].values():
         assert 1.8 < q["compression_ratio"] < 2.0 and 0.003 < q["rel_rms_error"] < 0.03
+    # the decomposed linear layer: its own roofline object, parity on sampled rows of the full-size call, no kernel error
+    m = d["mmd"]
+    mr = m["roofline"]
+    assert mr["bound"] == "tensor" and mr["unit"] == "TOP/s" and 0.3 < mr["frac"] < 1.1 and abs(mr["frac"] - mr["achieved"] / mr["peak"]) < 1e-3
+    assert m["kernel_status"] == 0 and m["parity"]["outputs_equal_to_oracle_bits"] > 0.99 and m["parity"]["weight_codes_exact_first_256_rows"]
+    assert 0 < m["e2e"]["tops"] < m["tops"] and m["e2e"]["h2d_bytes_per_call"] > 0 and m["cpu_baseline"]["kind"] == "oracle"
+    assert 1.9 < m["quality"]["weight_bytes_ratio"] < 2.0 and m["gpu_launches"] > 0
