@@ -1,0 +1,267 @@
+// bq4_kernels.cuh -- device code of the 4-bit variant (sm_100a).
+//
+//   q4_fast    : power-of-two blocks of 8..256 elements.  One thread per 8 elements (one or two
+//                128-bit loads), block absmax by a segmented shuffle over block / 8 lanes, codes
+//                by a 4-step branch-free search over the 15 thresholds in shared memory, eight
+//                nibbles per 32-bit store.  Two chunks per thread and trip, persistent grid.
+//   q4_wide    : power-of-two blocks of 512..65536: one warp per block, two passes over it (the
+//                second hits L1 / L2).
+//   dq4_fast   : 16 codes per 64-bit load, values from shared memory, 256-bit or 2 x 256-bit stores.
+//   *_general  : any block, any alignment: absmax per block, then one thread per byte.
+//
+// Arithmetic contract, as for the 8-bit kernels: exact fp32 absmax; the correctly rounded
+// quotient (for 16-bit inputs and divisors within [2^-64, 2^64] through the reciprocal route
+// whose exactness the CPU tests check over every pair of significands; IEEE division
+// otherwise); code = #{ j : t_j < xhat } over midpoints rounded toward -inf; one fp32 multiply
+// and a round-to-nearest-even narrowing on the way back.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace bq4k {
+
+enum { kF32 = 0, kF16 = 1, kBF16 = 2 };
+
+struct Tables4 {
+    float thr[16];      // [0..14] midpoints rounded toward -inf, [15] = +inf
+    float val[16];      // the codebook
+};
+
+template <int DT>
+__device__ __forceinline__ float load1(const void* x, size_t i) {
+    if constexpr (DT == kF32) return static_cast<const float*>(x)[i];
+    else if constexpr (DT == kBF16) return __uint_as_float(uint32_t(static_cast<const uint16_t*>(x)[i]) << 16);
+    else return __half2float(static_cast<const __half*>(x)[i]);
+}
+template <int DT>
+__device__ __forceinline__ void store1(void* y, size_t i, float v) {
+    if constexpr (DT == kF32) static_cast<float*>(y)[i] = v;
+    else if constexpr (DT == kBF16) static_cast<__nv_bfloat16*>(y)[i] = __float2bfloat16_rn(v);
+    else static_cast<__half*>(y)[i] = __float2half_rn(v);
+}
+
+// eight consecutive elements starting at element 8 c
+template <int DT>
+__device__ __forceinline__ void load8(const void* x, size_t c, float (&f)[8]) {
+    if constexpr (DT == kF32) {
+        const float4* p = reinterpret_cast<const float4*>(x) + 2 * c;
+        const float4 a = p[0], b = p[1];
+        f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+    } else {
+        const uint4 w = reinterpret_cast<const uint4*>(x)[c];
+        const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if constexpr (DT == kBF16) {
+                f[2 * i] = __uint_as_float(u[i] << 16);
+                f[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
+            } else {
+                const float2 p = __half22float2(*reinterpret_cast<const __half2*>(&u[i]));
+                f[2 * i] = p.x;
+                f[2 * i + 1] = p.y;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ uint32_t search16(const float* thr, float xhat) {
+    uint32_t q = 0;
+#pragma unroll
+    for (int s = 8; s >= 1; s >>= 1) q += (thr[q + s - 1] < xhat) ? s : 0;
+    return q;
+}
+
+// xhat = RN32(x / d).  16-bit inputs with d in [2^-64, 2^64]: q0 = RN(x r), e = x - d q0 (exact
+// in one fma), q = RN(q0 + e r) from the approximate reciprocal r; otherwise the IEEE division.
+template <int DT>
+__device__ __forceinline__ float quotient(float x, float d, float r, bool quick) {
+    if (DT != kF32 && quick) {
+        const float q0 = __fmul_rn(x, r);
+        const float e = __fmaf_rn(-d, q0, x);
+        return __fmaf_rn(e, r, q0);
+    }
+    return __fdiv_rn(x, d);
+}
+
+__device__ __forceinline__ void fill_tables(const Tables4& tab, float* thr, float* val) {
+    if (threadIdx.x < 16) { thr[threadIdx.x] = tab.thr[threadIdx.x]; val[threadIdx.x] = tab.val[threadIdx.x]; }
+    __syncthreads();
+}
+
+template <int DT>
+__global__ void __launch_bounds__(256)
+q4_fast(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restrict__ absmax, size_t nchunks, int lpb /* lanes per block = block / 8 */,
+        int log2_lpb, const __grid_constant__ Tables4 tab) {
+    __shared__ float thr[16], val[16];
+    fill_tables(tab, thr, val);
+    const size_t stride = size_t(gridDim.x) * 256;
+    // two chunks per trip, both loaded before either is used; the trip count is the same for the
+    // whole warp because chunk indices start at a multiple of 32 and the shuffles need every lane
+    const size_t first = size_t(blockIdx.x) * 256 + threadIdx.x;
+    const size_t warp_first = first - (threadIdx.x & 31);
+    for (size_t c0 = first, w0 = warp_first; w0 < nchunks; c0 += 2 * stride, w0 += 2 * stride) {
+        float f[2][8];
+        size_t c[2] = {c0, c0 + stride};
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            if (c[u] < nchunks) load8<DT>(x, c[u], f[u]);
+            else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) f[u][i] = 0.0f;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            float a = 0.0f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) a = fmaxf(a, fabsf(f[u][i]));
+            for (int s = 1; s < lpb; s <<= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, s));
+            const float d = (a != 0.0f) ? a : 1.0f;
+            const bool quick = (d >= 5.421010862427522e-20f) && (d <= 1.8446744073709552e19f);
+            float r;
+            asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(d));
+            uint32_t word = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) word |= search16(thr, quotient<DT>(f[u][i], d, r, quick)) << (4 * i);
+            if (c[u] < nchunks) {
+                reinterpret_cast<uint32_t*>(packed)[c[u]] = word;
+                if ((c[u] & size_t(lpb - 1)) == 0) absmax[c[u] >> log2_lpb] = a;
+            }
+        }
+    }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(256)
+q4_wide(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restrict__ absmax, size_t nblocks, int chunks_per_block,
+        const __grid_constant__ Tables4 tab) {
+    __shared__ float thr[16], val[16];
+    fill_tables(tab, thr, val);
+    const int lane = threadIdx.x & 31;
+    const size_t wstride = size_t(gridDim.x) * 8;
+    for (size_t b = size_t(blockIdx.x) * 8 + (threadIdx.x >> 5); b < nblocks; b += wstride) {
+        const size_t cbase = b * size_t(chunks_per_block);
+        float a = 0.0f;
+        for (int k = lane; k < chunks_per_block; k += 32) {
+            float f[8];
+            load8<DT>(x, cbase + k, f);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) a = fmaxf(a, fabsf(f[i]));
+        }
+#pragma unroll
+        for (int s = 1; s < 32; s <<= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, s));
+        const float d = (a != 0.0f) ? a : 1.0f;
+        const bool quick = (d >= 5.421010862427522e-20f) && (d <= 1.8446744073709552e19f);
+        float r;
+        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(d));
+        for (int k = lane; k < chunks_per_block; k += 32) {
+            float f[8];
+            load8<DT>(x, cbase + k, f);
+            uint32_t word = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) word |= search16(thr, quotient<DT>(f[i], d, r, quick)) << (4 * i);
+            reinterpret_cast<uint32_t*>(packed)[cbase + k] = word;
+        }
+        if (lane == 0) absmax[b] = a;
+    }
+}
+
+// General quantize, step 1: absmax of blocks first_block .. (one warp per block).
+template <int DT>
+__global__ void __launch_bounds__(256)
+q4_general_absmax(const void* __restrict__ x, float* __restrict__ absmax, size_t n, size_t block, size_t first_block) {
+    const int lane = threadIdx.x & 31;
+    const size_t nb = (n + block - 1) / block;
+    for (size_t b = first_block + size_t(blockIdx.x) * 8 + (threadIdx.x >> 5); b < nb; b += size_t(gridDim.x) * 8) {
+        const size_t lo = b * block, hi = (lo + block < n) ? lo + block : n;
+        float a = 0.0f;
+        for (size_t i = lo + lane; i < hi; i += 32) a = fmaxf(a, fabsf(load1<DT>(x, i)));
+#pragma unroll
+        for (int s = 1; s < 32; s <<= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, s));
+        if (lane == 0) absmax[b] = a;
+    }
+}
+
+// General quantize, step 2: one thread per output byte from byte first_byte on.
+template <int DT>
+__global__ void __launch_bounds__(256)
+q4_general_codes(const void* __restrict__ x, const float* __restrict__ absmax, uint8_t* __restrict__ packed, size_t n, size_t block,
+                 size_t first_byte, const __grid_constant__ Tables4 tab) {
+    __shared__ float thr[16], val[16];
+    fill_tables(tab, thr, val);
+    const size_t nbytes = (n + 1) / 2;
+    for (size_t j = first_byte + size_t(blockIdx.x) * 256 + threadIdx.x; j < nbytes; j += size_t(gridDim.x) * 256) {
+        uint32_t byte = 0;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const size_t i = 2 * j + h;
+            if (i < n) {
+                const float a = absmax[i / block];
+                const float d = (a != 0.0f) ? a : 1.0f;
+                byte |= search16(thr, __fdiv_rn(load1<DT>(x, i), d)) << (4 * h);
+            }
+        }
+        packed[j] = uint8_t(byte);
+    }
+}
+
+__device__ __forceinline__ void st32(void* p, const uint32_t (&w)[8]) {
+    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]),
+                 "r"(w[6]), "r"(w[7]) : "memory");
+}
+
+// 16 elements per thread; block is a power of two >= 16, so the 16 share one absmax.
+template <int DT>
+__global__ void __launch_bounds__(256)
+dq4_fast(const uint8_t* __restrict__ packed, const float* __restrict__ absmax, void* __restrict__ y, size_t n16, int log2_block,
+         const __grid_constant__ Tables4 tab) {
+    __shared__ float thr[16], val[16];
+    fill_tables(tab, thr, val);
+    for (size_t c = size_t(blockIdx.x) * 256 + threadIdx.x; c < n16; c += size_t(gridDim.x) * 256) {
+        const uint2 w = reinterpret_cast<const uint2*>(packed)[c];
+        const float a = __ldg(absmax + ((c * 16) >> log2_block));
+        float v[16];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            v[i] = __fmul_rn(val[(w.x >> (4 * i)) & 15u], a);
+            v[8 + i] = __fmul_rn(val[(w.y >> (4 * i)) & 15u], a);
+        }
+        if constexpr (DT == kF32) {
+            uint32_t lo[8], hi[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { lo[i] = __float_as_uint(v[i]); hi[i] = __float_as_uint(v[8 + i]); }
+            st32(static_cast<char*>(y) + c * 64, lo);
+            st32(static_cast<char*>(y) + c * 64 + 32, hi);
+        } else {
+            uint32_t pk[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if constexpr (DT == kBF16) {
+                    const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+                    pk[i] = *reinterpret_cast<const uint32_t*>(&h);
+                } else {
+                    const __half2 h = __floats2half2_rn(v[2 * i], v[2 * i + 1]);
+                    pk[i] = *reinterpret_cast<const uint32_t*>(&h);
+                }
+            }
+            st32(static_cast<char*>(y) + c * 32, pk);
+        }
+    }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(256)
+dq4_general(const uint8_t* __restrict__ packed, const float* __restrict__ absmax, void* __restrict__ y, size_t n, size_t block, size_t first_elem,
+            const __grid_constant__ Tables4 tab) {
+    __shared__ float thr[16], val[16];
+    fill_tables(tab, thr, val);
+    for (size_t i = first_elem + size_t(blockIdx.x) * 256 + threadIdx.x; i < n; i += size_t(gridDim.x) * 256) {
+        const uint32_t code = (packed[i >> 1] >> (4 * (i & 1))) & 15u;
+        store1<DT>(y, i, __fmul_rn(val[code], absmax[i / block]));
+    }
+}
+
+}  // namespace bq4k

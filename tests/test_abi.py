@@ -26,7 +26,41 @@ def test_every_declared_symbol_is_exported(bq):
 
 
 def test_every_header_is_covered():
-    assert sorted(os.listdir(os.path.join(ROOT, "include"))) == ["bq.h", "mmd.h"]
+    assert sorted(os.listdir(os.path.join(ROOT, "include"))) == ["bq.h", "bq4.h", "mmd.h"]
+
+
+def test_every_declared_bq4_symbol_is_exported(bq):
+    from paper_2407_19775_b200 import binding, bq4
+    L = binding.lib()
+    names = _declared("bq4.h", "bq4_")
+    assert {"bq4_make_codebook", "bq4_free_codebook", "bq4_quantize", "bq4_dequantize"} == set(names)
+    for name in names:
+        assert hasattr(L, name), name
+    assert set(bq4.SYMBOLS) == set(names)
+
+
+def test_bq4_argument_errors_and_host_codebook(bq):
+    import numpy as np
+    from paper_2407_19775_b200 import bq4
+    from oracle import bq4_oracle
+    L = bq4._lib()
+    one = ctypes.c_void_p(64)        # never dereferenced: every call below fails a check first
+    assert L.bq4_quantize(one, 9, 4, 64, one, one, one, None) == 2
+    assert L.bq4_quantize(one, 0, 4, 0, one, one, one, None) == 3
+    assert L.bq4_quantize(one, 0, 1 << 41, 64, one, one, one, None) == 4
+    assert L.bq4_quantize(one, 0, 4, 64, None, one, one, None) == 5
+    assert L.bq4_quantize(None, 0, 0, 64, one, None, None, None) == 0
+    assert L.bq4_quantize(None, 0, 4, 64, one, one, one, None) == 1
+    assert L.bq4_dequantize(one, one, 4, 64, one, None, 0, None) == 1
+    assert L.bq4_dequantize(one, one, 4, 64, one, one, 7, None) == 2
+    out = ctypes.c_void_p()
+    assert L.bq4_make_codebook(5, None, None, ctypes.byref(out)) == 5
+    assert L.bq4_make_codebook(0, None, None, None) == 1
+    assert L.bq4_free_codebook(None) == 0
+    cb = bq4.Codebook4()             # host only: no device is touched
+    assert np.array_equal(cb.values.view(np.uint32), bq4_oracle.make_codebook().view(np.uint32))
+    bad = cb.values.copy(); bad[3] = bad[4]
+    assert L.bq4_make_codebook(1, bad.ctypes.data, None, ctypes.byref(out)) == 5
 
 
 def test_every_declared_mmd_symbol_is_exported(bq):

@@ -1,0 +1,135 @@
+"""GPU parity of the 4-bit variant against its CPU oracle, through the C ABI: packed codes,
+absmax and dequantised output are compared bit for bit (integer and byte work; the floating
+point that decides a code is the same correctly rounded fp32 quotient on both sides)."""
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+from helpers import frac_of, round_down32
+from oracle import bq4_oracle as o4
+from paper_2407_19775_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+F32, F16, BF16 = 0, 1, 2
+DT = {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}
+
+
+def bits(t: torch.Tensor) -> np.ndarray:
+    return workloads.as_numpy_bits(t.cpu())
+
+
+def check(bq, x: torch.Tensor, block: int, ydt=None):
+    """x: a CPU tensor (any shape).  Quantize and dequantize on the GPU, compare with the oracle."""
+    cb = bq.Codebook4()
+    cb_ref = o4.make_codebook()
+    flat = x.reshape(-1)
+    dt = DT[flat.dtype]
+    p_ref, a_ref = o4.quantize(bits(flat), dt, block, cb_ref)
+    xd = flat.cuda()
+    p, a = bq.bq4_quantize(xd, block, cb)
+    torch.cuda.synchronize()
+    assert np.array_equal(p.cpu().numpy(), p_ref)
+    assert np.array_equal(a.cpu().numpy().view(np.uint32), a_ref.view(np.uint32))
+    for out in ([flat.dtype, torch.float32] if ydt is None else [ydt]):
+        y = bq.bq4_dequantize(p, a, flat.numel(), block, cb, out)
+        y_ref = o4.dequantize(p_ref, a_ref, flat.numel(), block, cb_ref, DT[out])
+        got = bits(y)
+        assert np.array_equal(got.view(np.uint32 if out == torch.float32 else np.uint16), y_ref.view(np.uint32 if out == torch.float32 else np.uint16))
+    return p_ref, a_ref
+
+
+@pytest.mark.parametrize("name,rows,block", [("tiny", None, 64), ("prefill7b", 96, 256), ("decode70b", 64, 64), ("moe_prefill", 40, 2048),
+                                             ("sweep1g", 24, 128), ("sweep1g", 24, 8), ("sweep1g", 16, 65536), ("prefill7b", 40, 16)])
+def test_workloads(bq, name, rows, block):
+    x = workloads.make(name, rows=rows)
+    check(bq, x, block)
+
+
+@pytest.mark.parametrize("tdt", [torch.float32, torch.bfloat16, torch.float16])
+def test_ragged_and_general_cases(bq, tdt):
+    g = torch.Generator().manual_seed(7)
+    x = (torch.randn(5000, generator=g) * 1.5).to(tdt)
+    x[100:164] = 0
+    for n, block in [(4999, 64), (5000, 24), (37, 64), (1, 8), (2, 1), (777, 3), (4097, 4096), (513, 512), (1023, 32), (5000, 131072)]:
+        check(bq, x[:n].clone(), block)
+
+
+def test_unaligned_pointers(bq):
+    cb = bq.Codebook4()
+    cb_ref = o4.make_codebook()
+    g = torch.Generator().manual_seed(9)
+    base = (torch.randn(4096 + 8, generator=g)).to(torch.bfloat16)
+    xd = base.cuda()[3:3 + 4096]                                 # 6 bytes off a 16-byte boundary
+    p_ref, a_ref = o4.quantize(bits(base[3:3 + 4096]), BF16, 64, cb_ref)
+    pbuf = torch.empty(2048 + 4, dtype=torch.uint8, device="cuda")
+    p, a = bq.bq4_quantize(xd, 64, cb, packed_out=pbuf[1:2049])
+    assert np.array_equal(p.cpu().numpy(), p_ref) and np.array_equal(a.cpu().numpy(), a_ref)
+    ybuf = torch.empty(4096 + 8, dtype=torch.bfloat16, device="cuda")
+    y = bq.bq4_dequantize(p, a, 4096, 64, cb, torch.bfloat16, y_out=ybuf[5:5 + 4096])
+    assert np.array_equal(bits(y), o4.dequantize(p_ref, a_ref, 4096, 64, cb_ref, BF16))
+
+
+def test_breakpoints_and_division(bq):
+    """Values on both sides of every breakpoint, with absmax 1 (block of 2: the absmax element and the value), and pairs
+    whose quotient a multiplication by the reciprocal would move across a breakpoint."""
+    cb_ref = o4.make_codebook()
+    xs = []
+    for j in range(15):
+        lo = round_down32((frac_of(cb_ref[j]) + frac_of(cb_ref[j + 1])) / 2)
+        xs += [1.0, float(lo), 1.0, float(np.nextafter(lo, np.float32(np.inf)))]
+    check(bq, torch.tensor(xs, dtype=torch.float32), 2)
+    rng = np.random.default_rng(0)
+    vals = []
+    for j in range(15):
+        lo = round_down32((frac_of(cb_ref[j]) + frac_of(cb_ref[j + 1])) / 2)
+        a = (1.0 + rng.random(6000)).astype(np.float32)
+        for target in (lo, np.nextafter(lo, np.float32(np.inf))):
+            x = (target * a).astype(np.float32)
+            differ = ((x / a).astype(np.float32) != (x * (np.float32(1) / a)).astype(np.float32)) & (np.abs(x) <= a)
+            for i in np.flatnonzero(differ)[:3]:
+                vals += [float(a[i]), float(x[i])]
+    assert len(vals) > 40
+    check(bq, torch.tensor(vals, dtype=torch.float32), 2)
+    # 16-bit absmax significands through the reciprocal route: every bf16 significand as the divisor
+    sig = torch.arange(128, 256, dtype=torch.float32) / 128.0
+    rows = torch.cat([sig[:, None], sig[:, None] * torch.linspace(-1, 1, 63)[None, :]], dim=1).to(torch.bfloat16)
+    check(bq, rows, 64)
+
+
+def test_scales_outside_the_reciprocal_window(bq):
+    g = torch.Generator().manual_seed(11)
+    x = torch.randn(8, 256, generator=g)
+    x[0] *= 1e-30; x[1] *= 1e30; x[2] *= 2.0 ** -64; x[3] *= 2.0 ** 64; x[4] *= 2.0 ** -65; x[5] = 0
+    check(bq, x.to(torch.bfloat16), 256)
+    check(bq, x.to(torch.bfloat16), 1024)
+    check(bq, x, 64)
+
+
+def test_user_codebook(bq):
+    lin = np.linspace(-1, 1, 16).astype(np.float32)              # a uniform map (no exact zero: allowed for user maps)
+    cb = bq.Codebook4(bq.USER, lin)
+    g = torch.Generator().manual_seed(13)
+    x = torch.randn(4096, generator=g).to(torch.float16)
+    p_ref, a_ref = o4.quantize(bits(x), F16, 128, lin)
+    p, a = bq.bq4_quantize(x.cuda(), 128, cb)
+    assert np.array_equal(p.cpu().numpy(), p_ref) and np.array_equal(a.cpu().numpy(), a_ref)
+    y = bq.bq4_dequantize(p, a, 4096, 128, cb, torch.float16)
+    assert np.array_equal(bits(y), o4.dequantize(p_ref, a_ref, 4096, 128, lin, F16))
+    with pytest.raises(bq.BqError):
+        bq.Codebook4(bq.USER, lin[::-1].copy())
+
+
+def test_kv_cache_shaped_tensor(bq):
+    """The other large activation-like tensor of the paper's system is the KV cache (2 x head_dim x heads x layers values
+    per token): the same calls with one block per head vector."""
+    g = torch.Generator().manual_seed(17)
+    kv = (torch.randn(2, 4, 8, 96, 128, generator=g) * 0.7).to(torch.bfloat16)      # [k/v, layers, heads, tokens, head_dim]
+    kv[:, :, 3, :, 17] *= 12                                                        # a heavy channel in one head
+    check(bq, kv, 128)
+    cb8 = bq.Codebook()
+    import oracle
+    ref_c, ref_a = oracle.quantize(bits(kv.reshape(-1)), BF16, 128, oracle.make_codebook())
+    c, a = bq.bq_quantize(kv.cuda().reshape(-1), 128, cb8)
+    assert np.array_equal(c.cpu().numpy(), ref_c) and np.array_equal(a.cpu().numpy(), ref_a)
