@@ -66,6 +66,37 @@ void build_thresholds(bq4k::Tables4& t) {
     t.thr[15] = std::numeric_limits<float>::infinity();
 }
 
+uint32_t f2u(float f) { uint32_t u; std::memcpy(&u, &f, 4); return u; }
+
+// The folded search tables (see Tables4); left invalid when the codebook does not mirror or two thresholds share a cell.
+void build_folded(bq4k::Tables4& t) {
+    t.folded = 0;
+    std::memset(t.entry, 0, sizeof t.entry);
+    if (t.val[7] != 0.0f) return;
+    for (int j = 0; j < 7; ++j)
+        if (t.val[j] != -t.val[14 - j]) return;
+    uint32_t tk[8];
+    for (int p = 0; p < 8; ++p) {
+        const double mid = (double(t.val[7 + p]) + double(t.val[8 + p])) / 2.0;            // exact
+        float f = float(mid);
+        if (double(f) > mid) f = std::nextafterf(f, 0.0f);                                 // positive: toward zero = toward -inf
+        tk[p] = 2u * f2u(f) + ((double(f) != mid) ? 1u : 0u);
+        if (tk[p] <= bq4k::kFoldKeyLow || tk[p] >= 0x7F000000u) return;                    // must lie inside the table's span
+    }
+    for (int i = 0; i < bq4k::kFoldCells; ++i) {
+        const uint32_t S = (bq4k::kFoldCellBase + uint32_t(i)) << 21;
+        uint32_t p0 = 0, inside = 0, off = 0x1FFFFFu;
+        for (int p = 0; p < 8; ++p) {
+            if (tk[p] < S) ++p0;
+            else if (tk[p] - S < (1u << 21)) { ++inside; off = tk[p] - S; }
+        }
+        if (inside > 1) return;
+        if (inside == 1 && off == 0x1FFFFFu) return;                                       // would look like an empty cell
+        t.entry[i] = (((7u + p0) << 24) | 0xE00000u | (0x1FFFFFu - off)) - S;
+    }
+    t.folded = 1;
+}
+
 int sm_count_of_current(int* sms) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -83,9 +114,13 @@ cudaError_t quantize_t(const void* x, size_t n, size_t B, const bq4k::Tables4& t
         const size_t nblocks = n / B, n_full = nblocks * B;
         if (l2 <= 8) {
             const size_t nchunks = n_full / 8;
-            bq4k::q4_fast<DT><<<capped((nchunks + 511) / 512, size_t(sms) * 8), 256, 0, s>>>(x, packed, absmax, nchunks, int(B / 8), l2 - 3, tab);
+            const unsigned grid = capped((nchunks + 511) / 512, size_t(sms) * 8);
+            if (tab.folded) bq4k::q4_fast<DT, true><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, int(B / 8), l2 - 3, tab);
+            else bq4k::q4_fast<DT, false><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, int(B / 8), l2 - 3, tab);
         } else {
-            bq4k::q4_wide<DT><<<capped((nblocks + 7) / 8, size_t(sms) * 8), 256, 0, s>>>(x, packed, absmax, nblocks, int(B / 8), tab);
+            const unsigned grid = capped((nblocks + 7) / 8, size_t(sms) * 8);
+            if (tab.folded) bq4k::q4_wide<DT, true><<<grid, 256, 0, s>>>(x, packed, absmax, nblocks, int(B / 8), tab);
+            else bq4k::q4_wide<DT, false><<<grid, 256, 0, s>>>(x, packed, absmax, nblocks, int(B / 8), tab);
         }
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
@@ -142,6 +177,7 @@ int bq4_make_codebook(int kind, const float* user_values16, float* host_values_o
         return BQ_ERR_CODEBOOK;
     }
     build_thresholds(cb->tab);
+    build_folded(cb->tab);
     if (host_values_out16) std::memcpy(host_values_out16, cb->tab.val, 16 * sizeof(float));
     *out = cb;
     return BQ_OK;

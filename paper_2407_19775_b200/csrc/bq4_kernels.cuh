@@ -25,9 +25,23 @@ namespace bq4k {
 
 enum { kF32 = 0, kF16 = 1, kBF16 = 2 };
 
+constexpr int kFoldCells = 73;          // cells of 2^21 keys from the key of 2^-9 up to the key of -1.0
+constexpr uint32_t kFoldKeyLow = 0x76000000u;      // key of +2^-9 (twice its bit pattern)
+constexpr uint32_t kFoldCellBase = kFoldKeyLow >> 21;
+
 struct Tables4 {
     float thr[16];      // [0..14] midpoints rounded toward -inf, [15] = +inf
     float val[16];      // the codebook
+    // Folded search, valid when `folded` is set (a codebook that mirrors around code 7 with one extra top value, such as
+    // the dynamic tree).  key = rotate-left-by-one of xhat's bits = 2 bits(|xhat|) + sign.  With the threshold keys
+    // TK[p] = 2 bits(round_down(theta_p)) + (theta_p is not an fp32) of the 8 positive midpoints, P = #{TK[p] < key} is
+    // #{theta_p < |xhat|} for xhat >= 0 and #{theta_p <= |xhat|} for xhat < 0: the tie rule on either side.  Keys are
+    // clamped from below to kFoldKeyLow and cut into cells of 2^21 keys (exponent and 3 fraction bits); no cell holds
+    // two thresholds.  The entry of the cell that starts at key S, with P0 thresholds below S and the threshold TK in it, is
+    //     E = ((7 + P0) << 24 | 0xE00000 | (0x1FFFFF - (TK - S))) - S
+    // so that (E + key) >> 24 = 7 + P0 + [key > TK]: one lookup and one addition.  (No threshold in the cell: TK - S = 0x1FFFFF.)
+    uint32_t entry[kFoldCells];
+    int folded;
 };
 
 template <int DT>
@@ -67,6 +81,28 @@ __device__ __forceinline__ void load8(const void* x, size_t c, float (&f)[8]) {
     }
 }
 
+// the same eight elements from the raw 128-bit words of a chunk (one word for 16-bit types, two for fp32)
+template <int DT, int W>
+__device__ __forceinline__ void widen_chunk(const uint4 (&w)[W], float (&f)[8]) {
+    if constexpr (DT == kF32) {
+        f[0] = __uint_as_float(w[0].x); f[1] = __uint_as_float(w[0].y); f[2] = __uint_as_float(w[0].z); f[3] = __uint_as_float(w[0].w);
+        f[4] = __uint_as_float(w[1].x); f[5] = __uint_as_float(w[1].y); f[6] = __uint_as_float(w[1].z); f[7] = __uint_as_float(w[1].w);
+    } else {
+        const uint32_t u[4] = {w[0].x, w[0].y, w[0].z, w[0].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if constexpr (DT == kBF16) {
+                f[2 * i] = __uint_as_float(u[i] << 16);
+                f[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
+            } else {
+                const float2 p = __half22float2(*reinterpret_cast<const __half2*>(&u[i]));
+                f[2 * i] = p.x;
+                f[2 * i + 1] = p.y;
+            }
+        }
+    }
+}
+
 __device__ __forceinline__ uint32_t search16(const float* thr, float xhat) {
     uint32_t q = 0;
 #pragma unroll
@@ -86,46 +122,77 @@ __device__ __forceinline__ float quotient(float x, float d, float r, bool quick)
     return __fdiv_rn(x, d);
 }
 
+// code of xhat through the folded table; `ent_lane` is this lane's column of the per-lane replicated entries, rebased
+// by the index of the first cell.  7 + P for xhat >= 0; 7 - min(P, 7) for xhat < 0 (there is no code for -1.0).
+__device__ __forceinline__ uint32_t search_folded16(uint32_t ent_lane, float xhat) {
+    const uint32_t b = __float_as_uint(xhat);
+    const uint32_t key = max(__funnelshift_l(b, b, 1), kFoldKeyLow);
+    uint32_t e;
+    asm("ld.shared.u32 %0, [%1];" : "=r"(e) : "r"(ent_lane + (key >> 21) * 128u));
+    const uint32_t c = (e + key) >> 24;
+    return (b >> 31) ? 14u - min(c, 14u) : c;
+}
+
 __device__ __forceinline__ void fill_tables(const Tables4& tab, float* thr, float* val) {
     if (threadIdx.x < 16) { thr[threadIdx.x] = tab.thr[threadIdx.x]; val[threadIdx.x] = tab.val[threadIdx.x]; }
     __syncthreads();
 }
 
-template <int DT>
+template <int DT, bool FOLDED>
 __global__ void __launch_bounds__(256)
 q4_fast(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restrict__ absmax, size_t nchunks, int lpb /* lanes per block = block / 8 */,
         int log2_lpb, const __grid_constant__ Tables4 tab) {
     __shared__ float thr[16], val[16];
+    __shared__ __align__(128) uint32_t ent[FOLDED ? kFoldCells * 32 : 1];      // every entry once per lane, in that lane's bank
     fill_tables(tab, thr, val);
+    uint32_t ent_lane = 0;
+    if constexpr (FOLDED) {
+        for (int i = threadIdx.x; i < kFoldCells * 32; i += 256) ent[i] = tab.entry[i >> 5];
+        __syncthreads();
+        ent_lane = uint32_t(__cvta_generic_to_shared(ent)) + (threadIdx.x & 31) * 4u - kFoldCellBase * 128u;
+    }
     const size_t stride = size_t(gridDim.x) * 256;
-    // two chunks per trip, both loaded before either is used; the trip count is the same for the
-    // whole warp because chunk indices start at a multiple of 32 and the shuffles need every lane
+    // Two chunks per trip; the loads of the next trip are issued before this trip's arithmetic.  The trip count is the
+    // same for the whole warp because chunk indices start at a multiple of 32 and the shuffles need every lane.
     const size_t first = size_t(blockIdx.x) * 256 + threadIdx.x;
     const size_t warp_first = first - (threadIdx.x & 31);
-    for (size_t c0 = first, w0 = warp_first; w0 < nchunks; c0 += 2 * stride, w0 += 2 * stride) {
-        float f[2][8];
-        size_t c[2] = {c0, c0 + stride};
+    constexpr int W = (DT == kF32) ? 2 : 1;                      // 128-bit loads per chunk
+    uint4 nxt[2][W];
+    auto fetch = [&](size_t c0) {
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
-            if (c[u] < nchunks) load8<DT>(x, c[u], f[u]);
-            else {
+            const size_t c = c0 + size_t(u) * stride;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) f[u][i] = 0.0f;
-            }
+            for (int k = 0; k < W; ++k)
+                nxt[u][k] = (c < nchunks) ? __ldg(reinterpret_cast<const uint4*>(x) + c * W + k) : make_uint4(0, 0, 0, 0);
         }
+    };
+    if (warp_first < nchunks) fetch(first);
+    for (size_t c0 = first, w0 = warp_first; w0 < nchunks; c0 += 2 * stride, w0 += 2 * stride) {
+        float f[2][8];
+        const size_t c[2] = {c0, c0 + stride};
+#pragma unroll
+        for (int u = 0; u < 2; ++u) widen_chunk<DT>(nxt[u], f[u]);
+        if (w0 + 2 * stride < nchunks) fetch(c0 + 2 * stride);
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
             float a = 0.0f;
 #pragma unroll
             for (int i = 0; i < 8; ++i) a = fmaxf(a, fabsf(f[u][i]));
-            for (int s = 1; s < lpb; s <<= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, s));
+#pragma unroll
+            for (int s = 1; s < 32; s <<= 1)
+                if (s < lpb) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, s));       // uniform over the warp
             const float d = (a != 0.0f) ? a : 1.0f;
             const bool quick = (d >= 5.421010862427522e-20f) && (d <= 1.8446744073709552e19f);
             float r;
             asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(d));
             uint32_t word = 0;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) word |= search16(thr, quotient<DT>(f[u][i], d, r, quick)) << (4 * i);
+            for (int i = 0; i < 8; ++i) {
+                const float xhat = quotient<DT>(f[u][i], d, r, quick);
+                const uint32_t q = FOLDED ? search_folded16(ent_lane, xhat) : search16(thr, xhat);
+                word |= q << (4 * i);
+            }
             if (c[u] < nchunks) {
                 reinterpret_cast<uint32_t*>(packed)[c[u]] = word;
                 if ((c[u] & size_t(lpb - 1)) == 0) absmax[c[u] >> log2_lpb] = a;
@@ -134,12 +201,19 @@ q4_fast(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restr
     }
 }
 
-template <int DT>
+template <int DT, bool FOLDED>
 __global__ void __launch_bounds__(256)
 q4_wide(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restrict__ absmax, size_t nblocks, int chunks_per_block,
         const __grid_constant__ Tables4 tab) {
     __shared__ float thr[16], val[16];
+    __shared__ __align__(128) uint32_t ent[FOLDED ? kFoldCells * 32 : 1];
     fill_tables(tab, thr, val);
+    uint32_t ent_lane = 0;
+    if constexpr (FOLDED) {
+        for (int i = threadIdx.x; i < kFoldCells * 32; i += 256) ent[i] = tab.entry[i >> 5];
+        __syncthreads();
+        ent_lane = uint32_t(__cvta_generic_to_shared(ent)) + (threadIdx.x & 31) * 4u - kFoldCellBase * 128u;
+    }
     const int lane = threadIdx.x & 31;
     const size_t wstride = size_t(gridDim.x) * 8;
     for (size_t b = size_t(blockIdx.x) * 8 + (threadIdx.x >> 5); b < nblocks; b += wstride) {
@@ -162,7 +236,11 @@ q4_wide(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restr
             load8<DT>(x, cbase + k, f);
             uint32_t word = 0;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) word |= search16(thr, quotient<DT>(f[i], d, r, quick)) << (4 * i);
+            for (int i = 0; i < 8; ++i) {
+                const float xhat = quotient<DT>(f[i], d, r, quick);
+                const uint32_t q = FOLDED ? search_folded16(ent_lane, xhat) : search16(thr, xhat);
+                word |= q << (4 * i);
+            }
             reinterpret_cast<uint32_t*>(packed)[cbase + k] = word;
         }
         if (lane == 0) absmax[b] = a;

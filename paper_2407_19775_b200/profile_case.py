@@ -12,13 +12,13 @@ import argparse
 
 import torch
 
-from . import Codebook, bq_dequantize, bq_quantize, bq_roundtrip, workloads
+from . import Codebook, Codebook4, bq4_dequantize, bq4_quantize, bq_dequantize, bq_quantize, bq_roundtrip, workloads
 
 
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="sweep1g")
-    ap.add_argument("--op", default="roundtrip", choices=["quantize", "dequantize", "roundtrip", "roundtrip_side"])
+    ap.add_argument("--op", default="roundtrip", choices=["quantize", "dequantize", "roundtrip", "roundtrip_side", "quantize4", "dequantize4"])
     ap.add_argument("--block", type=int, default=4096)
     ap.add_argument("--rows", type=int, default=8192)
     ap.add_argument("--launches", type=int, default=3)
@@ -33,8 +33,12 @@ def main() -> None:
     codes = torch.empty(n, dtype=torch.uint8, device=dev)
     absmax = torch.empty((n + args.block - 1) // args.block, dtype=torch.float32, device=dev)
     y = torch.empty_like(x)
+    cb4 = Codebook4()
+    packed = codes[: (n + 1) // 2]
     if args.op == "dequantize":
         bq_quantize(x, args.block, cb, codes, absmax)
+    if args.op == "dequantize4":
+        bq4_quantize(x, args.block, cb4, packed, absmax)
     torch.cuda.synchronize()
     for i in range(args.launches):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -43,6 +47,10 @@ def main() -> None:
             bq_quantize(x, args.block, cb, codes, absmax)
         elif args.op == "dequantize":
             bq_dequantize(codes, absmax, args.block, cb, x.dtype, y)
+        elif args.op == "quantize4":
+            bq4_quantize(x, args.block, cb4, packed, absmax)
+        elif args.op == "dequantize4":
+            bq4_dequantize(packed, absmax, n, args.block, cb4, x.dtype, y)
         elif args.op == "roundtrip":
             bq_roundtrip(x, args.block, cb, y_out=y)
         else:

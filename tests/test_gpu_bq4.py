@@ -98,6 +98,31 @@ def test_breakpoints_and_division(bq):
     check(bq, rows, 64)
 
 
+def test_vectorised_search_on_and_around_every_breakpoint(bq):
+    """The vectorised kernels find the code with one table lookup on the bits of xhat.  Blocks of 8 whose first element is
+    1.0 (so xhat = x) carry, for every breakpoint and both signs, the 2049 floats around it; plus a dense sweep of [-1, 1]
+    and the values next to zero and to the table's lower end."""
+    cb_ref = o4.make_codebook()
+    vals = []
+    for j in range(15):
+        lo = round_down32((frac_of(cb_ref[j]) + frac_of(cb_ref[j + 1])) / 2)
+        u = np.float32(lo).view(np.uint32).astype(np.int64)
+        vals.append((u + np.arange(-1024, 1025)).astype(np.uint32).view(np.float32))
+    vals.append(np.linspace(-1, 1, 200001).astype(np.float32))
+    vals.append((np.float32(2.0 ** -9).view(np.uint32).astype(np.int64) + np.arange(-64, 65)).astype(np.uint32).view(np.float32))
+    vals.append(np.array([0.0, -0.0, 1e-45, -1e-45, 1e-30, -1e-30, 1.0, -1.0, 0.99999994, -0.99999994], np.float32))
+    v = np.concatenate(vals)
+    v = np.concatenate([v, -v])
+    v = v[np.abs(v) <= 1]
+    v = v[: (v.size // 7) * 7].reshape(-1, 7)
+    x = np.concatenate([np.ones((v.shape[0], 1), np.float32), v], axis=1)       # [1.0, seven values] per block of 8
+    check(bq, torch.from_numpy(x), 8, ydt=torch.float32)
+    x16 = np.concatenate([np.ones((v.shape[0], 1), np.float32), v], axis=1).reshape(-1)
+    x16 = x16[: (x16.size // 1024) * 1024]                                      # the same through the one-warp-per-block kernel
+    x16.reshape(-1, 1024)[:, 0] = 1.0
+    check(bq, torch.from_numpy(x16), 1024, ydt=torch.float32)
+
+
 def test_scales_outside_the_reciprocal_window(bq):
     g = torch.Generator().manual_seed(11)
     x = torch.randn(8, 256, generator=g)
