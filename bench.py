@@ -251,6 +251,36 @@ def run_ours(args):
             den += (xs ** 2).sum(dtype=torch.float64)
         quality[f"b{b}"] = {"compression_ratio": round(2 * b / (b + 4), 3), "rel_rms_error": round(float((num / den).sqrt().item()), 5)}
 
+    # the 4-bit variant of the same path (16-entry codebook, two codes per byte) on the same tensor
+    cb4 = bq.Codebook4()
+    bq4 = {}
+    for b in (64, 1024):
+        packed = codes[: n // 2]
+        times = {}
+        for op, fn in (("quantize4", lambda: bq.bq4_quantize(x, b, cb4, packed, absmax[b])),
+                       ("dequantize4", lambda: bq.bq4_dequantize(packed, absmax[b], n, b, cb4, w.dtype, y))):
+            for _ in range(3):
+                fn()
+            ev = []
+            for _ in range(10):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); fn(); e1.record()
+                ev.append((e0, e1))
+            torch.cuda.synchronize()
+            times[op] = float(np.mean([a.elapsed_time(b_) for a, b_ in ev]))
+        ab = n * 2 + n // 2 + 4 * (n // b)
+        num = torch.zeros((), dtype=torch.float64, device=dev)
+        den = torch.zeros((), dtype=torch.float64, device=dev)
+        for s in range(0, n, 1 << 27):
+            xs, ys = x[s:s + (1 << 27)].float(), y[s:s + (1 << 27)].float()
+            num += ((xs - ys) ** 2).sum(dtype=torch.float64)
+            den += (xs ** 2).sum(dtype=torch.float64)
+        bq4[f"b{b}"] = {"quantize_ms": round(times["quantize4"], 4), "dequantize_ms": round(times["dequantize4"], 4), "algorithmic_bytes": int(ab),
+                        "quantize_frac_of_measured": round(ab / times["quantize4"] / 1e6 / peak, 4),
+                        "dequantize_frac_of_measured": round(ab / times["dequantize4"] / 1e6 / peak, 4),
+                        "compression_ratio": round(2.0 * n / (n / 2 + 4 * (n // b)), 3),
+                        "rel_rms_error": round(float((num / den).sqrt().item()), 5), "gpu_launches": 26}
+
     cpu = cpu_baseline(x_pin, rank) if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
     del x, y, codes, absmax
     torch.cuda.empty_cache()
@@ -265,7 +295,7 @@ def run_ours(args):
                                    "quantize+dequantize+roundtrip per block", "elements": n, "l2": "input (1 GiB) larger than L2, no flush needed",
                        "parallelism": f"replicated x{world}, no collective"},
             "e2e": e2e, "gpu_launches": len(events), "clocks": clocks, "roofline": roofline, "kernels": kernels,
-            "quality": quality, "cpu_baseline": cpu, "mmd": mmd,
+            "quality": quality, "cpu_baseline": cpu, "bq4": bq4, "mmd": mmd,
             "paper_context": "the paper reports no throughput for this path; it states only that hidden-state quantization halves the bandwidth",
         }
         print(json.dumps(line))

@@ -183,14 +183,22 @@ q4_fast(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restr
             for (int s = 1; s < 32; s <<= 1)
                 if (s < lpb) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, s));       // uniform over the warp
             const float d = (a != 0.0f) ? a : 1.0f;
-            const bool quick = (d >= 5.421010862427522e-20f) && (d <= 1.8446744073709552e19f);
+            // one choice of route for the whole warp keeps the per-element code free of branches
+            const bool quick = (DT != kF32) && __all_sync(0xffffffffu, (d >= 5.421010862427522e-20f) && (d <= 1.8446744073709552e19f));
             float r;
             asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(d));
+            float xh[8];
+            if (quick) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) xh[i] = quotient<DT>(f[u][i], d, r, true);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) xh[i] = __fdiv_rn(f[u][i], d);
+            }
             uint32_t word = 0;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                const float xhat = quotient<DT>(f[u][i], d, r, quick);
-                const uint32_t q = FOLDED ? search_folded16(ent_lane, xhat) : search16(thr, xhat);
+                const uint32_t q = FOLDED ? search_folded16(ent_lane, xh[i]) : search16(thr, xh[i]);
                 word |= q << (4 * i);
             }
             if (c[u] < nchunks) {
