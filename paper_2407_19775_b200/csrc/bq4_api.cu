@@ -85,14 +85,17 @@ void build_folded(bq4k::Tables4& t) {
     }
     for (int i = 0; i < bq4k::kFoldCells; ++i) {
         const uint32_t S = (bq4k::kFoldCellBase + uint32_t(i)) << 21;
-        uint32_t p0 = 0, inside = 0, off = 0x1FFFFFu;
-        for (int p = 0; p < 8; ++p) {
-            if (tk[p] < S) ++p0;
-            else if (tk[p] - S < (1u << 21)) { ++inside; off = tk[p] - S; }
+        for (int neg = 0; neg < 2; ++neg) {
+            const int nthr = neg ? 7 : 8;                                                  // no code below -val[14]: the top midpoint is one-sided
+            uint32_t p0 = 0, inside = 0, off = 0x1FFFFFu;
+            for (int p = 0; p < nthr; ++p) {
+                if (tk[p] < S) ++p0;
+                else if (tk[p] - S < (1u << 21)) { ++inside; off = tk[p] - S; }
+            }
+            if (inside > 1) return;
+            if (inside == 1 && off == 0x1FFFFFu) return;                                   // would look like an empty cell
+            t.entry[neg][i] = neg ? ((((7u - p0) << 24) | off) + S + 1u) : ((((7u + p0) << 24) | 0xE00000u | (0x1FFFFFu - off)) - S);
         }
-        if (inside > 1) return;
-        if (inside == 1 && off == 0x1FFFFFu) return;                                       // would look like an empty cell
-        t.entry[i] = (((7u + p0) << 24) | 0xE00000u | (0x1FFFFFu - off)) - S;
     }
     t.folded = 1;
 }
@@ -106,6 +109,26 @@ int sm_count_of_current(int* sms) {
 
 unsigned capped(size_t want, size_t cap) { return unsigned(want < 1 ? 1 : (want > cap ? cap : want)); }
 
+template <int DT, bool FOLDED>
+void launch_q4_fast_f(int log2_lpb, unsigned grid, cudaStream_t s, const void* x, uint8_t* packed, float* absmax, size_t nchunks,
+                      const bq4k::Tables4& tab) {
+    switch (log2_lpb) {
+        case 0: bq4k::q4_fast<DT, FOLDED, 0><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, tab); break;
+        case 1: bq4k::q4_fast<DT, FOLDED, 1><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, tab); break;
+        case 2: bq4k::q4_fast<DT, FOLDED, 2><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, tab); break;
+        case 3: bq4k::q4_fast<DT, FOLDED, 3><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, tab); break;
+        case 4: bq4k::q4_fast<DT, FOLDED, 4><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, tab); break;
+        default: bq4k::q4_fast<DT, FOLDED, 5><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, tab); break;
+    }
+}
+
+template <int DT>
+void launch_q4_fast(int log2_lpb, bool folded, unsigned grid, cudaStream_t s, const void* x, uint8_t* packed, float* absmax, size_t nchunks,
+                    const bq4k::Tables4& tab) {
+    if (folded) launch_q4_fast_f<DT, true>(log2_lpb, grid, s, x, packed, absmax, nchunks, tab);
+    else launch_q4_fast_f<DT, false>(log2_lpb, grid, s, x, packed, absmax, nchunks, tab);
+}
+
 template <int DT>
 cudaError_t quantize_t(const void* x, size_t n, size_t B, const bq4k::Tables4& tab, uint8_t* packed, float* absmax, int sms, cudaStream_t s) {
     size_t done = 0;
@@ -115,8 +138,7 @@ cudaError_t quantize_t(const void* x, size_t n, size_t B, const bq4k::Tables4& t
         if (l2 <= 8) {
             const size_t nchunks = n_full / 8;
             const unsigned grid = capped((nchunks + 511) / 512, size_t(sms) * 8);
-            if (tab.folded) bq4k::q4_fast<DT, true><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, int(B / 8), l2 - 3, tab);
-            else bq4k::q4_fast<DT, false><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, int(B / 8), l2 - 3, tab);
+            launch_q4_fast<DT>(l2 - 3, tab.folded != 0, grid, s, x, packed, absmax, nchunks, tab);
         } else {
             const unsigned grid = capped((nblocks + 7) / 8, size_t(sms) * 8);
             if (tab.folded) bq4k::q4_wide<DT, true><<<grid, 256, 0, s>>>(x, packed, absmax, nblocks, int(B / 8), tab);

@@ -34,13 +34,17 @@ struct Tables4 {
     float val[16];      // the codebook
     // Folded search, valid when `folded` is set (a codebook that mirrors around code 7 with one extra top value, such as
     // the dynamic tree).  key = rotate-left-by-one of xhat's bits = 2 bits(|xhat|) + sign.  With the threshold keys
-    // TK[p] = 2 bits(round_down(theta_p)) + (theta_p is not an fp32) of the 8 positive midpoints, P = #{TK[p] < key} is
+    // TK[p] = 2 bits(round_down(theta_p)) + (theta_p is not an fp32) of the positive midpoints, P = #{TK[p] < key} is
     // #{theta_p < |xhat|} for xhat >= 0 and #{theta_p <= |xhat|} for xhat < 0: the tie rule on either side.  Keys are
     // clamped from below to kFoldKeyLow and cut into cells of 2^21 keys (exponent and 3 fraction bits); no cell holds
-    // two thresholds.  The entry of the cell that starts at key S, with P0 thresholds below S and the threshold TK in it, is
-    //     E = ((7 + P0) << 24 | 0xE00000 | (0x1FFFFF - (TK - S))) - S
-    // so that (E + key) >> 24 = 7 + P0 + [key > TK]: one lookup and one addition.  (No threshold in the cell: TK - S = 0x1FFFFF.)
-    uint32_t entry[kFoldCells];
+    // two thresholds.  For the cell that starts at key S, with P0 thresholds below S and the threshold TK in it:
+    //   xhat >= 0 (8 thresholds, codes 7 + P):  E = ((7 + P0) << 24 | 0xE00000 | (0x1FFFFF - (TK - S))) - S, and
+    //             (E + key) >> 24 = 7 + P0 + [key > TK]: the low 21 bits carry through the three set bits into the code;
+    //   xhat <  0 (7 thresholds: there is no code for -1.0; codes 7 - P):  E = ((7 - P0) << 24 | (TK - S)) + S + 1, and
+    //             (E + ~key) >> 24 = (E - 1 - key) >> 24 = 7 - P0 - [key > TK]: the borrow runs through three clear bits.
+    // One lookup and one addition either way; the sign picks the half of the table and complements the key.
+    // (No threshold in the cell: TK - S = 0x1FFFFF, which neither carries nor borrows.)
+    uint32_t entry[2][kFoldCells];      // [0] xhat >= 0, [1] xhat < 0
     int folded;
 };
 
@@ -122,15 +126,60 @@ __device__ __forceinline__ float quotient(float x, float d, float r, bool quick)
     return __fdiv_rn(x, d);
 }
 
-// code of xhat through the folded table; `ent_lane` is this lane's column of the per-lane replicated entries, rebased
-// by the index of the first cell.  7 + P for xhat >= 0; 7 - min(P, 7) for xhat < 0 (there is no code for -1.0).
+// code of xhat through the folded table; `ent_lane` is this lane's column of the per-lane replicated entries (the
+// non-negative half first, the negative half kFoldCells rows later), rebased by the index of the first cell.  The two
+// address steps are multiply-adds on purpose: the integer ALU is the busiest pipe of these kernels, the fp32 pipe has room.
 __device__ __forceinline__ uint32_t search_folded16(uint32_t ent_lane, float xhat) {
     const uint32_t b = __float_as_uint(xhat);
     const uint32_t key = max(__funnelshift_l(b, b, 1), kFoldKeyLow);
-    uint32_t e;
-    asm("ld.shared.u32 %0, [%1];" : "=r"(e) : "r"(ent_lane + (key >> 21) * 128u));
-    const uint32_t c = (e + key) >> 24;
-    return (b >> 31) ? 14u - min(c, 14u) : c;
+    const uint32_t smask = uint32_t(int32_t(b) >> 31);
+    uint32_t addr, e;
+    asm("mad.lo.u32 %0, %1, 128, %2;" : "=r"(addr) : "r"(key >> 21), "r"(ent_lane));
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(addr) : "r"(smask), "r"(0u - uint32_t(kFoldCells) * 128u), "r"(addr));
+    asm("ld.shared.u32 %0, [%1];" : "=r"(e) : "r"(addr));
+    return (e + (key ^ smask)) >> 24;
+}
+// word + (q << shift) as one multiply-add (the nibbles of a word never overlap)
+__device__ __forceinline__ uint32_t put_nibble(uint32_t word, uint32_t q, int shift) {
+    uint32_t r;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(q), "r"(1u << shift), "r"(word));
+    return r;
+}
+
+// two fp32 lanes per instruction (sm_100 packed fp32 arithmetic)
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+    uint64_t v;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(a), "f"(b));
+    return v;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
+// xhat of eight elements by one route for all of them (`quick` is uniform over the warp): the reciprocal route two
+// quotients per instruction (q0 = x r; e = x - d q0; q = q0 + e r), or the IEEE division.
+__device__ __forceinline__ void quotients8(const float (&f)[8], float d, float r, bool quick, float (&xh)[8]) {
+    if (quick) {
+        const uint64_t r2 = pack2(r, r), nd2 = pack2(-d, -d);
+#pragma unroll
+        for (int i = 0; i < 8; i += 2) {
+            const uint64_t x2 = pack2(f[i], f[i + 1]);
+            const uint64_t q0 = mul2(x2, r2);
+            const uint64_t e = fma2(nd2, q0, x2);
+            unpack2(fma2(e, r2, q0), xh[i], xh[i + 1]);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) xh[i] = __fdiv_rn(f[i], d);
+    }
 }
 
 __device__ __forceinline__ void fill_tables(const Tables4& tab, float* thr, float* val) {
@@ -138,16 +187,17 @@ __device__ __forceinline__ void fill_tables(const Tables4& tab, float* thr, floa
     __syncthreads();
 }
 
-template <int DT, bool FOLDED>
+template <int DT, bool FOLDED, int LOG2_LPB /* log2 of the lanes per block = log2(block / 8) */>
 __global__ void __launch_bounds__(256)
-q4_fast(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restrict__ absmax, size_t nchunks, int lpb /* lanes per block = block / 8 */,
-        int log2_lpb, const __grid_constant__ Tables4 tab) {
+q4_fast(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restrict__ absmax, size_t nchunks, const __grid_constant__ Tables4 tab) {
+    constexpr int lpb = 1 << LOG2_LPB;
+    constexpr int log2_lpb = LOG2_LPB;
     __shared__ float thr[16], val[16];
-    __shared__ __align__(128) uint32_t ent[FOLDED ? kFoldCells * 32 : 1];      // every entry once per lane, in that lane's bank
+    __shared__ __align__(128) uint32_t ent[FOLDED ? 2 * kFoldCells * 32 : 1];  // every entry once per lane, in that lane's bank
     fill_tables(tab, thr, val);
     uint32_t ent_lane = 0;
     if constexpr (FOLDED) {
-        for (int i = threadIdx.x; i < kFoldCells * 32; i += 256) ent[i] = tab.entry[i >> 5];
+        for (int i = threadIdx.x; i < 2 * kFoldCells * 32; i += 256) ent[i] = (&tab.entry[0][0])[i >> 5];
         __syncthreads();
         ent_lane = uint32_t(__cvta_generic_to_shared(ent)) + (threadIdx.x & 31) * 4u - kFoldCellBase * 128u;
     }
@@ -180,26 +230,19 @@ q4_fast(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restr
 #pragma unroll
             for (int i = 0; i < 8; ++i) a = fmaxf(a, fabsf(f[u][i]));
 #pragma unroll
-            for (int s = 1; s < 32; s <<= 1)
-                if (s < lpb) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, s));       // uniform over the warp
+            for (int s = 1; s < lpb; s <<= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, s));
             const float d = (a != 0.0f) ? a : 1.0f;
             // one choice of route for the whole warp keeps the per-element code free of branches
             const bool quick = (DT != kF32) && __all_sync(0xffffffffu, (d >= 5.421010862427522e-20f) && (d <= 1.8446744073709552e19f));
             float r;
             asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(d));
             float xh[8];
-            if (quick) {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) xh[i] = quotient<DT>(f[u][i], d, r, true);
-            } else {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) xh[i] = __fdiv_rn(f[u][i], d);
-            }
+            quotients8(f[u], d, r, quick, xh);
             uint32_t word = 0;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const uint32_t q = FOLDED ? search_folded16(ent_lane, xh[i]) : search16(thr, xh[i]);
-                word |= q << (4 * i);
+                word = put_nibble(word, q, 4 * i);
             }
             if (c[u] < nchunks) {
                 reinterpret_cast<uint32_t*>(packed)[c[u]] = word;
@@ -214,11 +257,11 @@ __global__ void __launch_bounds__(256)
 q4_wide(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restrict__ absmax, size_t nblocks, int chunks_per_block,
         const __grid_constant__ Tables4 tab) {
     __shared__ float thr[16], val[16];
-    __shared__ __align__(128) uint32_t ent[FOLDED ? kFoldCells * 32 : 1];
+    __shared__ __align__(128) uint32_t ent[FOLDED ? 2 * kFoldCells * 32 : 1];
     fill_tables(tab, thr, val);
     uint32_t ent_lane = 0;
     if constexpr (FOLDED) {
-        for (int i = threadIdx.x; i < kFoldCells * 32; i += 256) ent[i] = tab.entry[i >> 5];
+        for (int i = threadIdx.x; i < 2 * kFoldCells * 32; i += 256) ent[i] = (&tab.entry[0][0])[i >> 5];
         __syncthreads();
         ent_lane = uint32_t(__cvta_generic_to_shared(ent)) + (threadIdx.x & 31) * 4u - kFoldCellBase * 128u;
     }
@@ -236,18 +279,18 @@ q4_wide(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restr
 #pragma unroll
         for (int s = 1; s < 32; s <<= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, s));
         const float d = (a != 0.0f) ? a : 1.0f;
-        const bool quick = (d >= 5.421010862427522e-20f) && (d <= 1.8446744073709552e19f);
+        const bool quick = (DT != kF32) && (d >= 5.421010862427522e-20f) && (d <= 1.8446744073709552e19f);      // one block per warp: uniform
         float r;
         asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(d));
         for (int k = lane; k < chunks_per_block; k += 32) {
-            float f[8];
+            float f[8], xh[8];
             load8<DT>(x, cbase + k, f);
+            quotients8(f, d, r, quick, xh);
             uint32_t word = 0;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                const float xhat = quotient<DT>(f[i], d, r, quick);
-                const uint32_t q = FOLDED ? search_folded16(ent_lane, xhat) : search16(thr, xhat);
-                word |= q << (4 * i);
+                const uint32_t q = FOLDED ? search_folded16(ent_lane, xh[i]) : search16(thr, xh[i]);
+                word = put_nibble(word, q, 4 * i);
             }
             reinterpret_cast<uint32_t*>(packed)[cbase + k] = word;
         }
