@@ -31,6 +31,9 @@ def test_bench_line_has_the_contract_keys(bq):
     assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
     for q in d["quality"].values():
         assert 1.8 < q["compression_ratio"] < 2.0 and 0.003 < q["rel_rms_error"] < 0.03
+    for v in d["bq4"].values():
+        assert 0.2 < v["quantize_frac_of_measured"] < 1.1 and 0.5 < v["dequantize_frac_of_measured"] < 1.1
+        assert 3.5 < v["compression_ratio"] < 4.0 and 0.05 < v["rel_rms_error"] < 0.3
     # the decomposed linear layer: its own roofline object, parity on sampled rows of the full-size call, no kernel error
     m = d["mmd"]
     mr = m["roofline"]
