@@ -116,23 +116,31 @@ int bn_slot(int bn) { return bn == 256 ? 0 : (bn == 128 ? 1 : 2); }
 // Rows of the activation tiles the one-tile-per-CTA kernel loads: a decode step's few rows need only half a tile.
 int activation_box_rows(int M) { return M <= 64 ? 64 : 128; }
 
-template <int XDT, int YDT, int BN>
-cudaError_t launch_tc(const mmd_weights* w, const CUtensorMap& mqx, const CUtensorMap& msx, const float* sx, void* y, int M,
-                      cudaStream_t stream) {
-    using Cfg = mmdk::TcCfg<BN>;
+template <int XDT, int YDT, int BN, int BM>
+cudaError_t launch_tc_bm(const mmd_weights* w, const CUtensorMap& mqx, const CUtensorMap& msx, const float* sx, void* y, int M,
+                         cudaStream_t stream) {
+    using Cfg = mmdk::TcCfg<BN, BM>;
     static bool opted[64] = {};
     if (w->device < 0 || w->device >= 64 || !opted[w->device]) {
-        const cudaError_t e = cudaFuncSetAttribute(mmdk::gemm_tc<XDT, YDT, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::kSmemBytes));
+        const cudaError_t e = cudaFuncSetAttribute(mmdk::gemm_tc<XDT, YDT, BN, BM>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::kSmemBytes));
         if (e != cudaSuccess) return e;
         if (w->device >= 0 && w->device < 64) opted[w->device] = true;
     }
-    const dim3 grid(unsigned((M + 127) / 128), unsigned((w->N + BN - 1) / BN));
+    const dim3 grid(unsigned((M + BM - 1) / BM), unsigned((w->N + BN - 1) / BN));
     const int kblocks = (w->K + 127) / 128, sblocks = w->side_cols / 64;
     const int slot = bn_slot(BN);
-    const uint32_t tx = uint32_t(activation_box_rows(M) + BN) * 128u;
-    mmdk::gemm_tc<XDT, YDT, BN><<<grid, mmdk::kTcThreads, Cfg::kSmemBytes, stream>>>(
+    const uint32_t tx = uint32_t(BM + BN) * 128u;
+    mmdk::gemm_tc<XDT, YDT, BN, BM><<<grid, mmdk::kTcThreads, Cfg::kSmemBytes, stream>>>(
         mqx, w->map_q[slot], sblocks ? msx : mqx, sblocks ? w->map_side[slot] : w->map_q[slot], sx, w->scale, y, M, w->N, kblocks, sblocks, tx, w->status);
     return cudaGetLastError();
+}
+
+// At most 64 activation rows: 64-row MMAs and 64-row activation boxes (the host's maps are made to match).
+template <int XDT, int YDT, int BN>
+cudaError_t launch_tc(const mmd_weights* w, const CUtensorMap& mqx, const CUtensorMap& msx, const float* sx, void* y, int M,
+                      cudaStream_t stream) {
+    return activation_box_rows(M) == 64 ? launch_tc_bm<XDT, YDT, BN, 64>(w, mqx, msx, sx, y, M, stream)
+                                        : launch_tc_bm<XDT, YDT, BN, 128>(w, mqx, msx, sx, y, M, stream);
 }
 
 template <int XDT, int YDT>

@@ -216,9 +216,11 @@ constexpr int kTcBM = 128;
 constexpr int kTcRowBytes = 128;
 constexpr long long kWaitLimitCycles = 4000000000ll;            // about two seconds
 
-template <int BN> struct TcCfg {
-    static constexpr int kStages = (BN >= 256) ? 4 : (BN >= 128 ? 6 : 8);
-    static constexpr uint32_t kABytes = kTcBM * kTcRowBytes;
+// BM = rows of the MMA: 128, or 64 for calls with at most 64 activation rows (a decode step), whose ring stages then
+// spend 8 KB instead of 16 KB on activations and hold more steps of the weight stream in flight.
+template <int BN, int BM = kTcBM> struct TcCfg {
+    static constexpr int kStages = (BM == 64) ? (BN >= 256 ? 4 : (BN >= 128 ? 8 : 12)) : ((BN >= 256) ? 4 : (BN >= 128 ? 6 : 8));
+    static constexpr uint32_t kABytes = BM * kTcRowBytes;
     static constexpr uint32_t kBBytes = BN * kTcRowBytes;
     static constexpr uint32_t kStageBytes = kABytes + kBBytes;
     static constexpr uint32_t kTmemCols = (2 * BN <= 32) ? 32 : 2 * BN;          // a power of two >= 32
@@ -299,14 +301,14 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         : "r"(taddr) : "memory");
 }
 
-template <int XDT, int YDT, int BN>
+template <int XDT, int YDT, int BN, int BM>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUtensorMap map_qw,
         const __grid_constant__ CUtensorMap map_sidex, const __grid_constant__ CUtensorMap map_sidew,
         const float* __restrict__ sx, const float* __restrict__ sw, void* __restrict__ y,
         int M, int N, int kblocks /* int8 steps of 128 features */, int sblocks /* side steps of 64 columns */,
         uint32_t stage_tx_bytes /* bytes the two loads of a stage bring: (activation rows in the map's box + BN) * 128 */, int* status) {
-    using Cfg = TcCfg<BN>;
+    using Cfg = TcCfg<BN, BM>;
     constexpr int S = Cfg::kStages;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;               // swizzled tiles need 1024-byte alignment
@@ -319,7 +321,7 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
     float* sw_s = reinterpret_cast<float*>(ctrl + 256);                         // BN scales of this tile's columns
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * kTcBM, n0 = blockIdx.y * BN;
+    const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
     const int steps = kblocks + sblocks;
 
     if (threadIdx.x == 0) {
@@ -345,8 +347,6 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
                 const uint32_t round = uint32_t(i / S);
                 if (!mbar_wait(empty0 + 8u * s, (round & 1u) ^ 1u, abort_flag, status, 1)) break;
                 const uint32_t a_dst = tiles + uint32_t(s) * Cfg::kStageBytes, b_dst = a_dst + Cfg::kABytes;
-                // with at most 64 activation rows the host's maps load 64-row boxes: the MMA still reads 128 rows of
-                // shared memory, and what it makes of the stale upper half lands in accumulator rows that are never stored
                 mbar_expect_tx(full0 + 8u * s, stage_tx_bytes);
                 if (i < kblocks) {
                     tma_load_2d(a_dst, &map_qx, i * 128, m0, full0 + 8u * s);
@@ -360,8 +360,8 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
         __syncwarp();
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc_i8 = umma_idesc(2, 1, kTcBM, BN);                   // int32 <- int8 x int8
-            constexpr uint32_t idesc_16 = umma_idesc(1, XDT == kBF16 ? 1u : 0u, kTcBM, BN);     // fp32 <- 16-bit x 16-bit
+            constexpr uint32_t idesc_i8 = umma_idesc(2, 1, BM, BN);                      // int32 <- int8 x int8
+            constexpr uint32_t idesc_16 = umma_idesc(1, XDT == kBF16 ? 1u : 0u, BM, BN);        // fp32 <- 16-bit x 16-bit
             bool ok = true;
             for (int i = 0; i < steps && ok; ++i) {
                 const int s = i % S;
@@ -391,7 +391,10 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
         for (int c = et; c < BN; c += 128) sw_s[c] = (n0 + c < N) ? sw[n0 + c] : 0.0f;
         asm volatile("bar.sync 1, 128;" ::: "memory");
         const int quarter = warp & 3;
-        const int m = m0 + quarter * 32 + lane;
+        // a 128-row accumulator has row r in lane r; a 64-row one keeps rows 16 q .. 16 q + 15 in the first 16 lanes of
+        // quarter q (the other lanes of the quarter hold nothing of it)
+        const bool row_lane = (BM == 128) || lane < 16;
+        const int m = row_lane ? m0 + quarter * (BM / 4) + lane : M;
         const float sxm = (m < M) ? sx[m] : 0.0f;
         bool ok = true;
         if (lane == 0) ok = mbar_wait(accbar, 0, abort_flag, status, 3);
