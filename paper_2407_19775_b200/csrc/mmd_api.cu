@@ -117,7 +117,7 @@ int bn_slot(int bn) { return bn == 256 ? 0 : (bn == 128 ? 1 : 2); }
 int activation_box_rows(int M) { return M <= 64 ? 64 : 128; }
 
 template <int XDT, int YDT, int BN, int BM>
-cudaError_t launch_tc_bm(const mmd_weights* w, const CUtensorMap& mqx, const CUtensorMap& msx, const float* sx, void* y, int M,
+cudaError_t launch_tc_bm(const mmd_weights* w, const CUtensorMap& mqx, const CUtensorMap& msx, const float* sx, void* y, int M, int split,
                          cudaStream_t stream) {
     using Cfg = mmdk::TcCfg<BN, BM>;
     static bool opted[64] = {};
@@ -126,21 +126,38 @@ cudaError_t launch_tc_bm(const mmd_weights* w, const CUtensorMap& mqx, const CUt
         if (e != cudaSuccess) return e;
         if (w->device >= 0 && w->device < 64) opted[w->device] = true;
     }
-    const dim3 grid(unsigned((M + BM - 1) / BM), unsigned((w->N + BN - 1) / BN));
-    const int kblocks = (w->K + 127) / 128, sblocks = w->side_cols / 64;
+    int kblocks = (w->K + 127) / 128, sblocks = w->side_cols / 64;
     const int slot = bn_slot(BN);
-    const uint32_t tx = uint32_t(BM + BN) * 128u;
-    mmdk::gemm_tc<XDT, YDT, BN, BM><<<grid, mmdk::kTcThreads, Cfg::kSmemBytes, stream>>>(
-        mqx, w->map_q[slot], sblocks ? msx : mqx, sblocks ? w->map_side[slot] : w->map_q[slot], sx, w->scale, y, M, w->N, kblocks, sblocks, tx, w->status);
-    return cudaGetLastError();
+    uint32_t tx = uint32_t(BM + BN) * 128u;
+    int* status = w->status;
+    int Mv = M, Nv = w->N;
+    const float* swv = w->scale;
+    // the ranks' partial sums must fit into rank 0's ring
+    if (split > 1 && size_t(split - 1) * BM * BN * 4 > size_t(Cfg::kStages) * Cfg::kStageBytes) split = 1;
+    if (split > kblocks) split = kblocks;
+    if (split < 1) split = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(unsigned((M + BM - 1) / BM), unsigned((w->N + BN - 1) / BN), unsigned(split));
+    cfg.blockDim = dim3(mmdk::kTcThreads, 1, 1);
+    cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 1;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = unsigned(split);
+    cfg.attrs = &attr;
+    cfg.numAttrs = split > 1 ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, mmdk::gemm_tc<XDT, YDT, BN, BM>, mqx, w->map_q[slot], sblocks ? msx : mqx,
+                              sblocks ? w->map_side[slot] : w->map_q[slot], sx, swv, y, Mv, Nv, kblocks, sblocks, tx, status);
 }
 
 // At most 64 activation rows: 64-row MMAs and 64-row activation boxes (the host's maps are made to match).
 template <int XDT, int YDT, int BN>
-cudaError_t launch_tc(const mmd_weights* w, const CUtensorMap& mqx, const CUtensorMap& msx, const float* sx, void* y, int M,
+cudaError_t launch_tc(const mmd_weights* w, const CUtensorMap& mqx, const CUtensorMap& msx, const float* sx, void* y, int M, int split,
                       cudaStream_t stream) {
-    return activation_box_rows(M) == 64 ? launch_tc_bm<XDT, YDT, BN, 64>(w, mqx, msx, sx, y, M, stream)
-                                        : launch_tc_bm<XDT, YDT, BN, 128>(w, mqx, msx, sx, y, M, stream);
+    return activation_box_rows(M) == 64 ? launch_tc_bm<XDT, YDT, BN, 64>(w, mqx, msx, sx, y, M, split, stream)
+                                        : launch_tc_bm<XDT, YDT, BN, 128>(w, mqx, msx, sx, y, M, split, stream);
 }
 
 template <int XDT, int YDT>
@@ -199,13 +216,20 @@ cudaError_t launch_tc_bn(const mmd_weights* w, const CUtensorMap& mqx, const CUt
     // tile (few rows, as in a decode step, where the weights are read once and the kernel is
     // bound by that stream) narrower tiles put more CTAs on the weight stream.
     const long mt = (M + 127) / 128;
-    if (w->N >= 256 && mt * ((w->N + 255) / 256) >= w->sm_count) return launch_tc<XDT, YDT, 256>(w, mqx, msx, sx, y, M, stream);
-    if (w->N >= 128 && mt * ((w->N + 127) / 128) >= w->sm_count) return launch_tc<XDT, YDT, 128>(w, mqx, msx, sx, y, M, stream);
-    // One row of tiles over a wide layer (a decode step) streams every weight once from DRAM and is bound by the bytes
-    // its CTAs keep in flight: 128-row weight tiles hold 6 x 16 KB per CTA against 8 x 8 KB for 64-row tiles (measured
-    // on 64 x 6144 -> 16384: 21.7 us against 35.3 us; equal at 8192 output features).
-    if (mt == 1 && w->N >= 8192) return launch_tc<XDT, YDT, 128>(w, mqx, msx, sx, y, M, stream);
-    return launch_tc<XDT, YDT, 64>(w, mqx, msx, sx, y, M, stream);
+    if (w->N >= 256 && mt * ((w->N + 255) / 256) >= w->sm_count) return launch_tc<XDT, YDT, 256>(w, mqx, msx, sx, y, M, 1, stream);
+    if (w->N >= 128 && mt * ((w->N + 127) / 128) >= w->sm_count) return launch_tc<XDT, YDT, 128>(w, mqx, msx, sx, y, M, 1, stream);
+    // One row of tiles (a decode step) streams every weight once from DRAM, and an SM streams only as fast as the bytes it
+    // keeps in flight.  128-row weight tiles hold the most per CTA; when they leave SMs idle, 2-4 CTAs share each tile's K
+    // steps (clusters along z) so that about one CTA per SM is streaming.
+    if (mt == 1 && w->N >= 1024) {
+        const long tiles = (w->N + 127) / 128;
+        int split = int(w->sm_count / tiles);
+        if (split > 4) split = 4;
+        if (split < 1) split = 1;
+        while (split > 1 && (w->K + 127) / 128 < 8 * split) --split;            // at least 8 steps per CTA
+        return launch_tc<XDT, YDT, 128>(w, mqx, msx, sx, y, M, split, stream);
+    }
+    return launch_tc<XDT, YDT, 64>(w, mqx, msx, sx, y, M, 1, stream);
 }
 
 template <int XDT, int YDT>

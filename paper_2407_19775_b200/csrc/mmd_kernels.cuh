@@ -210,6 +210,15 @@ gemm_general(const int8_t* __restrict__ qx, const int8_t* __restrict__ qw, const
 //
 // Every wait is bounded: a wait that runs out records a code in *status, raises the CTA's
 // abort flag and the kernel winds down (no further stores, tensor memory freed).
+//
+// Split K.  A call with one row of tiles over a narrow layer (a decode step) has fewer tiles
+// than the GPU has SMs, and an SM streams weights from DRAM only as fast as the bytes it can
+// keep in flight.  Such calls are launched in clusters of 2-4 CTAs along z: the CTAs of a
+// cluster work on the same tile, each on its own share of the K steps (the side steps go to
+// rank 0), and afterwards ranks 1.. write their int32 accumulators into rank 0's ring memory
+// (distributed shared memory; the ring is free by then, which the first cluster barrier
+// establishes), a second cluster barrier publishes them, and rank 0 adds them to its own and
+// runs the epilogue.  Integer sums do not depend on the order, so the result is the same bits.
 
 constexpr int kTcThreads = 192;
 constexpr int kTcBM = 128;
@@ -301,12 +310,36 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         : "r"(taddr) : "memory");
 }
 
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// the address, in the cluster's shared window, of this CTA's shared address `addr` in CTA `rank`
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_size() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+
 template <int XDT, int YDT, int BN, int BM>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUtensorMap map_qw,
         const __grid_constant__ CUtensorMap map_sidex, const __grid_constant__ CUtensorMap map_sidew,
         const float* __restrict__ sx, const float* __restrict__ sw, void* __restrict__ y,
-        int M, int N, int kblocks /* int8 steps of 128 features */, int sblocks /* side steps of 64 columns */,
+        int M, int N, int kblocks_all /* int8 steps of 128 features */, int sblocks_all /* side steps of 64 columns */,
         uint32_t stage_tx_bytes /* bytes the two loads of a stage bring: (activation rows in the map's box + BN) * 128 */, int* status) {
     using Cfg = TcCfg<BN, BM>;
     constexpr int S = Cfg::kStages;
@@ -322,6 +355,10 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
+    const uint32_t nsplit = cluster_size(), rank = cluster_rank();              // 1 and 0 without a cluster launch
+    const int kb_lo = int((long(kblocks_all) * rank) / nsplit), kb_hi = int((long(kblocks_all) * (rank + 1)) / nsplit);
+    const int kblocks = kb_hi - kb_lo;                                          // this CTA's share of the int8 steps
+    const int sblocks = (rank == 0) ? sblocks_all : 0;
     const int steps = kblocks + sblocks;
 
     if (threadIdx.x == 0) {
@@ -349,8 +386,8 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
                 const uint32_t a_dst = tiles + uint32_t(s) * Cfg::kStageBytes, b_dst = a_dst + Cfg::kABytes;
                 mbar_expect_tx(full0 + 8u * s, stage_tx_bytes);
                 if (i < kblocks) {
-                    tma_load_2d(a_dst, &map_qx, i * 128, m0, full0 + 8u * s);
-                    tma_load_2d(b_dst, &map_qw, i * 128, n0, full0 + 8u * s);
+                    tma_load_2d(a_dst, &map_qx, (kb_lo + i) * 128, m0, full0 + 8u * s);
+                    tma_load_2d(b_dst, &map_qw, (kb_lo + i) * 128, n0, full0 + 8u * s);
                 } else {
                     tma_load_2d(a_dst, &map_sidex, (i - kblocks) * 64, m0, full0 + 8u * s);
                     tma_load_2d(b_dst, &map_sidew, (i - kblocks) * 64, n0, full0 + 8u * s);
@@ -358,6 +395,7 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
             }
         }
         __syncwarp();
+        if (nsplit > 1) { cluster_sync_all(); cluster_sync_all(); }              // the two barriers of the exchange (see the epilogue)
     } else if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc_i8 = umma_idesc(2, 1, BM, BN);                      // int32 <- int8 x int8
@@ -385,6 +423,7 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
             if (ok) umma_commit(accbar);
         }
         __syncwarp();
+        if (nsplit > 1) { cluster_sync_all(); cluster_sync_all(); }
     } else {
         // epilogue: 128 threads, one accumulator row each
         const int et = threadIdx.x - 64;
@@ -400,14 +439,44 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
         if (lane == 0) ok = mbar_wait(accbar, 0, abort_flag, status, 3);
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (ok) {
-            const uint32_t lane_base = tmem + (uint32_t(quarter * 32) << 16);
+        const uint32_t lane_base = tmem + (uint32_t(quarter * 32) << 16);
+        const uint32_t row_in_tile = uint32_t(quarter * (BM / 4) + lane);       // meaningful where row_lane holds
+        constexpr uint32_t kPartBytes = uint32_t(BM) * BN * 4u;                  // one rank's accumulator, stored [column][row]
+        if (nsplit > 1) {
+            cluster_sync_all();                                                  // every CTA of the cluster is through its main loop: rank 0's ring is free
+            if (rank > 0) {
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    uint32_t ai[32];
+                    tmem_ld32(lane_base + uint32_t(c0), ai);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (ok && row_lane) {
+                        const uint32_t dst = map_to_cta(tiles + (rank - 1u) * kPartBytes + uint32_t(c0) * BM * 4u + row_in_tile * 4u, 0);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) st_cluster_u32(dst + uint32_t(j) * BM * 4u, ai[j]);
+                    }
+                }
+            }
+            cluster_sync_all();                                                  // the partial sums are in rank 0's shared memory
+        }
+        if (ok && rank == 0) {
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t ai[32], af[32];
                 tmem_ld32(lane_base + uint32_t(c0), ai);
                 if (sblocks > 0) tmem_ld32(lane_base + uint32_t(BN + c0), af);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (nsplit > 1 && row_lane) {
+                    for (uint32_t r = 1; r < nsplit; ++r) {
+                        const uint32_t src = tiles + (r - 1u) * kPartBytes + uint32_t(c0) * BM * 4u + row_in_tile * 4u;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            uint32_t v;
+                            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(src + uint32_t(j) * BM * 4u) : "memory");
+                            ai[j] += v;
+                        }
+                    }
+                }
                 float out[32];
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
@@ -720,21 +789,6 @@ constexpr uint32_t kPairHalfBytes = 128 * kTcRowBytes;                        //
 constexpr uint32_t kPairStageBytes = 2 * kPairHalfBytes;
 constexpr uint32_t kPairSmemBytes = kPairStages * kPairStageBytes + 1024 + kTcpCtrlBytes + kTcpSwBytes + kTcpWoBytes;
 
-__device__ __forceinline__ uint32_t cluster_rank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// the address, in the cluster's shared window, of this CTA's shared address `addr` in CTA `rank`
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
-    return r;
-}
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }

@@ -187,6 +187,24 @@ def test_linear_tensor_path(bq, name, M, K, N, tdt, ko):
         lin.close()
 
 
+@pytest.mark.parametrize("M,K,N,ko", [(64, 4096, 7688, 4), (100, 4096, 5120, 0), (7, 1024, 2048, 9), (64, 8192, 1024, 8), (128, 2048, 3000, 3)])
+def test_linear_one_row_of_tiles_shares_k_steps(bq, M, K, N, ko):
+    """Decode-size calls over narrow layers: clusters of 2-4 CTAs split a tile's K steps and add their integer sums
+    through shared memory; both the 64-row and the 128-row accumulator shapes, ragged N."""
+    g = torch.Generator().manual_seed(M * 7 + N)
+    X = (torch.randn(M, K, generator=g) * 0.6).to(torch.float16)
+    W = (torch.randn(N, K, generator=g) * 0.03).to(torch.float16)
+    idx = np.sort(torch.randperm(K, generator=g)[:ko].numpy()).astype(np.int32)
+    X[:, idx.tolist()] *= 25
+    lin = bq.DecomposedLinear(W.cuda(), idx)
+    for out in (torch.float32, None):
+        y = lin.linear(X.cuda(), out, path=3)
+        assert lin.kernel_status() == 0
+        check_output(y, X, W, idx, F16, exact_expected=(ko == 0))
+    assert torch.equal(lin.linear(X.cuda(), torch.float32, path=3)[:, :8], lin.linear(X.cuda(), torch.float32, path=3)[:, :8])
+    lin.close()
+
+
 def test_linear_seeded_fuzz(bq):
     """Random small shapes, feature counts, element types and value scales through every kernel that takes them."""
     rng = np.random.default_rng(2024)
