@@ -187,10 +187,12 @@ def test_linear_tensor_path(bq, name, M, K, N, tdt, ko):
         lin.close()
 
 
-@pytest.mark.parametrize("M,K,N,ko", [(64, 4096, 7688, 4), (100, 4096, 5120, 0), (7, 1024, 2048, 9), (64, 8192, 1024, 8), (128, 2048, 3000, 3)])
+@pytest.mark.parametrize("M,K,N,ko", [(64, 4096, 7688, 4), (100, 4096, 5120, 0), (7, 1024, 2048, 9), (64, 8192, 1024, 8), (128, 2048, 3000, 3),
+                                      (64, 1024, 20488, 5), (100, 512, 30000, 0), (33, 256, 37888, 70)])
 def test_linear_one_row_of_tiles_shares_k_steps(bq, M, K, N, ko):
-    """Decode-size calls over narrow layers: clusters of 2-4 CTAs split a tile's K steps and add their integer sums
-    through shared memory; both the 64-row and the 128-row accumulator shapes, ragged N."""
+    """Decode-size calls: over narrow layers clusters of 2-4 CTAs split a tile's K steps and add their integer sums
+    through shared memory; layers with more 128-row tiles than SMs run without the split.  Both the 64-row and the
+    128-row accumulator shapes, ragged N."""
     g = torch.Generator().manual_seed(M * 7 + N)
     X = (torch.randn(M, K, generator=g) * 0.6).to(torch.float16)
     W = (torch.randn(N, K, generator=g) * 0.03).to(torch.float16)
