@@ -415,6 +415,26 @@ def run_mmd(bq, dev, args):
     rec = mo.reconstruct(qw[:1024], sw[:1024], wo[:1024], mo.BF16, idx)
     wf = W[:1024].double().numpy()
     lin.close()
+
+    # a decode step through a 70B-class layer: 64 tokens, every weight read once (HBM-bound)
+    dX, dW, didx = workloads.make_linear("mmd_decode70b")
+    dM, dK, dN = dX.shape[0], dX.shape[1], dW.shape[0]
+    dXd = dX.to(dev)
+    dlin = bq.DecomposedLinear(dW.to(dev), didx)
+    dy = torch.empty((dM, dN), dtype=dX.dtype, device=dev)
+    dws = dlin.workspace(dM)
+    dlin.linear(dXd, y_out=dy, workspace=dws)
+    torch.cuda.synchronize()
+    ms_dec = timed_gpu(lambda: dlin.linear(dXd, y_out=dy, workspace=dws), 8)
+    dstatus = dlin.kernel_status()
+    dqw, dsw, dwo = mo.rowquant(workloads.bits_2d(dW[:512]), mo.F16, didx)
+    d_ref = mo.linear(workloads.bits_2d(dX), mo.F16, dqw, dsw, dwo, didx, mo.F16)
+    d_agree = float(np.mean(workloads.bits_2d(dy[:, :512].cpu().contiguous()) == d_ref))
+    dec_bytes = dN * dK + dM * dK * 3 + dM * dN * 2
+    decode = {"workload": f"mmd_decode70b: X [{dM},{dK}] x W [{dN},{dK}]^T fp16, {didx.size} critical features", "us_per_call": round(ms_dec * 1e3, 2),
+              "algorithmic_bytes": int(dec_bytes), "gbs": round(dec_bytes / ms_dec / 1e6, 1), "frac_of_measured_hbm": round(dec_bytes / ms_dec / 1e6 / hbm, 4),
+              "kernel_status": dstatus, "outputs_equal_to_oracle_bits_first_512_columns": round(d_agree, 5)}
+    dlin.close()
     return {
         "workload": f"{MMD_WORKLOAD}: X [{M},{K}] x W [{N},{K}]^T bf16, {idx.size} critical features; {wl.recipe}",
         "ms_per_call": round(ms_call, 4), "tops": round(ops / ms_call / 1e9, 1), "kernel_status": status,
@@ -430,7 +450,8 @@ def run_mmd(bq, dev, args):
                     "weight_rel_rms_error": round(float(np.sqrt(((rec - wf) ** 2).sum() / (wf ** 2).sum())), 5)},
         "cpu_baseline": {"value": round(2.0 * 256 * N * K / cpu_s / 1e12, 4), "unit": "TOP/s", "cores": os.cpu_count(), "kind": "oracle",
                          "sample": "first 256 tokens through the whole layer (weights already decomposed); numpy/BLAS threads"},
-        "gpu_launches": (2 * 2 + 8) * reps + 2 * (reps + 3),
+        "decode": decode,
+        "gpu_launches": (2 * 2 + 8 + 2 * 8) * reps + 2 * (reps + 3),
     }
 
 

@@ -41,3 +41,5 @@ def test_bench_line_has_the_contract_keys(bq):
     assert m["kernel_status"] == 0 and m["parity"]["outputs_equal_to_oracle_bits"] > 0.99 and m["parity"]["weight_codes_exact_first_256_rows"]
     assert 0 < m["e2e"]["tops"] < m["tops"] and m["e2e"]["h2d_bytes_per_call"] > 0 and m["cpu_baseline"]["kind"] == "oracle"
     assert 1.9 < m["quality"]["weight_bytes_ratio"] < 2.0 and m["gpu_launches"] > 0
+    dec = m["decode"]
+    assert dec["kernel_status"] == 0 and dec["outputs_equal_to_oracle_bits_first_512_columns"] > 0.99 and 0.2 < dec["frac_of_measured_hbm"] < 1.1
