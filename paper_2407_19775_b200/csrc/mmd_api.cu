@@ -141,13 +141,17 @@ cudaError_t launch_tc_bm(const mmd_weights* w, const CUtensorMap& mqx, const CUt
     cfg.blockDim = dim3(mmdk::kTcThreads, 1, 1);
     cfg.dynamicSmemBytes = Cfg::kSmemBytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = 1;
-    attr.val.clusterDim.y = 1;
-    attr.val.clusterDim.z = unsigned(split);
-    cfg.attrs = &attr;
-    cfg.numAttrs = split > 1 ? 1 : 0;
+    // The row kernel launched just before lets this kernel start early (its set-up and first weight loads overlap the row
+    // kernel); the kernel itself waits for the row kernel's results before it touches them.
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 1;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = unsigned(split);
+    cfg.attrs = attr;
+    cfg.numAttrs = split > 1 ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, mmdk::gemm_tc<XDT, YDT, BN, BM>, mqx, w->map_q[slot], sblocks ? msx : mqx,
                               sblocks ? w->map_side[slot] : w->map_q[slot], sx, swv, y, Mv, Nv, kblocks, sblocks, tx, status);
 }

@@ -53,6 +53,9 @@ rowquant(const void* __restrict__ v, int R, int K, const int32_t* __restrict__ i
          int8_t* __restrict__ q_out, float* __restrict__ scale_out, void* __restrict__ side_out) {
     extern __shared__ __align__(16) unsigned char mask[];       // K / 8 bytes
     __shared__ float red[8];
+    // A product kernel launched behind this one with programmatic stream serialization may start its set-up and its
+    // weight loads now; it waits (griddepcontrol.wait) for this grid's results before it reads them.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int nchunks = K / 8;
     for (int c = threadIdx.x; c < (nchunks + 3) / 4; c += 256) reinterpret_cast<uint32_t*>(mask)[c] = 0u;
     __syncthreads();
@@ -379,7 +382,22 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int i = 0; i < steps; ++i) {
+            // The first ring-full of weight tiles does not depend on the row kernel that runs before this one: their loads
+            // go out at once; the activation tiles of those stages follow when that kernel's results are visible.
+            const int pre = steps < S ? steps : S;
+            for (int i = 0; i < pre; ++i) {
+                const uint32_t b_dst = tiles + uint32_t(i) * Cfg::kStageBytes + Cfg::kABytes;
+                mbar_expect_tx(full0 + 8u * i, stage_tx_bytes);
+                if (i < kblocks) tma_load_2d(b_dst, &map_qw, (kb_lo + i) * 128, n0, full0 + 8u * i);
+                else tma_load_2d(b_dst, &map_sidew, (i - kblocks) * 64, n0, full0 + 8u * i);
+            }
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            for (int i = 0; i < pre; ++i) {
+                const uint32_t a_dst = tiles + uint32_t(i) * Cfg::kStageBytes;
+                if (i < kblocks) tma_load_2d(a_dst, &map_qx, (kb_lo + i) * 128, m0, full0 + 8u * i);
+                else tma_load_2d(a_dst, &map_sidex, (i - kblocks) * 64, m0, full0 + 8u * i);
+            }
+            for (int i = pre; i < steps; ++i) {
                 const int s = i % S;
                 const uint32_t round = uint32_t(i / S);
                 if (!mbar_wait(empty0 + 8u * s, (round & 1u) ^ 1u, abort_flag, status, 1)) break;
@@ -429,6 +447,7 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
         const int et = threadIdx.x - 64;
         for (int c = et; c < BN; c += 128) sw_s[c] = (n0 + c < N) ? sw[n0 + c] : 0.0f;
         asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("griddepcontrol.wait;" ::: "memory");       // the activations' row scales come from the kernel before this one
         const int quarter = warp & 3;
         // a 128-row accumulator has row r in lane r; a 64-row one keeps rows 16 q .. 16 q + 15 in the first 16 lanes of
         // quarter q (the other lanes of the quarter hold nothing of it)
