@@ -68,13 +68,23 @@ rowquant(const void* __restrict__ v, int R, int K, const int32_t* __restrict__ i
     for (int r = blockIdx.x; r < R; r += gridDim.x) {
         const uint4* row = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(v) + size_t(r) * K);
         float a = 0.0f;
-        for (int c = threadIdx.x; c < nchunks; c += 256) {
-            const uint4 w = row[c];
-            const uint32_t mk = mask[c];
-            float f[8];
-            widen8<DT>(w, f);
+        for (int c0 = threadIdx.x; c0 < nchunks; c0 += 256 * 4) {               // four loads in flight per thread
+            uint4 w[4];
+            uint32_t mk[4];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) a = fmaxf(a, ((mk >> i) & 1u) ? 0.0f : fabsf(f[i]));
+            for (int u = 0; u < 4; ++u) {
+                const int c = c0 + 256 * u;
+                const bool in = c < nchunks;
+                w[u] = in ? row[c] : make_uint4(0, 0, 0, 0);
+                mk[u] = in ? uint32_t(mask[c]) : 0xffu;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                float f[8];
+                widen8<DT>(w[u], f);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) a = fmaxf(a, ((mk[u] >> i) & 1u) ? 0.0f : fabsf(f[i]));
+            }
         }
 #pragma unroll
         for (int s = 16; s >= 1; s >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, s));
@@ -84,6 +94,14 @@ rowquant(const void* __restrict__ v, int R, int K, const int32_t* __restrict__ i
         for (int i = 0; i < 8; ++i) a = fmaxf(a, red[i]);
         const float d = (a != 0.0f) ? a : 1.0f;
         if (threadIdx.x == 0) scale_out[r] = __fdiv_rn(a, 127.0f);
+        // t = RN32(127 v / d).  n = 127 v is exact; for d within [2^-64, 2^64]: q0 = RN(n rc), e = n - d q0 (exact in one
+        // fma), t = RN(q0 + e rc) from the approximate reciprocal rc (within 1 ulp of 1 / d).  q0 + e rc is within a relative
+        // 2^-44 of n / d while a quotient with an 11-bit divisor that is not itself an fp32 stays a relative 2^-36 away from
+        // every rounding boundary, so t is the IEEE quotient (the CPU tests check every pair of 16-bit significands with rc
+        // off by up to 2 ulp).  Outside the window: the IEEE division.  d is the same for the whole CTA.
+        const bool quick = (d >= 5.421010862427522e-20f) && (d <= 1.8446744073709552e19f);
+        float rc;
+        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc) : "f"(d));
 
         uint2* qrow = reinterpret_cast<uint2*>(q_out + size_t(r) * K);
         for (int c = threadIdx.x; c < nchunks; c += 256) {
@@ -94,7 +112,15 @@ rowquant(const void* __restrict__ v, int R, int K, const int32_t* __restrict__ i
             uint32_t b[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                const int qi = __float2int_rn(__fdiv_rn(__fmul_rn(f[i], 127.0f), d));
+                const float n = __fmul_rn(f[i], 127.0f);
+                float t;
+                if (quick) {
+                    const float q0 = __fmul_rn(n, rc);
+                    t = __fmaf_rn(__fmaf_rn(-d, q0, n), rc, q0);
+                } else {
+                    t = __fdiv_rn(n, d);
+                }
+                const int qi = __float2int_rn(t);
                 b[i] = ((mk >> i) & 1u) ? 0u : (uint32_t(qi) & 0xffu);
             }
             qrow[c] = make_uint2(b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24), b[4] | (b[5] << 8) | (b[6] << 16) | (b[7] << 24));

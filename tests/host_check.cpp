@@ -127,4 +127,41 @@ long hc_check_quick_division(int sig_bits, int max_gap, int d_exp, long* code_mi
     return bad;
 }
 
+// The row kernel of the mixed matrix decomposition needs t = RN32(127 x / d) for 16-bit x and d
+// with |x| <= d.  It computes n = 127 x (exact), q0 = RN(n r), e = n - d q0 (one fma, exact),
+// t = RN(q0 + e r) from an approximate reciprocal r.  Same exhaustive check as above with the
+// 18-bit numerators 127 x: returns how many t differ in any bit from n / d; *int_mismatch
+// counts those whose rounding to an integer (ties to even) differs too.
+long hc_check_rowquant_division(int sig_bits, int max_gap, int d_exp, long* int_mismatch, long* checked) {
+    const int half = 1 << (sig_bits - 1);
+    long bad = 0, bad_int = 0, cnt = 0;
+    for (int md = 0; md < half; ++md) {
+        const float d = std::ldexp(float(half + md), d_exp - (sig_bits - 1));
+        for (int dr = -2; dr <= 2; ++dr) {
+            const float r = bqt::u2f(bqt::f2u(1.0f / d) + uint32_t(dr));
+            for (int gap = 0; gap <= max_gap; ++gap) {
+                for (int mx = 0; mx < half; ++mx) {
+                    const float x = std::ldexp(float(half + mx), d_exp - gap - (sig_bits - 1));
+                    if (x > d) continue;
+                    for (int sgn = 0; sgn < 2; ++sgn) {
+                        const float n = (sgn ? -x : x) * 127.0f;
+                        const float q0 = n * r;
+                        const float e = std::fmaf(-d, q0, n);
+                        const float t = std::fmaf(e, r, q0);
+                        const float ref = n / d;
+                        ++cnt;
+                        if (bqt::f2u(t) != bqt::f2u(ref)) {
+                            ++bad;
+                            if (std::nearbyintf(t) != std::nearbyintf(ref)) ++bad_int;
+                        }
+                    }
+                }
+            }
+        }
+    }
+    *int_mismatch = bad_int;
+    *checked = cnt;
+    return bad;
+}
+
 }  // extern "C"

@@ -25,6 +25,7 @@ def hc():
         os.replace(tmp, LIB)
     L = ctypes.CDLL(LIB)
     L.hc_check_quick_division.restype = ctypes.c_long
+    L.hc_check_rowquant_division.restype = ctypes.c_long
     L.hc_code_folded.argtypes = [ctypes.c_float]
     L.hc_code_general.argtypes = [ctypes.c_float]
     L.hc_value_folded.argtypes = [ctypes.c_float, ctypes.c_float]
@@ -118,6 +119,16 @@ def test_reciprocal_quotient_is_the_ieee_quotient_for_16bit_inputs(hc, sig_bits,
     cm, ck = ctypes.c_long(), ctypes.c_long()
     bad = hc.hc_check_quick_division(sig_bits, 34, d_exp, ctypes.byref(cm), ctypes.byref(ck))
     assert ck.value > 4_000_000 and bad == 0 and cm.value == 0
+
+
+@pytest.mark.parametrize("sig_bits,d_exp", [(8, 0), (11, 0), (11, -64), (11, 64)])
+def test_reciprocal_route_of_the_row_kernel_is_the_ieee_quotient(hc, sig_bits, d_exp):
+    """RN32(127 x / d) from an approximate reciprocal, for every pair of 16-bit significands, both signs, exponent gaps
+    down to 127 x / d ~ 2^-19 (everything below rounds to the integer 0 on either route) and every reciprocal within 2 ulp
+    of the correctly rounded one."""
+    im, ck = ctypes.c_long(), ctypes.c_long()
+    bad = hc.hc_check_rowquant_division(sig_bits, 26, d_exp, ctypes.byref(im), ctypes.byref(ck))
+    assert ck.value > 3_000_000 and bad == 0 and im.value == 0
 
 
 def test_user_codebook_rules(hc, cb):
