@@ -618,7 +618,7 @@ gemm_tcp(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUt
     const uint32_t acce0 = accf0 + 16u;                                         // 2: accumulator drained
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl + 8 * (2 * S + 4));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 8 * (2 * S + 4) + 8);
-    volatile int* epi_ok = reinterpret_cast<volatile int*>(ctrl + 8 * (2 * S + 4) + 12);     // the epilogue's shared verdict of its wait
+    volatile int* epi_ok = reinterpret_cast<volatile int*>(ctrl + 8 * (2 * S + 4) + 12);     // what the epilogue thread that waited found, for the other 127
     float* sw_s = reinterpret_cast<float*>(ctrl + kTcpCtrlBytes);               // [2][BN]
     float* wo_s = sw_s + 2 * BN;                                                // [BN][kTcpSide]
 
@@ -733,7 +733,7 @@ gemm_tcp(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUt
                 }
             }
             const float sxm = (m < M) ? sx[m] : 0.0f;
-            // one thread waits for the accumulator, with the bound; its verdict reaches the other 127 through the
+            // one thread waits for the accumulator, with the bound; what it found reaches the other 127 through the
             // barrier that also publishes the scales above, so the four warps always take the same way
             if (et == 0) *epi_ok = mbar_wait(accf0 + 8u * buf, (lt >> 1) & 1u, abort_flag, status, 3) ? 1 : 0;
             asm volatile("bar.sync 1, 128;" ::: "memory");
