@@ -257,3 +257,37 @@ def test_decode_workload_rows(bq):
         check_output(y, X, W, idx, F16, exact_expected=False)
     y16 = lin.linear(X.cuda(), None)
     check_output(y16, X, W, idx, F16, exact_expected=False)
+
+
+def test_full_size_layer_all_tensor_kernels_and_sampled_rows(bq):
+    """The benchmark's layer at full size (4096 x 6144 -> 16384, bf16, 6 critical features) in the launch configurations
+    bench.py times: the CTA-pair and the single-CTA persistent kernels add the side features in the same order, so they
+    must agree bit for bit; the one-tile-per-CTA kernel accumulates them on the tensor cores (other order); rows sampled
+    across tiles and CTA pairs are checked against the oracle."""
+    X, W, idx = workloads.make_linear("mmd_prefill_moe")
+    Xd = X.cuda()
+    lin = bq.DecomposedLinear(W.cuda(), idx)
+    y_pair = lin.linear(Xd, path=2)
+    assert lin.kernel_status() == 0
+    y_solo = lin.linear(Xd, path=4)
+    assert lin.kernel_status() == 0
+    assert torch.equal(y_pair, y_solo)
+    y_tile = lin.linear(Xd, path=3)
+    assert lin.kernel_status() == 0
+    assert (y_tile == y_pair).float().mean().item() > 0.999
+    rows = np.array([0, 127, 128, 255, 256, 1500, 2047, 2048, 4095])
+    qw, sw, wo = mo.rowquant(bits(W), BF16, idx)
+    q_dev, s_dev, _, _ = lin.view()
+    assert np.array_equal(q_dev[-300:].cpu().numpy(), qw[-300:]) and np.array_equal(s_dev.cpu().numpy(), sw)
+    Xr = X[rows]
+    y_ref, _, _, sabs = mo.linear(bits(Xr), BF16, qw, sw, wo, idx, BF16, parts=True)
+    y32 = mo.linear(bits(Xr), BF16, qw, sw, wo, idx, F32).astype(np.float64)
+    tol = 2.0 ** -23 * np.abs(y32) + (wo.shape[1] + 2) * 2.0 ** -22 * sabs
+    lo = mo.widen(mo.narrow((y32 - tol).astype(np.float32), BF16), BF16)
+    hi = mo.widen(mo.narrow((y32 + tol).astype(np.float32), BF16), BF16)
+    for y in (y_pair, y_tile):
+        got = bits(y[torch.from_numpy(rows).cuda()])
+        g = mo.widen(got, BF16)
+        assert np.all((g >= lo) & (g <= hi))
+        assert np.mean(got == y_ref) > 0.999
+    lin.close()
