@@ -158,3 +158,37 @@ def test_kv_cache_shaped_tensor(bq):
     ref_c, ref_a = oracle.quantize(bits(kv.reshape(-1)), BF16, 128, oracle.make_codebook())
     c, a = bq.bq_quantize(kv.cuda().reshape(-1), 128, cb8)
     assert np.array_equal(c.cpu().numpy(), ref_c) and np.array_equal(a.cpu().numpy(), ref_a)
+
+
+def test_full_size_tensor_sampled_blocks(bq):
+    """The benchmark's 1 GiB tensor at full size through the vectorised kernels (blocks 64 and 1024, as bench.py times them):
+    absmax of every block against a device-side max, the error bound on every element, and sampled whole blocks (first, last,
+    random) bit for bit against the oracle."""
+    cb = bq.Codebook4()
+    cb_ref = o4.make_codebook()
+    x_cpu = workloads.make("sweep1g").view(-1)
+    n = x_cpu.numel()
+    xd = x_cpu.cuda()
+    xb = bits(x_cpu)
+    rng = np.random.default_rng(321)
+    for block in (64, 1024):
+        nb = n // block
+        p, a = bq.bq4_quantize(xd, block, cb)
+        y = bq.bq4_dequantize(p, a, n, block, cb, torch.bfloat16)
+        torch.cuda.synchronize()
+        assert torch.equal(a.view(torch.int32), xd.view(nb, block).abs().amax(dim=1).float().view(torch.int32))
+        step = 1 << 26
+        for s0 in range(0, n, step):
+            e0 = min(n, s0 + step)
+            a_el = a[s0 // block:(e0 + block - 1) // block].repeat_interleave(block)[: e0 - s0]
+            err = (xd[s0:e0].float() - y[s0:e0].float()).abs()
+            bound = a_el * (0.1125 + 2.0 ** -20) + y[s0:e0].float().abs() * 2.0 ** -8          # half the widest gap + bf16 rounding of y
+            assert bool((err <= bound).all().item())
+        pick = np.unique(np.concatenate([[0, 1, nb - 2, nb - 1], rng.integers(0, nb, max(8, 65536 // block))]))
+        for b in pick:
+            seg = np.ascontiguousarray(xb[b * block:(b + 1) * block])
+            p_ref, a_ref = o4.quantize(seg, BF16, block, cb_ref)
+            assert np.array_equal(p[b * block // 2:(b + 1) * block // 2].cpu().numpy(), p_ref)
+            assert a[b].item() == a_ref[0]
+            assert np.array_equal(bits(y[b * block:(b + 1) * block]), o4.dequantize(p_ref, a_ref, block, block, cb_ref, BF16))
+        del p, a, y
