@@ -46,6 +46,19 @@ bool make_map(CUtensorMap* map, const void* base, int elem_bytes, uint64_t rows,
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same matrix (K a multiple of 128, 1-byte elements) seen as (128 bytes, rows, K / 128): one load then brings
+// `box_kblocks` K blocks of `box_rows` rows, laid out block after block, each with the 128-byte swizzle.
+bool make_map_kblocks(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_kblocks) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn || cols % 128 != 0) return false;
+    const cuuint64_t dims[3] = {128, rows, cols / 128};
+    const cuuint64_t strides[2] = {cols, 128};
+    const cuuint32_t box[3] = {128, box_rows, box_kblocks};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int DT>
 cudaError_t launch_rowquant(const void* v, int R, int K, const int32_t* idx, int ko, int8_t* q, float* scale, void* side, int sm_count,
                             cudaStream_t stream) {
@@ -91,6 +104,8 @@ struct mmd_weights {
     int* status;
     bool have_maps;
     CUtensorMap map_q[3], map_side[3];       // weight tiles of 256, 128 and 64 rows
+    bool have_pair_map;                      // K a multiple of 128: the CTA-pair kernel's view of the codes
+    CUtensorMap map_q_pair;                  // (128 bytes, rows, K / 128), boxes of 128 rows x 2 K blocks
 };
 
 namespace {
@@ -204,7 +219,7 @@ cudaError_t launch_tc2(const mmd_weights* w, const CUtensorMap& mqx, const float
     const long total = long(mpairs) * ntiles;
     const unsigned pairs = unsigned(total < max_pairs[d] ? total : max_pairs[d]);
     mmdk::gemm_tc2<XDT, YDT><<<2 * pairs, mmdk::kTcThreads, mmdk::kPairSmemBytes, stream>>>(
-        mqx, w->map_q[1], sx, w->scale, sidex, w->side, w->side_cols, w->ko, y, M, w->N, (w->K + 127) / 128, mpairs, ntiles, w->status);
+        mqx, w->map_q_pair, sx, w->scale, sidex, w->side, w->side_cols, w->ko, y, M, w->N, (w->K + 127) / 128, mpairs, ntiles, w->status);
     return cudaGetLastError();
 }
 
@@ -312,6 +327,7 @@ int mmd_decompose(const void* W, bq_dtype dt, int N, int K, const int32_t* idx_h
     if (e == cudaSuccess) e = rowquant_any(dt, W, N, K, w->idx, n_features, w->q, w->scale, w->side, w->sm_count, stream);
     if (e != cudaSuccess) { cudaFree(w->blob); delete w; return cuda_fail(e); }
     w->have_maps = true;
+    w->have_pair_map = make_map_kblocks(&w->map_q_pair, w->q, uint64_t(N), uint64_t(K), 128, mmdk::kPairStepBlocks);
     const uint32_t boxes[3] = {256, 128, 64};
     for (int s = 0; s < 3; ++s) {
         w->have_maps = w->have_maps && make_map(&w->map_q[s], w->q, 1, uint64_t(N), uint64_t(K), boxes[s]);
@@ -368,7 +384,7 @@ int mmd_linear(const mmd_weights* w, const void* X, int M, void* Y, bq_dtype ydt
     if (path == MMD_PATH_TENSOR_SOLO && !wants_persistent(w, M)) return MMD_ERR_PATH;
     const bool use_tc = (path >= MMD_PATH_TENSOR) || (path == MMD_PATH_AUTO && tc_ok);
     const bool persistent = use_tc && path != MMD_PATH_TENSOR_TILE && wants_persistent(w, M);
-    const bool pairs = persistent && path != MMD_PATH_TENSOR_SOLO;
+    const bool pairs = persistent && path != MMD_PATH_TENSOR_SOLO && w->have_pair_map;      // the pair kernel's loads need K % 128 == 0
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     char* ws = static_cast<char*>(workspace);
@@ -381,7 +397,7 @@ int mmd_linear(const mmd_weights* w, const void* X, int M, void* Y, bq_dtype ydt
     const bool bf = (w->dtype == BQ_BF16), f32out = (ydt == BQ_F32);
     if (pairs) {
         CUtensorMap mqx;
-        if (!make_map(&mqx, qx, 1, uint64_t(M), uint64_t(w->K), 128)) return MMD_ERR_PATH;
+        if (!make_map_kblocks(&mqx, qx, uint64_t(M), uint64_t(w->K), 128, mmdk::kPairStepBlocks)) return MMD_ERR_PATH;
         if (bf) e = f32out ? launch_tc2<mmdk::kBF16, mmdk::kF32>(w, mqx, sx, sidex, Y, M, stream) : launch_tc2<mmdk::kBF16, mmdk::kBF16>(w, mqx, sx, sidex, Y, M, stream);
         else e = f32out ? launch_tc2<mmdk::kF16, mmdk::kF32>(w, mqx, sx, sidex, Y, M, stream) : launch_tc2<mmdk::kF16, mmdk::kF16>(w, mqx, sx, sidex, Y, M, stream);
     } else if (persistent) {

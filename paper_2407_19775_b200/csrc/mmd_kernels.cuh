@@ -829,17 +829,20 @@ gemm_tcp(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUt
 // are signalled in both CTAs by one multicast tcgen05.commit; "accumulator drained" lives in
 // the even CTA and takes one arrival per epilogue warp of both CTAs.  No load is multicast.
 
-constexpr int kPairStages = 6;
-constexpr uint32_t kPairHalfBytes = 128 * kTcRowBytes;                        // 128 rows of activations, or of weights
+constexpr int kPairStages = 3;
+constexpr int kPairStepBlocks = 2;                                            // K blocks of 128 features one TMA load brings
+constexpr uint32_t kPairSlabBytes = 128 * kTcRowBytes;                        // 128 rows x 128 features
+constexpr uint32_t kPairHalfBytes = kPairStepBlocks * kPairSlabBytes;         // a stage's activations, or its weights
 constexpr uint32_t kPairStageBytes = 2 * kPairHalfBytes;
 constexpr uint32_t kPairSmemBytes = kPairStages * kPairStageBytes + 1024 + kTcpCtrlBytes + kTcpSwBytes + kTcpWoBytes;
 
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar_cluster_addr) {
-    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar_cluster_addr) : "memory");
+// one load of a [K blocks][rows][128 bytes] box from a map that views the matrix as (128 bytes, rows, K / 128)
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, int row, int kblock, uint32_t bar_cluster_addr) {
+    asm volatile("cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(dst), "l"(map), "r"(0), "r"(row), "r"(kblock), "r"(bar_cluster_addr) : "memory");
 }
 __device__ __forceinline__ void umma_i8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
@@ -973,6 +976,7 @@ gemm_tc2(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUt
     const uint32_t rank = cluster_rank();
     const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
     const int total_tiles = mpairs * ntiles;
+    const int ksteps = (kblocks + kPairStepBlocks - 1) / kPairStepBlocks;      // ring steps per tile
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, 1); }
@@ -998,15 +1002,15 @@ gemm_tc2(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUt
             for (int t = pair; t < total_tiles && ok; t += npairs) {
                 const int m0 = (t % mpairs) * 256 + int(rank) * 128;             // this CTA's activation rows
                 const int nb0 = (t / mpairs) * BN + int(rank) * 128;             // this CTA's half of the weight rows
-                for (int i = 0; i < kblocks; ++i, ++it) {
+                for (int i = 0; i < ksteps; ++i, ++it) {
                     const uint32_t s = it % S, round = it / S;
                     ok = mbar_wait(empty0 + 8u * s, (round & 1u) ^ 1u, abort_flag, status, 1);
                     if (!ok) break;
                     const uint32_t a_dst = tiles_sm + s * kPairStageBytes, b_dst = a_dst + kPairHalfBytes;
                     const uint32_t full_even = map_to_cta(full0 + 8u * s, 0);
                     if (rank == 0) mbar_expect_tx(full0 + 8u * s, 2 * kPairStageBytes);      // both CTAs' bytes
-                    tma_load_2d_pair(a_dst, &map_qx, i * 128, m0, full_even);
-                    tma_load_2d_pair(b_dst, &map_qw, i * 128, nb0, full_even);
+                    tma_load_3d_pair(a_dst, &map_qx, m0, i * kPairStepBlocks, full_even);     // a K block past the end reads as zeros
+                    tma_load_3d_pair(b_dst, &map_qw, nb0, i * kPairStepBlocks, full_even);
                 }
             }
         }
@@ -1022,16 +1026,19 @@ gemm_tc2(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUt
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t d_tmem = tmem + buf * uint32_t(BN);
-                for (int i = 0; i < kblocks; ++i, ++it) {
+                for (int i = 0; i < ksteps; ++i, ++it) {
                     const uint32_t s = it % S, round = it / S;
                     ok = mbar_wait(full0 + 8u * s, round & 1u, abort_flag, status, 2);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t a_src = tiles_sm + s * kPairStageBytes, b_src = a_src + kPairHalfBytes;
-                    const uint64_t adesc = umma_smem_desc(a_src), bdesc = umma_smem_desc(b_src);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        umma_i8_pair(d_tmem, adesc + uint64_t(2 * k), bdesc + uint64_t(2 * k), idesc_i8, (i > 0 || k > 0) ? 1u : 0u);
+                    for (int j = 0; j < kPairStepBlocks; ++j) {
+                        const uint64_t adesc = umma_smem_desc(a_src + uint32_t(j) * kPairSlabBytes), bdesc = umma_smem_desc(b_src + uint32_t(j) * kPairSlabBytes);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            umma_i8_pair(d_tmem, adesc + uint64_t(2 * k), bdesc + uint64_t(2 * k), idesc_i8, (i > 0 || j > 0 || k > 0) ? 1u : 0u);
+                    }
                     umma_commit_pair(empty0 + 8u * s);
                 }
                 if (ok) umma_commit_pair(accf0 + 8u * buf);
