@@ -131,25 +131,27 @@ int bn_slot(int bn) { return bn == 256 ? 0 : (bn == 128 ? 1 : 2); }
 // Rows of the activation tiles the one-tile-per-CTA kernel loads: a decode step's few rows need only half a tile.
 int activation_box_rows(int M) { return M <= 64 ? 64 : 128; }
 
-template <int XDT, int YDT, int BN, int BM>
+template <int XDT, int YDT, int BN, int BM, int KPB>
 cudaError_t launch_tc_bm(const mmd_weights* w, const CUtensorMap& mqx, const CUtensorMap& msx, const float* sx, void* y, int M, int split,
                          cudaStream_t stream) {
-    using Cfg = mmdk::TcCfg<BN, BM>;
+    using Cfg = mmdk::TcCfg<BN, BM, KPB>;
     static bool opted[64] = {};
     if (w->device < 0 || w->device >= 64 || !opted[w->device]) {
-        const cudaError_t e = cudaFuncSetAttribute(mmdk::gemm_tc<XDT, YDT, BN, BM>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::kSmemBytes));
+        const cudaError_t e = cudaFuncSetAttribute(mmdk::gemm_tc<XDT, YDT, BN, BM, KPB>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::kSmemBytes));
         if (e != cudaSuccess) return e;
         if (w->device >= 0 && w->device < 64) opted[w->device] = true;
     }
     int kblocks = (w->K + 127) / 128, sblocks = w->side_cols / 64;
+    const int ksteps = (kblocks + KPB - 1) / KPB;
     const int slot = bn_slot(BN);
-    uint32_t tx = uint32_t(BM + BN) * 128u;
+    CUtensorMap mqw = w->map_q[slot];
+    if (KPB > 1 && !make_map_kblocks(&mqw, w->q, uint64_t(w->N), uint64_t(w->K), BN, KPB)) return cudaErrorInvalidValue;
     int* status = w->status;
     int Mv = M, Nv = w->N;
     const float* swv = w->scale;
     // the ranks' partial sums must fit into rank 0's ring
     if (split > 1 && size_t(split - 1) * BM * BN * 4 > size_t(Cfg::kStages) * Cfg::kStageBytes) split = 1;
-    if (split > kblocks) split = kblocks;
+    if (split > ksteps) split = ksteps;
     if (split < 1) split = 1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(unsigned((M + BM - 1) / BM), unsigned((w->N + BN - 1) / BN), unsigned(split));
@@ -167,16 +169,25 @@ cudaError_t launch_tc_bm(const mmd_weights* w, const CUtensorMap& mqx, const CUt
     attr[1].val.clusterDim.z = unsigned(split);
     cfg.attrs = attr;
     cfg.numAttrs = split > 1 ? 2 : 1;
-    return cudaLaunchKernelEx(&cfg, mmdk::gemm_tc<XDT, YDT, BN, BM>, mqx, w->map_q[slot], sblocks ? msx : mqx,
-                              sblocks ? w->map_side[slot] : w->map_q[slot], sx, swv, y, Mv, Nv, kblocks, sblocks, tx, status);
+    return cudaLaunchKernelEx(&cfg, mmdk::gemm_tc<XDT, YDT, BN, BM, KPB>, mqx, mqw, sblocks ? msx : mqx,
+                              sblocks ? w->map_side[slot] : w->map_q[slot], sx, swv, y, Mv, Nv, kblocks, sblocks, status);
 }
 
 // At most 64 activation rows: 64-row MMAs and 64-row activation boxes (the host's maps are made to match).
 template <int XDT, int YDT, int BN>
 cudaError_t launch_tc(const mmd_weights* w, const CUtensorMap& mqx, const CUtensorMap& msx, const float* sx, void* y, int M, int split,
                       cudaStream_t stream) {
-    return activation_box_rows(M) == 64 ? launch_tc_bm<XDT, YDT, BN, 64>(w, mqx, msx, sx, y, M, split, stream)
-                                        : launch_tc_bm<XDT, YDT, BN, 128>(w, mqx, msx, sx, y, M, split, stream);
+    return activation_box_rows(M) == 64 ? launch_tc_bm<XDT, YDT, BN, 64, 1>(w, mqx, msx, sx, y, M, split, stream)
+                                        : launch_tc_bm<XDT, YDT, BN, 128, 1>(w, mqx, msx, sx, y, M, split, stream);
+}
+
+// Decode-size calls (one row of tiles) with K a multiple of 128: two K blocks per load.  `mqx2` is the activations'
+// three-dimensional map with boxes of activation_box_rows(M) rows x 2 K blocks.
+template <int XDT, int YDT>
+cudaError_t launch_tc_decode(const mmd_weights* w, const CUtensorMap& mqx2, const CUtensorMap& msx, const float* sx, void* y, int M, int split,
+                             cudaStream_t stream) {
+    return activation_box_rows(M) == 64 ? launch_tc_bm<XDT, YDT, 128, 64, 2>(w, mqx2, msx, sx, y, M, split, stream)
+                                        : launch_tc_bm<XDT, YDT, 128, 128, 2>(w, mqx2, msx, sx, y, M, split, stream);
 }
 
 template <int XDT, int YDT>
@@ -229,7 +240,7 @@ bool wants_persistent(const mmd_weights* w, int M) {
 }
 
 template <int XDT, int YDT>
-cudaError_t launch_tc_bn(const mmd_weights* w, const CUtensorMap& mqx, const CUtensorMap& msx, const float* sx, void* y, int M,
+cudaError_t launch_tc_bn(const mmd_weights* w, const CUtensorMap& mqx, const CUtensorMap& msx, const int8_t* qx, const float* sx, void* y, int M,
                          cudaStream_t stream) {
     // The widest tile has the highest arithmetic intensity; when it would leave SMs without a
     // tile (few rows, as in a decode step, where the weights are read once and the kernel is
@@ -245,6 +256,12 @@ cudaError_t launch_tc_bn(const mmd_weights* w, const CUtensorMap& mqx, const CUt
         int split = int(w->sm_count / tiles);
         if (split > 4) split = 4;
         if (split < 1) split = 1;
+        if (w->have_pair_map) {                                                  // K a multiple of 128: two K blocks per load
+            while (split > 1 && (w->K + 255) / 256 < 4 * split) --split;        // at least 4 steps per CTA
+            CUtensorMap mqx2;
+            if (make_map_kblocks(&mqx2, qx, uint64_t(M), uint64_t(w->K), uint32_t(activation_box_rows(M)), 2))
+                return launch_tc_decode<XDT, YDT>(w, mqx2, msx, sx, y, M, split, stream);
+        }
         while (split > 1 && (w->K + 127) / 128 < 8 * split) --split;            // at least 8 steps per CTA
         return launch_tc<XDT, YDT, 128>(w, mqx, msx, sx, y, M, split, stream);
     }
@@ -411,8 +428,8 @@ int mmd_linear(const mmd_weights* w, const void* X, int M, void* Y, bq_dtype ydt
         if (!make_map(&mqx, qx, 1, uint64_t(M), uint64_t(w->K), arows)) return MMD_ERR_PATH;
         if (w->side_cols > 0 && !make_map(&msx, sidex, 2, uint64_t(M), uint64_t(w->side_cols), arows)) return MMD_ERR_PATH;
         if (w->side_cols == 0) msx = mqx;
-        if (bf) e = f32out ? launch_tc_bn<mmdk::kBF16, mmdk::kF32>(w, mqx, msx, sx, Y, M, stream) : launch_tc_bn<mmdk::kBF16, mmdk::kBF16>(w, mqx, msx, sx, Y, M, stream);
-        else e = f32out ? launch_tc_bn<mmdk::kF16, mmdk::kF32>(w, mqx, msx, sx, Y, M, stream) : launch_tc_bn<mmdk::kF16, mmdk::kF16>(w, mqx, msx, sx, Y, M, stream);
+        if (bf) e = f32out ? launch_tc_bn<mmdk::kBF16, mmdk::kF32>(w, mqx, msx, qx, sx, Y, M, stream) : launch_tc_bn<mmdk::kBF16, mmdk::kBF16>(w, mqx, msx, qx, sx, Y, M, stream);
+        else e = f32out ? launch_tc_bn<mmdk::kF16, mmdk::kF32>(w, mqx, msx, qx, sx, Y, M, stream) : launch_tc_bn<mmdk::kF16, mmdk::kF16>(w, mqx, msx, qx, sx, Y, M, stream);
     } else {
         if (bf) e = f32out ? launch_general<mmdk::kBF16, mmdk::kF32>(w, qx, sx, sidex, Y, M, stream) : launch_general<mmdk::kBF16, mmdk::kBF16>(w, qx, sx, sidex, Y, M, stream);
         else e = f32out ? launch_general<mmdk::kF16, mmdk::kF32>(w, qx, sx, sidex, Y, M, stream) : launch_general<mmdk::kF16, mmdk::kF16>(w, qx, sx, sidex, Y, M, stream);

@@ -256,11 +256,15 @@ constexpr long long kWaitLimitCycles = 4000000000ll;            // about two sec
 
 // BM = rows of the MMA: 128, or 64 for calls with at most 64 activation rows (a decode step), whose ring stages then
 // spend 8 KB instead of 16 KB on activations and hold more steps of the weight stream in flight.
-template <int BN, int BM = kTcBM> struct TcCfg {
-    static constexpr int kStages = (BM == 64) ? (BN >= 256 ? 4 : (BN >= 128 ? 8 : 12)) : ((BN >= 256) ? 4 : (BN >= 128 ? 6 : 8));
-    static constexpr uint32_t kABytes = BM * kTcRowBytes;
-    static constexpr uint32_t kBBytes = BN * kTcRowBytes;
+// KPB = K blocks of 128 features one ring step (one TMA load per operand) brings: 1, or 2 for decode-size calls, where
+// the pace is set by the number of loads rather than by their bytes.
+template <int BN, int BM = kTcBM, int KPB = 1> struct TcCfg {
+    static constexpr uint32_t kASlabBytes = BM * kTcRowBytes;                   // one K block of the activation tile
+    static constexpr uint32_t kBSlabBytes = BN * kTcRowBytes;
+    static constexpr uint32_t kABytes = KPB * kASlabBytes;
+    static constexpr uint32_t kBBytes = KPB * kBSlabBytes;
     static constexpr uint32_t kStageBytes = kABytes + kBBytes;
+    static constexpr int kStages = (196608u / kStageBytes) > 12u ? 12 : int(196608u / kStageBytes);
     static constexpr uint32_t kTmemCols = (2 * BN <= 32) ? 32 : 2 * BN;          // a power of two >= 32
     static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 2048 /* barriers, scales */;
 };
@@ -299,6 +303,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// a [K blocks][rows][128 bytes] box from a map that views the matrix as (128 bytes, rows, K / 128)
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int row, int kblock, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(dst), "l"(map), "r"(0), "r"(row), "r"(kblock), "r"(bar) : "memory");
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                  ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
@@ -363,14 +372,15 @@ __device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v
     asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
 }
 
-template <int XDT, int YDT, int BN, int BM>
+template <int XDT, int YDT, int BN, int BM, int KPB>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUtensorMap map_qw,
         const __grid_constant__ CUtensorMap map_sidex, const __grid_constant__ CUtensorMap map_sidew,
         const float* __restrict__ sx, const float* __restrict__ sw, void* __restrict__ y,
-        int M, int N, int kblocks_all /* int8 steps of 128 features */, int sblocks_all /* side steps of 64 columns */,
-        uint32_t stage_tx_bytes /* bytes the two loads of a stage bring: (activation rows in the map's box + BN) * 128 */, int* status) {
-    using Cfg = TcCfg<BN, BM>;
+        int M, int N, int kblocks_all /* K blocks of 128 int8 features */, int sblocks_all /* side steps of 64 columns */, int* status) {
+    using Cfg = TcCfg<BN, BM, KPB>;
+    constexpr uint32_t kTxMain = Cfg::kStageBytes;                              // bytes of an int8 step's two loads (boxes of BM and BN rows)
+    constexpr uint32_t kTxSide = Cfg::kASlabBytes + Cfg::kBSlabBytes;           // bytes of a side step's two loads
     constexpr int S = Cfg::kStages;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;               // swizzled tiles need 1024-byte alignment
@@ -385,7 +395,8 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
     const uint32_t nsplit = cluster_size(), rank = cluster_rank();              // 1 and 0 without a cluster launch
-    const int kb_lo = int((long(kblocks_all) * rank) / nsplit), kb_hi = int((long(kblocks_all) * (rank + 1)) / nsplit);
+    const int ksteps_all = (kblocks_all + KPB - 1) / KPB;                       // int8 ring steps of KPB K blocks each
+    const int kb_lo = int((long(ksteps_all) * rank) / nsplit), kb_hi = int((long(ksteps_all) * (rank + 1)) / nsplit);
     const int kblocks = kb_hi - kb_lo;                                          // this CTA's share of the int8 steps
     const int sblocks = (rank == 0) ? sblocks_all : 0;
     const int steps = kblocks + sblocks;
@@ -405,6 +416,11 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = *tmem_slot;
+    // the load of one int8 step of one operand: KPB K blocks of `rows` rows from K block `step * KPB` on
+    auto load_main = [&](uint32_t dst, const CUtensorMap* map, int row0, int step, uint32_t bar) {
+        if constexpr (KPB == 1) tma_load_2d(dst, map, step * 128, row0, bar);
+        else tma_load_3d(dst, map, row0, step * KPB, bar);                      // a K block past the end reads as zeros
+    };
 
     if (warp == 0) {
         if (lane == 0) {
@@ -413,14 +429,14 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
             const int pre = steps < S ? steps : S;
             for (int i = 0; i < pre; ++i) {
                 const uint32_t b_dst = tiles + uint32_t(i) * Cfg::kStageBytes + Cfg::kABytes;
-                mbar_expect_tx(full0 + 8u * i, stage_tx_bytes);
-                if (i < kblocks) tma_load_2d(b_dst, &map_qw, (kb_lo + i) * 128, n0, full0 + 8u * i);
+                mbar_expect_tx(full0 + 8u * i, i < kblocks ? kTxMain : kTxSide);
+                if (i < kblocks) load_main(b_dst, &map_qw, n0, kb_lo + i, full0 + 8u * i);
                 else tma_load_2d(b_dst, &map_sidew, (i - kblocks) * 64, n0, full0 + 8u * i);
             }
             asm volatile("griddepcontrol.wait;" ::: "memory");
             for (int i = 0; i < pre; ++i) {
                 const uint32_t a_dst = tiles + uint32_t(i) * Cfg::kStageBytes;
-                if (i < kblocks) tma_load_2d(a_dst, &map_qx, (kb_lo + i) * 128, m0, full0 + 8u * i);
+                if (i < kblocks) load_main(a_dst, &map_qx, m0, kb_lo + i, full0 + 8u * i);
                 else tma_load_2d(a_dst, &map_sidex, (i - kblocks) * 64, m0, full0 + 8u * i);
             }
             for (int i = pre; i < steps; ++i) {
@@ -428,10 +444,10 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
                 const uint32_t round = uint32_t(i / S);
                 if (!mbar_wait(empty0 + 8u * s, (round & 1u) ^ 1u, abort_flag, status, 1)) break;
                 const uint32_t a_dst = tiles + uint32_t(s) * Cfg::kStageBytes, b_dst = a_dst + Cfg::kABytes;
-                mbar_expect_tx(full0 + 8u * s, stage_tx_bytes);
+                mbar_expect_tx(full0 + 8u * s, i < kblocks ? kTxMain : kTxSide);
                 if (i < kblocks) {
-                    tma_load_2d(a_dst, &map_qx, (kb_lo + i) * 128, m0, full0 + 8u * s);
-                    tma_load_2d(b_dst, &map_qw, (kb_lo + i) * 128, n0, full0 + 8u * s);
+                    load_main(a_dst, &map_qx, m0, kb_lo + i, full0 + 8u * s);
+                    load_main(b_dst, &map_qw, n0, kb_lo + i, full0 + 8u * s);
                 } else {
                     tma_load_2d(a_dst, &map_sidex, (i - kblocks) * 64, m0, full0 + 8u * s);
                     tma_load_2d(b_dst, &map_sidew, (i - kblocks) * 64, n0, full0 + 8u * s);
@@ -455,8 +471,12 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
                 const uint64_t adesc = umma_smem_desc(a_src), bdesc = umma_smem_desc(b_src);
                 if (i < kblocks) {
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)                       // 32 int8 features = 32 bytes per MMA
-                        umma_i8(tmem, adesc + uint64_t(2 * k), bdesc + uint64_t(2 * k), idesc_i8, (i > 0 || k > 0) ? 1u : 0u);
+                    for (int j = 0; j < KPB; ++j) {
+                        const uint64_t aj = umma_smem_desc(a_src + uint32_t(j) * Cfg::kASlabBytes), bj = umma_smem_desc(b_src + uint32_t(j) * Cfg::kBSlabBytes);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)                   // 32 int8 features = 32 bytes per MMA
+                            umma_i8(tmem, aj + uint64_t(2 * k), bj + uint64_t(2 * k), idesc_i8, (i > 0 || j > 0 || k > 0) ? 1u : 0u);
+                    }
                 } else {
 #pragma unroll
                     for (int k = 0; k < 4; ++k)                       // 16 side columns = 32 bytes per MMA
