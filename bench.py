@@ -310,9 +310,9 @@ MMD_WORKLOAD = "mmd_prefill_moe"
 NOMINAL_INT8_OVER_BF16 = 2.0          # dense int8 (4.5 POP/s) over dense bf16 (2.25 PFLOP/s)
 FALLBACK_BF16_TFLOPS = 1590.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch of the product kernel (a one-pass ncu capture of
-# the full layer: 130.44 MB read for 128.5 MB of codes, side columns and scales; 105.09 MB written, the rest of the 134.2 MB
+# the full layer: 130.28 MB read for 128.5 MB of codes, side columns and scales; 104.04 MB written, the rest of the 134.2 MB
 # of Y still being dirty lines in L2 when the kernel ends).  Set to None when the kernel changes until it is re-measured.
-MMD_TRAFFIC_BYTES = 235530000
+MMD_TRAFFIC_BYTES = 234320000
 
 
 def measured_tensor_peak():

@@ -181,8 +181,8 @@ cudaError_t launch_tc(const mmd_weights* w, const CUtensorMap& mqx, const CUtens
                                         : launch_tc_bm<XDT, YDT, BN, 128, 1>(w, mqx, msx, sx, y, M, split, stream);
 }
 
-// Decode-size calls (one row of tiles) with K a multiple of 128: two K blocks per load.  `mqx2` is the activations'
-// three-dimensional map with boxes of activation_box_rows(M) rows x 2 K blocks.
+// 128-column tiles with K a multiple of 128: two K blocks per load (decode-size calls and mid-size products).  `mqx2` is
+// the activations' three-dimensional map with boxes of activation_box_rows(M) rows x 2 K blocks.
 template <int XDT, int YDT>
 cudaError_t launch_tc_decode(const mmd_weights* w, const CUtensorMap& mqx2, const CUtensorMap& msx, const float* sx, void* y, int M, int split,
                              cudaStream_t stream) {
@@ -236,7 +236,8 @@ cudaError_t launch_tc2(const mmd_weights* w, const CUtensorMap& mqx, const float
 
 // Large products with few critical features take the persistent kernels.
 bool wants_persistent(const mmd_weights* w, int M) {
-    return w->ko <= mmdk::kTcpSide && w->N >= 256 && long((M + 127) / 128) * ((w->N + 255) / 256) >= w->sm_count;
+    // from about half a wave of 128 x 256 tiles on: below that the one-tile-per-CTA kernel's narrower tiles fill the SMs better
+    return w->ko <= mmdk::kTcpSide && w->N >= 256 && long((M + 127) / 128) * ((w->N + 255) / 256) >= w->sm_count / 2;
 }
 
 template <int XDT, int YDT>
@@ -247,7 +248,12 @@ cudaError_t launch_tc_bn(const mmd_weights* w, const CUtensorMap& mqx, const CUt
     // bound by that stream) narrower tiles put more CTAs on the weight stream.
     const long mt = (M + 127) / 128;
     if (w->N >= 256 && mt * ((w->N + 255) / 256) >= w->sm_count) return launch_tc<XDT, YDT, 256>(w, mqx, msx, sx, y, M, 1, stream);
-    if (w->N >= 128 && mt * ((w->N + 127) / 128) >= w->sm_count) return launch_tc<XDT, YDT, 128>(w, mqx, msx, sx, y, M, 1, stream);
+    if (w->N >= 128 && mt * ((w->N + 127) / 128) >= w->sm_count) {
+        CUtensorMap mqx2;                                                        // K a multiple of 128: two K blocks per load
+        if (w->have_pair_map && make_map_kblocks(&mqx2, qx, uint64_t(M), uint64_t(w->K), uint32_t(activation_box_rows(M)), 2))
+            return launch_tc_decode<XDT, YDT>(w, mqx2, msx, sx, y, M, 1, stream);
+        return launch_tc<XDT, YDT, 128>(w, mqx, msx, sx, y, M, 1, stream);
+    }
     // One row of tiles (a decode step) streams every weight once from DRAM, and an SM streams only as fast as the bytes it
     // keeps in flight.  128-row weight tiles hold the most per CTA; when they leave SMs idle, 2-4 CTAs share each tile's K
     // steps (clusters along z) so that about one CTA per SM is streaming.
