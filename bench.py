@@ -413,22 +413,35 @@ def run_mmd(bq, dev, args):
     cpu_s = time.perf_counter() - t
     lin.close()
 
-    # a decode step through a 70B-class layer: 64 tokens, every weight read once (HBM-bound)
+    # a decode step through a 70B-class layer: 64 tokens, every weight read once (HBM-bound).  The codes of one layer (67 MB)
+    # would stay in the 126 MB L2 from call to call, so the timed graph cycles through four copies of the layer (268 MB):
+    # every call streams its weights from DRAM, as consecutive layers of a model do.
     dX, dW, didx = workloads.make_linear("mmd_decode70b")
     dM, dK, dN = dX.shape[0], dX.shape[1], dW.shape[0]
     dXd = dX.to(dev)
-    dlin = bq.DecomposedLinear(dW.to(dev), didx)
+    dWd = dW.to(dev)
+    dlins = [bq.DecomposedLinear(dWd, didx) for _ in range(DECODE_LAYER_COPIES)]
     dy = torch.empty((dM, dN), dtype=dX.dtype, device=dev)
-    dws = dlin.workspace(dM)
-    dlin.linear(dXd, y_out=dy, workspace=dws)
+    dws = dlins[0].workspace(dM)
+    for dl in dlins:
+        dl.linear(dXd, y_out=dy, workspace=dws)
     torch.cuda.synchronize()
-    ms_dec = timed_gpu(lambda: dlin.linear(dXd, y_out=dy, workspace=dws), 8)
-    dstatus = dlin.kernel_status()
+    turn = [0]
+
+    def decode_call():
+        dlins[turn[0] % DECODE_LAYER_COPIES].linear(dXd, y_out=dy, workspace=dws)
+        turn[0] += 1
+
+    ms_dec = timed_gpu(decode_call, 2 * DECODE_LAYER_COPIES)
+    dstatus = max(dl.kernel_status() for dl in dlins)
     dec_bytes = dN * dK + dM * dK * 3 + dM * dN * 2
-    decode = {"workload": f"mmd_decode70b: X [{dM},{dK}] x W [{dN},{dK}]^T fp16, {didx.size} critical features", "us_per_call": round(ms_dec * 1e3, 2),
+    decode = {"workload": f"mmd_decode70b: X [{dM},{dK}] x W [{dN},{dK}]^T fp16, {didx.size} critical features; "
+                          f"{DECODE_LAYER_COPIES} copies of the layer in turn ({DECODE_LAYER_COPIES * dN * dK >> 20} MiB of codes, larger than L2)",
+              "us_per_call": round(ms_dec * 1e3, 2),
               "algorithmic_bytes": int(dec_bytes), "gbs": round(dec_bytes / ms_dec / 1e6, 1), "frac_of_measured_hbm": round(dec_bytes / ms_dec / 1e6 / hbm, 4),
               "kernel_status": dstatus}
-    dlin.close()
+    for dl in dlins:
+        dl.close()
     return {
         "workload": f"{MMD_WORKLOAD}: X [{M},{K}] x W [{N},{K}]^T bf16, {idx.size} critical features; {wl.recipe}",
         "ms_per_call": round(ms_call, 4), "tops": round(ops / ms_call / 1e9, 1), "kernel_status": status,
@@ -447,6 +460,8 @@ def run_mmd(bq, dev, args):
         "gpu_launches": (2 * 2 + 8 + 2 * 8) * reps + 2 * (reps + 3),
     }
 
+
+DECODE_LAYER_COPIES = 4
 
 # DRAM bytes per full-size launch (dram__bytes_read.sum + dram__bytes_write.sum), from ncu
 # captures of the first 8192 rows scaled to 65536 rows: reads scale with the rows (they equal

@@ -133,7 +133,7 @@ int activation_box_rows(int M) { return M <= 64 ? 64 : 128; }
 
 template <int XDT, int YDT, int BN, int BM, int KPB>
 cudaError_t launch_tc_bm(const mmd_weights* w, const CUtensorMap& mqx, const CUtensorMap& msx, const float* sx, void* y, int M, int split,
-                         cudaStream_t stream) {
+                         cudaStream_t stream, int n_tile_base = 0, int n_tile_count = -1) {
     using Cfg = mmdk::TcCfg<BN, BM, KPB>;
     static bool opted[64] = {};
     if (w->device < 0 || w->device >= 64 || !opted[w->device]) {
@@ -154,23 +154,43 @@ cudaError_t launch_tc_bm(const mmd_weights* w, const CUtensorMap& mqx, const CUt
     if (split > ksteps) split = ksteps;
     if (split < 1) split = 1;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(unsigned((M + BM - 1) / BM), unsigned((w->N + BN - 1) / BN), unsigned(split));
+    if (n_tile_count < 0) n_tile_count = (w->N + BN - 1) / BN - n_tile_base;
     cfg.blockDim = dim3(mmdk::kTcThreads, 1, 1);
     cfg.dynamicSmemBytes = Cfg::kSmemBytes;
     cfg.stream = stream;
-    // The row kernel launched just before lets this kernel start early (its set-up and first weight loads overlap the row
-    // kernel); the kernel itself waits for the row kernel's results before it touches them.
     cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
     attr[1].id = cudaLaunchAttributeClusterDimension;
     attr[1].val.clusterDim.x = 1;
     attr[1].val.clusterDim.y = 1;
+    // The split is there to put one CTA on every SM at the same time.  A cluster's CTAs must sit in one GPC, so fewer
+    // clusters of 3 or 4 fit on the device than its SM count suggests; a split whose clusters would not all run at once
+    // (a second, nearly empty wave) is lowered until they do.
+    static int max_clusters[64][5] = {};
+    const long clusters = long((M + BM - 1) / BM) * n_tile_count;
+    for (; split > 1; --split) {
+        const int d = (w->device >= 0 && w->device < 64) ? w->device : 0;
+        if (max_clusters[d][split] == 0) {
+            cfg.gridDim = dim3(1, unsigned(w->sm_count / split), unsigned(split));
+            attr[1].val.clusterDim.z = unsigned(split);
+            cfg.attrs = &attr[1];
+            cfg.numAttrs = 1;
+            int n = 0;
+            const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, mmdk::gemm_tc<XDT, YDT, BN, BM, KPB>, &cfg);
+            if (e != cudaSuccess) return e;
+            max_clusters[d][split] = n > 0 ? n : -1;
+        }
+        if (clusters <= max_clusters[d][split]) break;
+    }
+    cfg.gridDim = dim3(unsigned((M + BM - 1) / BM), unsigned(n_tile_count), unsigned(split));
+    // The row kernel launched just before lets this kernel start early (its set-up and first weight loads overlap the row
+    // kernel); the kernel itself waits for the row kernel's results before it touches them.
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
     attr[1].val.clusterDim.z = unsigned(split);
     cfg.attrs = attr;
     cfg.numAttrs = split > 1 ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, mmdk::gemm_tc<XDT, YDT, BN, BM, KPB>, mqx, mqw, sblocks ? msx : mqx,
-                              sblocks ? w->map_side[slot] : w->map_q[slot], sx, swv, y, Mv, Nv, kblocks, sblocks, status);
+                              sblocks ? w->map_side[slot] : w->map_q[slot], sx, swv, y, Mv, Nv, kblocks, sblocks, n_tile_base, status);
 }
 
 // At most 64 activation rows: 64-row MMAs and 64-row activation boxes (the host's maps are made to match).
@@ -185,9 +205,9 @@ cudaError_t launch_tc(const mmd_weights* w, const CUtensorMap& mqx, const CUtens
 // the activations' three-dimensional map with boxes of activation_box_rows(M) rows x 2 K blocks.
 template <int XDT, int YDT>
 cudaError_t launch_tc_decode(const mmd_weights* w, const CUtensorMap& mqx2, const CUtensorMap& msx, const float* sx, void* y, int M, int split,
-                             cudaStream_t stream) {
-    return activation_box_rows(M) == 64 ? launch_tc_bm<XDT, YDT, 128, 64, 2>(w, mqx2, msx, sx, y, M, split, stream)
-                                        : launch_tc_bm<XDT, YDT, 128, 128, 2>(w, mqx2, msx, sx, y, M, split, stream);
+                             cudaStream_t stream, int n_tile_base = 0, int n_tile_count = -1) {
+    return activation_box_rows(M) == 64 ? launch_tc_bm<XDT, YDT, 128, 64, 2>(w, mqx2, msx, sx, y, M, split, stream, n_tile_base, n_tile_count)
+                                        : launch_tc_bm<XDT, YDT, 128, 128, 2>(w, mqx2, msx, sx, y, M, split, stream, n_tile_base, n_tile_count);
 }
 
 template <int XDT, int YDT>
@@ -236,8 +256,9 @@ cudaError_t launch_tc2(const mmd_weights* w, const CUtensorMap& mqx, const float
 
 // Large products with few critical features take the persistent kernels.
 bool wants_persistent(const mmd_weights* w, int M) {
-    // from about half a wave of 128 x 256 tiles on: below that the one-tile-per-CTA kernel's narrower tiles fill the SMs better
-    return w->ko <= mmdk::kTcpSide && w->N >= 256 && long((M + 127) / 128) * ((w->N + 255) / 256) >= w->sm_count / 2;
+    // from about half a wave of 128 x 256 tiles on: below that the one-tile-per-CTA kernel's narrower tiles fill the SMs better.
+    // One row of tiles (a decode step) is bound by the weight stream, not by the tensor cores: it stays with that kernel too.
+    return w->ko <= mmdk::kTcpSide && w->N >= 256 && M > 128 && long((M + 127) / 128) * ((w->N + 255) / 256) >= w->sm_count / 2;
 }
 
 template <int XDT, int YDT>
@@ -250,8 +271,24 @@ cudaError_t launch_tc_bn(const mmd_weights* w, const CUtensorMap& mqx, const CUt
     if (w->N >= 256 && mt * ((w->N + 255) / 256) >= w->sm_count) return launch_tc<XDT, YDT, 256>(w, mqx, msx, sx, y, M, 1, stream);
     if (w->N >= 128 && mt * ((w->N + 127) / 128) >= w->sm_count) {
         CUtensorMap mqx2;                                                        // K a multiple of 128: two K blocks per load
-        if (w->have_pair_map && make_map_kblocks(&mqx2, qx, uint64_t(M), uint64_t(w->K), uint32_t(activation_box_rows(M)), 2))
+        if (w->have_pair_map && make_map_kblocks(&mqx2, qx, uint64_t(M), uint64_t(w->K), uint32_t(activation_box_rows(M)), 2)) {
+            // One row of tiles that does not fill whole waves (a decode step through a wide layer): the whole waves run one
+            // tile per CTA, and the tiles left over share their K steps among 2-4 CTAs each, so that the last wave also
+            // keeps about one CTA per SM on the weight stream instead of running at full length on a few SMs.
+            const long tiles = (w->N + 127) / 128;
+            const long rest = tiles % w->sm_count;
+            if (mt == 1 && rest > 0 && rest <= w->sm_count / 2) {
+                int split = int(w->sm_count / rest);
+                if (split > 4) split = 4;
+                while (split > 1 && (w->K + 255) / 256 < 4 * split) --split;    // at least 4 steps per CTA
+                if (split > 1) {
+                    const cudaError_t e = launch_tc_decode<XDT, YDT>(w, mqx2, msx, sx, y, M, 1, stream, 0, int(tiles - rest));
+                    if (e != cudaSuccess) return e;
+                    return launch_tc_decode<XDT, YDT>(w, mqx2, msx, sx, y, M, split, stream, int(tiles - rest), int(rest));
+                }
+            }
             return launch_tc_decode<XDT, YDT>(w, mqx2, msx, sx, y, M, 1, stream);
+        }
         return launch_tc<XDT, YDT, 128>(w, mqx, msx, sx, y, M, 1, stream);
     }
     // One row of tiles (a decode step) streams every weight once from DRAM, and an SM streams only as fast as the bytes it

@@ -377,7 +377,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUtensorMap map_qw,
         const __grid_constant__ CUtensorMap map_sidex, const __grid_constant__ CUtensorMap map_sidew,
         const float* __restrict__ sx, const float* __restrict__ sw, void* __restrict__ y,
-        int M, int N, int kblocks_all /* K blocks of 128 int8 features */, int sblocks_all /* side steps of 64 columns */, int* status) {
+        int M, int N, int kblocks_all /* K blocks of 128 int8 features */, int sblocks_all /* side steps of 64 columns */,
+        int n_tile_base /* first column tile of this launch */, int* status) {
     using Cfg = TcCfg<BN, BM, KPB>;
     constexpr uint32_t kTxMain = Cfg::kStageBytes;                              // bytes of an int8 step's two loads (boxes of BM and BN rows)
     constexpr uint32_t kTxSide = Cfg::kASlabBytes + Cfg::kBSlabBytes;           // bytes of a side step's two loads
@@ -393,7 +394,7 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
     float* sw_s = reinterpret_cast<float*>(ctrl + 256);                         // BN scales of this tile's columns
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
+    const int m0 = blockIdx.x * BM, n0 = (n_tile_base + int(blockIdx.y)) * BN;
     const uint32_t nsplit = cluster_size(), rank = cluster_rank();              // 1 and 0 without a cluster launch
     const int ksteps_all = (kblocks_all + KPB - 1) / KPB;                       // int8 ring steps of KPB K blocks each
     const int kb_lo = int((long(ksteps_all) * rank) / nsplit), kb_hi = int((long(ksteps_all) * (rank + 1)) / nsplit);

@@ -188,10 +188,14 @@ def test_linear_tensor_path(bq, name, M, K, N, tdt, ko):
 
 
 @pytest.mark.parametrize("M,K,N,ko", [(64, 4096, 7688, 4), (100, 4096, 5120, 0), (7, 1024, 2048, 9), (64, 8192, 1024, 8), (128, 2048, 3000, 3),
-                                      (64, 1024, 20488, 5), (100, 512, 30000, 0), (33, 256, 37888, 70)])
+                                      (64, 1024, 20488, 5), (100, 512, 30000, 0), (33, 256, 37888, 70),
+                                      (64, 2048, 20488, 5), (40, 4096, 19208, 3), (128, 2048, 24000, 0),
+                                      (64, 4096, 4736, 2), (48, 3072, 6272, 0)])
 def test_linear_one_row_of_tiles_shares_k_steps(bq, M, K, N, ko):
     """Decode-size calls: over narrow layers clusters of 2-4 CTAs split a tile's K steps and add their integer sums
-    through shared memory; layers with more 128-row tiles than SMs run without the split.  Both the 64-row and the
+    through shared memory; layers with more 128-row tiles than SMs run their whole waves without the split and, in a
+    second launch, the few tiles left over with it (13, 3 and 40 tiles left); 37 and 49 tiles ask for clusters of 4 and
+    3 on every SM, more than a device with uneven GPCs runs at once, so the split is lowered.  Both the 64-row and the
     128-row accumulator shapes, ragged N."""
     g = torch.Generator().manual_seed(M * 7 + N)
     X = (torch.randn(M, K, generator=g) * 0.6).to(torch.float16)
