@@ -254,11 +254,17 @@ def run_ours(args):
     # the 4-bit variant of the same path (16-entry codebook, two codes per byte) on the same tensor
     cb4 = bq.Codebook4()
     bq4 = {}
-    for b in (64, 1024):
+    for b, s16 in ((64, False), (1024, False), (64, True)):       # s16: the block scale stored as a bf16 (2 bytes instead of 4)
         packed = codes[: n // 2]
+        scale16 = absmax[b].view(torch.bfloat16)[: n // b]
         times = {}
-        for op, fn in (("quantize4", lambda: bq.bq4_quantize(x, b, cb4, packed, absmax[b])),
-                       ("dequantize4", lambda: bq.bq4_dequantize(packed, absmax[b], n, b, cb4, w.dtype, y))):
+        if s16:
+            ops = (("quantize4", lambda: bq.bq4_quantize_s16(x, b, cb4, packed, scale16)),
+                   ("dequantize4", lambda: bq.bq4_dequantize_s16(packed, scale16, n, b, cb4, w.dtype, y)))
+        else:
+            ops = (("quantize4", lambda: bq.bq4_quantize(x, b, cb4, packed, absmax[b])),
+                   ("dequantize4", lambda: bq.bq4_dequantize(packed, absmax[b], n, b, cb4, w.dtype, y)))
+        for op, fn in ops:
             for _ in range(3):
                 fn()
             ev = []
@@ -268,18 +274,20 @@ def run_ours(args):
                 ev.append((e0, e1))
             torch.cuda.synchronize()
             times[op] = float(np.mean([a.elapsed_time(b_) for a, b_ in ev]))
-        ab = n * 2 + n // 2 + 4 * (n // b)
+        scale_bytes = 2 if s16 else 4
+        ab = n * 2 + n // 2 + scale_bytes * (n // b)
         num = torch.zeros((), dtype=torch.float64, device=dev)
         den = torch.zeros((), dtype=torch.float64, device=dev)
         for s in range(0, n, 1 << 27):
             xs, ys = x[s:s + (1 << 27)].float(), y[s:s + (1 << 27)].float()
             num += ((xs - ys) ** 2).sum(dtype=torch.float64)
             den += (xs ** 2).sum(dtype=torch.float64)
-        bq4[f"b{b}"] = {"quantize_ms": round(times["quantize4"], 4), "dequantize_ms": round(times["dequantize4"], 4), "algorithmic_bytes": int(ab),
-                        "quantize_frac_of_measured": round(ab / times["quantize4"] / 1e6 / peak, 4),
-                        "dequantize_frac_of_measured": round(ab / times["dequantize4"] / 1e6 / peak, 4),
-                        "compression_ratio": round(2.0 * n / (n / 2 + 4 * (n // b)), 3),
-                        "rel_rms_error": round(float((num / den).sqrt().item()), 5), "gpu_launches": 26}
+        bq4[f"b{b}" + ("_scale16" if s16 else "")] = {
+            "quantize_ms": round(times["quantize4"], 4), "dequantize_ms": round(times["dequantize4"], 4), "algorithmic_bytes": int(ab),
+            "quantize_frac_of_measured": round(ab / times["quantize4"] / 1e6 / peak, 4),
+            "dequantize_frac_of_measured": round(ab / times["dequantize4"] / 1e6 / peak, 4),
+            "compression_ratio": round(2.0 * n / (n / 2 + scale_bytes * (n // b)), 3),
+            "rel_rms_error": round(float((num / den).sqrt().item()), 5), "gpu_launches": 26}
 
     cpu = cpu_baseline(x_pin, rank) if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
     del x, y, codes, absmax

@@ -62,6 +62,25 @@ int bq4_quantize(const void* x, bq_dtype xdt, size_t n, int block, const bq4_cod
 int bq4_dequantize(const uint8_t* packed, const float* absmax, size_t n, int block, const bq4_codebook* cb,
                    void* y_out, bq_dtype ydt, void* cuda_stream);
 
+/*
+ * bq4_quantize_s16 / bq4_dequantize_s16 -- the same codec with the block scale stored in two
+ * bytes instead of four (at block 64 the fp32 absmax is 11 % of the 4-bit payload, the 16-bit
+ * scale 6 %).  The paper fixes no format for the scale; this is a variant of its "Dynamic
+ * Quantization" item.
+ *   scale_b = the block's absmax rounded toward +infinity to a bf16 (1 sign, 8 exponent, 7
+ *   fraction bits), so that no |x_i| / scale_b exceeds 1; never above the largest finite bf16
+ *   (inputs above it are outside the contract); 0 for an all-zero block.  scale_out[b] holds the
+ *   bf16's 16 bits.  xhat_i = x_i / scale_b as one IEEE fp32 division (divisor 1 for a zero
+ *   block); codes and packing as in bq4_quantize.  Dequantize: y_i = round-to-nearest-even to
+ *   ydt of the fp32 product value[code_i] * scale_b.
+ *   scale_out / scale: ceil(n / block) 16-bit words, device memory, 2-byte aligned.
+ * Arguments, errors and kernels otherwise as bq4_quantize / bq4_dequantize.
+ */
+int bq4_quantize_s16(const void* x, bq_dtype xdt, size_t n, int block, const bq4_codebook* cb,
+                     uint8_t* packed_out, uint16_t* scale_out, void* cuda_stream);
+int bq4_dequantize_s16(const uint8_t* packed, const uint16_t* scale, size_t n, int block, const bq4_codebook* cb,
+                       void* y_out, bq_dtype ydt, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

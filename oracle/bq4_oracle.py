@@ -17,6 +17,10 @@ payload), one of the natural variants of the path.  Readings, all stated:
              high nibble of a last odd element is 0.
   inverse    y = narrow(RN32(value[code] * absmax)).
 
+  16-bit scale (the *_s16 pair) the block's scale is its absmax rounded toward +infinity to a bf16
+             (never above the largest finite bf16), stored as the bf16's 16 bits; x is divided by
+             that scale and the inverse multiplies by it; everything else as above.
+
 Nothing here is imported by the CUDA library or its binding; it shares no code with it.
 fp16 / bf16 arrays are ``uint16`` bit patterns, fp32 arrays are ``float32``.
 Pins: tests/test_oracle_bq4.py (exact rationals, both sides of all 15 breakpoints, torch
@@ -85,3 +89,38 @@ def dequantize(packed: np.ndarray, absmax: np.ndarray, n: int, block: int, cb: n
     scale = np.repeat(np.ascontiguousarray(absmax, np.float32), block)[:n]
     v = (cb[codes] * scale).astype(np.float32)                   # one fp32 multiply per element
     return narrow(v, ydt)
+
+
+BF16_MAX_BITS = 0x7F7F                                           # the largest finite bf16
+
+
+def scale16_of(absmax: float) -> int:
+    """The 16 bits of the smallest bf16 that is >= absmax (absmax >= 0, finite), capped at the largest finite bf16."""
+    bits = int(np.float32(absmax).view(np.uint32))
+    top, low = bits >> 16, bits & 0xFFFF
+    if low:
+        top += 1                                                 # the next bf16 up: magnitudes order like their bit patterns
+    return min(top, BF16_MAX_BITS)
+
+
+def quantize_s16(x: np.ndarray, dt: int, block: int, cb: np.ndarray):
+    """-> (packed uint8 [ceil(n / 2)], scale uint16 [ceil(n / block)])."""
+    v = _as_f32(x, dt)
+    n = v.size
+    nb = (n + block - 1) // block
+    scale = np.zeros(nb, np.uint16)
+    codes = np.zeros(n + (n & 1), np.uint8)
+    for b in range(nb):
+        seg = v[b * block:min(n, (b + 1) * block)]
+        s16 = scale16_of(np.max(np.abs(seg)))
+        scale[b] = s16
+        s = widen(np.array([s16], np.uint16), BF16)[0]
+        d = s if s != 0 else np.float32(1.0)
+        xhat = np.divide(seg, d, dtype=np.float32)               # one fp32 division per element, by the stored scale
+        codes[b * block:b * block + seg.size] = nearest(xhat, cb)
+    low, high = codes[0::2], codes[1::2]                          # element 2i in the low nibble of byte i
+    return (low + np.uint8(16) * high).astype(np.uint8), scale
+
+
+def dequantize_s16(packed: np.ndarray, scale: np.ndarray, n: int, block: int, cb: np.ndarray, ydt: int) -> np.ndarray:
+    return dequantize(packed, widen(np.ascontiguousarray(scale, np.uint16), BF16), n, block, cb, ydt)

@@ -109,27 +109,27 @@ int sm_count_of_current(int* sms) {
 
 unsigned capped(size_t want, size_t cap) { return unsigned(want < 1 ? 1 : (want > cap ? cap : want)); }
 
-template <int DT, bool FOLDED>
+template <int DT, bool FOLDED, bool S16>
 void launch_q4_fast_f(int log2_lpb, unsigned grid, cudaStream_t s, const void* x, uint8_t* packed, float* absmax, size_t nchunks,
                       const bq4k::Tables4& tab) {
     switch (log2_lpb) {
-        case 0: bq4k::q4_fast<DT, FOLDED, 0><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, tab); break;
-        case 1: bq4k::q4_fast<DT, FOLDED, 1><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, tab); break;
-        case 2: bq4k::q4_fast<DT, FOLDED, 2><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, tab); break;
-        case 3: bq4k::q4_fast<DT, FOLDED, 3><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, tab); break;
-        case 4: bq4k::q4_fast<DT, FOLDED, 4><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, tab); break;
-        default: bq4k::q4_fast<DT, FOLDED, 5><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, tab); break;
+        case 0: bq4k::q4_fast<DT, FOLDED, 0, S16><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, tab); break;
+        case 1: bq4k::q4_fast<DT, FOLDED, 1, S16><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, tab); break;
+        case 2: bq4k::q4_fast<DT, FOLDED, 2, S16><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, tab); break;
+        case 3: bq4k::q4_fast<DT, FOLDED, 3, S16><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, tab); break;
+        case 4: bq4k::q4_fast<DT, FOLDED, 4, S16><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, tab); break;
+        default: bq4k::q4_fast<DT, FOLDED, 5, S16><<<grid, 256, 0, s>>>(x, packed, absmax, nchunks, tab); break;
     }
 }
 
-template <int DT>
+template <int DT, bool S16>
 void launch_q4_fast(int log2_lpb, bool folded, unsigned grid, cudaStream_t s, const void* x, uint8_t* packed, float* absmax, size_t nchunks,
                     const bq4k::Tables4& tab) {
-    if (folded) launch_q4_fast_f<DT, true>(log2_lpb, grid, s, x, packed, absmax, nchunks, tab);
-    else launch_q4_fast_f<DT, false>(log2_lpb, grid, s, x, packed, absmax, nchunks, tab);
+    if (folded) launch_q4_fast_f<DT, true, S16>(log2_lpb, grid, s, x, packed, absmax, nchunks, tab);
+    else launch_q4_fast_f<DT, false, S16>(log2_lpb, grid, s, x, packed, absmax, nchunks, tab);
 }
 
-template <int DT>
+template <int DT, bool S16 = false>
 cudaError_t quantize_t(const void* x, size_t n, size_t B, const bq4k::Tables4& tab, uint8_t* packed, float* absmax, int sms, cudaStream_t s) {
     size_t done = 0;
     const int l2 = log2_exact(B);
@@ -138,11 +138,11 @@ cudaError_t quantize_t(const void* x, size_t n, size_t B, const bq4k::Tables4& t
         if (l2 <= 8) {
             const size_t nchunks = n_full / 8;
             const unsigned grid = capped((nchunks + 511) / 512, size_t(sms) * 8);
-            launch_q4_fast<DT>(l2 - 3, tab.folded != 0, grid, s, x, packed, absmax, nchunks, tab);
+            launch_q4_fast<DT, S16>(l2 - 3, tab.folded != 0, grid, s, x, packed, absmax, nchunks, tab);
         } else {
             const unsigned grid = capped((nblocks + 7) / 8, size_t(sms) * 8);
-            if (tab.folded) bq4k::q4_wide<DT, true><<<grid, 256, 0, s>>>(x, packed, absmax, nblocks, int(B / 8), tab);
-            else bq4k::q4_wide<DT, false><<<grid, 256, 0, s>>>(x, packed, absmax, nblocks, int(B / 8), tab);
+            if (tab.folded) bq4k::q4_wide<DT, true, S16><<<grid, 256, 0, s>>>(x, packed, absmax, nblocks, int(B / 8), tab);
+            else bq4k::q4_wide<DT, false, S16><<<grid, 256, 0, s>>>(x, packed, absmax, nblocks, int(B / 8), tab);
         }
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
@@ -150,29 +150,29 @@ cudaError_t quantize_t(const void* x, size_t n, size_t B, const bq4k::Tables4& t
     }
     if (done < n) {
         const size_t nb = (n + B - 1) / B, first_block = done / B;
-        bq4k::q4_general_absmax<DT><<<capped((nb - first_block + 7) / 8, size_t(sms) * 8), 256, 0, s>>>(x, absmax, n, B, first_block);
+        bq4k::q4_general_absmax<DT, S16><<<capped((nb - first_block + 7) / 8, size_t(sms) * 8), 256, 0, s>>>(x, absmax, n, B, first_block);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         const size_t nbytes = (n + 1) / 2, first_byte = done / 2;
-        bq4k::q4_general_codes<DT><<<capped((nbytes - first_byte + 255) / 256, size_t(sms) * 8), 256, 0, s>>>(x, absmax, packed, n, B, first_byte, tab);
+        bq4k::q4_general_codes<DT, S16><<<capped((nbytes - first_byte + 255) / 256, size_t(sms) * 8), 256, 0, s>>>(x, absmax, packed, n, B, first_byte, tab);
         return cudaGetLastError();
     }
     return cudaSuccess;
 }
 
-template <int DT>
+template <int DT, bool S16 = false>
 cudaError_t dequantize_t(const uint8_t* packed, const float* absmax, size_t n, size_t B, const bq4k::Tables4& tab, void* y, int sms, cudaStream_t s) {
     size_t done = 0;
     const int l2 = log2_exact(B);
     if (l2 >= 4 && aligned(packed, 8) && aligned(y, 32) && n >= 16) {
         const size_t n16 = n / 16;
-        bq4k::dq4_fast<DT><<<capped((n16 + 255) / 256, size_t(sms) * 16), 256, 0, s>>>(packed, absmax, y, n16, l2, tab);
+        bq4k::dq4_fast<DT, S16><<<capped((n16 + 255) / 256, size_t(sms) * 16), 256, 0, s>>>(packed, absmax, y, n16, l2, tab);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         done = n16 * 16;
     }
     if (done < n) {
-        bq4k::dq4_general<DT><<<capped((n - done + 255) / 256, size_t(sms) * 8), 256, 0, s>>>(packed, absmax, y, n, B, done, tab);
+        bq4k::dq4_general<DT, S16><<<capped((n - done + 255) / 256, size_t(sms) * 8), 256, 0, s>>>(packed, absmax, y, n, B, done, tab);
         return cudaGetLastError();
     }
     return cudaSuccess;
@@ -248,6 +248,50 @@ int bq4_dequantize(const uint8_t* packed, const float* absmax, size_t n, int blo
         case BQ_F32: e = dequantize_t<bq4k::kF32>(packed, absmax, n, size_t(block), cb->tab, y_out, sms, s); break;
         case BQ_F16: e = dequantize_t<bq4k::kF16>(packed, absmax, n, size_t(block), cb->tab, y_out, sms, s); break;
         default: e = dequantize_t<bq4k::kBF16>(packed, absmax, n, size_t(block), cb->tab, y_out, sms, s); break;
+    }
+    return e == cudaSuccess ? BQ_OK : cuda_fail(e);
+}
+
+int bq4_quantize_s16(const void* x, bq_dtype xdt, size_t n, int block, const bq4_codebook* cb, uint8_t* packed_out, uint16_t* scale_out,
+                     void* cuda_stream) {
+    if (!known_dtype(xdt)) return BQ_ERR_DTYPE;
+    if (block < 1) return BQ_ERR_BLOCK;
+    if (n >= kMaxElems) return BQ_ERR_SIZE;
+    if (!cb) return BQ_ERR_CODEBOOK;
+    if (n == 0) return BQ_OK;
+    if (!x || !packed_out || !scale_out) return BQ_ERR_NULL;
+    int sms = 0;
+    const int rc = sm_count_of_current(&sms);
+    if (rc != BQ_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    float* scales = reinterpret_cast<float*>(scale_out);          // the S16 kernels address it as 16-bit words
+    cudaError_t e;
+    switch (xdt) {
+        case BQ_F32: e = quantize_t<bq4k::kF32, true>(x, n, size_t(block), cb->tab, packed_out, scales, sms, s); break;
+        case BQ_F16: e = quantize_t<bq4k::kF16, true>(x, n, size_t(block), cb->tab, packed_out, scales, sms, s); break;
+        default: e = quantize_t<bq4k::kBF16, true>(x, n, size_t(block), cb->tab, packed_out, scales, sms, s); break;
+    }
+    return e == cudaSuccess ? BQ_OK : cuda_fail(e);
+}
+
+int bq4_dequantize_s16(const uint8_t* packed, const uint16_t* scale, size_t n, int block, const bq4_codebook* cb, void* y_out, bq_dtype ydt,
+                       void* cuda_stream) {
+    if (!known_dtype(ydt)) return BQ_ERR_DTYPE;
+    if (block < 1) return BQ_ERR_BLOCK;
+    if (n >= kMaxElems) return BQ_ERR_SIZE;
+    if (!cb) return BQ_ERR_CODEBOOK;
+    if (n == 0) return BQ_OK;
+    if (!packed || !scale || !y_out) return BQ_ERR_NULL;
+    int sms = 0;
+    const int rc = sm_count_of_current(&sms);
+    if (rc != BQ_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const float* scales = reinterpret_cast<const float*>(scale);
+    cudaError_t e;
+    switch (ydt) {
+        case BQ_F32: e = dequantize_t<bq4k::kF32, true>(packed, scales, n, size_t(block), cb->tab, y_out, sms, s); break;
+        case BQ_F16: e = dequantize_t<bq4k::kF16, true>(packed, scales, n, size_t(block), cb->tab, y_out, sms, s); break;
+        default: e = dequantize_t<bq4k::kBF16, true>(packed, scales, n, size_t(block), cb->tab, y_out, sms, s); break;
     }
     return e == cudaSuccess ? BQ_OK : cuda_fail(e);
 }

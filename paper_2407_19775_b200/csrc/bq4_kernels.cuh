@@ -182,12 +182,31 @@ __device__ __forceinline__ void quotients8(const float (&f)[8], float d, float r
     }
 }
 
+// The scale of a block.  Plain form: its absmax as an fp32.  S16 form: the absmax rounded toward +infinity to a bf16 (so
+// that no |x| / scale exceeds 1), never above the largest finite bf16; the two stored bytes are the bf16 itself.  The
+// `absmax` arguments of the kernels point at floats or, with S16, at 16-bit words.
+template <bool S16>
+__device__ __forceinline__ float block_scale(float a /* >= 0 */) {
+    if constexpr (!S16) return a;
+    else return __uint_as_float(min((__float_as_uint(a) + 0xFFFFu) & 0xFFFF0000u, 0x7F7F0000u));
+}
+template <bool S16>
+__device__ __forceinline__ void store_scale(float* p, size_t i, float s) {
+    if constexpr (!S16) p[i] = s;
+    else reinterpret_cast<uint16_t*>(p)[i] = uint16_t(__float_as_uint(s) >> 16);
+}
+template <bool S16>
+__device__ __forceinline__ float load_scale(const float* p, size_t i) {
+    if constexpr (!S16) return __ldg(p + i);
+    else return __uint_as_float(uint32_t(__ldg(reinterpret_cast<const uint16_t*>(p) + i)) << 16);
+}
+
 __device__ __forceinline__ void fill_tables(const Tables4& tab, float* thr, float* val) {
     if (threadIdx.x < 16) { thr[threadIdx.x] = tab.thr[threadIdx.x]; val[threadIdx.x] = tab.val[threadIdx.x]; }
     __syncthreads();
 }
 
-template <int DT, bool FOLDED, int LOG2_LPB /* log2 of the lanes per block = log2(block / 8) */>
+template <int DT, bool FOLDED, int LOG2_LPB /* log2 of the lanes per block = log2(block / 8) */, bool S16 = false>
 __global__ void __launch_bounds__(256)
 q4_fast(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restrict__ absmax, size_t nchunks, const __grid_constant__ Tables4 tab) {
     constexpr int lpb = 1 << LOG2_LPB;
@@ -231,6 +250,7 @@ q4_fast(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restr
             for (int i = 0; i < 8; ++i) a = fmaxf(a, fabsf(f[u][i]));
 #pragma unroll
             for (int s = 1; s < lpb; s <<= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, s));
+            a = block_scale<S16>(a);
             const float d = (a != 0.0f) ? a : 1.0f;
             // one choice of route for the whole warp keeps the per-element code free of branches
             const bool quick = (DT != kF32) && __all_sync(0xffffffffu, (d >= 5.421010862427522e-20f) && (d <= 1.8446744073709552e19f));
@@ -246,13 +266,13 @@ q4_fast(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restr
             }
             if (c[u] < nchunks) {
                 reinterpret_cast<uint32_t*>(packed)[c[u]] = word;
-                if ((c[u] & size_t(lpb - 1)) == 0) absmax[c[u] >> log2_lpb] = a;
+                if ((c[u] & size_t(lpb - 1)) == 0) store_scale<S16>(absmax, c[u] >> log2_lpb, a);
             }
         }
     }
 }
 
-template <int DT, bool FOLDED>
+template <int DT, bool FOLDED, bool S16 = false>
 __global__ void __launch_bounds__(256)
 q4_wide(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restrict__ absmax, size_t nblocks, int chunks_per_block,
         const __grid_constant__ Tables4 tab) {
@@ -278,6 +298,7 @@ q4_wide(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restr
         }
 #pragma unroll
         for (int s = 1; s < 32; s <<= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, s));
+        a = block_scale<S16>(a);
         const float d = (a != 0.0f) ? a : 1.0f;
         const bool quick = (DT != kF32) && (d >= 5.421010862427522e-20f) && (d <= 1.8446744073709552e19f);      // one block per warp: uniform
         float r;
@@ -294,12 +315,12 @@ q4_wide(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restr
             }
             reinterpret_cast<uint32_t*>(packed)[cbase + k] = word;
         }
-        if (lane == 0) absmax[b] = a;
+        if (lane == 0) store_scale<S16>(absmax, b, a);
     }
 }
 
 // General quantize, step 1: absmax of blocks first_block .. (one warp per block).
-template <int DT>
+template <int DT, bool S16 = false>
 __global__ void __launch_bounds__(256)
 q4_general_absmax(const void* __restrict__ x, float* __restrict__ absmax, size_t n, size_t block, size_t first_block) {
     const int lane = threadIdx.x & 31;
@@ -310,12 +331,12 @@ q4_general_absmax(const void* __restrict__ x, float* __restrict__ absmax, size_t
         for (size_t i = lo + lane; i < hi; i += 32) a = fmaxf(a, fabsf(load1<DT>(x, i)));
 #pragma unroll
         for (int s = 1; s < 32; s <<= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, s));
-        if (lane == 0) absmax[b] = a;
+        if (lane == 0) store_scale<S16>(absmax, b, block_scale<S16>(a));
     }
 }
 
 // General quantize, step 2: one thread per output byte from byte first_byte on.
-template <int DT>
+template <int DT, bool S16 = false>
 __global__ void __launch_bounds__(256)
 q4_general_codes(const void* __restrict__ x, const float* __restrict__ absmax, uint8_t* __restrict__ packed, size_t n, size_t block,
                  size_t first_byte, const __grid_constant__ Tables4 tab) {
@@ -328,7 +349,7 @@ q4_general_codes(const void* __restrict__ x, const float* __restrict__ absmax, u
         for (int h = 0; h < 2; ++h) {
             const size_t i = 2 * j + h;
             if (i < n) {
-                const float a = absmax[i / block];
+                const float a = load_scale<S16>(absmax, i / block);
                 const float d = (a != 0.0f) ? a : 1.0f;
                 byte |= search16(thr, __fdiv_rn(load1<DT>(x, i), d)) << (4 * h);
             }
@@ -343,7 +364,7 @@ __device__ __forceinline__ void st32(void* p, const uint32_t (&w)[8]) {
 }
 
 // 16 elements per thread; block is a power of two >= 16, so the 16 share one absmax.
-template <int DT>
+template <int DT, bool S16 = false>
 __global__ void __launch_bounds__(256)
 dq4_fast(const uint8_t* __restrict__ packed, const float* __restrict__ absmax, void* __restrict__ y, size_t n16, int log2_block,
          const __grid_constant__ Tables4 tab) {
@@ -351,7 +372,7 @@ dq4_fast(const uint8_t* __restrict__ packed, const float* __restrict__ absmax, v
     fill_tables(tab, thr, val);
     for (size_t c = size_t(blockIdx.x) * 256 + threadIdx.x; c < n16; c += size_t(gridDim.x) * 256) {
         const uint2 w = reinterpret_cast<const uint2*>(packed)[c];
-        const float a = __ldg(absmax + ((c * 16) >> log2_block));
+        const float a = load_scale<S16>(absmax, (c * 16) >> log2_block);
         float v[16];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -381,7 +402,7 @@ dq4_fast(const uint8_t* __restrict__ packed, const float* __restrict__ absmax, v
     }
 }
 
-template <int DT>
+template <int DT, bool S16 = false>
 __global__ void __launch_bounds__(256)
 dq4_general(const uint8_t* __restrict__ packed, const float* __restrict__ absmax, void* __restrict__ y, size_t n, size_t block, size_t first_elem,
             const __grid_constant__ Tables4 tab) {
@@ -389,7 +410,7 @@ dq4_general(const uint8_t* __restrict__ packed, const float* __restrict__ absmax
     fill_tables(tab, thr, val);
     for (size_t i = first_elem + size_t(blockIdx.x) * 256 + threadIdx.x; i < n; i += size_t(gridDim.x) * 256) {
         const uint32_t code = (packed[i >> 1] >> (4 * (i & 1))) & 15u;
-        store1<DT>(y, i, __fmul_rn(val[code], absmax[i / block]));
+        store1<DT>(y, i, __fmul_rn(val[code], load_scale<S16>(absmax, i / block)));
     }
 }
 

@@ -33,7 +33,7 @@ def test_every_declared_bq4_symbol_is_exported(bq):
     from paper_2407_19775_b200 import binding, bq4
     L = binding.lib()
     names = _declared("bq4.h", "bq4_")
-    assert {"bq4_make_codebook", "bq4_free_codebook", "bq4_quantize", "bq4_dequantize"} == set(names)
+    assert {"bq4_make_codebook", "bq4_free_codebook", "bq4_quantize", "bq4_dequantize", "bq4_quantize_s16", "bq4_dequantize_s16"} == set(names)
     for name in names:
         assert hasattr(L, name), name
     assert set(bq4.SYMBOLS) == set(names)
@@ -53,6 +53,13 @@ def test_bq4_argument_errors_and_host_codebook(bq):
     assert L.bq4_quantize(None, 0, 4, 64, one, one, one, None) == 1
     assert L.bq4_dequantize(one, one, 4, 64, one, None, 0, None) == 1
     assert L.bq4_dequantize(one, one, 4, 64, one, one, 7, None) == 2
+    assert L.bq4_quantize_s16(one, 9, 4, 64, one, one, one, None) == 2
+    assert L.bq4_quantize_s16(one, 0, 4, 0, one, one, one, None) == 3
+    assert L.bq4_quantize_s16(one, 0, 4, 64, None, one, one, None) == 5
+    assert L.bq4_quantize_s16(one, 0, 4, 64, one, one, None, None) == 1
+    assert L.bq4_quantize_s16(None, 0, 0, 64, one, None, None, None) == 0
+    assert L.bq4_dequantize_s16(one, None, 4, 64, one, one, 0, None) == 1
+    assert L.bq4_dequantize_s16(one, one, 4, 64, one, one, 7, None) == 2
     out = ctypes.c_void_p()
     assert L.bq4_make_codebook(5, None, None, ctypes.byref(out)) == 5
     assert L.bq4_make_codebook(0, None, None, None) == 1

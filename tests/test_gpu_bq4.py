@@ -192,3 +192,65 @@ def test_full_size_tensor_sampled_blocks(bq):
             assert a[b].item() == a_ref[0]
             assert np.array_equal(bits(y[b * block:(b + 1) * block]), o4.dequantize(p_ref, a_ref, block, block, cb_ref, BF16))
         del p, a, y
+
+
+def check_s16(bq, x: torch.Tensor, block: int):
+    """The 16-bit-scale pair against its oracle: packed codes, scale words and both outputs bit for bit."""
+    cb = bq.Codebook4()
+    cb_ref = o4.make_codebook()
+    flat = x.reshape(-1)
+    dt = DT[flat.dtype]
+    p_ref, s_ref = o4.quantize_s16(bits(flat), dt, block, cb_ref)
+    p, s = bq.bq4_quantize_s16(flat.cuda(), block, cb)
+    torch.cuda.synchronize()
+    assert s.dtype == torch.bfloat16
+    assert np.array_equal(p.cpu().numpy(), p_ref)
+    assert np.array_equal(bits(s), s_ref)
+    for out in (flat.dtype, torch.float32):
+        y = bq.bq4_dequantize_s16(p, s, flat.numel(), block, cb, out)
+        y_ref = o4.dequantize_s16(p_ref, s_ref, flat.numel(), block, cb_ref, DT[out])
+        view = np.uint32 if out == torch.float32 else np.uint16
+        assert np.array_equal(bits(y).view(view), y_ref.view(view))
+    return p_ref, s_ref
+
+
+@pytest.mark.parametrize("name,rows,block", [("tiny", None, 64), ("prefill7b", 64, 256), ("decode70b", 64, 64), ("moe_prefill", 24, 2048),
+                                             ("sweep1g", 16, 8), ("sweep1g", 16, 65536)])
+def test_scale16_workloads(bq, name, rows, block):
+    check_s16(bq, workloads.make(name, rows=rows), block)
+
+
+@pytest.mark.parametrize("tdt", [torch.float32, torch.bfloat16, torch.float16])
+def test_scale16_ragged_general_and_extreme_scales(bq, tdt):
+    """Ragged tails and odd blocks (the general kernels), zero blocks, and blocks whose absmax sits on, just above and
+    just below a bf16, in the subnormal range and near the top of the type's range."""
+    g = torch.Generator().manual_seed(17)
+    x = (torch.randn(6000, generator=g) * 1.5).to(tdt)
+    x[100:164] = 0
+    for n, block in [(5999, 64), (6000, 24), (37, 64), (1, 8), (777, 3), (4097, 4096), (1023, 32)]:
+        check_s16(bq, x[:n].clone(), block)
+    top = {torch.float32: 3.0e38, torch.bfloat16: 3.0e38, torch.float16: 60000.0}[tdt]
+    tiny = {torch.float32: 1e-41, torch.bfloat16: 1e-39, torch.float16: 6e-8}[tdt]
+    peaks = [1.0, 1.0000001, 0.99999994, 1.0078125, 1.00390625, 255.0, 256.5, top, tiny, 3 * tiny, 2.0 ** -126, 1.5 * 2.0 ** -126]
+    blocks = []
+    for k, pk in enumerate(peaks):
+        b = torch.rand(64, generator=g) * 2 - 1
+        b[k % 64] = 1.0 if k % 2 else -1.0
+        blocks.append((b.double() * pk).to(tdt))
+    check_s16(bq, torch.cat(blocks), 64)
+    check_s16(bq, torch.cat(blocks)[:64 * len(peaks) - 8], 16)
+
+
+def test_scale16_is_close_to_the_fp32_scale(bq):
+    """Property at a size the oracle does not reach: every stored scale is a bf16 in [absmax, absmax (1 + 2^-7)) and the
+    reconstruction error stays within the 4-bit bound against that scale."""
+    cb = bq.Codebook4()
+    x = workloads.make("sweep1g", rows=4096).reshape(-1).cuda()
+    block = 64
+    p, s = bq.bq4_quantize_s16(x, block, cb)
+    _, a = bq.bq4_quantize(x, block, cb)
+    sf = s.float()
+    assert bool((sf >= a).all()) and bool((sf.double() < a.double() * (1 + 2.0 ** -7) + 1e-300).all())
+    y = bq.bq4_dequantize_s16(p, s, x.numel(), block, cb, torch.float32)
+    err = (x.float() - y).abs().view(-1, block) / sf.clamp_min(1e-30)[:, None]
+    assert float(err.max()) <= 0.1125 * (1 + 1e-5)

@@ -155,7 +155,63 @@ def pin_error_bound(m) -> bool:
     return bool(ok)
 
 
-PINS = {"codebook": pin_codebook, "breakpoints": pin_breakpoints, "quantize": pin_quantize, "packing": pin_packing,
+def pin_scale16(m) -> bool:
+    """The 16-bit scale: the smallest bf16 >= absmax (torch's bf16 grid and exact rationals say which), the codes of
+    x / scale against the exact nearest value, the inverse against torch, and the bound |x| <= scale < absmax (1 + 2^-7)."""
+    cb = exact_codebook()
+    ok = True
+    # the rounding itself, on values torch can narrow: scale is a bf16, >= a, and the bf16 just below it is < a
+    rng = np.random.default_rng(11)
+    vals = np.concatenate([np.abs(rng.standard_normal(400)).astype(np.float32) * np.float32(10.0) ** rng.integers(-20, 20, 400).astype(np.float32),
+                           np.array([0.0, 1.0, 1.0000001, 0.99999994, 3.0, 2.0 ** -126, 2.0 ** -140, 3.3895314e38, 3.4e38], np.float32)])
+    for a in vals:
+        bits = m.scale16_of(a)
+        s = torch.tensor([bits], dtype=torch.int32).to(torch.int16).view(torch.bfloat16).float().item()
+        if a > 3.3895314e38:
+            ok &= bits == 0x7F7F
+            continue
+        ok &= frac_of(np.float32(s)) >= frac_of(a)
+        if bits > 0:
+            below = torch.tensor([bits - 1], dtype=torch.int32).to(torch.int16).view(torch.bfloat16).float().item()
+            ok &= frac_of(np.float32(below)) < frac_of(a)
+        else:
+            ok &= a == 0
+        if torch.tensor([float(a)]).to(torch.bfloat16).float().item() == float(a):
+            ok &= np.float32(s) == a                               # a bf16 stays itself
+    g = torch.Generator().manual_seed(21)
+    x = torch.randn(32 * 9 + 5, generator=g) * 3.0
+    x[32:64] = 0
+    x[70] = -7.3
+    # a block whose absmax 1.001 is stored as 1.0078125: 0.9475 / 1.001 lies above the breakpoint 0.94375 between the two
+    # top codes, 0.9475 / 1.0078125 below it
+    x[96:128] *= 0.05
+    x[96], x[97] = 1.001, 0.9475
+    for dt, tdt in ((F32, torch.float32), (BF16, torch.bfloat16), (F16, torch.float16)):
+        xt = x.to(tdt)
+        bits = xt.numpy() if dt == F32 else xt.view(torch.int16).numpy().view(np.uint16)
+        packed, sc = m.quantize_s16(bits, dt, 32, cb)
+        f = xt.float().numpy()
+        n = f.size
+        ok &= sc.dtype == np.uint16 and sc.size == (n + 31) // 32 and sc[1] == 0
+        sf = torch.from_numpy(sc.astype(np.int32)).to(torch.int16).view(torch.bfloat16).float().numpy()
+        pad = np.concatenate([np.abs(f), np.zeros((-n) % 32, np.float32)]).reshape(-1, 32).max(axis=1)
+        ok &= bool(np.all(sf >= pad)) and bool(np.all(sf.astype(np.float64) < pad.astype(np.float64) * (1 + 2.0 ** -7) + 1e-300))
+        codes = m.unpack(packed, n)
+        for i in range(n):
+            d = sf[i // 32]
+            xhat = rn32(frac_of(f[i]) / frac_of(d)) if d != 0 else np.float32(f[i])
+            ok &= int(codes[i]) == nearest_exact16(xhat, cb)
+        ok &= bool(np.all(codes[32:64] == 7))
+        if dt != BF16:
+            ok &= int(codes[97]) == 14 and int(sc[3]) == 0x3F81
+        y = m.dequantize_s16(packed, sc, n, 32, cb, dt)
+        want = (torch.from_numpy(cb)[torch.from_numpy(codes.astype(np.int64))] * torch.from_numpy(np.repeat(sf, 32)[:n])).to(tdt)
+        wb = want.numpy() if dt == F32 else want.view(torch.int16).numpy().view(np.uint16)
+        ok &= np.array_equal(y.view(np.uint32 if dt == F32 else np.uint16), wb.view(np.uint32 if dt == F32 else np.uint16))
+    return bool(ok)
+
+
+PINS = {"scale16": pin_scale16, "codebook": pin_codebook, "breakpoints": pin_breakpoints, "quantize": pin_quantize, "packing": pin_packing,
         "dequantize": pin_dequantize, "error_bound": pin_error_bound}
 
 
@@ -172,6 +228,8 @@ MUTATIONS = {
     "multiply_by_reciprocal": ("xhat = (seg / d).astype(np.float32)", "xhat = (seg * (np.float32(1.0) / d)).astype(np.float32)", {"quantize"}),
     "nibbles_swapped": ("packed = (codes[0::2] | (codes[1::2] << np.uint8(4)))", "packed = (codes[1::2] | (codes[0::2] << np.uint8(4)))", {"packing"}),
     "wrong_block_scale": ("scale = np.repeat(np.ascontiguousarray(absmax, np.float32), block)[:n]", "scale = np.repeat(np.ascontiguousarray(absmax, np.float32), block)[1:n + 1]", {"dequantize"}),
+    "scale16_rounds_to_nearest": ("    if low:\n        top += 1", "    if low >= 0x8000:\n        top += 1", {"scale16"}),
+    "scale16_divides_by_absmax": ("        s = widen(np.array([s16], np.uint16), BF16)[0]\n", "        s = np.float32(np.max(np.abs(seg)))\n", {"scale16"}),
     "unpack_high_first": ("codes[0::2] = packed & np.uint8(15)\n    codes[1::2] = packed >> np.uint8(4)", "codes[1::2] = packed & np.uint8(15)\n    codes[0::2] = packed >> np.uint8(4)", {"packing", "dequantize"}),
 }
 
