@@ -289,6 +289,27 @@ def run_ours(args):
             "compression_ratio": round(2.0 * n / (n / 2 + scale_bytes * (n // b)), 3),
             "rel_rms_error": round(float((num / den).sqrt().item()), 5), "gpu_launches": 26}
 
+    # block-size selection on the same tensor: the roundtrip and the error sums of four candidates in one call
+    tune_blocks = [64, 256, 1024, 4096]
+    tune_ws = torch.empty(bq.tune.workspace_bytes(w.dtype, n), dtype=torch.uint8, device=dev)
+    tune_sums = torch.empty(len(tune_blocks) + 1, dtype=torch.float64, device=dev)
+    for _ in range(2):
+        bq.tune.block_errors(x, tune_blocks, cb, tune_ws, tune_sums)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(5):
+        bq.tune.block_errors(x, tune_blocks, cb, tune_ws, tune_sums)
+    e1.record()
+    torch.cuda.synchronize()
+    tune_ms = e0.elapsed_time(e1) / 5
+    tune_bytes = len(tune_blocks) * 4 * n * 2                     # per candidate: roundtrip reads x and writes y, the sums read both
+    sums_host = tune_sums.cpu().numpy()
+    tune = {"blocks": tune_blocks, "ms_per_call": round(tune_ms, 4), "algorithmic_bytes": int(tune_bytes),
+            "frac_of_measured": round(tune_bytes / tune_ms / 1e6 / peak, 4),
+            "rel_rms_error": [round(float(v), 5) for v in np.sqrt(sums_host[:-1] / sums_host[-1])],
+            "picked_for_rel_rms_0.01": bq.tune.pick_block(tune_blocks, sums_host, 0.01), "gpu_launches": 7 * 3 * len(tune_blocks)}
+    del tune_ws
+
     cpu = cpu_baseline(x_pin, rank) if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
     del x, y, codes, absmax
     torch.cuda.empty_cache()
@@ -303,7 +324,7 @@ def run_ours(args):
                                    "quantize+dequantize+roundtrip per block", "elements": n, "l2": "input (1 GiB) larger than L2, no flush needed",
                        "parallelism": f"replicated x{world}, no collective"},
             "e2e": e2e, "gpu_launches": len(events), "clocks": clocks, "roofline": roofline, "kernels": kernels,
-            "quality": quality, "cpu_baseline": cpu, "bq4": bq4, "mmd": mmd,
+            "quality": quality, "cpu_baseline": cpu, "bq4": bq4, "autotune": tune, "mmd": mmd,
             "paper_context": "the paper reports no throughput for this path; it states only that hidden-state quantization halves the bandwidth",
         }
         print(json.dumps(line))

@@ -30,7 +30,7 @@ def _sources():
 
 def _newest_header() -> float:
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
-    deps.append(os.path.join(INCLUDE, "bq.h"))
+    deps += [os.path.join(INCLUDE, f) for f in os.listdir(INCLUDE) if f.endswith(".h")]
     return max(os.path.getmtime(p) for p in deps)
 
 

@@ -26,7 +26,7 @@ def test_every_declared_symbol_is_exported(bq):
 
 
 def test_every_header_is_covered():
-    assert sorted(os.listdir(os.path.join(ROOT, "include"))) == ["bq.h", "bq4.h", "mmd.h"]
+    assert sorted(os.listdir(os.path.join(ROOT, "include"))) == ["bq.h", "bq4.h", "bq_tune.h", "mmd.h"]
 
 
 def test_every_declared_bq4_symbol_is_exported(bq):
@@ -68,6 +68,43 @@ def test_bq4_argument_errors_and_host_codebook(bq):
     assert np.array_equal(cb.values.view(np.uint32), bq4_oracle.make_codebook().view(np.uint32))
     bad = cb.values.copy(); bad[3] = bad[4]
     assert L.bq4_make_codebook(1, bad.ctypes.data, None, ctypes.byref(out)) == 5
+
+
+def test_every_declared_tune_symbol_is_exported_and_host_rule(bq):
+    import numpy as np
+    from paper_2407_19775_b200 import binding, tune
+    L = binding.lib()
+    names = _declared("bq_tune.h", "bqt_")
+    assert {"bqt_workspace_bytes", "bqt_block_errors", "bqt_pick_block"} == set(names)
+    for name in names:
+        assert hasattr(L, name), name
+    assert set(tune.SYMBOLS) == set(names)
+    T = tune._lib()
+    assert T.bqt_workspace_bytes(2, 1000) == 2048 + 16384 and T.bqt_workspace_bytes(0, 64) == 256 + 16384 and T.bqt_workspace_bytes(7, 64) == 0
+    one = ctypes.c_void_p(256)       # never dereferenced: every call below fails a check first
+    blocks = np.array([64, 256], np.int32)
+    bad = np.array([64, 0], np.int32)
+    assert T.bqt_block_errors(one, 9, 4, one, blocks.ctypes.data, 2, one, 1 << 20, one, None) == 2
+    assert T.bqt_block_errors(one, 0, 4, one, None, 2, one, 1 << 20, one, None) == 1
+    assert T.bqt_block_errors(one, 0, 4, one, blocks.ctypes.data, 0, one, 1 << 20, one, None) == 3
+    assert T.bqt_block_errors(one, 0, 4, one, blocks.ctypes.data, 17, one, 1 << 20, one, None) == 3
+    assert T.bqt_block_errors(one, 0, 4, one, bad.ctypes.data, 2, one, 1 << 20, one, None) == 3
+    assert T.bqt_block_errors(one, 0, 4, None, blocks.ctypes.data, 2, one, 1 << 20, one, None) == 5
+    assert T.bqt_block_errors(None, 0, 4, one, blocks.ctypes.data, 2, one, 1 << 20, one, None) == 1
+    assert T.bqt_block_errors(one, 0, 4, one, blocks.ctypes.data, 2, one, 100, one, None) == 4
+    assert T.bqt_block_errors(one, 0, 4, one, blocks.ctypes.data, 2, ctypes.c_void_p(264), 1 << 20, one, None) == 4
+    # the host rule against the oracle's statement of it, every branch
+    from oracle import tune_oracle
+    cases = [([64, 256, 1024], [1.0, 2.0, 5.0], 100.0, 0.15), ([64, 256, 1024], [1.0, 2.0, 5.0], 100.0, 0.3), ([64, 256, 1024], [1.0, 2.0, 5.0], 100.0, 0.05),
+             ([1024, 64, 256], [5.0, 1.0, 2.0], 100.0, 0.15), ([64, 256], [3.0, 3.0], 100.0, 0.01), ([64, 256], [0.0, 0.0], 0.0, 0.0),
+             ([256, 64], [4.0, 4.0], 100.0, 0.2), ([32], [7.0], 1.0, 0.0)]
+    for cand, err2, norm2, tol in cases:
+        assert tune.pick_block(cand, err2 + [norm2], tol) == tune_oracle.pick_block(cand, err2, norm2, tol), (cand, err2, tol)
+    out = ctypes.c_int()
+    sums = np.array([1.0, 2.0, 9.0])
+    assert T.bqt_pick_block(blocks.ctypes.data, sums.ctypes.data, 2, -1.0, ctypes.byref(out)) == 4
+    assert T.bqt_pick_block(blocks.ctypes.data, sums.ctypes.data, 2, float("nan"), ctypes.byref(out)) == 4
+    assert T.bqt_pick_block(None, sums.ctypes.data, 2, 0.1, ctypes.byref(out)) == 1
 
 
 def test_every_declared_mmd_symbol_is_exported(bq):

@@ -34,6 +34,10 @@ def test_bench_line_has_the_contract_keys(bq):
     for v in d["bq4"].values():
         assert 0.2 < v["quantize_frac_of_measured"] < 1.1 and 0.5 < v["dequantize_frac_of_measured"] < 1.1
         assert 3.5 < v["compression_ratio"] < 4.0 and 0.05 < v["rel_rms_error"] < 0.3
+    assert set(d["bq4"]) == {"b64", "b1024", "b64_scale16"} and d["bq4"]["b64_scale16"]["compression_ratio"] > d["bq4"]["b64"]["compression_ratio"]
+    t = d["autotune"]
+    assert 0.3 < t["frac_of_measured"] < 1.1 and t["picked_for_rel_rms_0.01"] in t["blocks"] and len(t["rel_rms_error"]) == len(t["blocks"])
+    assert all(abs(a - q["rel_rms_error"]) < 2e-5 for a, q in zip(t["rel_rms_error"], d["quality"].values()))
     # the decomposed linear layer: its own roofline object, no kernel error (its full-size parity is tests/test_gpu_mmd.py's)
     m = d["mmd"]
     mr = m["roofline"]
