@@ -12,13 +12,13 @@ import argparse
 
 import torch
 
-from . import Codebook, Codebook4, bq4_dequantize, bq4_quantize, bq_dequantize, bq_quantize, bq_roundtrip, workloads
+from . import Codebook, Codebook4, bq4_dequantize, bq4_quantize, bq_dequantize, bq_quantize, bq_roundtrip, tune, workloads
 
 
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="sweep1g")
-    ap.add_argument("--op", default="roundtrip", choices=["quantize", "dequantize", "roundtrip", "roundtrip_side", "quantize4", "dequantize4"])
+    ap.add_argument("--op", default="roundtrip", choices=["quantize", "dequantize", "roundtrip", "roundtrip_side", "quantize4", "dequantize4", "block_errors"])
     ap.add_argument("--block", type=int, default=4096)
     ap.add_argument("--rows", type=int, default=8192)
     ap.add_argument("--launches", type=int, default=3)
@@ -39,6 +39,9 @@ def main() -> None:
         bq_quantize(x, args.block, cb, codes, absmax)
     if args.op == "dequantize4":
         bq4_quantize(x, args.block, cb4, packed, absmax)
+    if args.op == "block_errors":                                # one candidate: the roundtrip, then the two kernels of the sums
+        tune_ws = torch.empty(tune.workspace_bytes(x.dtype, n), dtype=torch.uint8, device=dev)
+        tune_sums = torch.empty(2, dtype=torch.float64, device=dev)
     torch.cuda.synchronize()
     for i in range(args.launches):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -51,6 +54,8 @@ def main() -> None:
             bq4_quantize(x, args.block, cb4, packed, absmax)
         elif args.op == "dequantize4":
             bq4_dequantize(packed, absmax, n, args.block, cb4, x.dtype, y)
+        elif args.op == "block_errors":
+            tune.block_errors(x, [args.block], cb, tune_ws, tune_sums)
         elif args.op == "roundtrip":
             bq_roundtrip(x, args.block, cb, y_out=y)
         else:
