@@ -47,12 +47,57 @@ __device__ __forceinline__ void widen8(const uint4& w, float (&f)[8]) {
 // rowquant: one CTA of 256 threads per row.  A bit mask of the critical features sits in
 // shared memory, one byte per 16-byte chunk of the row, so the regular path costs one byte
 // load per eight elements.  The row is read twice (the second pass hits L1 / L2).
+//
+// The kernel is bound by instruction issue, so both passes are written for few instructions:
+// the absmax pass works on the packed 16-bit patterns (the magnitudes of finite fp16 / bf16
+// values order like their bit patterns: one mask and one two-lane unsigned max per pair), the
+// code pass does its fp32 arithmetic two elements per instruction, rounds to an integer by
+// adding 1.5 * 2^23 (round-to-nearest-even, the low byte of the sum's bit pattern is the int8
+// code) and gathers the four low bytes of a word with byte permutes.  A chunk that holds a
+// critical feature (rare) takes a slower masked path.
+__device__ __forceinline__ uint64_t rq_pack2(float a, float b) {
+    uint64_t v;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(a), "f"(b));
+    return v;
+}
+__device__ __forceinline__ uint64_t rq_mul2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t rq_fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t rq_add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint32_t rq_prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+// 0xffff in the halves of word j (elements 2j, 2j + 1 of the chunk) whose mask bit is clear
+__device__ __forceinline__ uint32_t rq_keep_halves(uint32_t mk, int j) {
+    return (((mk >> (2 * j)) & 1u) ? 0u : 0x0000ffffu) | (((mk >> (2 * j + 1)) & 1u) ? 0u : 0xffff0000u);
+}
+// 0xff in the bytes of code word h (elements 4h .. 4h + 3 of the chunk) whose mask bit is clear
+__device__ __forceinline__ uint32_t rq_keep_bytes(uint32_t mk, int h) {
+    uint32_t keep = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) keep |= ((mk >> (4 * h + i)) & 1u) ? 0u : (0xffu << (8 * i));
+    return keep;
+}
+
 template <int DT>
 __global__ void __launch_bounds__(256)
 rowquant(const void* __restrict__ v, int R, int K, const int32_t* __restrict__ idx, int ko, int side_cols,
          int8_t* __restrict__ q_out, float* __restrict__ scale_out, void* __restrict__ side_out) {
     extern __shared__ __align__(16) unsigned char mask[];       // K / 8 bytes
-    __shared__ float red[8];
+    __shared__ uint32_t red[8];
     // A product kernel launched behind this one with programmatic stream serialization may start its set-up and its
     // weight loads now; it waits (griddepcontrol.wait) for this grid's results before it reads them.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -67,7 +112,7 @@ rowquant(const void* __restrict__ v, int R, int K, const int32_t* __restrict__ i
 
     for (int r = blockIdx.x; r < R; r += gridDim.x) {
         const uint4* row = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(v) + size_t(r) * K);
-        float a = 0.0f;
+        uint32_t m2 = 0u;                                                       // two running maxima of 15-bit magnitudes
         for (int c0 = threadIdx.x; c0 < nchunks; c0 += 256 * 4) {               // four loads in flight per thread
             uint4 w[4];
             uint32_t mk[4];
@@ -76,22 +121,27 @@ rowquant(const void* __restrict__ v, int R, int K, const int32_t* __restrict__ i
                 const int c = c0 + 256 * u;
                 const bool in = c < nchunks;
                 w[u] = in ? row[c] : make_uint4(0, 0, 0, 0);
-                mk[u] = in ? uint32_t(mask[c]) : 0xffu;
+                mk[u] = in ? uint32_t(mask[c]) : 0u;
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                float f[8];
-                widen8<DT>(w[u], f);
+                uint32_t x[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
+                if (mk[u] != 0u) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) a = fmaxf(a, ((mk[u] >> i) & 1u) ? 0.0f : fabsf(f[i]));
+                    for (int j = 0; j < 4; ++j) x[j] &= rq_keep_halves(mk[u], j);
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) m2 = __vmaxu2(m2, x[j] & 0x7fff7fffu);
             }
         }
+        m2 = max(m2 & 0xffffu, m2 >> 16);
 #pragma unroll
-        for (int s = 16; s >= 1; s >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, s));
-        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = a;
+        for (int s = 16; s >= 1; s >>= 1) m2 = max(m2, __shfl_xor_sync(0xffffffffu, m2, s));
+        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m2;
         __syncthreads();
 #pragma unroll
-        for (int i = 0; i < 8; ++i) a = fmaxf(a, red[i]);
+        for (int i = 0; i < 8; ++i) m2 = max(m2, red[i]);
+        const float a = widen16<DT>(m2);
         const float d = (a != 0.0f) ? a : 1.0f;
         if (threadIdx.x == 0) scale_out[r] = __fdiv_rn(a, 127.0f);
         // t = RN32(127 v / d).  n = 127 v is exact; for d within [2^-64, 2^64]: q0 = RN(n rc), e = n - d q0 (exact in one
@@ -102,6 +152,8 @@ rowquant(const void* __restrict__ v, int R, int K, const int32_t* __restrict__ i
         const bool quick = (d >= 5.421010862427522e-20f) && (d <= 1.8446744073709552e19f);
         float rc;
         asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc) : "f"(d));
+        constexpr float kMagic = 12582912.0f;                                   // 1.5 * 2^23: t + kMagic rounds t to an integer, ties to even
+        const uint64_t c127 = rq_pack2(127.0f, 127.0f), rc2 = rq_pack2(rc, rc), nd2 = rq_pack2(-d, -d), magic2 = rq_pack2(kMagic, kMagic);
 
         uint2* qrow = reinterpret_cast<uint2*>(q_out + size_t(r) * K);
         for (int c = threadIdx.x; c < nchunks; c += 256) {
@@ -109,21 +161,28 @@ rowquant(const void* __restrict__ v, int R, int K, const int32_t* __restrict__ i
             const uint32_t mk = mask[c];
             float f[8];
             widen8<DT>(w, f);
-            uint32_t b[8];
+            uint32_t b[8];                                                      // bit patterns whose low byte is the code
+            if (quick) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const float n = __fmul_rn(f[i], 127.0f);
-                float t;
-                if (quick) {
-                    const float q0 = __fmul_rn(n, rc);
-                    t = __fmaf_rn(__fmaf_rn(-d, q0, n), rc, q0);
-                } else {
-                    t = __fdiv_rn(n, d);
+                for (int i = 0; i < 8; i += 2) {
+                    const uint64_t n2 = rq_mul2(rq_pack2(f[i], f[i + 1]), c127);
+                    const uint64_t q0 = rq_mul2(n2, rc2);
+                    const uint64_t t2 = rq_fma2(rq_fma2(nd2, q0, n2), rc2, q0);
+                    const uint64_t s2 = rq_add2(t2, magic2);
+                    b[i] = uint32_t(s2);
+                    b[i + 1] = uint32_t(s2 >> 32);
                 }
-                const int qi = __float2int_rn(t);
-                b[i] = ((mk >> i) & 1u) ? 0u : (uint32_t(qi) & 0xffu);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) b[i] = __float_as_uint(__fadd_rn(__fdiv_rn(__fmul_rn(f[i], 127.0f), d), kMagic));
             }
-            qrow[c] = make_uint2(b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24), b[4] | (b[5] << 8) | (b[6] << 16) | (b[7] << 24));
+            uint32_t lo = rq_prmt(rq_prmt(b[0], b[1], 0x0040u), rq_prmt(b[2], b[3], 0x0040u), 0x5410u);
+            uint32_t hi = rq_prmt(rq_prmt(b[4], b[5], 0x0040u), rq_prmt(b[6], b[7], 0x0040u), 0x5410u);
+            if (mk != 0u) {                                                     // critical features hold no code
+                lo &= rq_keep_bytes(mk, 0);
+                hi &= rq_keep_bytes(mk, 1);
+            }
+            qrow[c] = make_uint2(lo, hi);
         }
         uint16_t* srow = static_cast<uint16_t*>(side_out) + size_t(r) * side_cols;
         const uint16_t* vrow = static_cast<const uint16_t*>(v) + size_t(r) * K;
