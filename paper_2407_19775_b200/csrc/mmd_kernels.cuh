@@ -93,7 +93,7 @@ __device__ __forceinline__ uint32_t rq_keep_bytes(uint32_t mk, int h) {
 }
 
 template <int DT>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 6)                        // six CTAs per SM: the row's second read then mostly hits L1 / L2 while others load
 rowquant(const void* __restrict__ v, int R, int K, const int32_t* __restrict__ idx, int ko, int side_cols,
          int8_t* __restrict__ q_out, float* __restrict__ scale_out, void* __restrict__ side_out) {
     extern __shared__ __align__(16) unsigned char mask[];       // K / 8 bytes
