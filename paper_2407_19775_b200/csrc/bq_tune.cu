@@ -12,6 +12,7 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include "bq_error.h"
 #include "bq_tune.h"
 
 namespace {
@@ -116,6 +117,11 @@ cudaError_t launch_sums(const void* x, const void* y, size_t n, double* partial,
     return cudaGetLastError();
 }
 
+int cuda_fail(cudaError_t e) {
+    bql::set_last_cuda_error(cudaGetErrorString(e));
+    return BQ_ERR_CUDA;
+}
+
 size_t elem_bytes(bq_dtype dt) { return dt == BQ_F32 ? 4 : ((dt == BQ_F16 || dt == BQ_BF16) ? 2 : 0); }
 
 }  // namespace
@@ -136,7 +142,10 @@ int bqt_block_errors(const void* x, bq_dtype xdt, size_t n, const bq_codebook* c
         if (blocks[c] < 1) return BQ_ERR_BLOCK;
     if (!cb) return BQ_ERR_CODEBOOK;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    if (n == 0) return cudaMemsetAsync(sums_out, 0, size_t(n_blocks + 1) * sizeof(double), s) == cudaSuccess ? BQ_OK : BQ_ERR_CUDA;
+    if (n == 0) {
+        const cudaError_t e = cudaMemsetAsync(sums_out, 0, size_t(n_blocks + 1) * sizeof(double), s);
+        return e == cudaSuccess ? BQ_OK : cuda_fail(e);
+    }
     if (!x || !workspace) return BQ_ERR_NULL;
     if (workspace_bytes < bqt_workspace_bytes(xdt, n) || reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return BQ_ERR_SIZE;
     void* y = workspace;
@@ -151,7 +160,7 @@ int bqt_block_errors(const void* x, bq_dtype xdt, size_t n, const bq_codebook* c
             case BQ_F16: e = launch_sums<BQ_F16>(x, y, n, partial, sums_out + c, norm_out, s); break;
             default: e = launch_sums<BQ_BF16>(x, y, n, partial, sums_out + c, norm_out, s); break;
         }
-        if (e != cudaSuccess) return BQ_ERR_CUDA;
+        if (e != cudaSuccess) return cuda_fail(e);
     }
     return BQ_OK;
 }
