@@ -80,6 +80,12 @@ __device__ __forceinline__ uint32_t rq_prmt(uint32_t a, uint32_t b, uint32_t sel
     asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
     return d;
 }
+// per-halfword unsigned maximum
+__device__ __forceinline__ uint32_t rq_max_u16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("max.u16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
 // 0xffff in the halves of word j (elements 2j, 2j + 1 of the chunk) whose mask bit is clear
 __device__ __forceinline__ uint32_t rq_keep_halves(uint32_t mk, int j) {
     return (((mk >> (2 * j)) & 1u) ? 0u : 0x0000ffffu) | (((mk >> (2 * j + 1)) & 1u) ? 0u : 0xffff0000u);
@@ -131,7 +137,7 @@ rowquant(const void* __restrict__ v, int R, int K, const int32_t* __restrict__ i
                     for (int j = 0; j < 4; ++j) x[j] &= rq_keep_halves(mk[u], j);
                 }
 #pragma unroll
-                for (int j = 0; j < 4; ++j) m2 = __vmaxu2(m2, x[j] & 0x7fff7fffu);
+                for (int j = 0; j < 4; ++j) m2 = rq_max_u16x2(m2, x[j] & 0x7fff7fffu);
             }
         }
         m2 = max(m2 & 0xffffu, m2 >> 16);
