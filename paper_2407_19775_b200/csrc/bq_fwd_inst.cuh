@@ -25,7 +25,7 @@ template <int XDT, int B, int RMAX> struct Shape {
 // Below this many elements the per-CTA table set-up of the tuned kernel (193 KB of shared
 // memory to fill) costs more than it saves; the LITE kernels read the tables through L1.
 #ifndef BQ_LITE_MAX_LOG2
-#define BQ_LITE_MAX_LOG2 21
+#define BQ_LITE_MAX_LOG2 23
 #endif
 constexpr size_t kLiteMaxElems = size_t(1) << BQ_LITE_MAX_LOG2;
 
