@@ -337,10 +337,11 @@ def run_ours(args):
 # ------------------------------------------------------------------------------------------ the small configurations
 
 def run_small(bq, dev):
-    """GPU time of the fused roundtrip on the configurations that fit in L2, twice: `warm_us` replays the call on the same
-    buffers (input and output stay in L2: the launch-bound figure), `cold_us` writes a 256 MiB buffer before every call (the
-    tensor then comes from DRAM, and the call also pays for the flush buffer's dirty lines it displaces) and subtracts the
-    time of the writes alone.  CUDA-graph replays, so no host launch gap is in either."""
+    """GPU time per call of the three operations on the four configurations beside the headline one, each with its own
+    block size.  `warm_us` replays the call on the same buffers (for the three configurations that fit in L2 the tensors
+    stay there: the launch-bound figure); for those, the roundtrip also gets `cold_us`: a 256 MiB buffer is written before
+    every call (the tensor then comes from DRAM, and the call also pays for the flush buffer's dirty lines it displaces) and
+    the time of the writes alone is subtracted.  CUDA-graph replays, so no host launch gap is in any figure."""
     cb = bq.Codebook(device=dev)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     side = torch.cuda.Stream()
@@ -366,21 +367,38 @@ def run_small(bq, dev):
 
     out = {}
     inner = 8
+    peak, _ = measured_peak()
     t_flush = replay_time([lambda: flush.fill_(1)] * inner) / inner
-    for name in ("tiny", "decode70b", "prefill7b"):
+    for name in ("tiny", "decode70b", "prefill7b", "moe_prefill"):
         w = workloads.WORKLOADS[name]
         x = workloads.make(name).reshape(-1).to(dev)
+        n = x.numel()
         y = torch.empty_like(x)
         b = w.blocks[0]
-        call = lambda: bq.bq_roundtrip(x, b, cb, y_out=y)
-        warm = replay_time([call] * inner) / inner
-        both = []
-        for _ in range(inner):
-            both += [lambda: flush.fill_(1), call]
-        cold = replay_time(both) / inner - t_flush
-        nbytes = 2 * x.numel() * x.element_size()
-        out[name] = {"shape": list(w.shape), "dtype": str(x.dtype)[6:], "block": b, "warm_us": round(warm * 1e3, 2), "cold_us": round(cold * 1e3, 2),
-                     "algorithmic_bytes": int(nbytes), "cold_gbs": round(nbytes / max(cold, 1e-6) / 1e6, 1), "gpu_launches": 2 * inner * 22}
+        codes = torch.empty(n, dtype=torch.uint8, device=dev)
+        absmax = torch.empty(n // b, dtype=torch.float32, device=dev)
+        calls = {"quantize": lambda: bq.bq_quantize(x, b, cb, codes, absmax),
+                 "dequantize": lambda: bq.bq_dequantize(codes, absmax, b, cb, x.dtype, y),
+                 "roundtrip": lambda: bq.bq_roundtrip(x, b, cb, y_out=y)}
+        es = x.element_size()
+        nbytes = {"quantize": n * es + n + 4 * (n // b), "dequantize": n + 4 * (n // b) + n * es, "roundtrip": 2 * n * es}
+        entry = {"shape": list(w.shape), "dtype": str(x.dtype)[6:], "block": b, "fits_l2": bool(2 * n * es < (100 << 20))}
+        launches = 0
+        for op, call in calls.items():
+            warm = replay_time([call] * inner) / inner
+            launches += inner * 22
+            entry[op] = {"warm_us": round(warm * 1e3, 2), "algorithmic_bytes": int(nbytes[op]), "gbs": round(nbytes[op] / warm / 1e6, 1),
+                         "frac_of_measured": round(nbytes[op] / warm / 1e6 / peak, 4)}
+            if entry["fits_l2"] and op == "roundtrip":
+                both = []
+                for _ in range(inner):
+                    both += [lambda: flush.fill_(1), call]
+                cold = replay_time(both) / inner - t_flush
+                launches += inner * 22
+                entry[op]["cold_us"] = round(cold * 1e3, 2)
+        entry["gpu_launches"] = launches
+        out[name] = entry
+        del x, y, codes, absmax
     return out
 
 

@@ -39,7 +39,11 @@ def test_bench_line_has_the_contract_keys(bq):
     assert 0.3 < t["frac_of_measured"] < 1.1 and t["picked_for_rel_rms_0.01"] in t["blocks"] and len(t["rel_rms_error"]) == len(t["blocks"])
     assert all(abs(a - q["rel_rms_error"]) < 2e-5 for a, q in zip(t["rel_rms_error"], d["quality"].values()))
     sc = d["small_configs"]
-    assert set(sc) == {"tiny", "decode70b", "prefill7b"} and all(0 < v["warm_us"] < 100 and 0 < v["cold_us"] < 200 for v in sc.values())
+    assert set(sc) == {"tiny", "decode70b", "prefill7b", "moe_prefill"}
+    for v in sc.values():
+        assert all(0 < v[op]["warm_us"] < 1000 and 0 < v[op]["frac_of_measured"] < 1.1 for op in ("quantize", "dequantize", "roundtrip"))
+        assert ("cold_us" in v["roundtrip"]) == v["fits_l2"]
+    assert sc["moe_prefill"]["roundtrip"]["frac_of_measured"] > 0.5 and not sc["moe_prefill"]["fits_l2"]
     # the decomposed linear layer: its own roofline object, no kernel error (its full-size parity is tests/test_gpu_mmd.py's)
     m = d["mmd"]
     mr = m["roofline"]
