@@ -67,8 +67,20 @@ cudaError_t launch_rowquant(const void* v, int R, int K, const int32_t* idx, int
     int grid = R;
     const int cap = sm_count * 16;
     if (grid > cap) grid = cap;
-    mmdk::rowquant<DT><<<grid, 256, smem, stream>>>(v, R, K, idx, ko, mmd_side_columns(ko), q, scale, side);
-    return cudaGetLastError();
+    // launched with programmatic stream serialization: the kernel waits (griddepcontrol.wait) for the kernels before it
+    // before it touches global memory; behind a kernel that never signals its dependents this is an ordinary launch
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(unsigned(grid), 1, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int side_cols = mmd_side_columns(ko);
+    return cudaLaunchKernelEx(&cfg, mmdk::rowquant<DT>, v, R, K, idx, ko, side_cols, q, scale, side);
 }
 
 cudaError_t rowquant_any(int dt, const void* v, int R, int K, const int32_t* idx, int ko, int8_t* q, float* scale, void* side, int sm_count,

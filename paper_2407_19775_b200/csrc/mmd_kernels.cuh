@@ -109,6 +109,11 @@ rowquant(const void* __restrict__ v, int R, int K, const int32_t* __restrict__ i
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int nchunks = K / 8;
     for (int c = threadIdx.x; c < (nchunks + 3) / 4; c += 256) reinterpret_cast<uint32_t*>(mask)[c] = 0u;
+    // This kernel is itself launched with programmatic stream serialization: behind a product kernel that lets its
+    // dependents start early (a chain of layers) its CTAs are already resident when that kernel ends.  Everything it reads
+    // from or writes to global memory comes after this wait for the kernels before it (the product kernel of the previous
+    // call may still be reading the buffers written below).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     __syncthreads();
     for (int j = threadIdx.x; j < ko; j += 256) {
         const int k = idx[j];
@@ -458,6 +463,10 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
     volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 8 * (2 * S + 1) + 8);
     float* sw_s = reinterpret_cast<float*>(ctrl + 256);                         // BN scales of this tile's columns
 
+    // Kernels launched behind this one with programmatic stream serialization (the row kernel of the next call, or this
+    // call's second launch for the tiles left over) may become resident as SMs free up; each waits for this grid to
+    // complete before it touches global memory that this grid reads or writes.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m0 = blockIdx.x * BM, n0 = (n_tile_base + int(blockIdx.y)) * BN;
     const uint32_t nsplit = cluster_size(), rank = cluster_rank();              // 1 and 0 without a cluster launch

@@ -295,3 +295,26 @@ def test_full_size_layer_all_tensor_kernels_and_sampled_rows(bq):
         assert np.all((g >= lo) & (g <= hi))
         assert np.mean(got == y_ref) > 0.999
     lin.close()
+
+
+@pytest.mark.parametrize("M,K,N", [(64, 2048, 4096), (64, 2048, 20488), (128, 1024, 1536)])
+def test_back_to_back_calls_share_a_workspace(bq, M, K, N):
+    """A chain of calls with different activations through one workspace and no synchronisation in between: the row kernel
+    and the product kernel of consecutive calls are launched so that each may become resident before the one before it has
+    ended, and each must still wait before it touches the shared buffers.  Without critical features the tensor-core path
+    and the general kernel agree bit for bit, so every output of the chain is compared with a call of its own."""
+    g = torch.Generator().manual_seed(M + N)
+    W = (torch.randn(N, K, generator=g) * 0.03).to(torch.float16)
+    lin = bq.DecomposedLinear(W.cuda(), np.zeros(0, np.int32))
+    ws = lin.workspace(M)
+    xs = [(torch.randn(M, K, generator=g) * (0.2 + 0.3 * i)).to(torch.float16).cuda() for i in range(8)]
+    ys = [torch.empty(M, N, dtype=torch.float32, device="cuda") for _ in xs]
+    for _ in range(3):
+        for x, y in zip(xs, ys):
+            lin.linear(x, y_out=y, workspace=ws)
+    torch.cuda.synchronize()
+    assert lin.kernel_status() == 0
+    for x, y in zip(xs, ys):
+        assert torch.equal(y, lin.linear(x, torch.float32, path=1))
+    check_output(ys[3], xs[3].cpu(), W, np.zeros(0, np.int32), F16, exact_expected=True)
+    lin.close()
