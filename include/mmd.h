@@ -113,11 +113,15 @@ int mmd_workspace_layout(const mmd_weights* w, int M, size_t* offsets3, size_t* 
 
 /*
  * mmd_linear -- Y = X W^T through the decomposition: one row kernel over X into the
- * workspace, then one product kernel.
+ * workspace, then the product kernel (two launches of it for one row of tiles that does not
+ * fill whole waves of the device: the whole waves, then the tiles left over).  Consecutive
+ * calls on one stream are ordered as usual; the kernels of a call and of the next may become
+ * resident early (programmatic stream serialization) but wait for the kernels before them
+ * before they touch global memory.
  *   X: [M, K] of the handle's element type (16-byte aligned).  Y: [M, N] of type ydt.
  *   workspace: at least mmd_workspace_layout's total, 256-byte aligned; its contents after
  *   the call are the decomposition of X (tests read them back).  Calls that share a
- *   workspace must not overlap on the device.
+ *   workspace must not overlap on the device (different streams): order them.
  *   path: MMD_PATH_*.  The two kernels give identical integer sums; their fp32 side sums may
  *   differ in the order of the additions.
  */

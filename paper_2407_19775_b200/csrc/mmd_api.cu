@@ -164,6 +164,7 @@ cudaError_t launch_tc_bm(const mmd_weights* w, const CUtensorMap& mqx, const CUt
     // the ranks' partial sums must fit into rank 0's ring
     if (split > 1 && size_t(split - 1) * BM * BN * 4 > size_t(Cfg::kStages) * Cfg::kStageBytes) split = 1;
     if (split > ksteps) split = ksteps;
+    if (split > 4) split = 4;                                    // the largest cluster the exchange is written for (and the table below holds)
     if (split < 1) split = 1;
     cudaLaunchConfig_t cfg = {};
     if (n_tile_count < 0) n_tile_count = (w->N + BN - 1) / BN - n_tile_base;
