@@ -514,32 +514,40 @@ def run_mmd(bq, dev, args):
     # a decode step through a 70B-class layer: 64 tokens, every weight read once (HBM-bound).  The codes of one layer (67 MB)
     # would stay in the 126 MB L2 from call to call, so the timed graph cycles through four copies of the layer (268 MB):
     # every call streams its weights from DRAM, as consecutive layers of a model do.
-    dX, dW, didx = workloads.make_linear("mmd_decode70b")
-    dM, dK, dN = dX.shape[0], dX.shape[1], dW.shape[0]
-    dXd = dX.to(dev)
-    dWd = dW.to(dev)
-    dlins = [bq.DecomposedLinear(dWd, didx) for _ in range(DECODE_LAYER_COPIES)]
-    dy = torch.empty((dM, dN), dtype=dX.dtype, device=dev)
-    dws = dlins[0].workspace(dM)
-    for dl in dlins:
-        dl.linear(dXd, y_out=dy, workspace=dws)
-    torch.cuda.synchronize()
-    turn = [0]
+    def decode_entry(out_features, copies):
+        dX, dW, didx = workloads.make_linear("mmd_decode70b")
+        dXd = dX.to(dev)
+        dWd = dW.to(dev)
+        if out_features is not None:                             # a wider layer: the workload's rows repeated (timing only)
+            dWd = dWd.repeat((out_features + dWd.shape[0] - 1) // dWd.shape[0], 1)[:out_features].contiguous()
+        dM, dK, dN = dX.shape[0], dX.shape[1], dWd.shape[0]
+        dlins = [bq.DecomposedLinear(dWd, didx) for _ in range(copies)]
+        del dWd
+        dy = torch.empty((dM, dN), dtype=dX.dtype, device=dev)
+        dws = dlins[0].workspace(dM)
+        for dl in dlins:
+            dl.linear(dXd, y_out=dy, workspace=dws)
+        torch.cuda.synchronize()
+        turn = [0]
 
-    def decode_call():
-        dlins[turn[0] % DECODE_LAYER_COPIES].linear(dXd, y_out=dy, workspace=dws)
-        turn[0] += 1
+        def decode_call():
+            dlins[turn[0] % copies].linear(dXd, y_out=dy, workspace=dws)
+            turn[0] += 1
 
-    ms_dec = timed_gpu(decode_call, 2 * DECODE_LAYER_COPIES)
-    dstatus = max(dl.kernel_status() for dl in dlins)
-    dec_bytes = dN * dK + dM * dK * 3 + dM * dN * 2
-    decode = {"workload": f"mmd_decode70b: X [{dM},{dK}] x W [{dN},{dK}]^T fp16, {didx.size} critical features; "
-                          f"{DECODE_LAYER_COPIES} copies of the layer in turn ({DECODE_LAYER_COPIES * dN * dK >> 20} MiB of codes, larger than L2)",
-              "us_per_call": round(ms_dec * 1e3, 2),
-              "algorithmic_bytes": int(dec_bytes), "gbs": round(dec_bytes / ms_dec / 1e6, 1), "frac_of_measured_hbm": round(dec_bytes / ms_dec / 1e6 / hbm, 4),
-              "kernel_status": dstatus}
-    for dl in dlins:
-        dl.close()
+        ms_dec = timed_gpu(decode_call, 2 * copies)
+        dstatus = max(dl.kernel_status() for dl in dlins)
+        dec_bytes = dN * dK + dM * dK * 3 + dM * dN * 2
+        entry = {"workload": f"mmd_decode70b{'' if out_features is None else ' (weight rows repeated)'}: X [{dM},{dK}] x W [{dN},{dK}]^T fp16, {didx.size} critical features; "
+                             f"{copies} copies of the layer in turn ({copies * dN * dK >> 20} MiB of codes, larger than L2)",
+                 "us_per_call": round(ms_dec * 1e3, 2),
+                 "algorithmic_bytes": int(dec_bytes), "gbs": round(dec_bytes / ms_dec / 1e6, 1),
+                 "frac_of_measured_hbm": round(dec_bytes / ms_dec / 1e6 / hbm, 4), "kernel_status": dstatus}
+        for dl in dlins:
+            dl.close()
+        return entry
+
+    decode = decode_entry(None, DECODE_LAYER_COPIES)            # the 8192 -> 8192 projection
+    decode_wide = decode_entry(28672, 2)                        # the 8192 -> 28672 projection: more tiles than SMs
     return {
         "workload": f"{MMD_WORKLOAD}: X [{M},{K}] x W [{N},{K}]^T bf16, {idx.size} critical features; {wl.recipe}",
         "ms_per_call": round(ms_call, 4), "tops": round(ops / ms_call / 1e9, 1), "kernel_status": status,
@@ -554,8 +562,8 @@ def run_mmd(bq, dev, args):
                     "weight_rel_rms_error": round(w_err, 5)},
         "cpu_baseline": {"value": round(2.0 * 256 * N * K / cpu_s / 1e12, 4), "unit": "TOP/s", "cores": os.cpu_count(), "kind": "oracle",
                          "sample": "first 256 tokens through the whole layer (weights already decomposed); numpy/BLAS threads"},
-        "decode": decode,
-        "gpu_launches": (2 * 2 + 8 + 2 * 8) * reps + 2 * (reps + 3),
+        "decode": decode, "decode_wide": decode_wide,
+        "gpu_launches": (2 * 2 + 8 + 2 * 8 + 2 * 4) * reps + 2 * (reps + 3),
     }
 
 

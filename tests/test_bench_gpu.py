@@ -53,3 +53,5 @@ def test_bench_line_has_the_contract_keys(bq):
     assert 1.9 < m["quality"]["weight_bytes_ratio"] < 2.0 and m["gpu_launches"] > 0
     dec = m["decode"]
     assert dec["kernel_status"] == 0 and 0.2 < dec["frac_of_measured_hbm"] < 1.1
+    wide = m["decode_wide"]
+    assert wide["kernel_status"] == 0 and 0.3 < wide["frac_of_measured_hbm"] < 1.1 and wide["algorithmic_bytes"] > 3 * dec["algorithmic_bytes"]
