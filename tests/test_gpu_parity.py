@@ -151,13 +151,13 @@ def test_config_sweep1g_full_size(bq, gcb, cb):
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.float16, torch.bfloat16])
 @pytest.mark.parametrize("block", [64, 128, 256, 512, 1024, 2048, 4096])
-@pytest.mark.parametrize("size", ["small", "large"])
+@pytest.mark.parametrize("size", ["small", "medium", "large"])
 def test_tuned_blocks_many_tiles_and_ragged_tail(bq, gcb, cb, dtype, block, size):
-    """Several tiles per warp, then blocks that do not fill a tile, then a short block.  "small"
-    stays below the 8 Mi-element switch of the forward kernels (tables read through L1), "large" is above it
-    (persistent kernels with the tables in shared memory)."""
+    """Several tiles per warp, then blocks that do not fill a tile, then a short block.  "small" and
+    "medium" (a thousand CTAs) stay below the 8 Mi-element switch of the forward kernels (tables read
+    through L1), "large" is above it (persistent kernels with the tables in shared memory)."""
     g = torch.Generator().manual_seed(block + 17)
-    n = (300_000 if size == "small" else (1 << 23) + 150_000)
+    n = {"small": 300_000, "medium": (1 << 22) + 150_000, "large": (1 << 23) + 150_000}[size]
     n = (n // block) * block + 3 * block + 37
     x = (torch.randn(n, generator=g) * (1.0 + 30.0 * (torch.rand(n, generator=g) < 0.002))).to(dtype)
     check_all_ops(bq, gcb, cb, x, block)
