@@ -38,19 +38,19 @@ cudaError_t fwd_general_y(int ydt, bool wy, bool wq, const void* x, void* y, uin
 constexpr int kDeqNT = BQ_DEQ_NT;
 constexpr int kDeqU = BQ_DEQ_U;
 
-template <int YDT>
+template <int YDT, bool WIDE>
 cudaError_t deq_fast_go(const uint8_t* codes, const float* absmax, void* y, size_t n16, int log2_block, const bqk::DeviceTables& tab,
                         int sm_count, cudaStream_t stream) {
     if (n16 <= (size_t(1) << (BQ_LITE_MAX_LOG2 + 2 - 4))) {      // up to 8 Mi elements: no shared-memory table, one chunk per thread
         const size_t grid = (n16 + 255) / 256;
-        bqk::deq_fast<YDT, 256, 1, true><<<unsigned(grid), 256, 0, stream>>>(codes, absmax, y, n16, log2_block, tab);
+        bqk::deq_fast<YDT, 256, 1, true, WIDE><<<unsigned(grid), 256, 0, stream>>>(codes, absmax, y, n16, log2_block, tab);
         return cudaGetLastError();
     }
     const size_t tile = size_t(kDeqNT) * kDeqU;
     size_t grid = (n16 + tile - 1) / tile;
     const size_t cap = size_t(sm_count) * BQ_DEQ_CTAS;
     if (grid > cap) grid = cap;
-    bqk::deq_fast<YDT, kDeqNT, kDeqU, false><<<unsigned(grid), kDeqNT, bqk::kDeqSmemBytes, stream>>>(codes, absmax, y, n16, log2_block, tab);
+    bqk::deq_fast<YDT, kDeqNT, kDeqU, false, WIDE><<<unsigned(grid), kDeqNT, bqk::kDeqSmemBytes, stream>>>(codes, absmax, y, n16, log2_block, tab);
     return cudaGetLastError();
 }
 
@@ -73,10 +73,16 @@ cudaError_t launch_fwd_general(int xdt, int ydt, bool write_y, bool write_q, con
 
 cudaError_t launch_deq_fast(int ydt, const uint8_t* codes, const float* absmax, void* y, size_t n16, int log2_block,
                             const bqk::DeviceTables& tab, int sm_count, int /*device*/, cudaStream_t stream) {
+    // the 256-bit stores of the kernel need y on a 32-byte boundary; a y that is only 16-byte
+    // aligned (a tensor sliced at 8 16-bit elements, say) takes the variant with 128-bit stores
+    const bool wide = (reinterpret_cast<uintptr_t>(y) & 31u) == 0;
     switch (ydt) {
-        case BQ_F32: return deq_fast_go<bqk::kF32>(codes, absmax, y, n16, log2_block, tab, sm_count, stream);
-        case BQ_F16: return deq_fast_go<bqk::kF16>(codes, absmax, y, n16, log2_block, tab, sm_count, stream);
-        default: return deq_fast_go<bqk::kBF16>(codes, absmax, y, n16, log2_block, tab, sm_count, stream);
+#define BQ_DEQ_CASE(DT) (wide ? deq_fast_go<DT, true>(codes, absmax, y, n16, log2_block, tab, sm_count, stream) \
+                              : deq_fast_go<DT, false>(codes, absmax, y, n16, log2_block, tab, sm_count, stream))
+        case BQ_F32: return BQ_DEQ_CASE(bqk::kF32);
+        case BQ_F16: return BQ_DEQ_CASE(bqk::kF16);
+        default: return BQ_DEQ_CASE(bqk::kBF16);
+#undef BQ_DEQ_CASE
     }
 }
 

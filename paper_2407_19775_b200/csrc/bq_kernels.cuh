@@ -77,6 +77,16 @@ __device__ __forceinline__ void stg_stream_16(void* p, uint4 v) {
 __device__ __forceinline__ void stg_stream_32(void* p, uint4 a, uint4 b) {
     asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w) : "memory");
 }
+// 32 contiguous bytes: one 256-bit store when p is 32-byte aligned (WIDE), else two 128-bit ones
+template <bool WIDE>
+__device__ __forceinline__ void store_32(void* p, uint4 a, uint4 b) {
+    if constexpr (WIDE) {
+        stg_stream_32(p, a, b);
+    } else {
+        stg_stream_16(p, a);
+        stg_stream_16(static_cast<char*>(p) + 16, b);
+    }
+}
 __device__ __forceinline__ void stg_stream_8(void* p, uint2 v) {
     asm volatile("st.global.cs.v2.u32 [%0], {%1,%2};" ::"l"(p), "r"(v.x), "r"(v.y) : "memory");
 }
@@ -534,11 +544,13 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
 #ifndef BQ_DEQ_MINB
 #define BQ_DEQ_MINB 3
 #endif
-template <int YDT, int NT, int U, bool LITE>
+// WIDE: y is 32-byte aligned, so 16 outputs of a 16-bit type (8 of fp32) go out as one 256-bit
+// store; otherwise (y only 16-byte aligned) the same bytes leave as two 128-bit stores.
+template <int YDT, int NT, int U, bool LITE, bool WIDE>
 __global__ void __launch_bounds__(NT, LITE ? 1 : BQ_DEQ_MINB)
 deq_fast(const uint8_t* __restrict__ codes, const float* __restrict__ absmax, void* __restrict__ y, size_t n16 /* n / 16 */,
          int log2_block, DeviceTables tab) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
+    extern __shared__ __align__(128) unsigned char smem_raw[];
     const uint32_t sm_base = uint32_t(__cvta_generic_to_shared(smem_raw));
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t sm_lane = sm_base + uint32_t(lane) * 4u;
@@ -604,12 +616,12 @@ deq_fast(const uint8_t* __restrict__ codes, const float* __restrict__ absmax, vo
                 for (int k = 0; k < 2; ++k) {
                     const float t0[4] = {v[8 * k], v[8 * k + 1], v[8 * k + 2], v[8 * k + 3]};
                     const float t1[4] = {v[8 * k + 4], v[8 * k + 5], v[8 * k + 6], v[8 * k + 7]};
-                    stg_stream_32(out + 32 * k, narrow_chunk<kF32>(t0), narrow_chunk<kF32>(t1));
+                    store_32<WIDE>(out + 32 * k, narrow_chunk<kF32>(t0), narrow_chunk<kF32>(t1));
                 }
             } else {
                 const float t0[8] = {v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]};
                 const float t1[8] = {v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15]};
-                stg_stream_32(out, narrow_chunk<YDT>(t0), narrow_chunk<YDT>(t1));
+                store_32<WIDE>(out, narrow_chunk<YDT>(t0), narrow_chunk<YDT>(t1));
             }
         }
     }

@@ -3,6 +3,8 @@
 
 #include <cuda_runtime.h>
 
+#include <mutex>
+
 #include "../../include/bq.h"
 #include "bq_kernels.cuh"
 #include "bq_tables.h"
@@ -37,12 +39,17 @@ cudaError_t launch_deq_general(int ydt, const uint8_t* codes, const float* absma
                                const bqk::DeviceTables& tab, int sm_count, cudaStream_t stream);
 
 // Kernels that need more than 48 KB of dynamic shared memory must opt in once per device.
+// The per-device "already done" table is written under a lock (two host threads may make their
+// first call together); a device beyond the table simply opts in on every call.
 template <auto Kernel>
 inline cudaError_t allow_smem(int bytes, int device) {
+    static std::mutex lock;
     static bool done[64] = {};
-    if (device >= 0 && device < 64 && done[device]) return cudaSuccess;
+    const bool tracked = device >= 0 && device < 64;
+    std::lock_guard<std::mutex> guard(lock);
+    if (tracked && done[device]) return cudaSuccess;
     const cudaError_t e = cudaFuncSetAttribute(Kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    if (e == cudaSuccess && device >= 0 && device < 64) done[device] = true;
+    if (e == cudaSuccess && tracked) done[device] = true;
     return e;
 }
 

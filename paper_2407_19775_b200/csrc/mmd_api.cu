@@ -5,6 +5,7 @@
 #include "mmd_kernels.cuh"
 
 #include <cstring>
+#include <mutex>
 #include <new>
 
 namespace {
@@ -23,15 +24,22 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
+    // a function-local static is initialised once, under the language's own lock, however many threads arrive together
+    static const EncodeTiledFn fn = [] {
         void* p = nullptr;
         cudaDriverEntryPointQueryResult qres;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess && qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
+            return reinterpret_cast<EncodeTiledFn>(p);
+        return EncodeTiledFn(nullptr);
+    }();
     return fn;
 }
+
+// Per-device facts that the launchers look up on first use (shared-memory opt-ins, how many clusters run at once) are
+// kept in small tables indexed by the device ordinal and written under this lock: two host threads may issue their
+// first call at the same time.  mmd_decompose refuses devices beyond the tables, so an index is always in range.
+constexpr int kMaxDevices = 64;
+std::mutex g_cache_lock;
 
 // Row-major [rows, cols] matrix of 1- or 2-byte elements, tiles of box_rows x 128 bytes, 128-byte swizzle.
 bool make_map(CUtensorMap* map, const void* base, int elem_bytes, uint64_t rows, uint64_t cols, uint32_t box_rows) {
@@ -147,11 +155,15 @@ template <int XDT, int YDT, int BN, int BM, int KPB>
 cudaError_t launch_tc_bm(const mmd_weights* w, const CUtensorMap& mqx, const CUtensorMap& msx, const float* sx, void* y, int M, int split,
                          cudaStream_t stream, int n_tile_base = 0, int n_tile_count = -1) {
     using Cfg = mmdk::TcCfg<BN, BM, KPB>;
-    static bool opted[64] = {};
-    if (w->device < 0 || w->device >= 64 || !opted[w->device]) {
+    static bool opted[kMaxDevices] = {};
+    static int max_clusters[kMaxDevices][5] = {};
+    if (w->device < 0 || w->device >= kMaxDevices) return cudaErrorInvalidDevice;
+    const int d = w->device;
+    std::lock_guard<std::mutex> guard(g_cache_lock);              // held to the end: the tables are read on the way to the launch
+    if (!opted[d]) {
         const cudaError_t e = cudaFuncSetAttribute(mmdk::gemm_tc<XDT, YDT, BN, BM, KPB>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::kSmemBytes));
         if (e != cudaSuccess) return e;
-        if (w->device >= 0 && w->device < 64) opted[w->device] = true;
+        opted[d] = true;
     }
     int kblocks = (w->K + 127) / 128, sblocks = w->side_cols / 64;
     const int ksteps = (kblocks + KPB - 1) / KPB;
@@ -178,10 +190,8 @@ cudaError_t launch_tc_bm(const mmd_weights* w, const CUtensorMap& mqx, const CUt
     // The split is there to put one CTA on every SM at the same time.  A cluster's CTAs must sit in one GPC, so fewer
     // clusters of 3 or 4 fit on the device than its SM count suggests; a split whose clusters would not all run at once
     // (a second, nearly empty wave) is lowered until they do.
-    static int max_clusters[64][5] = {};
     const long clusters = long((M + BM - 1) / BM) * n_tile_count;
     for (; split > 1; --split) {
-        const int d = (w->device >= 0 && w->device < 64) ? w->device : 0;
         if (max_clusters[d][split] == 0) {
             cfg.gridDim = dim3(1, unsigned(w->sm_count / split), unsigned(split));
             attr[1].val.clusterDim.z = unsigned(split);
@@ -225,11 +235,15 @@ cudaError_t launch_tc_decode(const mmd_weights* w, const CUtensorMap& mqx2, cons
 
 template <int XDT, int YDT>
 cudaError_t launch_tcp(const mmd_weights* w, const CUtensorMap& mqx, const float* sx, const void* sidex, void* y, int M, cudaStream_t stream) {
-    static bool opted[64] = {};
-    if (w->device < 0 || w->device >= 64 || !opted[w->device]) {
-        const cudaError_t e = cudaFuncSetAttribute(mmdk::gemm_tcp<XDT, YDT>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(mmdk::kTcpSmemBytes));
-        if (e != cudaSuccess) return e;
-        if (w->device >= 0 && w->device < 64) opted[w->device] = true;
+    static bool opted[kMaxDevices] = {};
+    if (w->device < 0 || w->device >= kMaxDevices) return cudaErrorInvalidDevice;
+    {
+        std::lock_guard<std::mutex> guard(g_cache_lock);
+        if (!opted[w->device]) {
+            const cudaError_t e = cudaFuncSetAttribute(mmdk::gemm_tcp<XDT, YDT>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(mmdk::kTcpSmemBytes));
+            if (e != cudaSuccess) return e;
+            opted[w->device] = true;
+        }
     }
     const int mtiles = (M + 127) / 128, ntiles = (w->N + mmdk::kTcpBN - 1) / mmdk::kTcpBN;
     const long total = long(mtiles) * ntiles;
@@ -241,9 +255,11 @@ cudaError_t launch_tcp(const mmd_weights* w, const CUtensorMap& mqx, const float
 
 template <int XDT, int YDT>
 cudaError_t launch_tc2(const mmd_weights* w, const CUtensorMap& mqx, const float* sx, const void* sidex, void* y, int M, cudaStream_t stream) {
-    static bool opted[64] = {};
-    static int max_pairs[64] = {};
-    const int d = (w->device >= 0 && w->device < 64) ? w->device : 0;
+    static bool opted[kMaxDevices] = {};
+    static int max_pairs[kMaxDevices] = {};
+    if (w->device < 0 || w->device >= kMaxDevices) return cudaErrorInvalidDevice;
+    const int d = w->device;
+    std::unique_lock<std::mutex> guard(g_cache_lock);
     if (!opted[d]) {
         cudaError_t e = cudaFuncSetAttribute(mmdk::gemm_tc2<XDT, YDT>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(mmdk::kPairSmemBytes));
         if (e != cudaSuccess) return e;
@@ -259,9 +275,11 @@ cudaError_t launch_tc2(const mmd_weights* w, const CUtensorMap& mqx, const float
         max_pairs[d] = n;
         opted[d] = true;
     }
+    const int pairs_at_once = max_pairs[d];
+    guard.unlock();
     const int mpairs = (M + 255) / 256, ntiles = (w->N + mmdk::kTcpBN - 1) / mmdk::kTcpBN;
     const long total = long(mpairs) * ntiles;
-    const unsigned pairs = unsigned(total < max_pairs[d] ? total : max_pairs[d]);
+    const unsigned pairs = unsigned(total < pairs_at_once ? total : pairs_at_once);
     mmdk::gemm_tc2<XDT, YDT><<<2 * pairs, mmdk::kTcThreads, mmdk::kPairSmemBytes, stream>>>(
         mqx, w->map_q_pair, sx, w->scale, sidex, w->side, w->side_cols, w->ko, y, M, w->N, (w->K + 127) / 128, mpairs, ntiles, w->status);
     return cudaGetLastError();
@@ -379,6 +397,7 @@ int mmd_decompose(const void* W, bq_dtype dt, int N, int K, const int32_t* idx_h
     w->N = N; w->K = K; w->ko = n_features; w->side_cols = mmd_side_columns(n_features); w->dtype = dt;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = cudaGetDevice(&w->device);
+    if (e == cudaSuccess && (w->device < 0 || w->device >= kMaxDevices)) e = cudaErrorInvalidDevice;     // beyond the per-device tables
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&w->sm_count, cudaDevAttrMultiProcessorCount, w->device);
     const size_t o_q = 0;
     const size_t o_scale = round_up(size_t(N) * K, kWsAlign);

@@ -461,6 +461,8 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
     const uint32_t accbar = empty0 + 8u * S;                                    // accumulators complete
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl + 8 * (2 * S + 1));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 8 * (2 * S + 1) + 8);
+    volatile int* peer_gave_up = reinterpret_cast<volatile int*>(ctrl + 8 * (2 * S + 1) + 12);   // split K: set in rank 0 by a rank that ran out of a wait
+    static_assert(8 * (2 * S + 1) + 16 <= 256, "control words end before the column scales");
     float* sw_s = reinterpret_cast<float*>(ctrl + 256);                         // BN scales of this tile's columns
 
     // Kernels launched behind this one with programmatic stream serialization (the row kernel of the next call, or this
@@ -480,6 +482,7 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
         for (int s = 0; s < S; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, 1); }
         mbar_init(accbar, 1);
         *abort_flag = 0;
+        *peer_gave_up = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -596,8 +599,11 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
                         for (int j = 0; j < 32; ++j) st_cluster_u32(dst + uint32_t(j) * BM * 4u, ai[j]);
                     }
                 }
+                // a rank whose wait ran out has no sums to give: it says so, and rank 0 then stores nothing for this tile
+                if (!ok && lane == 0) st_cluster_u32(map_to_cta(smem_u32(const_cast<int*>(peer_gave_up)), 0), 1u);
             }
             cluster_sync_all();                                                  // the partial sums are in rank 0's shared memory
+            if (rank == 0 && *peer_gave_up) ok = false;
         }
         if (ok && rank == 0) {
 #pragma unroll 1

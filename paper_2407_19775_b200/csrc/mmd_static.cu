@@ -43,6 +43,10 @@ cudaError_t scratch_address(void** out) {
 extern "C" int mmd_linear_static(const mmd_weights* w, const void* X, int M, void* Y, bq_dtype ydt, int path, void* cuda_stream) {
     if (!w) return BQ_ERR_NULL;
     if (M < 0) return BQ_ERR_SIZE;
+    // A call of mmd_linear with zero rows checks the element type and the path and launches nothing:
+    // both entry points then answer a bad argument with the same code, whatever M is.
+    const int checked = mmd_linear(w, X, 0, Y, ydt, nullptr, 0, path, cuda_stream);
+    if (checked != BQ_OK || M == 0) return checked;
     size_t need = 0;
     const int rc = mmd_workspace_layout(w, M, nullptr, &need);
     if (rc != BQ_OK) return rc;
@@ -53,7 +57,6 @@ extern "C" int mmd_linear_static(const mmd_weights* w, const void* X, int M, voi
         bql::set_last_cuda_error(text);
         return MMD_ERR_STATIC_LIMIT;
     }
-    if (M == 0) return BQ_OK;
     void* scratch = nullptr;
     const cudaError_t e = scratch_address(&scratch);
     if (e != cudaSuccess) {

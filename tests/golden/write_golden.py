@@ -10,6 +10,12 @@ codebook_dynamic_tree.txt : the 256 fp32 codes as hex bit patterns, one per line
                             techniques", item 1.
 thresholds_round_down.txt : the 255 midpoints between neighbouring codes, each rounded
                             toward -inf to fp32 (hex), plus their SHA-256.
+
+These files are REGRESSION pins: they hold what the oracle produced when they were written, so
+they catch a later change of the oracle, not a mistake it had from the start.  The checks of the
+codebook against its definition are elsewhere (tests/test_oracle_codebook.py): the rebuild of all
+256 values in exact rational arithmetic, the decoding of the eight bit fields, and the mirror /
+sum / decade invariants.
 """
 import hashlib
 import os
@@ -32,7 +38,7 @@ def hexf(v) -> str:
 def main() -> None:
     cb = oracle.make_codebook()
     with open(os.path.join(HERE, "codebook_dynamic_tree.txt"), "w") as f:
-        f.write("# dynamic-tree codebook, fp32 bit patterns, index ascending (written by write_golden.py from oracle/)\n")
+        f.write("# dynamic-tree codebook, fp32 bit patterns, index ascending (regression pin: written by write_golden.py from oracle/; the definition is checked by the exact-rational rebuild in test_oracle_codebook.py)\n")
         for v in cb:
             f.write(hexf(v) + "\n")
         f.write("sha256 " + hashlib.sha256(cb.astype("<f4").tobytes()).hexdigest() + "\n")
@@ -46,7 +52,7 @@ def main() -> None:
         down.append(g)
     down = np.array(down, np.float32)
     with open(os.path.join(HERE, "thresholds_round_down.txt"), "w") as f:
-        f.write("# midpoints between neighbouring codes, rounded toward -inf to fp32 (written by write_golden.py)\n")
+        f.write("# midpoints between neighbouring codes, rounded toward -inf to fp32 (regression pin: written by write_golden.py from the oracle's codes in exact rationals)\n")
         for v in down:
             f.write(hexf(v) + "\n")
         f.write("sha256 " + hashlib.sha256(down.astype("<f4").tobytes()).hexdigest() + "\n")

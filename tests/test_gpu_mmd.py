@@ -207,7 +207,6 @@ def test_linear_one_row_of_tiles_shares_k_steps(bq, M, K, N, ko):
         y = lin.linear(X.cuda(), out, path=3)
         assert lin.kernel_status() == 0
         check_output(y, X, W, idx, F16, exact_expected=(ko == 0))
-    assert torch.equal(lin.linear(X.cuda(), torch.float32, path=3)[:, :8], lin.linear(X.cuda(), torch.float32, path=3)[:, :8])
     lin.close()
 
 
@@ -263,11 +262,12 @@ def test_decode_workload_rows(bq):
     check_output(y16, X, W, idx, F16, exact_expected=False)
 
 
-def test_full_size_layer_all_tensor_kernels_and_sampled_rows(bq):
+def test_full_size_layer_all_tensor_kernels_every_row(bq):
     """The benchmark's layer at full size (4096 x 6144 -> 16384, bf16, 6 critical features) in the launch configurations
     bench.py times: the CTA-pair and the single-CTA persistent kernels add the side features in the same order, so they
-    must agree bit for bit; the one-tile-per-CTA kernel accumulates them on the tensor cores (other order); rows sampled
-    across tiles and CTA pairs are checked against the oracle."""
+    must agree bit for bit; the one-tile-per-CTA kernel accumulates them on the tensor cores (other order).  Every row of
+    every output is checked against the oracle (512 rows at a time, so that the oracle's float64 matrices stay small),
+    and so is every int8 code, scale and side column of the decomposed weights."""
     X, W, idx = workloads.make_linear("mmd_prefill_moe")
     Xd = X.cuda()
     lin = bq.DecomposedLinear(W.cuda(), idx)
@@ -278,22 +278,26 @@ def test_full_size_layer_all_tensor_kernels_and_sampled_rows(bq):
     assert torch.equal(y_pair, y_solo)
     y_tile = lin.linear(Xd, path=3)
     assert lin.kernel_status() == 0
-    assert (y_tile == y_pair).float().mean().item() > 0.999
-    rows = np.array([0, 127, 128, 255, 256, 1500, 2047, 2048, 4095])
+    y_gen = lin.linear(Xd, path=1)
     qw, sw, wo = mo.rowquant(bits(W), BF16, idx)
-    q_dev, s_dev, _, _ = lin.view()
-    assert np.array_equal(q_dev[-300:].cpu().numpy(), qw[-300:]) and np.array_equal(s_dev.cpu().numpy(), sw)
-    Xr = X[rows]
-    y_ref, _, _, sabs = mo.linear(bits(Xr), BF16, qw, sw, wo, idx, BF16, parts=True)
-    y32 = mo.linear(bits(Xr), BF16, qw, sw, wo, idx, F32).astype(np.float64)
-    tol = 2.0 ** -23 * np.abs(y32) + (wo.shape[1] + 2) * 2.0 ** -22 * sabs
-    lo = mo.widen(mo.narrow((y32 - tol).astype(np.float32), BF16), BF16)
-    hi = mo.widen(mo.narrow((y32 + tol).astype(np.float32), BF16), BF16)
-    for y in (y_pair, y_tile):
-        got = bits(y[torch.from_numpy(rows).cuda()])
-        g = mo.widen(got, BF16)
-        assert np.all((g >= lo) & (g <= hi))
-        assert np.mean(got == y_ref) > 0.999
+    q_dev, s_dev, side_dev, _ = lin.view()
+    assert np.array_equal(q_dev.cpu().numpy(), qw) and np.array_equal(s_dev.cpu().numpy().view(np.uint32), sw.view(np.uint32))
+    assert np.array_equal(bits(side_dev), wo)
+    same = {"pair": 0, "tile": 0, "general": 0}
+    for r0 in range(0, X.shape[0], 512):
+        Xr = bits(X[r0:r0 + 512])
+        y_ref, _, _, sabs = mo.linear(Xr, BF16, qw, sw, wo, idx, BF16, parts=True)
+        y32 = mo.linear(Xr, BF16, qw, sw, wo, idx, F32).astype(np.float64)
+        tol = 2.0 ** -23 * np.abs(y32) + (wo.shape[1] + 2) * 2.0 ** -22 * sabs
+        lo = mo.widen(mo.narrow((y32 - tol).astype(np.float32), BF16), BF16)
+        hi = mo.widen(mo.narrow((y32 + tol).astype(np.float32), BF16), BF16)
+        for name, y in (("pair", y_pair), ("tile", y_tile), ("general", y_gen)):
+            got = bits(y[r0:r0 + 512])
+            g = mo.widen(got, BF16)
+            assert np.all((g >= lo) & (g <= hi)), f"{name} kernel, rows {r0}..{r0 + 511}"
+            same[name] += int(np.sum(got == y_ref))
+    for name, cnt in same.items():
+        assert cnt > 0.999 * X.shape[0] * W.shape[0], name       # and nearly all are the oracle's own bits
     lin.close()
 
 

@@ -26,19 +26,24 @@ def _bits(t):
     return workloads.as_numpy_bits(t)
 
 
-def _padded(n, dtype, dev, pad=64):
-    """An output buffer with canary bytes after its n elements."""
+def _padded(n, dtype, dev, pad=64, lead=0):
+    """An output buffer of n elements that starts `lead` bytes into a (512-byte aligned) allocation,
+    with canary bytes before and after it."""
     esz = torch.empty(0, dtype=dtype).element_size()
-    raw = torch.full((n * esz + pad,), CANARY, dtype=torch.uint8, device=dev)
-    return raw, raw[: n * esz].view(dtype)
+    assert lead % esz == 0
+    raw = torch.full((lead + n * esz + pad,), CANARY, dtype=torch.uint8, device=dev)
+    return (raw, lead), raw[lead: lead + n * esz].view(dtype)
 
 
-def _canary_ok(raw, nbytes):
-    return bool((raw[nbytes:] == CANARY).all().item())
+def _canary_ok(raw_lead, nbytes):
+    raw, lead = raw_lead
+    return bool((raw[:lead] == CANARY).all().item()) and bool((raw[lead + nbytes:] == CANARY).all().item())
 
 
-def check_all_ops(bq, gcb, cb, x_cpu: torch.Tensor, block: int, ydtypes=None, offset_elems: int = 0):
-    """quantize, dequantize, roundtrip (with and without side outputs) against the oracle."""
+def check_all_ops(bq, gcb, cb, x_cpu: torch.Tensor, block: int, ydtypes=None, offset_elems: int = 0, out_lead=None):
+    """quantize, dequantize, roundtrip (with and without side outputs) against the oracle.
+    `out_lead` = bytes by which (y, codes, absmax) outputs are shifted off their allocation's base."""
+    ylead, clead, alead = out_lead or (0, 0, 0)
     dev = torch.device("cuda:0")
     x_cpu = x_cpu.contiguous().view(-1)
     n = x_cpu.numel()
@@ -50,8 +55,8 @@ def check_all_ops(bq, gcb, cb, x_cpu: torch.Tensor, block: int, ydtypes=None, of
         xd.copy_(x_cpu)
     else:
         xd = x_cpu.to(dev)
-    craw, codes = _padded(n, torch.uint8, dev)
-    araw, absmax = _padded(nb, torch.float32, dev)
+    craw, codes = _padded(n, torch.uint8, dev, lead=clead)
+    araw, absmax = _padded(nb, torch.float32, dev, lead=alead)
     bq.bq_quantize(xd, block, gcb, codes, absmax)
     ref_y, ref_c, ref_a = {}, None, None
     for ydt in (ydtypes or [xdt]):
@@ -63,13 +68,14 @@ def check_all_ops(bq, gcb, cb, x_cpu: torch.Tensor, block: int, ydtypes=None, of
     assert _canary_ok(craw, n) and _canary_ok(araw, nb * 4)
     for ydt, yref in ref_y.items():
         esz = torch.empty(0, dtype=ydt).element_size()
-        yraw, y = _padded(n, ydt, dev)
+        ylead_e = ylead - ylead % esz
+        yraw, y = _padded(n, ydt, dev, lead=ylead_e)
         bq.bq_dequantize(codes, absmax, block, gcb, ydt, y)
-        y2raw, y2 = _padded(n, ydt, dev)
+        y2raw, y2 = _padded(n, ydt, dev, lead=ylead_e)
         bq.bq_roundtrip(xd, block, gcb, y_out=y2)
-        y3raw, y3 = _padded(n, ydt, dev)
-        c3raw, c3 = _padded(n, torch.uint8, dev)
-        a3raw, a3 = _padded(nb, torch.float32, dev)
+        y3raw, y3 = _padded(n, ydt, dev, lead=ylead_e)
+        c3raw, c3 = _padded(n, torch.uint8, dev, lead=clead)
+        a3raw, a3 = _padded(nb, torch.float32, dev, lead=alead)
         bq.bq_roundtrip(xd, block, gcb, y_out=y3, codes_out=c3, absmax_out=a3)
         torch.cuda.synchronize()
         assert np.array_equal(_bits(y.cpu()), yref), f"dequantize {ydt}"
@@ -99,52 +105,56 @@ def test_config_decode70b(bq, gcb, cb):
     check_all_ops(bq, gcb, cb, workloads.make("decode70b"), 64)
 
 
-def _sampled_full_size(bq, gcb, cb, name, blocks, nsample=1536):
-    """Full-size run in the launch configuration the benchmark times; the oracle checks a
-    sample of whole blocks (first, last and random ones) bit for bit, and device-side
-    properties cover every element."""
+def _whole_tensor(bq, gcb, cb, name, blocks, chunk=1 << 26):
+    """Full-size run in the launch configuration the benchmark times.  EVERY code, every absmax and
+    every output element of quantize, dequantize, the fused roundtrip and the roundtrip with side
+    outputs is compared with the oracle, which runs on all host cores over contiguous ranges of
+    whole blocks, 64 Mi elements at a time so that host memory stays bounded.  Device-side
+    properties (textbook absmax, the error bound) are checked on every element as well."""
     dev = torch.device("cuda:0")
     x_cpu = workloads.make(name).view(-1)
     n = x_cpu.numel()
     xd = x_cpu.to(dev)
     xb = _bits(x_cpu)
     odt = ODT[x_cpu.dtype]
-    rng = np.random.default_rng(123)
     for block in blocks:
+        assert n % block == 0 and chunk % block == 0
         nb = n // block
         codes, absmax = bq.bq_quantize(xd, block, gcb)
         y = bq.bq_dequantize(codes, absmax, block, gcb, x_cpu.dtype)
-        y2 = bq.bq_roundtrip(xd, block, gcb)
+        y2 = bq.bq_roundtrip(xd, block, gcb).view(-1)
+        y3 = torch.empty_like(y)
+        c3, a3 = torch.empty_like(codes), torch.empty_like(absmax)
+        bq.bq_roundtrip(xd, block, gcb, y_out=y3, codes_out=c3, absmax_out=a3)
         torch.cuda.synchronize()
-        # every element: fused == separate; absmax == max|x| per block; error bound
-        assert torch.equal(y.view(torch.int16), y2.view(-1).view(torch.int16))
         ref_absmax = xd.view(nb, block).abs().amax(dim=1).float()
         assert torch.equal(absmax.view(torch.int32), ref_absmax.view(torch.int32))
-        step = 1 << 26
-        for s in range(0, n, step):
-            e = min(n, s + step)
-            a_el = absmax[s // block:(e + block - 1) // block].repeat_interleave(block)[: e - s]
+        for s in range(0, n, chunk):
+            e = min(n, s + chunk)
+            b0, b1 = s // block, e // block
+            a_el = absmax[b0:b1].repeat_interleave(block)
             err = (xd[s:e].float() - y[s:e].float()).abs()
             bound = a_el * (0.00703125 + 2.0 ** -22) + (y[s:e].float().abs() * 2.0 ** -8)    # code gap + bf16 rounding of y
             assert bool((err <= bound).all().item())
-        # sampled blocks, bit for bit
-        pick = np.unique(np.concatenate([[0, 1, nb - 2, nb - 1], rng.integers(0, nb, max(8, nsample * 64 // block))]))
-        idx = (pick[:, None] * block + np.arange(block)[None, :]).reshape(-1)
-        xs = np.ascontiguousarray(xb[idx])
-        ys, cs, as_ = oracle.roundtrip_sharded(xs, odt, block, cb, odt, THREADS)
-        tidx = torch.from_numpy(idx).to(dev)
-        assert np.array_equal(codes[tidx].cpu().numpy(), cs)
-        assert np.array_equal(absmax[torch.from_numpy(pick).to(dev)].cpu().numpy().view(np.uint32), as_.view(np.uint32))
-        assert np.array_equal(_bits(y[tidx].cpu()), ys)
-        del codes, absmax, y, y2
+            del a_el, err, bound
+            yr, cr, ar = oracle.roundtrip_sharded(xb[s:e], odt, block, cb, odt, THREADS)
+            where = f"{name} block {block} elements [{s}, {e})"
+            assert np.array_equal(codes[s:e].cpu().numpy(), cr), "quantize codes, " + where
+            assert np.array_equal(c3[s:e].cpu().numpy(), cr), "roundtrip side codes, " + where
+            assert np.array_equal(absmax[b0:b1].cpu().numpy().view(np.uint32), ar.view(np.uint32)), "absmax, " + where
+            assert np.array_equal(a3[b0:b1].cpu().numpy().view(np.uint32), ar.view(np.uint32)), "side absmax, " + where
+            assert np.array_equal(_bits(y[s:e].cpu()), yr), "dequantize, " + where
+            assert np.array_equal(_bits(y2[s:e].cpu()), yr), "roundtrip, " + where
+            assert np.array_equal(_bits(y3[s:e].cpu()), yr), "roundtrip with side outputs, " + where
+        del codes, absmax, y, y2, y3, c3, a3
 
 
 def test_config_moe_prefill_full_size(bq, gcb, cb):
-    _sampled_full_size(bq, gcb, cb, "moe_prefill", [2048])
+    _whole_tensor(bq, gcb, cb, "moe_prefill", [2048])
 
 
 def test_config_sweep1g_full_size(bq, gcb, cb):
-    _sampled_full_size(bq, gcb, cb, "sweep1g", [64, 256, 1024, 4096])
+    _whole_tensor(bq, gcb, cb, "sweep1g", [64, 256, 1024, 4096])
 
 
 # ------------------------------------------------------------------------------- shapes, tails, alignment
@@ -177,6 +187,23 @@ def test_unaligned_input_pointer(bq, gcb, cb, dtype, offset):
     g = torch.Generator().manual_seed(5)
     x = torch.randn(64 * 300 + 11, generator=g).to(dtype)
     check_all_ops(bq, gcb, cb, x, 64, offset_elems=offset)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("lead", [(16, 16, 16), (16, 0, 0), (0, 8, 4), (2, 1, 4), (4, 3, 8), (48, 24, 12), (32, 16, 4)])
+@pytest.mark.parametrize("n", [64 * 300 + 11, (1 << 23) + 64 * 40 + 5])
+def test_unaligned_output_pointers(bq, gcb, cb, dtype, lead, n):
+    if n > 100_000 and lead not in ((16, 16, 16), (2, 1, 4), (32, 16, 4)):
+        pytest.skip("the large size runs three of the offsets")
+    """Outputs that start off their allocation's base: y on a 16-byte but not 32-byte boundary (the wide
+    stores of the dequantize kernel must not be used), on an element boundary only, codes on odd bytes,
+    absmax on a 4-byte boundary; below and above the size where the persistent kernels take over."""
+    g = torch.Generator().manual_seed(sum(lead) + n % 97)
+    x = torch.randn(n, generator=g).to(dtype)
+    check_all_ops(bq, gcb, cb, x, 64, out_lead=lead)
+    if n < 100_000:
+        check_all_ops(bq, gcb, cb, x, 4096, out_lead=lead)
+        check_all_ops(bq, gcb, cb, x, 100, out_lead=lead)
 
 
 def test_mixed_output_types(bq, gcb, cb):
@@ -314,7 +341,8 @@ def test_random_shapes_types_and_offsets(bq, gcb, cb):
         if rng.random() < 0.3:
             x[:: max(1, n // 7)] = 0.0
         offset = int(rng.choice([0, 0, 0, 1, 2, 8]))
-        check_all_ops(bq, gcb, cb, x, block, offset_elems=offset)
+        lead = (int(rng.choice([0, 0, 4, 16, 32, 48])), int(rng.choice([0, 0, 1, 8, 16])), int(rng.choice([0, 0, 4, 16])))
+        check_all_ops(bq, gcb, cb, x, block, offset_elems=offset, out_lead=lead)
 
 
 @pytest.mark.parametrize("dtype,sig", [(torch.bfloat16, 8), (torch.float16, 11)])

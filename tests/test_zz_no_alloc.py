@@ -59,3 +59,25 @@ def test_static_scratch_rejects_what_does_not_fit(bq):
     _, fits = lin.workspace_layout(64)
     assert fits <= bq.mmd.STATIC_SCRATCH_BYTES
     lin.close()
+
+
+def test_static_entry_answers_bad_arguments_like_the_workspace_entry(bq):
+    """Bad element type, bad path and zero rows: the two entry points return the same status, before any launch,
+    whether or not the row count would fit the built-in array."""
+    from paper_2407_19775_b200.mmd import _lib
+    X, W, idx = workloads.make_linear("mmd_decode70b", out_features=64)
+    lin = bq.DecomposedLinear(W.cuda(), idx)
+    L = _lib()
+    x = X.cuda()
+    y = torch.empty((x.shape[0], lin.N), dtype=torch.float32, device="cuda")
+    ws = lin.workspace(x.shape[0])
+    stream = torch.cuda.current_stream().cuda_stream
+    BF16, F32 = 2, 0                                                             # the weights are fp16: bf16 output is refused
+    for M in (0, x.shape[0], 600):                                               # 600 rows do not fit the built-in array
+        for ydt, path in ((BF16, 0), (F32, 99), (F32, -1), (BF16, 99)):
+            a = L.mmd_linear(lin.handle, x.data_ptr(), M, y.data_ptr(), ydt, ws.data_ptr(), ws.numel(), path, stream)
+            b = L.mmd_linear_static(lin.handle, x.data_ptr(), M, y.data_ptr(), ydt, path, stream)
+            assert a == b and a != 0, (M, ydt, path, a, b)
+    assert L.mmd_linear_static(lin.handle, x.data_ptr(), 0, y.data_ptr(), F32, 0, stream) == 0
+    assert L.mmd_linear_static(None, x.data_ptr(), 4, y.data_ptr(), F32, 0, stream) == L.mmd_linear(None, x.data_ptr(), 4, y.data_ptr(), F32, ws.data_ptr(), ws.numel(), 0, stream)
+    lin.close()
