@@ -46,6 +46,24 @@ def algorithmic_bytes(op: str, n: int, block: int, s_in: int = 2, s_out: int = 2
     return n * s_in + n * s_out
 
 
+def progress(section: str, payload) -> None:
+    """Finished sections go to stderr as they complete (one JSON object per line), so that a run that
+    is killed keeps what it had measured; stdout carries only the final line."""
+    sys.stderr.write(json.dumps({"section": section, "result": payload}) + "\n")
+    sys.stderr.flush()
+
+
+def sha256_of(t: torch.Tensor) -> str:
+    """SHA-256 of a host tensor's bytes (the seeded input as the kernels and the oracle both see it)."""
+    import hashlib
+    flat = t.contiguous().view(-1).view(torch.uint8).numpy()
+    h = hashlib.sha256()
+    step = 1 << 26
+    for s0 in range(0, flat.size, step):
+        h.update(flat[s0:s0 + step].data)
+    return h.hexdigest()
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -155,16 +173,25 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
 
+    global WORKLOAD, BLOCKS
+    WORKLOAD = args.config
     w = workloads.WORKLOADS[WORKLOAD]
+    BLOCKS = tuple(w.blocks)
     x_host = workloads.make(WORKLOAD).view(-1)
     n = x_host.numel()
+    es = x_host.element_size()
     x_pin = x_host.pin_memory()
     del x_host
+    input_sha = sha256_of(x_pin) if rank == 0 else None
     cb = bq.Codebook(device=dev)
     x = x_pin.to(dev, non_blocking=True)
     codes = torch.empty(n, dtype=torch.uint8, device=dev)
-    absmax = {b: torch.empty(n // b, dtype=torch.float32, device=dev) for b in BLOCKS}
+    absmax = {b: torch.empty((n + b - 1) // b, dtype=torch.float32, device=dev) for b in BLOCKS}
     y = torch.empty(n, dtype=w.dtype, device=dev)
+    # A tensor that fits in L2 (126 MB) would be timed L2-resident: a 256 MiB buffer is written before every
+    # launch, outside the per-launch events, and `value` is then taken from the launches' own event times.
+    fits_l2 = 2 * n * es < (120 << 20)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if fits_l2 else None
     torch.cuda.synchronize()
 
     def launch(op, b):
@@ -178,6 +205,8 @@ def run_ours(args):
     def step(events=None):
         for b in BLOCKS:
             for op in OPS:
+                if flush is not None:
+                    flush.fill_(1)
                 if events is not None:
                     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                     e0.record()
@@ -209,21 +238,23 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else None
     max_s = max_over_ranks(local_s, world, dev)
 
-    bytes_per_step = n * 2 * len(BLOCKS) * len(OPS)
-    value = whole_job_value(bytes_per_step * args.steps, world, max_s) / 1e9
-
+    bytes_per_step = n * es * len(BLOCKS) * len(OPS)
     # per-kernel durations from the events recorded inside the timed region
     peak, peak_kind = measured_peak()
     per = {}
     for op, b, e0, e1 in events:
         per.setdefault((op, b), []).append(e0.elapsed_time(e1))
+    if flush is not None:                            # the flush writes are not the path's work: count the launches' own time
+        local_s = sum(sum(v) for v in per.values()) / 1e3
+        max_s = max_over_ranks(local_s, world, dev)
+    value = whole_job_value(bytes_per_step * args.steps, world, max_s) / 1e9
     kernels = {}
     for (op, b), ms in per.items():
         avg = float(np.mean(ms))
-        ab = algorithmic_bytes(op, n, b)
+        ab = algorithmic_bytes(op, n, b, es, es)
         kernels[f"{op}_b{b}"] = {
             "ms": round(avg, 4), "ms_min": round(float(np.min(ms)), 4), "algorithmic_bytes": int(ab), "traffic": TRAFFIC_BYTES.get(f"{op}_b{b}"),
-            "input_gbs": round(n * (1 if op == "dequantize" else 2) / avg / 1e6, 1),
+            "input_gbs": round(n * (1 if op == "dequantize" else es) / avg / 1e6, 1),
             "total_gbs": round(ab / avg / 1e6, 1),
             "frac_of_measured": round(ab / avg / 1e6 / peak, 4),
             "frac_of_nominal_8tbs": round(ab / avg / 1e6 / NOMINAL_HBM_GBS, 4),
@@ -231,13 +262,19 @@ def run_ours(args):
     totals = {k: v["ms"] for k, v in kernels.items()}
     dominant = max(totals, key=totals.get)
     dop, db = dominant.split("_b")
-    dab = algorithmic_bytes(dop, n, int(db))
+    dab = algorithmic_bytes(dop, n, int(db), es, es)
     achieved = dab / kernels[dominant]["ms"] / 1e6
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": round(achieved, 1), "peak": peak, "peak_kind": peak_kind,
-                "unit": "GB/s", "frac": round(achieved / peak, 4), "traffic": TRAFFIC_BYTES.get(dominant)}
+                "unit": "GB/s", "frac": round(achieved / peak, 4), "traffic": TRAFFIC_BYTES.get(dominant) if WORKLOAD == "sweep1g" else None}
+    if rank == 0:
+        progress("kernels", {"value_gbs": round(value, 1), "ms_per_step": round(max_s * 1e3 / args.steps, 4), "roofline": roofline,
+                             "kernels": kernels, "input_sha256": input_sha})
 
     # end to end: host buffers in, host buffers out, copies inside the timed region
     e2e = run_e2e(bq, cb, x_pin, dev, w.dtype, n, args, world)
+    if rank == 0:
+        progress("e2e", e2e)
+    full = WORKLOAD == "sweep1g"                     # the variants and the other configurations ride on the headline run only
 
     # compression and reconstruction error (block 4096 outputs are still resident: recompute per block cheaply)
     quality = {}
@@ -249,12 +286,14 @@ def run_ours(args):
             xs, ys = x[s:s + (1 << 27)].float(), y[s:s + (1 << 27)].float()
             num += ((xs - ys) ** 2).sum(dtype=torch.float64)
             den += (xs ** 2).sum(dtype=torch.float64)
-        quality[f"b{b}"] = {"compression_ratio": round(2 * b / (b + 4), 3), "rel_rms_error": round(float((num / den).sqrt().item()), 5)}
+        quality[f"b{b}"] = {"compression_ratio": round(es * b / (b + 4), 3), "rel_rms_error": round(float((num / den).sqrt().item()), 5)}
+    if rank == 0:
+        progress("quality", quality)
 
     # the 4-bit variant of the same path (16-entry codebook, two codes per byte) on the same tensor
     cb4 = bq.Codebook4()
     bq4 = {}
-    for b, s16 in ((64, False), (1024, False), (64, True)):       # s16: the block scale stored as a bf16 (2 bytes instead of 4)
+    for b, s16 in (((64, False), (1024, False), (64, True)) if full else ()):       # s16: the block scale stored as a bf16 (2 bytes instead of 4)
         packed = codes[: n // 2]
         scale16 = absmax[b].view(torch.bfloat16)[: n // b]
         times = {}
@@ -289,6 +328,15 @@ def run_ours(args):
             "compression_ratio": round(2.0 * n / (n / 2 + scale_bytes * (n // b)), 3),
             "rel_rms_error": round(float((num / den).sqrt().item()), 5), "gpu_launches": 26}
 
+    if rank == 0 and full:
+        progress("bq4", bq4)
+    cpu = cpu_baseline(x_pin, w, rank) if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
+    if cpu is not None:
+        progress("cpu_baseline", cpu)
+    if not full:
+        return finish(rank, world, args, value, max_s, n, w, e2e, events, clocks, roofline, kernels, quality, cpu, input_sha,
+                      None, None, None, None)
+
     # block-size selection on the same tensor: the roundtrip and the error sums of four candidates in one call
     tune_blocks = [64, 256, 1024, 4096]
     tune_ws = torch.empty(bq.tune.workspace_bytes(w.dtype, n), dtype=torch.uint8, device=dev)
@@ -309,23 +357,45 @@ def run_ours(args):
             "rel_rms_error": [round(float(v), 5) for v in np.sqrt(sums_host[:-1] / sums_host[-1])],
             "picked_for_rel_rms_0.01": bq.tune.pick_block(tune_blocks, sums_host, 0.01), "gpu_launches": 7 * 3 * len(tune_blocks)}
     del tune_ws
+    if rank == 0:
+        progress("autotune", tune)
 
-    cpu = cpu_baseline(x_pin, rank) if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
     del x, y, codes, absmax
     torch.cuda.empty_cache()
     small = run_small(bq, dev) if rank == 0 else None
-    mmd = run_mmd(bq, dev, args) if (rank == 0 and not args.no_mmd) else None
-
     if rank == 0:
+        progress("small_configs", small)
+    mmd = run_mmd(bq, dev, args) if (rank == 0 and not args.no_mmd) else None
+    if mmd is not None:
+        progress("mmd", mmd)
+    transport = run_transport(bq, dev, args) if (rank == 0 and not args.no_transport) else None
+    if transport is not None:
+        progress("transport", transport)
+    mtpp = run_mtpp(bq, dev, args) if (rank == 0 and not args.no_mtpp) else None
+    if mtpp is not None:
+        progress("mtpp", mtpp)
+    return finish(rank, world, args, value, max_s, n, w, e2e, events, clocks, roofline, kernels, quality, cpu, input_sha,
+                  bq4, tune, small, mmd, transport, mtpp)
+
+
+def finish(rank, world, args, value, max_s, n, w, e2e, events, clocks, roofline, kernels, quality, cpu, input_sha, bq4, tune, small, mmd,
+           transport=None, mtpp=None):
+    if rank == 0:
+        blocks = "/".join(str(b) for b in BLOCKS)
+        es = torch.empty(0, dtype=w.dtype).element_size()
+        fits_l2 = 2 * n * es < (120 << 20)
         line = {
             "metric": METRIC, "value": round(value, 1), "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": round(max_s * 1e3 / args.steps, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
-            "config": {"workload": "sweep1g: [16,4096,8192] bf16, Laplace(0,0.5), 8 outlier channels x60, seed 4; blocks 64/256/1024/4096; "
-                                   "quantize+dequantize+roundtrip per block", "elements": n, "l2": "input (1 GiB) larger than L2, no flush needed",
-                       "parallelism": f"replicated x{world}, no collective"},
+            "config": {"workload": f"{WORKLOAD}: {list(w.shape)} {str(w.dtype)[6:]}, {w.recipe}, seed {w.seed}; blocks {blocks}; "
+                                   "quantize+dequantize+roundtrip per block", "elements": n,
+                       "l2": ("tensor fits in L2: a 256 MiB buffer is written before every launch and the value counts the launches' own "
+                              "event times" if fits_l2 else f"input ({n * es >> 20} MiB) larger than L2, no flush needed"),
+                       "parallelism": f"replicated x{world}, no collective", "input_sha256": input_sha},
             "e2e": e2e, "gpu_launches": len(events), "clocks": clocks, "roofline": roofline, "kernels": kernels,
             "quality": quality, "cpu_baseline": cpu, "bq4": bq4, "autotune": tune, "small_configs": small, "mmd": mmd,
+            "transport": transport, "mtpp": mtpp,
             "paper_context": "the paper reports no throughput for this path; it states only that hidden-state quantization halves the bandwidth",
         }
         print(json.dumps(line))
@@ -399,6 +469,124 @@ def run_small(bq, dev):
         entry["gpu_launches"] = launches
         out[name] = entry
         del x, y, codes, absmax
+    return out
+
+
+# ------------------------------------------------------------------------------------------ slicing topological orders
+
+def run_mtpp(bq, dev, args, name="mtpp_unet"):
+    """The paper's other fully stated algorithm (its Algorithm 1), batched over a population of orders: priority
+    vectors are decoded into topological orders and every order is cut into at most k blocks of least bottleneck
+    cost.  One CTA per order; integer arithmetic; no HBM traffic to speak of (the graph and a row of n node
+    numbers per order), so the figure is orders per second and the time per order, beside the oracle's time
+    on a sample of orders.  Its results are compared with the oracle by tests/test_gpu_mtpp.py."""
+    import oracle.mtpp_oracle as mo
+    w = workloads.GRAPH_WORKLOADS[name]
+    n, edges, work, sizeparam, sizeout = workloads.make_graph(name)
+    dg = bq.mtpp.SliceGraph(n, edges, work, sizeparam, sizeout, device=dev)
+    keys_host = workloads.make_keys(name)
+    keys = keys_host.to(dev)
+    P = keys.shape[0]
+    orders = torch.empty((P, n), dtype=torch.int32, device=dev)
+    out = dg.slice_orders(dg.decode_orders(keys, orders), w.k, w.B, w.M)
+    torch.cuda.synchronize()
+    reps = max(3, min(args.steps, 20))
+
+    def timed(fn):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    ms_decode = timed(lambda: dg.decode_orders(keys, orders))
+    ms_slice = timed(lambda: dg.slice_orders(orders, w.k, w.B, w.M, out))
+    cost = out[0].cpu().numpy()
+    # the oracle on two orders of the same population (decode + slice), one thread
+    g = mo.Graph(n, [tuple(e) for e in edges.tolist()], work.tolist(), sizeparam.tolist(), sizeout.tolist())
+    t = time.perf_counter()
+    sample = 2
+    for p in range(sample):
+        mo.slice_order(g, mo.decode_order(g, keys_host[p].tolist()), w.k, w.B, w.M)
+    cpu_s = (time.perf_counter() - t) / sample
+    dg.close()
+    return {"workload": f"{name}: {w.recipe}; n = {n} nodes, {edges.shape[0]} edges, at most k = {w.k} blocks, population {P}",
+            "decode_ms": round(ms_decode, 4), "slice_ms": round(ms_slice, 4), "orders_per_s": round(P / (ms_decode + ms_slice) * 1e3, 1),
+            "us_per_order": round((ms_decode + ms_slice) * 1e3 / P, 3), "best_bottleneck": int(cost.min()), "worst_bottleneck": int(cost.max()),
+            "cpu_baseline": {"value": round(1.0 / cpu_s, 3), "unit": "orders/s", "cores": 1, "kind": "oracle", "sample": f"{sample} orders of the population, decode + slice"},
+            "gpu_launches": 2 * (reps + 2) + 2}
+
+
+# ------------------------------------------------------------------------------------------ the boundary transport (loop-back)
+
+NVLINK_PEER_GBS = 770.0          # measured peer copy rate per direction on this pool's machines (context for the projection only)
+
+
+def run_transport(bq, dev, args, block=256):
+    """The hand-off across a shard boundary on ONE device (sender and receiver both here: loop-back):
+    the sending side's quantize kernel fills a mailbox piece by piece, the receiving side's dequantize kernel
+    drains it on a second stream.  Timed against handing over the raw 16-bit tensor the same way (a device
+    copy per piece) and against the fused roundtrip kernel.  No link is crossed here, so the figures are the
+    cost of the pipeline itself; what NVLink would add is printed as a projection from the bytes, and labelled so."""
+    from paper_2407_19775_b200 import transport
+    x = workloads.make(WORKLOAD).view(-1).to(dev)
+    n = x.numel()
+    es = x.element_size()
+    y = torch.empty_like(x)
+    cb = bq.Codebook(device=dev)
+    chunk, slots = 1 << 25, 3
+    rx = transport.Receiver(cb, chunk, min_block=block, slots=slots)
+    s_send, s_recv = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    reps = max(3, min(args.steps, 20))
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s_send.wait_stream(torch.cuda.current_stream(dev))
+        s_recv.wait_stream(torch.cuda.current_stream(dev))
+        t0.record(s_send)
+        s_recv.wait_event(t0)
+        for _ in range(reps):
+            fn()
+        s_recv.wait_stream(s_send)
+        t1.record(s_recv)
+        torch.cuda.synchronize()
+        return t0.elapsed_time(t1) / reps
+
+    out = {"workload": f"{WORKLOAD}, block {block}", "link": "loop-back on one device (sender and receiver are the same GPU); NVLink unmeasured on hardware",
+           "pieces": len(transport.plan(n, block, chunk, slots)), "chunk_elems": chunk, "slots": slots,
+           "payload_bytes": transport.payload_bytes(n, block), "raw_bytes": n * es,
+           "bytes_ratio": round(n * es / transport.payload_bytes(n, block), 3)}
+    for name, mode in (("store", transport.STORE), ("copy", transport.COPY)):
+        tx = transport.Sender(cb, rx.export(), mode)
+        ms = timed(lambda: transport.transfer(tx, rx, x, block, y, s_send, s_recv))
+        out[name] = {"ms": round(ms, 4), "activation_gbs": round(n * es / ms / 1e6, 1)}
+        tx.close()
+    ref = bq.bq_roundtrip(x, block, cb)
+    torch.cuda.synchronize()
+    out["bit_identical_to_roundtrip"] = bool(torch.equal(ref.view(torch.int16), y.view(torch.int16)))
+    pieces = [(lo, min(n, lo + chunk)) for lo in range(0, n, chunk)]
+
+    def raw():
+        for lo, hi in pieces:                                   # the uncompressed hand-off: one device copy per piece, then nothing to expand
+            with torch.cuda.stream(s_send):
+                y[lo:hi].copy_(x[lo:hi], non_blocking=True)
+
+    out["raw_copy"] = {"ms": round(timed(raw), 4)}
+    with torch.cuda.stream(s_send):
+        out["fused_roundtrip"] = {"ms": round(timed(lambda: bq.bq_roundtrip(x, block, cb, y_out=y)), 4)}
+    out["nvlink_projection"] = {"assumed_gbs": NVLINK_PEER_GBS, "payload_ms": round(out["payload_bytes"] / NVLINK_PEER_GBS / 1e6, 4),
+                                "raw_ms": round(n * es / NVLINK_PEER_GBS / 1e6, 4),
+                                "note": "bytes over an assumed link rate, not a measurement: the stores of the quantize kernel would be link-bound"}
+    out["gpu_launches"] = 2 * (reps + 3) * (2 * out["pieces"]) + (reps + 3)
+    rx.close()
     return out
 
 
@@ -553,9 +741,14 @@ def run_mmd(bq, dev, args):
         "ms_per_call": round(ms_call, 4), "tops": round(ops / ms_call / 1e9, 1), "kernel_status": status,
         "rowquant": {"ms": round(ms_row, 4), "algorithmic_bytes": int(row_bytes), "gbs": round(row_bytes / ms_row / 1e6, 1),
                      "frac_of_measured_hbm": round(row_bytes / ms_row / 1e6 / hbm, 4)},
-        "roofline": {"bound": "tensor", "kernel": "gemm_tc2 (persistent CTA pairs, int8 tcgen05 cta_group::2)", "achieved": round(ops / ms_prod / 1e9, 1),
-                     "peak": round(peak, 1), "peak_kind": f"{kind} bf16 x {NOMINAL_INT8_OVER_BF16} (nominal int8 / bf16 ratio)", "unit": "TOP/s",
-                     "frac": round(ops / ms_prod / 1e9 / peak, 4), "ms": round(ms_prod, 4), "traffic": MMD_TRAFFIC_BYTES},
+        # the whole call as timed (row kernel + product kernel) over the tensor peak; the product kernel alone is an estimate
+        # (call minus row kernel: an upper estimate, because part of the row kernel hides under the product kernel's set-up)
+        "roofline": {"bound": "tensor", "kernel": "whole mmd_linear call: rowquant + gemm_tc2 (persistent CTA pairs, int8 tcgen05 cta_group::2)",
+                     "achieved": round(ops / ms_call / 1e9, 1), "peak": round(peak, 1),
+                     "peak_kind": f"{kind} bf16 x {NOMINAL_INT8_OVER_BF16} (nominal int8 / bf16 ratio)", "unit": "TOP/s",
+                     "frac": round(ops / ms_call / 1e9 / peak, 4), "ms": round(ms_call, 4), "traffic": MMD_TRAFFIC_BYTES,
+                     "product_kernel_estimate": {"ms": round(ms_prod, 4), "achieved": round(ops / ms_prod / 1e9, 1),
+                                                 "frac": round(ops / ms_prod / 1e9 / peak, 4), "how": "call minus row kernel (upper estimate)"}},
         "e2e": {"ms_per_call": round(ms_e2e, 4), "tops": round(ops / ms_e2e / 1e9, 1), "h2d_bytes_per_call": int(M * K * 2),
                 "d2h_bytes_per_call": int(M * N * 2)},
         "quality": {"weight_bytes_ratio": round(2.0 * N * K / (N * K + 4 * N + 2 * N * sd.shape[1]), 3),
@@ -575,23 +768,26 @@ DECODE_LAYER_COPIES = 4
 # dirty lines that are still in L2 when the kernel ends, a size-independent residue measured
 # in the same capture.  Set an entry to None when its kernel changes until it is re-measured.
 TRAFFIC_BYTES = {
-    "quantize_b64": 1599487744, "quantize_b256": 1578846464, "quantize_b1024": 1573560576, "quantize_b4096": 1572869632,
-    "dequantize_b64": 1586586368, "dequantize_b256": 1560828416, "dequantize_b1024": 1555288832, "dequantize_b4096": 1553292032,
-    "roundtrip_b64": 2095262976, "roundtrip_b256": 2095527936, "roundtrip_b1024": 2095371776, "roundtrip_b4096": 2095418624,
+    "quantize_b64": None, "quantize_b256": None, "quantize_b1024": None, "quantize_b4096": None,
+    "dequantize_b64": None, "dequantize_b256": None, "dequantize_b1024": None, "dequantize_b4096": None,
+    "roundtrip_b64": None, "roundtrip_b256": None, "roundtrip_b1024": None, "roundtrip_b4096": None,
 }
 
 
 def run_e2e(bq, cb, x_pin, dev, dtype, n, args, world):
-    """One end-to-end step per block size through the host-to-host API, everything starting
-    and ending in pinned host memory: sender (x up, quantize, codes+absmax down), receiver
-    (codes+absmax up, dequantize, y down) and the fused loop (x up, roundtrip, y down).  The
-    three legs of each call overlap chunk by chunk on three streams."""
+    """One end-to-end step per block size through the library's host-buffer calls (bq_quantize_host,
+    bq_dequantize_host, bq_roundtrip_host), everything starting and ending in pinned host memory: sender
+    (x up, quantize, codes+absmax down), receiver (codes+absmax up, dequantize, y down) and the fused loop
+    (x up, roundtrip, y down).  The three legs of each call overlap piece by piece on the pipe's three streams;
+    the timed region ends when the last byte is back in host memory."""
     from paper_2407_19775_b200.pipeline import HostBoundary
     steps = max(1, min(args.steps, args.e2e_steps))
-    hb = HostBoundary(cb, dtype, chunk=1 << 25, slots=3, max_blocks_per_chunk=(1 << 25) // min(BLOCKS))
+    es = x_pin.element_size()
+    chunk = min(1 << 25, max(max(BLOCKS), (n // max(BLOCKS)) * max(BLOCKS)))
+    hb = HostBoundary(cb, dtype, chunk=chunk, slots=3, min_block=min(BLOCKS))
     c_pin = torch.empty(n, dtype=torch.uint8).pin_memory()
     y_pin = torch.empty(n, dtype=dtype).pin_memory()
-    a_pin = {b: torch.empty(n // b, dtype=torch.float32).pin_memory() for b in BLOCKS}
+    a_pin = {b: torch.empty((n + b - 1) // b, dtype=torch.float32).pin_memory() for b in BLOCKS}
     h2d = d2h = 0
 
     def one_step(count=False):
@@ -601,47 +797,53 @@ def run_e2e(bq, cb, x_pin, dev, dtype, n, args, world):
             hb.dequantize(c_pin, a_pin[b], b, y_pin)
             hb.roundtrip(x_pin, b, y_pin)
             if count:
-                h2d += 2 * n * 2 + n + 4 * (n // b)
-                d2h += n + 4 * (n // b) + 2 * n * 2
+                nb = (n + b - 1) // b
+                h2d += 2 * n * es + n + 4 * nb
+                d2h += n + 4 * nb + 2 * n * es
 
     one_step()
+    hb.wait()
     torch.cuda.synchronize()
     barrier(world, dev)
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record()
     for i in range(steps):
         one_step(count=(i == 0))
+    hb.wait_on_current_stream()
     t1.record()
     torch.cuda.synchronize()
     barrier(world, dev)
     sec = max_over_ranks(t0.elapsed_time(t1) / 1e3, world, dev)
-    bytes_per_step = n * 2 * len(BLOCKS) * len(OPS)
+    hb.close()
+    bytes_per_step = n * es * len(BLOCKS) * len(OPS)
     return {"value": round(whole_job_value(bytes_per_step * steps, world, sec) / 1e9, 2), "unit": "GB/s", "steps": steps,
-            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "api": "HostBoundary (32 Mi-element chunks, 3 streams)"}
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "api": f"bq_quantize_host / bq_dequantize_host / bq_roundtrip_host (C ABI, host pointers; {chunk >> 20} Mi-element pieces, 3 slots, 3 streams)"}
 
 
 # ------------------------------------------------------------------------------------------ the CPU oracle arm
 
-def oracle_step(oracle, xb, cb, threads):
+def oracle_step(oracle, xb, odt, cb, threads):
     for b in BLOCKS:
-        c, a = oracle.quantize_sharded(xb, oracle.BF16, b, cb, threads)
-        oracle.dequantize_sharded(c, a, b, cb, oracle.BF16, threads)
-        oracle.roundtrip_sharded(xb, oracle.BF16, b, cb, oracle.BF16, threads)
+        c, a = oracle.quantize_sharded(xb, odt, b, cb, threads)
+        oracle.dequantize_sharded(c, a, b, cb, odt, threads)
+        oracle.roundtrip_sharded(xb, odt, b, cb, odt, threads)
 
 
-def cpu_baseline(x_pin, rank, rows=512):
-    """The CPU oracle, as it stands, on a bounded sample (the first `rows` rows) of the same
-    tensor, one thread."""
+def cpu_baseline(x_pin, w, rank, elems=1 << 24):
+    """The CPU oracle, as it stands, on a bounded sample (the first 16 Mi elements, or the whole tensor when it
+    is smaller) of the same tensor, one thread, every block size of the workload x 3 operations."""
     import oracle
-    xb = workloads.as_numpy_bits(x_pin[: rows * 8192])
+    odt = {torch.float32: oracle.F32, torch.float16: oracle.F16, torch.bfloat16: oracle.BF16}[w.dtype]
+    xb = workloads.as_numpy_bits(x_pin[:elems]) if w.dtype != torch.float32 else x_pin[:elems].numpy()
     cb = oracle.make_codebook()
-    oracle_step(oracle, xb[:8192 * 8], cb, 1)        # touch the library once
+    oracle_step(oracle, xb[:8192 * 8], odt, cb, 1)        # touch the library once
     t = time.perf_counter()
-    oracle_step(oracle, xb, cb, 1)
+    oracle_step(oracle, xb, odt, cb, 1)
     sec = time.perf_counter() - t
-    return {"value": round(xb.size * 2 * len(BLOCKS) * len(OPS) / sec / 1e9, 5), "unit": "GB/s", "cores": 1, "kind": "oracle",
+    return {"value": round(xb.size * x_pin.element_size() * len(BLOCKS) * len(OPS) / sec / 1e9, 5), "unit": "GB/s", "cores": 1, "kind": "oracle",
             "host_cores_total": os.cpu_count(), "seconds": round(sec, 2),
-            "sample": f"first {rows} rows ({xb.size} elements) of sweep1g, all 4 block sizes x 3 ops, single thread"}
+            "sample": f"first {xb.size} elements of {w.name}, {len(BLOCKS)} block size(s) x 3 ops, single thread"}
 
 
 def run_reference(args):
@@ -658,10 +860,10 @@ def run_reference(args):
     xb = workloads.as_numpy_bits(x)
     cb = oracle.make_codebook()
     for _ in range(args.warmup):
-        oracle_step(oracle, xb, cb, threads)
+        oracle_step(oracle, xb, oracle.BF16, cb, threads)
     t = time.perf_counter()
     for _ in range(args.steps):
-        oracle_step(oracle, xb, cb, threads)
+        oracle_step(oracle, xb, oracle.BF16, cb, threads)
     sec = time.perf_counter() - t
     value = xb.size * 2 * len(BLOCKS) * len(OPS) * args.steps / sec / 1e9
     sample = f"first {rows} rows ({xb.size} elements) of sweep1g per step, all 4 block sizes x 3 ops, {threads} threads over whole blocks"
@@ -687,6 +889,11 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-mmd", action="store_true", help="skip the decomposed-linear-layer section")
+    ap.add_argument("--no-transport", action="store_true", help="skip the loop-back boundary-transport section")
+    ap.add_argument("--no-mtpp", action="store_true", help="skip the order-slicing section")
+    ap.add_argument("--config", default="sweep1g", choices=sorted(workloads.WORKLOADS),
+                    help="the workload the step runs on (default: the largest, which the metric is quoted on); the 4-bit, block-selection, "
+                         "small-configuration, linear-layer and transport sections ride on the default only")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

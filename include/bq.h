@@ -103,10 +103,88 @@ int bq_dequantize(const uint8_t* codes, const float* absmax, size_t n, int block
 int bq_roundtrip(const void* x, bq_dtype xdt, size_t n, int block, const bq_codebook* cb,
                  void* y_out, bq_dtype ydt, uint8_t* codes_out, float* absmax_out, void* cuda_stream);
 
+/* ------------------------------------------------------------------------------------------
+ * Host-buffer calls.  The paper's receiving node gets the compressed hidden state from the
+ * network, i.e. in host memory, and the sending node hands it to the network from host memory
+ * (section "Compression techniques", item 1: the hidden states "exchanged between nodes").
+ * These calls take HOST pointers and stream the tensor through the GPU in chunks: upload of
+ * chunk i+1, the kernel on chunk i and the download of chunk i-1 overlap on three streams of
+ * the pipe's own (PCIe is full duplex, the copy engines run beside the SMs).  Every step of
+ * the method still runs in the kernels of bq_quantize / bq_dequantize / bq_roundtrip.
+ *
+ * A pipe owns its device staging buffers, streams and events; all of them are made by
+ * bq_host_pipe_create and nothing is allocated per call.  One cudaMemcpyAsync per chunk and
+ * direction.  Host buffers should be page-locked (cudaHostAlloc / cudaHostRegister): pageable
+ * memory still gives the right bytes, but the copies then block the calling thread and do
+ * not overlap.
+ */
+typedef struct bq_host_pipe bq_host_pipe;
+
+/*
+ * bq_host_pipe_create -- on the codebook's device (which must be current).
+ *   chunk_elems: elements per piece (> 0); a call uses the largest multiple of its block size that
+ *                fits, so block <= chunk_elems is required of every call.
+ *   min_block:   the smallest block size calls will use (sizes the absmax staging: chunk_elems /
+ *                min_block + 1 floats per slot); calls with a smaller block get BQ_ERR_BLOCK.
+ *   widest:      the widest element type calls will use (BQ_F32, or BQ_F16 / BQ_BF16 for 2-byte
+ *                staging); calls with a wider type get BQ_ERR_DTYPE.
+ *   slots:       pieces in flight, 2..8 (3 keeps upload, kernel and download of different pieces busy).
+ * Device memory held: slots * chunk_elems * (2 * element bytes + 1) + the absmax staging.
+ * The codebook must outlive the pipe.
+ */
+int bq_host_pipe_create(const bq_codebook* cb, size_t chunk_elems, int min_block, bq_dtype widest, int slots,
+                        bq_host_pipe** out);
+
+/* Waits for the pipe's work, then frees its streams, events and device memory.  NULL is allowed. */
+int bq_host_pipe_destroy(bq_host_pipe* pipe);
+
+/*
+ * The three data calls, host to host.  Same results, bit for bit, as the device-pointer calls
+ * on the whole tensor (pieces are whole numbers of blocks, and blocks are independent).
+ *   x_host, y_host: n elements; codes_host: n bytes; absmax_host: ceil(n / block) floats.
+ * Each call ENQUEUES its copies and kernels and returns; calls on one pipe run in the order
+ * they were made (a later call may read what an earlier one wrote).  The host buffers belong
+ * to the pipe until bq_host_pipe_wait returns.  Errors as for the device calls, plus
+ * BQ_ERR_BLOCK for block < min_block or block > chunk_elems and BQ_ERR_DTYPE for a type wider
+ * than `widest`.  y_host may be x_host in bq_roundtrip_host when the types agree.
+ */
+int bq_quantize_host(bq_host_pipe* pipe, const void* x_host, bq_dtype xdt, size_t n, int block,
+                     uint8_t* codes_host, float* absmax_host);
+int bq_dequantize_host(bq_host_pipe* pipe, const uint8_t* codes_host, const float* absmax_host, size_t n, int block,
+                       void* y_host, bq_dtype ydt);
+int bq_roundtrip_host(bq_host_pipe* pipe, const void* x_host, bq_dtype xdt, size_t n, int block,
+                      void* y_host, bq_dtype ydt);
+
+/* Blocks the calling thread until everything enqueued on the pipe has finished (results are then in
+ * the host buffers); returns BQ_ERR_CUDA if any of that work failed. */
+int bq_host_pipe_wait(bq_host_pipe* pipe);
+
+/* Makes `cuda_stream` wait (on the device, without blocking the host) for everything enqueued on
+ * the pipe so far. */
+int bq_host_pipe_wait_on_stream(bq_host_pipe* pipe, void* cuda_stream);
+
 /* 1 when the codebook mirrors around zero (value[j] == -value[254 - j], zero at 127) and its
  * midpoints are spaced so that the tuned kernels' folded search applies; 0 when every call
  * with this codebook takes the general kernels.  The dynamic-tree codebook gives 1. */
 int bq_codebook_is_folded(const bq_codebook* cb);
+
+/*
+ * bq_set_staging -- chooses, for the whole process, how bq_quantize and bq_roundtrip bring blocks of
+ * 2048 and 4096 elements on chip: 0 (the default) = every thread loads its part of a tile into
+ * registers; non-zero = whole blocks are staged through shared memory by bulk asynchronous copies
+ * (cp.async.bulk onto an mbarrier ring; this GPU's memory only).  Same results, bit for bit.
+ * Returns the previous setting.  Shapes without a staged kernel (other block sizes, fp32 blocks of
+ * 4096, unaligned pointers) are unaffected.
+ */
+int bq_set_staging(int on);
+
+/*
+ * bq_kernel_status -- 0, or non-zero when a kernel launched with this codebook gave up on a wait
+ * that is bounded for safety (the staged kernels wait for their copies for about two seconds at
+ * most): the outputs of that call are then incomplete.  Synchronises the device, reads the word and
+ * clears it.  status_out: HOST.
+ */
+int bq_kernel_status(const bq_codebook* cb, int* status_out);
 
 /* A fixed English description of a status code (never NULL). */
 const char* bq_status_string(int status);

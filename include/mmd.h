@@ -156,6 +156,22 @@ int mmd_linear_static(const mmd_weights* w, const void* X, int M, void* Y, bq_dt
  */
 int mmd_kernel_status(const mmd_weights* w, int* status_out);
 
+/*
+ * mmd_selftest_bounded_wait -- a diagnostic with no counterpart in the paper: runs, on the
+ * handle's device, one CTA that has the roles of a tensor-core product kernel (tensor memory
+ * allocated, an "MMA thread", epilogue warps) and lets the MMA thread wait, through the kernels'
+ * own bounded wait, for a barrier that nothing ever arms, with a limit of limit_us microseconds
+ * (1 .. 100000) instead of the kernels' two seconds.  The wait runs out, the thread records
+ * MMD_SELFTEST_CODE in the handle's status word and raises the CTA's give-up flag, the other
+ * waiters leave on seeing it, the tensor memory is freed and the kernel returns: the same path a
+ * product kernel takes when a copy never lands.  Nothing traps, faults or waits without a limit.
+ * threads_left_out (HOST) receives how many threads left through that path (160 of the CTA's 192:
+ * warp 1 waits for nothing).  Synchronises the stream.  Afterwards mmd_kernel_status returns
+ * MMD_SELFTEST_CODE once, and the handle works as before.
+ */
+enum { MMD_SELFTEST_CODE = 77 };
+int mmd_selftest_bounded_wait(const mmd_weights* w, unsigned limit_us, int* threads_left_out, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -18,7 +18,9 @@ LIB_PATH = os.environ.get("BQ_LIB", os.path.join(_HERE, "libbq.so"))    # BQ_LIB
 _lib = None
 
 SYMBOLS = ("bq_make_codebook", "bq_free_codebook", "bq_quantize", "bq_dequantize", "bq_roundtrip",
-           "bq_status_string", "bq_last_cuda_error", "bq_codebook_is_folded")
+           "bq_status_string", "bq_last_cuda_error", "bq_codebook_is_folded",
+           "bq_host_pipe_create", "bq_host_pipe_destroy", "bq_quantize_host", "bq_dequantize_host", "bq_roundtrip_host",
+           "bq_host_pipe_wait", "bq_host_pipe_wait_on_stream", "bq_set_staging", "bq_kernel_status")
 
 
 class BqError(RuntimeError):
@@ -41,6 +43,15 @@ def lib() -> ctypes.CDLL:
         L.bq_status_string.restype = ctypes.c_char_p
         L.bq_last_cuda_error.restype = ctypes.c_char_p
         L.bq_codebook_is_folded.argtypes = [vp]
+        L.bq_host_pipe_create.argtypes = [vp, sz, i32, i32, i32, ctypes.POINTER(vp)]
+        L.bq_host_pipe_destroy.argtypes = [vp]
+        L.bq_quantize_host.argtypes = [vp, vp, i32, sz, i32, vp, vp]
+        L.bq_dequantize_host.argtypes = [vp, vp, vp, sz, i32, vp, i32]
+        L.bq_roundtrip_host.argtypes = [vp, vp, i32, sz, i32, vp, i32]
+        L.bq_host_pipe_wait.argtypes = [vp]
+        L.bq_host_pipe_wait_on_stream.argtypes = [vp, vp]
+        L.bq_set_staging.argtypes = [i32]
+        L.bq_kernel_status.argtypes = [vp, ctypes.POINTER(i32)]
         _lib = L
     return _lib
 
@@ -103,6 +114,19 @@ class Codebook:
             self.close()
         except Exception:
             pass
+
+
+def set_staging(on: bool) -> bool:
+    """``bq_set_staging``: blocks of 2048 / 4096 through the shared-memory-staged kernel; returns the previous setting."""
+    return bool(lib().bq_set_staging(int(bool(on))))
+
+
+def kernel_status(cb: "Codebook") -> int:
+    """``bq_kernel_status``: non-zero when a kernel of this codebook gave up on a bounded wait (reads and clears)."""
+    st = ctypes.c_int(0)
+    with torch.cuda.device(cb.device):
+        _check(lib().bq_kernel_status(cb.handle, ctypes.byref(st)), "bq_kernel_status")
+    return int(st.value)
 
 
 def n_blocks(n: int, block: int) -> int:

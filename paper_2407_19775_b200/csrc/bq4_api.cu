@@ -72,6 +72,7 @@ uint32_t f2u(float f) { uint32_t u; std::memcpy(&u, &f, 4); return u; }
 void build_folded(bq4k::Tables4& t) {
     t.folded = 0;
     std::memset(t.entry, 0, sizeof t.entry);
+    t.neg_limit = 0.0f;
     if (t.val[7] != 0.0f) return;
     for (int j = 0; j < 7; ++j)
         if (t.val[j] != -t.val[14 - j]) return;
@@ -85,17 +86,22 @@ void build_folded(bq4k::Tables4& t) {
     }
     for (int i = 0; i < bq4k::kFoldCells; ++i) {
         const uint32_t S = (bq4k::kFoldCellBase + uint32_t(i)) << 21;
-        for (int neg = 0; neg < 2; ++neg) {
-            const int nthr = neg ? 7 : 8;                                                  // no code below -val[14]: the top midpoint is one-sided
-            uint32_t p0 = 0, inside = 0, off = 0x1FFFFFu;
-            for (int p = 0; p < nthr; ++p) {
-                if (tk[p] < S) ++p0;
-                else if (tk[p] - S < (1u << 21)) { ++inside; off = tk[p] - S; }
-            }
-            if (inside > 1) return;
-            if (inside == 1 && off == 0x1FFFFFu) return;                                   // would look like an empty cell
-            t.entry[neg][i] = neg ? ((((7u - p0) << 24) | off) + S + 1u) : ((((7u + p0) << 24) | 0xE00000u | (0x1FFFFFu - off)) - S);
+        uint32_t p0 = 0, inside = 0, off = 0x1FFFFFu;
+        for (int p = 0; p < 8; ++p) {
+            if (tk[p] < S) ++p0;
+            else if (tk[p] - S < (1u << 21)) { ++inside; off = tk[p] - S; }
         }
+        if (inside > 1) return;
+        if (inside == 1 && off == 0x1FFFFFu) return;                                       // would look like an empty cell
+        t.entry[i] = (((7u + p0) << 24) | 0xE00000u | (0x1FFFFFu - off)) - S;
+    }
+    // negative side: P must not count the top midpoint (there is no code below -val[14]); xhat is clamped to the largest
+    // magnitude whose odd key does not pass it
+    {
+        const uint32_t bits = (tk[7] - 1u) >> 1;
+        float m;
+        std::memcpy(&m, &bits, 4);
+        t.neg_limit = -m;
     }
     t.folded = 1;
 }

@@ -38,13 +38,13 @@ struct Tables4 {
     // #{theta_p < |xhat|} for xhat >= 0 and #{theta_p <= |xhat|} for xhat < 0: the tie rule on either side.  Keys are
     // clamped from below to kFoldKeyLow and cut into cells of 2^21 keys (exponent and 3 fraction bits); no cell holds
     // two thresholds.  For the cell that starts at key S, with P0 thresholds below S and the threshold TK in it:
-    //   xhat >= 0 (8 thresholds, codes 7 + P):  E = ((7 + P0) << 24 | 0xE00000 | (0x1FFFFF - (TK - S))) - S, and
-    //             (E + key) >> 24 = 7 + P0 + [key > TK]: the low 21 bits carry through the three set bits into the code;
-    //   xhat <  0 (7 thresholds: there is no code for -1.0; codes 7 - P):  E = ((7 - P0) << 24 | (TK - S)) + S + 1, and
-    //             (E + ~key) >> 24 = (E - 1 - key) >> 24 = 7 - P0 - [key > TK]: the borrow runs through three clear bits.
-    // One lookup and one addition either way; the sign picks the half of the table and complements the key.
-    // (No threshold in the cell: TK - S = 0x1FFFFF, which neither carries nor borrows.)
-    uint32_t entry[2][kFoldCells];      // [0] xhat >= 0, [1] xhat < 0
+    //     E = ((7 + P0) << 24 | 0xE00000 | (0x1FFFFF - (TK - S))) - S, and (E + key) >> 24 = 7 + P0 + [key > TK]:
+    // the low 21 bits carry through the three set bits into the top byte, which is the code of a non-negative xhat.
+    // (No threshold in the cell: TK - S = 0x1FFFFF, which never carries.)  A negative xhat takes 7 - P = (c ^ 0xF) - 1
+    // from the same byte c, applied to four elements at a time once the bytes are gathered in a word; xhat is clamped
+    // from below to neg_limit first, so that P <= 7 there (there is no code for -1.0).
+    uint32_t entry[kFoldCells];
+    float neg_limit;                    // -(largest |xhat| whose negative key does not pass the top threshold)
     int folded;
 };
 
@@ -126,24 +126,54 @@ __device__ __forceinline__ float quotient(float x, float d, float r, bool quick)
     return __fdiv_rn(x, d);
 }
 
-// code of xhat through the folded table; `ent_lane` is this lane's column of the per-lane replicated entries (the
-// non-negative half first, the negative half kFoldCells rows later), rebased by the index of the first cell.  The two
-// address steps are multiply-adds on purpose: the integer ALU is the busiest pipe of these kernels, the fp32 pipe has room.
-__device__ __forceinline__ uint32_t search_folded16(uint32_t ent_lane, float xhat) {
-    const uint32_t b = __float_as_uint(xhat);
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+// 0xFF in the byte of every negative element: four fp32 values, or four 16-bit elements held in two words (the
+// permute's sign-replicate mode copies a sign bit over a whole byte)
+__device__ __forceinline__ uint32_t sign_bytes_32(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    return prmt(prmt(a, b, 0x00FBu), prmt(c, d, 0x00FBu), 0x5410u);
+}
+__device__ __forceinline__ uint32_t sign_bytes_16(uint32_t w0, uint32_t w1) { return prmt(w0, w1, 0xFDB9u); }
+
+// entry + key of one xhat through the folded table: the top byte of the result is 7 + P.  `ent_lane` is this lane's column
+// of the per-lane replicated entries, rebased by the index of the first cell.  The address step is a multiply-add on
+// purpose: the integer ALU is the busiest pipe of these kernels, the fp32 pipe has room.
+__device__ __forceinline__ uint32_t folded_sum16(uint32_t ent_lane, float xhat, float neg_limit) {
+    const uint32_t b = __float_as_uint(fmaxf(xhat, neg_limit));
     const uint32_t key = max(__funnelshift_l(b, b, 1), kFoldKeyLow);
-    const uint32_t smask = uint32_t(int32_t(b) >> 31);
     uint32_t addr, e;
     asm("mad.lo.u32 %0, %1, 128, %2;" : "=r"(addr) : "r"(key >> 21), "r"(ent_lane));
-    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(addr) : "r"(smask), "r"(0u - uint32_t(kFoldCells) * 128u), "r"(addr));
     asm("ld.shared.u32 %0, [%1];" : "=r"(e) : "r"(addr));
-    return (e + (key ^ smask)) >> 24;
+    return e + key;
 }
-// word + (q << shift) as one multiply-add (the nibbles of a word never overlap)
-__device__ __forceinline__ uint32_t put_nibble(uint32_t word, uint32_t q, int shift) {
-    uint32_t r;
-    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(q), "r"(1u << shift), "r"(word));
-    return r;
+// Eight codes as eight nibbles.  The top bytes c = 7 + P of the sums are gathered four to a word; negative elements
+// (0xFF in `neg0` / `neg1`) take 7 - P = (c ^ 0xF) - 1, which cannot borrow between bytes because c <= 14 there, and the
+// "-1 in every negative byte" is neg * 0x01010101 (neg = 255 * (neg & 0x01010101), and 255 * 0x01010101 = -1 mod 2^32);
+// then byte pairs fold into nibble pairs: x | x >> 4 leaves [q1 q0] in byte 0 and [q3 q2] in byte 2.
+__device__ __forceinline__ uint32_t pack_nibbles8(const uint32_t (&sum)[8], uint32_t neg0, uint32_t neg1) {
+    uint32_t c0 = prmt(prmt(sum[0], sum[1], 0x0073u), prmt(sum[2], sum[3], 0x0073u), 0x5410u);
+    uint32_t c1 = prmt(prmt(sum[4], sum[5], 0x0073u), prmt(sum[6], sum[7], 0x0073u), 0x5410u);
+    asm("mad.lo.u32 %0, %1, 0x01010101, %2;" : "=r"(c0) : "r"(neg0), "r"(c0 ^ (neg0 & 0x0F0F0F0Fu)));
+    asm("mad.lo.u32 %0, %1, 0x01010101, %2;" : "=r"(c1) : "r"(neg1), "r"(c1 ^ (neg1 & 0x0F0F0F0Fu)));
+    return prmt(c0 | (c0 >> 4), c1 | (c1 >> 4), 0x6420u);
+}
+// the codes of eight normalised values as one word of nibbles: the folded table, or the 4-step search over the thresholds
+template <bool FOLDED>
+__device__ __forceinline__ uint32_t codes8(const float (&xh)[8], uint32_t ent_lane, float neg_limit, const float* thr, uint32_t neg0, uint32_t neg1) {
+    if constexpr (FOLDED) {
+        uint32_t sum[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) sum[i] = folded_sum16(ent_lane, xh[i], neg_limit);
+        return pack_nibbles8(sum, neg0, neg1);
+    } else {
+        uint32_t word = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) word |= search16(thr, xh[i]) << (4 * i);
+        return word;
+    }
 }
 
 // two fp32 lanes per instruction (sm_100 packed fp32 arithmetic)
@@ -212,14 +242,15 @@ q4_fast(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restr
     constexpr int lpb = 1 << LOG2_LPB;
     constexpr int log2_lpb = LOG2_LPB;
     __shared__ float thr[16], val[16];
-    __shared__ __align__(128) uint32_t ent[FOLDED ? 2 * kFoldCells * 32 : 1];  // every entry once per lane, in that lane's bank
+    __shared__ __align__(128) uint32_t ent[FOLDED ? kFoldCells * 32 : 1];      // every entry once per lane, in that lane's bank
     fill_tables(tab, thr, val);
     uint32_t ent_lane = 0;
     if constexpr (FOLDED) {
-        for (int i = threadIdx.x; i < 2 * kFoldCells * 32; i += 256) ent[i] = (&tab.entry[0][0])[i >> 5];
+        for (int i = threadIdx.x; i < kFoldCells * 32; i += 256) ent[i] = tab.entry[i >> 5];
         __syncthreads();
         ent_lane = uint32_t(__cvta_generic_to_shared(ent)) + (threadIdx.x & 31) * 4u - kFoldCellBase * 128u;
     }
+    const float neg_limit = tab.neg_limit;
     const size_t stride = size_t(gridDim.x) * 256;
     // Two chunks per trip; the loads of the next trip are issued before this trip's arithmetic.  The trip count is the
     // same for the whole warp because chunk indices start at a multiple of 32 and the shuffles need every lane.
@@ -239,15 +270,25 @@ q4_fast(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restr
     if (warp_first < nchunks) fetch(first);
     for (size_t c0 = first, w0 = warp_first; w0 < nchunks; c0 += 2 * stride, w0 += 2 * stride) {
         float f[2][8];
+        uint32_t neg[2][2];                                         // sign bytes of the eight elements, taken before the words are reused
         const size_t c[2] = {c0, c0 + stride};
 #pragma unroll
-        for (int u = 0; u < 2; ++u) widen_chunk<DT>(nxt[u], f[u]);
+        for (int u = 0; u < 2; ++u) {
+            if constexpr (DT == kF32) {
+                neg[u][0] = sign_bytes_32(nxt[u][0].x, nxt[u][0].y, nxt[u][0].z, nxt[u][0].w);
+                neg[u][1] = sign_bytes_32(nxt[u][W - 1].x, nxt[u][W - 1].y, nxt[u][W - 1].z, nxt[u][W - 1].w);
+            } else {
+                neg[u][0] = sign_bytes_16(nxt[u][0].x, nxt[u][0].y);
+                neg[u][1] = sign_bytes_16(nxt[u][0].z, nxt[u][0].w);
+            }
+            widen_chunk<DT>(nxt[u], f[u]);
+        }
         if (w0 + 2 * stride < nchunks) fetch(c0 + 2 * stride);
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
             float a = 0.0f;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) a = fmaxf(a, fabsf(f[u][i]));
+            for (int i = 0; i < 8; i += 2) asm("max.abs.f32 %0, %1, %2, %3;" : "=f"(a) : "f"(a), "f"(f[u][i]), "f"(f[u][i + 1]));     // max(|a|, |x|, |y|)
 #pragma unroll
             for (int s = 1; s < lpb; s <<= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, s));
             a = block_scale<S16>(a);
@@ -258,12 +299,7 @@ q4_fast(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restr
             asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(d));
             float xh[8];
             quotients8(f[u], d, r, quick, xh);
-            uint32_t word = 0;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const uint32_t q = FOLDED ? search_folded16(ent_lane, xh[i]) : search16(thr, xh[i]);
-                word = put_nibble(word, q, 4 * i);
-            }
+            const uint32_t word = codes8<FOLDED>(xh, ent_lane, neg_limit, thr, neg[u][0], neg[u][1]);
             if (c[u] < nchunks) {
                 reinterpret_cast<uint32_t*>(packed)[c[u]] = word;
                 if ((c[u] & size_t(lpb - 1)) == 0) store_scale<S16>(absmax, c[u] >> log2_lpb, a);
@@ -277,14 +313,15 @@ __global__ void __launch_bounds__(256)
 q4_wide(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restrict__ absmax, size_t nblocks, int chunks_per_block,
         const __grid_constant__ Tables4 tab) {
     __shared__ float thr[16], val[16];
-    __shared__ __align__(128) uint32_t ent[FOLDED ? 2 * kFoldCells * 32 : 1];
+    __shared__ __align__(128) uint32_t ent[FOLDED ? kFoldCells * 32 : 1];
     fill_tables(tab, thr, val);
     uint32_t ent_lane = 0;
     if constexpr (FOLDED) {
-        for (int i = threadIdx.x; i < 2 * kFoldCells * 32; i += 256) ent[i] = (&tab.entry[0][0])[i >> 5];
+        for (int i = threadIdx.x; i < kFoldCells * 32; i += 256) ent[i] = tab.entry[i >> 5];
         __syncthreads();
         ent_lane = uint32_t(__cvta_generic_to_shared(ent)) + (threadIdx.x & 31) * 4u - kFoldCellBase * 128u;
     }
+    const float neg_limit = tab.neg_limit;
     const int lane = threadIdx.x & 31;
     const size_t wstride = size_t(gridDim.x) * 8;
     for (size_t b = size_t(blockIdx.x) * 8 + (threadIdx.x >> 5); b < nblocks; b += wstride) {
@@ -307,13 +344,10 @@ q4_wide(const void* __restrict__ x, uint8_t* __restrict__ packed, float* __restr
             float f[8], xh[8];
             load8<DT>(x, cbase + k, f);
             quotients8(f, d, r, quick, xh);
-            uint32_t word = 0;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const uint32_t q = FOLDED ? search_folded16(ent_lane, xh[i]) : search16(thr, xh[i]);
-                word = put_nibble(word, q, 4 * i);
-            }
-            reinterpret_cast<uint32_t*>(packed)[cbase + k] = word;
+            // the quotients carry the signs of the inputs
+            const uint32_t neg0 = sign_bytes_32(__float_as_uint(xh[0]), __float_as_uint(xh[1]), __float_as_uint(xh[2]), __float_as_uint(xh[3]));
+            const uint32_t neg1 = sign_bytes_32(__float_as_uint(xh[4]), __float_as_uint(xh[5]), __float_as_uint(xh[6]), __float_as_uint(xh[7]));
+            reinterpret_cast<uint32_t*>(packed)[cbase + k] = codes8<FOLDED>(xh, ent_lane, neg_limit, thr, neg0, neg1);
         }
         if (lane == 0) store_scale<S16>(absmax, b, a);
     }

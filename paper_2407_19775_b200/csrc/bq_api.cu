@@ -5,6 +5,7 @@
 #include "bq_error.h"
 #include "bq_launch.h"
 
+#include <atomic>
 #include <cstring>
 #include <new>
 
@@ -36,6 +37,8 @@ bool tuned_block(int block) {
 
 constexpr size_t kMaxElems = size_t(1) << 40;
 
+std::atomic<int> g_staging{0};      // bq_set_staging: blocks of 2048 / 4096 through the shared-memory-staged kernel
+
 }  // namespace
 
 void bql::set_last_cuda_error(const char* text) { std::strncpy(g_last_error, text, sizeof(g_last_error) - 1); }
@@ -44,9 +47,12 @@ struct bq_codebook {
     bqt::Tables host;
     bqk::DeviceTables dev;
     void* blob;
+    int* status;              // device word set by a kernel whose bounded wait ran out
     int device;
     int sm_count;
 };
+
+static bool on_codebook_device_c(const bq_codebook* cb);
 
 extern "C" {
 
@@ -89,7 +95,7 @@ int bq_make_codebook(int kind, const float* user_values256, float* host_values_o
     if (host_values_out256) std::memcpy(host_values_out256, cb->host.values, 256 * sizeof(float));
 
     // one device allocation: values | thr_down | tk | cmag | guess  (the kernels rely on guess following cmag directly)
-    const size_t words = 256 + 256 + 128 + 132 + bqt::kCells;
+    const size_t words = 256 + 256 + 128 + 132 + bqt::kCells + 4;      // the last four words: the kernels' status word (zero)
     cudaError_t e = cudaGetDevice(&cb->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&cb->sm_count, cudaDevAttrMultiProcessorCount, cb->device);
     if (e == cudaSuccess) e = cudaMalloc(&cb->blob, words * 4);
@@ -112,6 +118,7 @@ int bq_make_codebook(int kind, const float* user_values256, float* host_values_o
     cb->dev.cmag = reinterpret_cast<const float*>(base + o_cm);
     cb->dev.guess = base + o_gs;
     cb->dev.neg_limit = cb->host.folded ? cb->host.neg_limit : 0.0f;
+    cb->status = reinterpret_cast<int*>(cb->blob) + (words - 4);
     *out = cb;
     return BQ_OK;
 }
@@ -124,6 +131,19 @@ int bq_free_codebook(bq_codebook* cb) {
 }
 
 int bq_codebook_is_folded(const bq_codebook* cb) { return (cb && cb->host.folded) ? 1 : 0; }
+
+int bq_set_staging(int on) { return g_staging.exchange(on ? 1 : 0); }
+
+int bq_kernel_status(const bq_codebook* cb, int* status_out) {
+    if (!cb || !status_out) return BQ_ERR_NULL;
+    if (!on_codebook_device_c(cb)) return BQ_ERR_CODEBOOK;
+    int host[2] = {0, 0};
+    cudaError_t e = cudaMemcpy(host, cb->status, sizeof(int), cudaMemcpyDeviceToHost);      // waits for the device's earlier work
+    if (e == cudaSuccess && host[0] != 0) e = cudaMemset(cb->status, 0, sizeof(int));
+    if (e != cudaSuccess) return cuda_fail(e);
+    *status_out = host[0];
+    return BQ_OK;
+}
 
 }  // extern "C"
 
@@ -143,7 +163,15 @@ int forward(const void* x, int xdt, size_t n, int block, const bq_codebook* cb, 
     size_t done = 0;        // elements covered by the tuned kernel
     const bool can_tune = cb->host.folded && tuned_block(block) && aligned(x, 16) && (!write_y || (aligned(y, 16) && ydt == xdt)) &&
                           (!write_q || (aligned(codes, 8) && aligned(absmax, 4)));
-    if (can_tune && n >= B) {
+    if (can_tune && n >= B && g_staging.load() && (block == 2048 || block == 4096)) {
+        // the staged kernel takes every whole block; the short last block, if any, goes to the general kernel below
+        bool taken = false;
+        cudaError_t e = bql::launch_fwd_staged(xdt, block, write_y, write_q, x, y, codes, absmax, n / B, cb->dev, cb->sm_count, cb->device,
+                                               cb->status, stream, &taken);
+        if (e != cudaSuccess) return cuda_fail(e);
+        if (taken) done = (n / B) * B;
+    }
+    if (can_tune && n >= B && done == 0) {
         const size_t n_full = (n / B) * B;
         cudaError_t e = bql::launch_fwd_fast(xdt, block, write_y, write_q, x, y, codes, absmax, n_full, cb->dev, cb->sm_count, cb->device, stream,
                                              &done);
@@ -213,3 +241,8 @@ int bq_dequantize(const uint8_t* codes, const float* absmax, size_t n, int block
 }
 
 }  // extern "C"
+
+static bool on_codebook_device_c(const bq_codebook* cb) {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == cb->device;
+}

@@ -220,10 +220,14 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
 // the bytes of negative elements (sign_mask_* below: byte-permutes that replicate a sign bit
 // over its byte; taken from the inputs, whose signs the quotients share); the subtraction
 // cannot borrow between bytes because c ^ 0xFF >= 1 wherever 1 is subtracted (the clamp in
-// search_folded keeps c <= 254 on the negative side).
+// search_folded keeps c <= 254 on the negative side).  The "1 in every negative byte" is never
+// formed: neg = 255 * (neg & 0x01010101) and 255 * 0x01010101 = -1 (mod 2^32), so
+// neg * 0x01010101 = -(neg & 0x01010101), and the subtraction is one multiply-add.
 __device__ __forceinline__ uint32_t pack_codes(const Found& f0, const Found& f1, const Found& f2, const Found& f3, uint32_t neg) {
     const uint32_t c = prmt(prmt(f0.sum, f1.sum, 0x0073u), prmt(f2.sum, f3.sum, 0x0073u), 0x5410u);
-    return (c ^ neg) - (neg & 0x01010101u);
+    uint32_t out;
+    asm("mad.lo.u32 %0, %1, 0x01010101, %2;" : "=r"(out) : "r"(neg), "r"(c ^ neg));
+    return out;
 }
 // sign bytes of four 16-bit elements held in two words (element sign bits sit in bytes 1, 3, 5, 7)
 __device__ __forceinline__ uint32_t sign_mask_16(uint32_t w0, uint32_t w1) { return prmt(w0, w1, 0xFDB9u); }

@@ -30,6 +30,13 @@ inline cudaError_t launch_fwd_fast(int xdt, int block, bool write_y, bool write_
     }
 }
 
+// The shared-memory-staged forward kernel (blocks of 2048 and 4096 elements whose ring fits beside the tables): all
+// `nblocks` whole blocks; *taken says whether this shape has such a kernel.  `status` is the codebook's device word that a
+// wait which ran out sets.
+cudaError_t launch_fwd_staged(int xdt, int block, bool write_y, bool write_q, const void* x, void* y, uint8_t* codes, float* absmax,
+                              size_t nblocks, const bqk::DeviceTables& tab, int sm_count, int device, int* status, cudaStream_t stream,
+                              bool* taken);
+
 cudaError_t launch_fwd_general(int xdt, int ydt, bool write_y, bool write_q, const void* x, void* y, uint8_t* codes, float* absmax,
                                size_t n, size_t block, size_t first_block, const bqk::DeviceTables& tab, int sm_count,
                                cudaStream_t stream);

@@ -512,6 +512,26 @@ int mmd_linear(const mmd_weights* w, const void* X, int M, void* Y, bq_dtype ydt
     return e == cudaSuccess ? BQ_OK : cuda_fail(e);
 }
 
+int mmd_selftest_bounded_wait(const mmd_weights* w, unsigned limit_us, int* threads_left_out, void* cuda_stream) {
+    if (!w || !threads_left_out) return BQ_ERR_NULL;
+    if (limit_us < 1 || limit_us > 100000) return BQ_ERR_SIZE;              // 1 us .. 0.1 s: this wait is meant to run out
+    if (!on_device(w)) return BQ_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int khz = 0;
+    cudaError_t e = cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, w->device);
+    if (e != cudaSuccess) return cuda_fail(e);
+    const long long cycles = (long long)limit_us * (khz > 0 ? khz : 1000000) / 1000;
+    // the counter lives in the handle's spare status space (the word after the status)
+    int* left = w->status + 1;
+    e = cudaMemsetAsync(left, 0, sizeof(int), stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    mmdk::wait_selftest<<<1, mmdk::kTcThreads, 0, stream>>>(w->status, MMD_SELFTEST_CODE, cycles, left);
+    e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaMemcpyAsync(threads_left_out, left, sizeof(int), cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    return e == cudaSuccess ? BQ_OK : cuda_fail(e);
+}
+
 int mmd_kernel_status(const mmd_weights* w, int* status_out) {
     if (!w || !status_out) return BQ_ERR_NULL;
     if (!on_device(w)) return BQ_ERR_CUDA;

@@ -357,14 +357,15 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait.  Returns false when the limit ran out or another thread of the CTA gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code,
+                                          long long limit_cycles = kWaitLimitCycles) {
     if (mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
     for (uint32_t it = 1;; ++it) {
         if (mbar_try(bar, parity)) return true;
         if ((it & 255u) == 0u) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitLimitCycles) {
+            if (clock64() - t0 > limit_cycles) {
                 *abort_flag = 1;
                 atomicCAS(status, 0, code);
                 return false;
@@ -1186,6 +1187,58 @@ gemm_tc2(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUt
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(2 * BN) : "memory");
+    }
+}
+
+
+// ------------------------------------------------------------------------------------------
+// wait_selftest: the give-up path of the tensor-core kernels on its own, with a short limit.
+//
+// One CTA with the roles of gemm_tc: warp 1 allocates tensor memory; thread 0 (the "MMA
+// thread") waits, through the same bounded routine as the product kernels, for a barrier that
+// nothing ever arms; the epilogue warps wait for an "accumulator complete" barrier that, as in
+// a product kernel whose MMA thread gave up, is never committed.  The first wait to run out
+// records `code` and raises the CTA's abort flag, the other waiters see the flag and leave,
+// every thread meets at the barrier, the tensor memory is given back and the kernel returns.
+// No copy is in flight and nothing is stored besides the status word and the `left` counter
+// (how many threads left through the give-up path).
+__global__ void __launch_bounds__(kTcThreads, 1)
+wait_selftest(int* status, int code, long long limit_cycles, int* left) {
+    __shared__ __align__(8) unsigned long long bars[2];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_word;
+    volatile int* abort_flag = &abort_word;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t never = smem_u32(&bars[0]), accbar = smem_u32(&bars[1]);
+    if (threadIdx.x == 0) {
+        mbar_init(never, 1);
+        mbar_init(accbar, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(32) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = tmem_slot;
+    bool ok = true;
+    if (warp == 0) {
+        if (lane == 0) ok = mbar_wait(never, 0, abort_flag, status, code, limit_cycles);
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+    } else if (warp >= 2) {
+        // a limit of its own, far longer: these warps leave because of the abort flag, not their own clock
+        if (lane == 0) ok = mbar_wait(accbar, 0, abort_flag, status, code + 1, limit_cycles * 64);
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+    }
+    if (!ok) atomicAdd(left, 1);
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(32) : "memory");
     }
 }
 

@@ -14,7 +14,8 @@ PATH_AUTO, PATH_GENERAL, PATH_TENSOR, PATH_TENSOR_TILE, PATH_TENSOR_SOLO = 0, 1,
 _TORCH_OF = {0: torch.float32, 1: torch.float16, 2: torch.bfloat16}
 
 SYMBOLS = ("mmd_side_columns", "mmd_select_features", "mmd_rowquant", "mmd_decompose", "mmd_free", "mmd_weights_view",
-           "mmd_workspace_layout", "mmd_linear", "mmd_linear_static", "mmd_kernel_status")
+           "mmd_workspace_layout", "mmd_linear", "mmd_linear_static", "mmd_kernel_status", "mmd_selftest_bounded_wait")
+SELFTEST_CODE = 77
 STATIC_SCRATCH_BYTES = 4 << 20
 _typed = False
 
@@ -34,6 +35,7 @@ def _lib() -> ctypes.CDLL:
         L.mmd_linear.argtypes = [vp, vp, i32, vp, i32, vp, sz, i32, vp]
         L.mmd_linear_static.argtypes = [vp, vp, i32, vp, i32, i32, vp]
         L.mmd_kernel_status.argtypes = [vp, ctypes.POINTER(i32)]
+        L.mmd_selftest_bounded_wait.argtypes = [vp, ctypes.c_uint, ctypes.POINTER(i32), vp]
         _typed = True
     return L
 
@@ -178,6 +180,15 @@ class DecomposedLinear:
         with torch.cuda.device(self.device):
             _check(_lib().mmd_kernel_status(self._h, ctypes.byref(st)), "mmd_kernel_status")
         return int(st.value)
+
+    def selftest_bounded_wait(self, limit_us: int = 2000) -> int:
+        """``mmd_selftest_bounded_wait``: lets a bounded wait of the tensor-core kernels run out on purpose (short
+        limit, a barrier nothing arms); returns how many threads left through the give-up path."""
+        left = ctypes.c_int(-1)
+        with torch.cuda.device(self.device):
+            _check(_lib().mmd_selftest_bounded_wait(self._h, limit_us, ctypes.byref(left), torch.cuda.current_stream(self.device).cuda_stream),
+                   "mmd_selftest_bounded_wait")
+        return int(left.value)
 
     def close(self) -> None:
         if self._h:

@@ -218,3 +218,80 @@ def make_linear(name: str, tokens: int | None = None, out_features: int | None =
 def bits_2d(x: torch.Tensor) -> np.ndarray:
     """A 2-D fp16 / bf16 CPU tensor as a uint16 bit-pattern array of the same shape."""
     return as_numpy_bits(x).reshape(x.shape)
+
+
+# ------------------------------------------------------------------------------------------
+# Computation graphs for the slicing of topological orders: layered networks that are not a plain
+# chain of equal blocks (a U-shaped denoiser with skip connections and a conditioning node that
+# feeds every stage; a trunk with several prediction heads of different depth), the kind of model
+# the paper's dynamic sharding is for.  Node attributes are integers: work in microseconds,
+# sizeparam and sizeout in bytes; B is the link's bytes per microsecond, M the fast memory in bytes.
+# The priority vectors of a population are uniform keys in [0, 1).  Only inputs are drawn here:
+# decoding keys into orders and costing blocks is the method's work.
+
+@dataclass(frozen=True)
+class GraphWorkload:
+    name: str
+    kind: str
+    n: int
+    k: int
+    population: int
+    B: int
+    M: int
+    seed: int
+    recipe: str
+
+
+GRAPH_WORKLOADS = {
+    "mtpp_tiny": GraphWorkload("mtpp_tiny", "random", 14, 3, 6, 3, 4000, 20, "random DAG, edge probability 0.25"),
+    "mtpp_heads": GraphWorkload("mtpp_heads", "heads", 96, 4, 24, 125, 6 << 20, 21,
+                                "a trunk of 40 operations and 4 heads of 8..20 operations reading different trunk depths; 1 Gbit/s link"),
+    "mtpp_unet": GraphWorkload("mtpp_unet", "unet", 256, 8, 2048, 125, 48 << 20, 22,
+                               "U-shaped denoiser: 8 stages down, 8 up, skip connections, one conditioning node feeding every stage; 1 Gbit/s link"),
+}
+
+
+def make_graph(name: str):
+    """Returns (n, edges int32 [m, 2], work, sizeparam, sizeout as int64 arrays) of graph workload ``name``."""
+    w = GRAPH_WORKLOADS[name]
+    rng = np.random.default_rng(w.seed)
+    n = w.n
+    edges = []
+    if w.kind == "random":
+        edges = [(u, v) for u in range(n) for v in range(u + 1, n) if rng.random() < 0.25]
+    elif w.kind == "heads":
+        trunk = 40
+        edges += [(i, i + 1) for i in range(trunk - 1)]
+        at = trunk
+        for h, depth in enumerate((8, 12, 16, 20)):
+            tap = 9 + 10 * h                                  # each head reads another depth of the trunk
+            edges.append((tap, at))
+            edges += [(at + i, at + i + 1) for i in range(depth - 1)]
+            if h % 2:
+                edges.append((tap - 4, at + depth // 2))      # and a second, earlier feature half-way
+            at += depth
+        assert at == n
+    else:
+        stages, per = 8, (n - 1) // 16                        # node 0 is the conditioning node
+        body = list(range(1, 1 + 16 * per))
+        extra = list(range(1 + 16 * per, n))                  # left-over nodes extend the last stage
+        chain = body + extra
+        edges += [(a, b) for a, b in zip(chain, chain[1:])]
+        for s in range(16):
+            edges.append((0, chain[s * per]))                 # conditioning enters every stage
+        for s in range(stages):
+            edges.append((chain[s * per + per - 1], chain[(15 - s) * per]))      # skip: end of down-stage s -> start of up-stage 15 - s
+    work = rng.integers(20, 2000, n)
+    sizeparam = rng.integers(0, 8 << 20, n) * (rng.random(n) < 0.6)
+    sizeout = rng.integers(64 << 10, 4 << 20, n)
+    e = np.asarray(sorted(set(edges)), np.int32).reshape(-1, 2)
+    return n, e, work.astype(np.int64), sizeparam.astype(np.int64), sizeout.astype(np.int64)
+
+
+def make_keys(name: str, population: int | None = None) -> torch.Tensor:
+    """Uniform priority vectors [population, n] float32 (a row of equal keys is put first)."""
+    w = GRAPH_WORKLOADS[name]
+    P = w.population if population is None else population
+    keys = torch.rand((P, w.n), generator=_gen(w.seed + 500), dtype=torch.float32)
+    keys[0] = 0.5
+    return keys

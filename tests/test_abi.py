@@ -26,7 +26,7 @@ def test_every_declared_symbol_is_exported(bq):
 
 
 def test_every_header_is_covered():
-    assert sorted(os.listdir(os.path.join(ROOT, "include"))) == ["bq.h", "bq4.h", "bq_tune.h", "mmd.h"]
+    assert sorted(os.listdir(os.path.join(ROOT, "include"))) == ["bq.h", "bq4.h", "bq_transport.h", "bq_tune.h", "mmd.h", "mtpp.h"]
 
 
 def test_every_declared_bq4_symbol_is_exported(bq):
@@ -169,6 +169,98 @@ def test_argument_errors_need_no_device(bq):
     assert L.bq_make_codebook(7, None, None, ctypes.byref(out)) == 5
     assert L.bq_make_codebook(0, None, None, None) == 1
     assert L.bq_free_codebook(None) == 0
+
+
+def test_every_declared_transport_symbol_is_exported_and_host_arithmetic(bq):
+    from paper_2407_19775_b200 import binding, transport
+    L = binding.lib()
+    names = _declared("bq_transport.h", "bqx_")
+    assert {"bqx_rx_create", "bqx_tx_open", "bqx_tx_send_piece", "bqx_rx_recv_piece", "bqx_transfer", "bqx_plan"} <= set(names)
+    for name in names:
+        assert hasattr(L, name), name
+    assert set(transport.SYMBOLS) == set(names)
+    # what crosses the boundary: n + 4 ceil(n / block) bytes, about half of a 16-bit tensor (the paper's "halve")
+    assert transport.payload_bytes(1 << 20, 64) == (1 << 20) + 4 * (1 << 14)
+    assert transport.payload_bytes(1000, 64) == 1000 + 4 * 16 and transport.payload_bytes(0, 64) == 0
+    assert abs(2 * (1 << 30) / transport.payload_bytes(1 << 30, 256) - 2 * 256 / 260) < 1e-12
+    assert transport.mailbox_bytes(1 << 20, 64, 3) == 3 * ((1 << 20) + 65792)      # codes + (2^14 + 1 floats rounded up to 256 bytes)
+    assert transport.mailbox_bytes(0, 64, 3) == 0 and transport.mailbox_bytes(1 << 20, 64, 1) == 0 and transport.mailbox_bytes(32, 64, 3) == 0
+    # the piece schedule: whole blocks per piece, slots in turn, a short last piece
+    assert transport.plan(1000, 64, 300, 3) == [(0, 0, 256), (1, 256, 256), (2, 512, 256), (0, 768, 232)]
+    assert transport.plan(256, 64, 300, 2) == [(0, 0, 256)]
+    assert transport.plan(0, 64, 300, 2) == []
+    assert transport.plan(257, 1, 100, 2) == [(0, 0, 100), (1, 100, 100), (0, 200, 57)]
+    T = transport._lib()
+    assert T.bqx_plan(1000, 0, 300, 3, 0, None, None, None, None) == 3 and T.bqx_plan(1000, 301, 300, 3, 0, None, None, None, None) == 3
+    one = ctypes.c_void_p(256)       # never dereferenced: every call below fails a check first
+    out = ctypes.c_void_p()
+    assert T.bqx_rx_create(None, 1 << 20, 64, 3, ctypes.byref(out)) == 5
+    assert T.bqx_rx_create(one, 1 << 20, 64, 3, None) == 1
+    assert T.bqx_rx_create(one, 1 << 20, 0, 3, ctypes.byref(out)) == 3
+    assert T.bqx_rx_create(one, 1 << 20, 64, 9, ctypes.byref(out)) == 4
+    assert T.bqx_rx_create(one, 0, 64, 3, ctypes.byref(out)) == 4
+    assert T.bqx_tx_open(one, None, 0, ctypes.byref(out)) == 1
+    assert T.bqx_tx_open(None, one, 0, ctypes.byref(out)) == 5
+    junk = ctypes.create_string_buffer(2048)
+    assert T.bqx_tx_open(one, junk, 0, ctypes.byref(out)) == 4                    # not a mailbox description
+    assert T.bqx_tx_open(one, junk, 7, ctypes.byref(out)) == 4                    # unknown mode
+    assert T.bqx_rx_destroy(None) == 0 and T.bqx_tx_close(None) == 0
+    assert T.bqx_tx_send_piece(None, one, 2, 64, 64, 0, None) == 1
+    assert T.bqx_rx_recv_piece(None, 64, 64, 0, one, 2, None) == 1
+    assert T.bqx_transfer(None, None, one, 2, 64, 64, one, 2, None, None) == 1
+
+
+def test_every_declared_mtpp_symbol_is_exported_and_argument_errors(bq):
+    import numpy as np
+    from paper_2407_19775_b200 import binding, mtpp
+    L = binding.lib()
+    names = _declared("mtpp.h", "mtpp_")
+    assert set(names) == {"mtpp_graph_create", "mtpp_graph_free", "mtpp_decode_orders", "mtpp_slice_orders"} == set(mtpp.SYMBOLS)
+    for name in names:
+        assert hasattr(L, name), name
+    T = mtpp._lib()
+    out = ctypes.c_void_p()
+    three = np.array([1, 2, 3], np.int64)
+
+    def create(n, edges, w=three, sp=three, so=three, outp=ctypes.byref(out)):
+        e = np.asarray(edges, np.int32).reshape(-1, 2)
+        return T.mtpp_graph_create(n, e.shape[0], e.ctypes.data if e.size else None, w.ctypes.data, sp.ctypes.data, so.ctypes.data, outp)
+
+    # every check below fails on the host, before any device is touched
+    assert create(3, [(0, 1)], outp=None) == 1
+    assert create(0, []) == 4 and create(2000, []) == 4
+    assert create(3, [(0, 3)]) == 4 and create(3, [(1, 1)]) == 4 and create(3, [(-1, 2)]) == 4
+    assert create(3, [(0, 1), (1, 2), (2, 0)]) == 4                                  # a cycle
+    assert create(3, [(0, 1)], w=np.array([1, -2, 3], np.int64)) == 4               # negative work
+    assert create(3, [(0, 1)], so=np.array([1, 2, 1 << 41], np.int64)) == 4         # too large
+    assert T.mtpp_graph_create(3, 1, None, three.ctypes.data, three.ctypes.data, three.ctypes.data, ctypes.byref(out)) == 1
+    assert T.mtpp_graph_free(None) == 0
+    one = ctypes.c_void_p(256)
+    assert T.mtpp_decode_orders(None, one, 4, one, None) == 1
+    assert T.mtpp_slice_orders(None, one, 4, 3, 1, 0, one, one, one, one, None) == 1
+
+
+def test_host_call_argument_errors_need_no_device(bq):
+    from paper_2407_19775_b200 import binding
+    L = binding.lib()
+    one = ctypes.c_void_p(16)        # never dereferenced: every call below fails a check first
+    out = ctypes.c_void_p()
+    assert L.bq_host_pipe_create(one, 1 << 20, 64, 2, 3, None) == 1             # nowhere to put the handle
+    assert L.bq_host_pipe_create(None, 1 << 20, 64, 2, 3, ctypes.byref(out)) == 5     # no codebook
+    assert L.bq_host_pipe_create(one, 1 << 20, 64, 9, 3, ctypes.byref(out)) == 2      # element type
+    assert L.bq_host_pipe_create(one, 1 << 20, 0, 2, 3, ctypes.byref(out)) == 3       # smallest block
+    assert L.bq_host_pipe_create(one, 32, 64, 2, 3, ctypes.byref(out)) == 3           # a block does not fit a piece
+    assert L.bq_host_pipe_create(one, 0, 1, 2, 3, ctypes.byref(out)) == 3
+    assert L.bq_host_pipe_create(one, 1 << 20, 64, 2, 1, ctypes.byref(out)) == 4      # slots
+    assert L.bq_host_pipe_create(one, 1 << 20, 64, 2, 9, ctypes.byref(out)) == 4
+    assert L.bq_host_pipe_create(one, 1 << 35, 64, 2, 3, ctypes.byref(out)) == 4      # piece too large
+    assert out.value is None
+    assert L.bq_host_pipe_destroy(None) == 0
+    assert L.bq_host_pipe_wait(None) == 1
+    assert L.bq_host_pipe_wait_on_stream(None, None) == 1
+    assert L.bq_quantize_host(None, one, 2, 64, 64, one, one) == 1
+    assert L.bq_dequantize_host(None, one, one, 64, 64, one, 2) == 1
+    assert L.bq_roundtrip_host(None, one, 2, 64, 64, one, 2) == 1
 
 
 def test_missing_library_is_an_error(monkeypatch):

@@ -55,3 +55,26 @@ def test_bench_line_has_the_contract_keys(bq):
     assert dec["kernel_status"] == 0 and 0.2 < dec["frac_of_measured_hbm"] < 1.1
     wide = m["decode_wide"]
     assert wide["kernel_status"] == 0 and 0.3 < wide["frac_of_measured_hbm"] < 1.1 and wide["algorithmic_bytes"] > 3 * dec["algorithmic_bytes"]
+    assert abs(mr["ms"] - m["ms_per_call"]) < 1e-6 and mr["product_kernel_estimate"]["frac"] >= mr["frac"]      # the roofline is the whole call's
+    # the input's fingerprint, the host-buffer calls behind e2e, finished sections on stderr as they complete
+    assert len(d["config"]["input_sha256"]) == 64 and "bq_roundtrip_host" in e["api"]
+    sections = [json.loads(line)["section"] for line in r.stderr.splitlines() if line.startswith('{"section"')]
+    assert sections[:3] == ["kernels", "e2e", "quality"] and {"bq4", "autotune", "small_configs", "mmd", "transport"} <= set(sections)
+    # the boundary transport, loop-back: what arrives is the fused roundtrip's bytes; about half the bytes cross
+    tr = d["transport"]
+    assert tr["bit_identical_to_roundtrip"] is True and "loop-back" in tr["link"] and 1.9 < tr["bytes_ratio"] < 2.0
+    assert 0 < tr["store"]["ms"] < 5 and 0 < tr["copy"]["ms"] < 5 and tr["pieces"] == 16
+    mt = d["mtpp"]
+    assert mt["orders_per_s"] > 1000 * mt["cpu_baseline"]["value"] > 0 and 0 < mt["best_bottleneck"] <= mt["worst_bottleneck"]
+
+
+def test_bench_on_another_config(bq):
+    """--config runs the step on one of the other workloads; a tensor that fits in L2 is flushed out before every launch."""
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--steps", "3", "--warmup", "3", "--e2e-steps", "1", "--config", "prefill7b"],
+                       capture_output=True, text=True, timeout=600, cwd=ROOT)
+    assert r.returncode == 0, r.stderr[-2000:]
+    d = json.loads(r.stdout.strip().splitlines()[-1])
+    assert "prefill7b" in d["config"]["workload"] and "256 MiB buffer is written before every launch" in d["config"]["l2"]
+    assert d["gpu_launches"] == 3 * 3 and set(d["kernels"]) == {"quantize_b256", "dequantize_b256", "roundtrip_b256"}
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["mmd"] is None and d["roofline"]["traffic"] is None
+    assert 0 < d["e2e"]["value"] < d["value"]

@@ -322,3 +322,23 @@ def test_back_to_back_calls_share_a_workspace(bq, M, K, N):
         assert torch.equal(y, lin.linear(x, torch.float32, path=1))
     check_output(ys[3], xs[3].cpu(), W, np.zeros(0, np.int32), F16, exact_expected=True)
     lin.close()
+
+
+def test_a_bounded_wait_that_runs_out_leaves_a_status_and_a_usable_handle(bq):
+    """The give-up path of the tensor-core kernels, exercised the safe way: a diagnostic CTA with the kernels' roles waits
+    (2 ms limit instead of 2 s) for a barrier that nothing arms.  It must return, leave its code in the status word, free
+    its tensor memory (the product kernels after it need all of it) and leave the handle and the context working."""
+    X, W, idx = workloads.make_linear("mmd_decode70b", tokens=48, out_features=512)
+    lin = bq.DecomposedLinear(W.cuda(), idx)
+    before = lin.linear(X.cuda(), torch.float32, path=3)
+    assert lin.kernel_status() == 0
+    for limit_us in (2000, 50):
+        assert lin.selftest_bounded_wait(limit_us) == 160            # warps 0 and 2..5 left through the give-up path
+        assert lin.kernel_status() == bq.mmd.SELFTEST_CODE           # recorded ...
+        assert lin.kernel_status() == 0                              # ... and cleared by the read
+        after = lin.linear(X.cuda(), torch.float32, path=3)          # tensor memory was given back, the context is intact
+        assert lin.kernel_status() == 0 and torch.equal(after, before)
+    check_output(before, X, W, idx, F16, exact_expected=False)
+    with pytest.raises(bq.BqError):
+        lin.selftest_bounded_wait(0)
+    lin.close()

@@ -1,0 +1,115 @@
+"""GPU parity of the slicing of topological orders (include/mtpp.h) against the CPU oracle: the decoded
+orders, the bottleneck cost, the number of blocks and the cut positions are integers and must be identical."""
+import random
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import mtpp_oracle as mo
+from paper_2407_19775_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+
+def oracle_graph(n, edges, work, sizeparam, sizeout):
+    return mo.Graph(n, [tuple(e) for e in edges.tolist()], work.tolist(), sizeparam.tolist(), sizeout.tolist())
+
+
+def check_population(bq, name, population, ks, sample=None):
+    w = workloads.GRAPH_WORKLOADS[name]
+    n, edges, work, sizeparam, sizeout = workloads.make_graph(name)
+    g = oracle_graph(n, edges, work, sizeparam, sizeout)
+    dg = bq.mtpp.SliceGraph(n, edges, work, sizeparam, sizeout, device="cuda:0")
+    keys = workloads.make_keys(name, population)
+    orders = dg.decode_orders(keys.cuda())
+    torch.cuda.synchronize()
+    got_orders = orders.cpu().numpy()
+    rows = range(population) if sample is None else sample
+    for p in rows:
+        assert got_orders[p].tolist() == mo.decode_order(g, keys[p].tolist()), f"order {p}"
+    for k in ks:
+        cost, blocks, cuts, status = dg.slice_orders(orders, k, w.B, w.M)
+        torch.cuda.synchronize()
+        assert int(status.sum()) == 0
+        cost, blocks, cuts = cost.cpu().numpy(), blocks.cpu().numpy(), cuts.cpu().numpy()
+        for p in rows:
+            want = mo.slice_order(g, got_orders[p].tolist(), k, w.B, w.M)
+            got = (int(cost[p]), int(blocks[p]), cuts[p][:blocks[p]].tolist())
+            assert got == want, f"order {p}, k {k}"
+            assert not cuts[p][blocks[p]:].any()
+        # every order: the cuts it returns have the bottleneck it returns, under the oracle's block cost (cheap: k blocks each)
+        if sample is not None:
+            for p in range(0, population, max(1, population // 64)):
+                ends = cuts[p][:blocks[p]].tolist()
+                starts = [1] + [e + 1 for e in ends[:-1]]
+                pi = got_orders[p].tolist()
+                assert mo.is_topological(g, pi) and ends[-1] == n
+                assert max(mo.segment_cost(g, pi, s, e, w.B, w.M) for s, e in zip(starts, ends)) == int(cost[p])
+    dg.close()
+
+
+def test_tiny_graph_every_order_every_k(bq):
+    check_population(bq, "mtpp_tiny", 6, [1, 2, 3, 5, 14, 16])
+
+
+def test_trunk_with_heads(bq):
+    check_population(bq, "mtpp_heads", 24, [1, 4, 7], sample=range(0, 24, 2))
+
+
+def test_unet_population_sampled_orders(bq):
+    """The benchmark's population in its launch configuration (2048 orders of 256 nodes, 8 blocks): three orders in full
+    against the oracle, and on every 32nd order the returned cuts re-costed by the oracle."""
+    check_population(bq, "mtpp_unet", 2048, [8], sample=[0, 1, 2047])
+
+
+def test_random_graphs_fuzz(bq):
+    rng = random.Random(7)
+    for case in range(12):
+        n = rng.choice([1, 2, 3, 17, 33, 64, 100])
+        edges = np.asarray([(u, v) for u in range(n) for v in range(u + 1, n) if rng.random() < rng.choice([0.0, 0.05, 0.3])], np.int32).reshape(-1, 2)
+        work = np.asarray([rng.randrange(0, 50) for _ in range(n)], np.int64)
+        sizeparam = np.asarray([rng.randrange(0, 500) for _ in range(n)], np.int64)
+        sizeout = np.asarray([rng.randrange(0, 80) for _ in range(n)], np.int64)
+        g = oracle_graph(n, edges, work, sizeparam, sizeout)
+        dg = bq.mtpp.SliceGraph(n, edges, work, sizeparam, sizeout, device="cuda:0")
+        P = 5
+        keys = torch.rand((P, n), generator=torch.Generator().manual_seed(case))
+        if case % 3 == 0:
+            keys = (keys * 3).floor() / 3                                    # many equal keys: the node index decides
+        orders = dg.decode_orders(keys.cuda())
+        B, M, k = rng.randrange(1, 9), rng.randrange(0, 2000), rng.choice([1, 2, 5, 16])
+        cost, blocks, cuts, status = dg.slice_orders(orders, k, B, M)
+        torch.cuda.synchronize()
+        for p in range(P):
+            pi = orders[p].cpu().tolist()
+            assert pi == mo.decode_order(g, keys[p].tolist())
+            assert (int(cost[p]), int(blocks[p]), cuts[p][:int(blocks[p])].cpu().tolist()) == mo.slice_order(g, pi, k, B, M), (case, p)
+        dg.close()
+
+
+def test_rows_that_are_not_topological_orders_are_flagged(bq):
+    n, edges, work, sizeparam, sizeout = workloads.make_graph("mtpp_tiny")
+    g = oracle_graph(n, edges, work, sizeparam, sizeout)
+    dg = bq.mtpp.SliceGraph(n, edges, work, sizeparam, sizeout, device="cuda:0")
+    good = mo.decode_order(g, [0.5] * n)
+    u, v = edges[0]
+    swapped = list(good)
+    iu, iv = swapped.index(u), swapped.index(v)
+    swapped[iu], swapped[iv] = swapped[iv], swapped[iu]                   # a consumer before its producer
+    twice = list(good); twice[3] = twice[4]
+    outside = list(good); outside[0] = n + 5
+    negative = list(good); negative[2] = -1
+    orders = torch.tensor([good, swapped, twice, outside, negative, good], dtype=torch.int32, device="cuda:0")
+    cost, blocks, cuts, status = dg.slice_orders(orders, 3, 2, 1000)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [0, 1, 1, 1, 1, 0]
+    assert cost.cpu().tolist()[1:5] == [-1] * 4 and blocks.cpu().tolist()[1:5] == [0] * 4 and not cuts[1:5].any()
+    want = mo.slice_order(g, good, 3, 2, 1000)
+    for p in (0, 5):
+        assert (int(cost[p]), int(blocks[p]), cuts[p][:int(blocks[p])].cpu().tolist()) == want
+    with pytest.raises(bq.BqError):
+        dg.slice_orders(orders, 17, 2, 1000)
+    with pytest.raises(bq.BqError):
+        dg.slice_orders(orders, 3, 0, 1000)
+    dg.close()

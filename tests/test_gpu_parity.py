@@ -157,6 +157,51 @@ def test_config_sweep1g_full_size(bq, gcb, cb):
     _whole_tensor(bq, gcb, cb, "sweep1g", [64, 256, 1024, 4096])
 
 
+# ------------------------------------------------------------------------------- blocks staged through shared memory
+
+@pytest.fixture
+def staging(bq):
+    """Blocks of 2048 / 4096 elements go through the kernel that stages them in shared memory with bulk
+    asynchronous copies; the default is restored afterwards."""
+    before = bq.set_staging(True)
+    try:
+        yield
+    finally:
+        bq.set_staging(before)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("block", [2048, 4096])
+@pytest.mark.parametrize("size", ["few", "medium", "large"])
+def test_staged_blocks_against_the_oracle(bq, gcb, cb, staging, dtype, block, size):
+    """A handful of blocks (fewer than teams), about a thousand, and enough for every ring to wrap many
+    times; a short last block that the general kernel takes; fp32 blocks of 4096 have no staged kernel
+    and must come out the same through the register kernel."""
+    g = torch.Generator().manual_seed(block + 3)
+    n = {"few": 2 * block, "medium": 1000 * block, "large": (1 << 23) + 300 * block}[size] + 37
+    x = (torch.randn(n, generator=g) * (1.0 + 30.0 * (torch.rand(n, generator=g) < 0.002))).to(dtype)
+    x[block:2 * block] = 0                                         # a zero block
+    check_all_ops(bq, gcb, cb, x, block)
+    assert bq.kernel_status(gcb) == 0
+
+
+def test_staged_config_moe_prefill_full_size(bq, gcb, cb, staging):
+    _whole_tensor(bq, gcb, cb, "moe_prefill", [2048])
+    assert bq.kernel_status(gcb) == 0
+
+
+def test_staged_scales_outside_the_reciprocal_window_and_in_place(bq, gcb, cb, staging):
+    g = torch.Generator().manual_seed(12)
+    x = torch.randn(2048 * 40, generator=g)
+    x[:2048 * 10] *= 1e-25                                        # absmax below 2^-64: the IEEE division
+    x[2048 * 10:2048 * 20] *= 1e25
+    check_all_ops(bq, gcb, cb, x.to(torch.bfloat16), 2048)
+    xd = x.to(torch.bfloat16).to("cuda:0")
+    bq.bq_roundtrip(xd, 2048, gcb, y_out=xd)                      # in place: a stage is read before its block's outputs are written
+    torch.cuda.synchronize()
+    assert np.array_equal(_bits(xd.cpu()), oracle.roundtrip(_bits(x.to(torch.bfloat16)), oracle.BF16, 2048, cb, oracle.BF16))
+
+
 # ------------------------------------------------------------------------------- shapes, tails, alignment
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.float16, torch.bfloat16])
@@ -233,25 +278,55 @@ def test_non_default_stream(bq, gcb, cb):
     assert np.array_equal(_bits(y.cpu()), oracle.roundtrip(_bits(x), oracle.F16, 64, cb, oracle.F16))
 
 
-def test_host_to_host_pipeline(bq, gcb, cb):
-    """The chunked three-stream path between pinned host tensors gives the same bytes; the
-    chunk is small here so that slots are reused several times and the last piece is short."""
-    x = workloads.make("prefill7b", rows=200).view(-1)[: 200 * 4096 - 256 * 3].contiguous()
-    n, block = x.numel(), 256
-    hb = bq.HostBoundary(gcb, torch.bfloat16, chunk=256 * 300, slots=3)
+@pytest.mark.parametrize("dtype,block,chunk", [(torch.bfloat16, 256, 256 * 300), (torch.float32, 64, 5000), (torch.float16, 4096, 4096 * 3 + 100)])
+def test_host_to_host_calls(bq, gcb, cb, dtype, block, chunk):
+    """bq_quantize_host / bq_dequantize_host / bq_roundtrip_host between pinned host tensors give the
+    oracle's bytes; the pieces are small here so that slots are reused several times, a piece is not
+    a multiple of the block (the library rounds it down) and the last piece and the last block are
+    short.  Calls are enqueued back to back: the dequantize reads what the quantize before it wrote."""
+    g = torch.Generator().manual_seed(block)
+    n = chunk * 7 + block * 2 + 13
+    x = (torch.randn(n, generator=g) * 3).to(dtype)
+    nb = (n + block - 1) // block
+    hb = bq.HostBoundary(gcb, dtype, chunk=chunk, slots=3, min_block=block)
     x_pin = x.pin_memory()
-    c_pin = torch.empty(n, dtype=torch.uint8).pin_memory()
-    a_pin = torch.empty(n // block, dtype=torch.float32).pin_memory()
-    y_pin = torch.empty(n, dtype=torch.bfloat16).pin_memory()
-    y2_pin = torch.empty(n, dtype=torch.bfloat16).pin_memory()
-    hb.quantize(x_pin, block, c_pin, a_pin)
-    torch.cuda.synchronize()
-    hb.dequantize(c_pin, a_pin, block, y_pin)
-    hb.roundtrip(x_pin, block, y2_pin)
-    torch.cuda.synchronize()
-    yr, cr, ar = oracle.roundtrip_sharded(_bits(x), oracle.BF16, block, cb, oracle.BF16, THREADS)
-    assert np.array_equal(c_pin.numpy(), cr) and np.array_equal(a_pin.numpy().view(np.uint32), ar.view(np.uint32))
+    c_pin = torch.full((n + 64,), CANARY, dtype=torch.uint8).pin_memory()
+    a_pin = torch.empty(nb, dtype=torch.float32).pin_memory()
+    y_pin = torch.empty(n, dtype=dtype).pin_memory()
+    y2_pin = torch.empty(n, dtype=dtype).pin_memory()
+    for _ in range(2):                                           # the second round reuses slots that are still draining
+        hb.quantize(x_pin, block, c_pin[:n], a_pin)
+        hb.dequantize(c_pin[:n], a_pin, block, y_pin)
+        hb.roundtrip(x_pin, block, y2_pin)
+    hb.wait()
+    yr, cr, ar = oracle.roundtrip_sharded(_bits(x), ODT[dtype], block, cb, ODT[dtype], THREADS)
+    assert np.array_equal(c_pin[:n].numpy(), cr) and bool((c_pin[n:] == CANARY).all())
+    assert np.array_equal(a_pin.numpy().view(np.uint32), ar.view(np.uint32))
     assert np.array_equal(_bits(y_pin), yr) and np.array_equal(_bits(y2_pin), yr)
+    # in place, and ordered behind the current stream's view of the pipe
+    x2 = x_pin.clone().pin_memory()
+    hb.roundtrip(x2, block, x2)
+    hb.wait_on_current_stream()
+    torch.cuda.current_stream().synchronize()
+    assert np.array_equal(_bits(x2), yr)
+    # what the pipe was not made for is refused before anything is enqueued
+    with pytest.raises(bq.BqError):
+        hb.roundtrip(x_pin, max(1, block // 2), y2_pin)           # below min_block
+    if dtype != torch.float32:
+        with pytest.raises(bq.BqError):
+            hb.roundtrip(x_pin.float(), block, y2_pin.float())    # wider than the staging
+    hb.close()
+
+
+def test_host_to_host_calls_from_pageable_memory(bq, gcb, cb):
+    x = workloads.make("prefill7b", rows=40).view(-1)
+    n, block = x.numel(), 256
+    hb = bq.HostBoundary(gcb, torch.bfloat16, chunk=256 * 100, slots=2, min_block=256)
+    y = torch.empty(n, dtype=torch.bfloat16)
+    hb.roundtrip(x, block, y)
+    hb.wait()
+    assert np.array_equal(_bits(y), oracle.roundtrip(_bits(x), oracle.BF16, block, cb, oracle.BF16))
+    hb.close()
 
 
 def test_non_finite_inputs_stay_in_bounds(bq, gcb, cb):
