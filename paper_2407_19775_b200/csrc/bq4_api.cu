@@ -3,6 +3,7 @@
 // of kernel.
 #include "../../include/bq4.h"
 #include "bq4_kernels.cuh"
+#include "bq_launch.h"
 #include "bq_error.h"
 
 #include <cmath>
@@ -135,23 +136,43 @@ void launch_q4_fast(int log2_lpb, bool folded, unsigned grid, cudaStream_t s, co
     else launch_q4_fast_f<DT, false, S16>(log2_lpb, grid, s, x, packed, absmax, nchunks, tab);
 }
 
+// Above this many elements the 8-bit path's persistent forward kernel, in its 4-bit flavour, takes the whole tiles (its
+// per-block scalars are computed once per block and its tiles keep eight chunks per thread in flight).
+constexpr size_t kFwd4MinElems = size_t(1) << 23;
+
 template <int DT, bool S16 = false>
 cudaError_t quantize_t(const void* x, size_t n, size_t B, const bq4k::Tables4& tab, uint8_t* packed, float* absmax, int sms, cudaStream_t s) {
     size_t done = 0;
     const int l2 = log2_exact(B);
+    constexpr size_t EB = (DT == bq4k::kF32) ? 4 : 2;
     if (l2 >= 3 && l2 <= 16 && aligned(x, 16) && aligned(packed, 4) && n >= B) {
         const size_t nblocks = n / B, n_full = nblocks * B;
-        if (l2 <= 8) {
-            const size_t nchunks = n_full / 8;
-            const unsigned grid = capped((nchunks + 511) / 512, size_t(sms) * 8);
-            launch_q4_fast<DT, S16>(l2 - 3, tab.folded != 0, grid, s, x, packed, absmax, nchunks, tab);
-        } else {
-            const unsigned grid = capped((nblocks + 7) / 8, size_t(sms) * 8);
-            if (tab.folded) bq4k::q4_wide<DT, true, S16><<<grid, 256, 0, s>>>(x, packed, absmax, nblocks, int(B / 8), tab);
-            else bq4k::q4_wide<DT, false, S16><<<grid, 256, 0, s>>>(x, packed, absmax, nblocks, int(B / 8), tab);
+        if (!S16 && DT != bq4k::kF32 && tab.folded && l2 >= 6 && l2 <= 12 && n_full > kFwd4MinElems && aligned(absmax, 4)) {
+            bqk::Tables4Fast fast;
+            std::memcpy(fast.entry, tab.entry, sizeof fast.entry);
+            fast.neg_limit = tab.neg_limit;
+            int dev = 0;
+            cudaError_t e = cudaGetDevice(&dev);
+            if (e == cudaSuccess) e = bql::launch_fwd4_fast(DT == bq4k::kF16 ? BQ_F16 : BQ_BF16, int(B), x, packed, absmax, n_full, fast, sms, dev, s, &done);
+            if (e != cudaSuccess) return e;
         }
-        cudaError_t e = cudaGetLastError();
-        if (e != cudaSuccess) return e;
+        if (done < n_full) {                                      // the whole blocks the tiles did not cover (all of them for small tensors)
+            const char* xr = static_cast<const char*>(x) + done * EB;
+            uint8_t* pr = packed + done / 2;
+            float* ar = S16 ? reinterpret_cast<float*>(reinterpret_cast<uint16_t*>(absmax) + done / B) : absmax + done / B;
+            const size_t rblocks = (n_full - done) / B;
+            if (l2 <= 8) {
+                const size_t nchunks = (n_full - done) / 8;
+                const unsigned grid = capped((nchunks + 511) / 512, size_t(sms) * 8);
+                launch_q4_fast<DT, S16>(l2 - 3, tab.folded != 0, grid, s, xr, pr, ar, nchunks, tab);
+            } else {
+                const unsigned grid = capped((rblocks + 7) / 8, size_t(sms) * 8);
+                if (tab.folded) bq4k::q4_wide<DT, true, S16><<<grid, 256, 0, s>>>(xr, pr, ar, rblocks, int(B / 8), tab);
+                else bq4k::q4_wide<DT, false, S16><<<grid, 256, 0, s>>>(xr, pr, ar, rblocks, int(B / 8), tab);
+            }
+            cudaError_t e = cudaGetLastError();
+            if (e != cudaSuccess) return e;
+        }
         done = n_full;
     }
     if (done < n) {

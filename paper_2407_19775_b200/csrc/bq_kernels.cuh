@@ -51,6 +51,22 @@ struct DeviceTables {
     float neg_limit;            // -(largest |xhat| whose negative key does not pass the last threshold)
 };
 
+// The 4-bit variant of the path (16 codes, two per byte) runs through the same forward kernel.  Its
+// folded table is small enough to travel in the kernel's parameters: cells of 2^21 keys from the
+// key of 2^-9 up, entry ((7 + P0) << 24 | 0xE00000 | (0x1FFFFF - (TK - S))) - S, so that the top byte
+// of entry + key is 7 + P (see bq4_kernels.cuh for the map and the table's construction).
+constexpr uint32_t kKeyLow4 = 0x76000000u;             // key of +2^-9
+constexpr uint32_t kCellBase4 = kKeyLow4 >> 21;
+constexpr int kCells4 = 73;
+struct Tables4Fast {
+    uint32_t entry[kCells4];
+    float neg_limit;
+};
+constexpr uint32_t kFwd4SmemBytes = uint32_t(kCells4) * 128u + 2u * 32u * 4u + 128u;
+constexpr uint32_t kRedOff4 = uint32_t(kCells4) * 128u;
+template <int BITS> struct TabArg { using type = DeviceTables; };
+template <> struct TabArg<4> { using type = Tables4Fast; };
+
 // ------------------------------------------------------------------------------------------
 // small helpers
 
@@ -174,6 +190,7 @@ struct Found {
 // tables straight from global memory through L1.
 template <bool LITE> struct TabRef;
 template <> struct TabRef<false> {
+    static constexpr uint32_t kLow = kKeyLow;
     uint32_t guess_lane;   // this lane's column of the entry table, rebased by the index of the first cell
     uint32_t cm_lane;      // this lane's column of the magnitude table, rebased by -127 rows
     __device__ __forceinline__ TabRef(const DeviceTables&, uint32_t sm_lane)
@@ -192,6 +209,7 @@ template <> struct TabRef<false> {
     }
 };
 template <> struct TabRef<true> {
+    static constexpr uint32_t kLow = kKeyLow;
     const uint32_t* guess;
     const float* cmag;
     __device__ __forceinline__ TabRef(const DeviceTables& t, uint32_t) : guess(t.guess - kCellBase), cmag(t.cmag - 127) {}
@@ -199,12 +217,24 @@ template <> struct TabRef<true> {
     __device__ __forceinline__ float magnitude(uint32_t sum) const { return __ldg(cmag + (sum >> 24)); }
 };
 
-template <bool LITE>
-__device__ __forceinline__ Found search_folded(float xhat, float neg_limit, const TabRef<LITE>& tab) {
+// the 4-bit table: per-lane copies in shared memory only (large tensors)
+struct TabRef4 {
+    static constexpr uint32_t kLow = kKeyLow4;
+    uint32_t guess_lane;
+    __device__ __forceinline__ TabRef4(uint32_t sm_lane) : guess_lane(sm_lane - kCellBase4 * 128u) {}
+    __device__ __forceinline__ uint32_t entry(uint32_t key) const {
+        uint32_t ga;
+        asm("mad.lo.u32 %0, %1, 128, %2;" : "=r"(ga) : "r"(key >> 21), "r"(guess_lane));
+        return lds_u32(ga);
+    }
+};
+
+template <class Tab>
+__device__ __forceinline__ Found search_folded(float xhat, float neg_limit, const Tab& tab) {
     Found f;
     xhat = fmaxf(xhat, neg_limit);
     f.bits = __float_as_uint(xhat);
-    const uint32_t key = max(__funnelshift_l(f.bits, f.bits, 1), kKeyLow);
+    const uint32_t key = max(__funnelshift_l(f.bits, f.bits, 1), Tab::kLow);
     f.sum = tab.entry(key) + key;
     return f;
 }
@@ -234,6 +264,19 @@ __device__ __forceinline__ uint32_t sign_mask_16(uint32_t w0, uint32_t w1) { ret
 // sign bytes of four fp32 elements
 __device__ __forceinline__ uint32_t sign_mask_32(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     return prmt(prmt(a, b, 0x00FBu), prmt(c, d, 0x00FBu), 0x5410u);
+}
+
+// Eight 4-bit codes as eight nibbles (element 2i in the low nibble of byte i).  The top bytes c = 7 + P of the
+// sums are gathered four to a word; negative elements (0xFF in `neg0` / `neg1`) take 7 - P = (c ^ 0xF) - 1, which
+// cannot borrow between bytes because c <= 14 there (the clamp keeps P <= 7 on that side), and the "-1 in every
+// negative byte" is neg * 0x01010101 as in pack_codes; then byte pairs fold into nibble pairs: x | x >> 4 leaves
+// [q1 q0] in byte 0 and [q3 q2] in byte 2.
+__device__ __forceinline__ uint32_t pack_nibbles8(const uint32_t (&sum)[8], uint32_t neg0, uint32_t neg1) {
+    uint32_t c0 = prmt(prmt(sum[0], sum[1], 0x0073u), prmt(sum[2], sum[3], 0x0073u), 0x5410u);
+    uint32_t c1 = prmt(prmt(sum[4], sum[5], 0x0073u), prmt(sum[6], sum[7], 0x0073u), 0x5410u);
+    asm("mad.lo.u32 %0, %1, 0x01010101, %2;" : "=r"(c0) : "r"(neg0), "r"(c0 ^ (neg0 & 0x0F0F0F0Fu)));
+    asm("mad.lo.u32 %0, %1, 0x01010101, %2;" : "=r"(c1) : "r"(neg1), "r"(c1 ^ (neg1 & 0x0F0F0F0Fu)));
+    return prmt(c0 | (c0 >> 4), c1 | (c1 >> 4), 0x6420u);
 }
 
 // Two fp32 lanes per instruction (sm_100 packed fp32 arithmetic).
@@ -328,10 +371,14 @@ __device__ __forceinline__ float rcp_approx(float d) {
 // rounding boundary, and never sits on one.  The CPU tests check every significand pair
 // with r perturbed by +-2 ulp.  Outside that window, and for fp32 inputs, the IEEE division
 // is used.
-template <int XDT, int B, int R, int TW, bool WRITE_Y, bool WRITE_Q, int NT, bool LITE>
+//   BITS         8: the 256-entry codebook, one code per byte.  4: the 16-entry codebook of the 4-bit variant, two
+//                codes per byte (quantize only, 16-bit inputs, the shared-memory flavour); everything up to
+//                the search is the same code.
+template <int XDT, int B, int R, int TW, bool WRITE_Y, bool WRITE_Q, int NT, bool LITE, int BITS = 8>
 __global__ void __launch_bounds__(NT, 1)
 fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__ codes, float* __restrict__ absmax_out,
-         size_t ntiles, DeviceTables tab) {
+         size_t ntiles, const __grid_constant__ typename TabArg<BITS>::type tab) {
+    static_assert(BITS == 8 || (BITS == 4 && !WRITE_Y && WRITE_Q && !LITE && Elem<XDT>::kPerChunk == 8), "the 4-bit flavour: quantize, 16-bit inputs, tables in shared memory");
     constexpr int EPC = Elem<XDT>::kPerChunk;
     constexpr int EB = Elem<XDT>::kBytes;
     constexpr int ROW = 32 * EPC;
@@ -347,10 +394,17 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
     const uint32_t sm_base = (uint32_t(__cvta_generic_to_shared(smem_raw)) + 127u) & ~127u;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t sm_lane = sm_base + uint32_t(lane) * 4u;
-    const TabRef<LITE> tref(tab, sm_lane);
-    constexpr uint32_t RED = LITE ? 0u : kRedOff;
+    auto make_tref = [&]() {
+        if constexpr (BITS == 4) return TabRef4(sm_lane);
+        else return TabRef<LITE>(tab, sm_lane);
+    };
+    const auto tref = make_tref();
+    constexpr uint32_t RED = (BITS == 4) ? kRedOff4 : (LITE ? 0u : kRedOff);
 
-    if constexpr (!LITE) {
+    if constexpr (BITS == 4) {
+        for (int i = threadIdx.x; i < kCells4 * 32; i += NT) sts_u32(sm_base + uint32_t(i) * 4u, tab.entry[i >> 5]);     // every entry once per lane
+        __syncthreads();
+    } else if constexpr (!LITE) {
         fill_fwd_tables<NT>(tab, sm_base);
         __syncthreads();
     }
@@ -524,7 +578,10 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
             {
                 if constexpr (WRITE_Y) stg_stream_16(yb + off * EB, narrow_chunk<XDT>(out));
                 if constexpr (WRITE_Q) {
-                    if constexpr (EPC == 8) {
+                    if constexpr (BITS == 4) {
+                        const uint32_t sums[8] = {fd[0].sum, fd[1].sum, fd[2].sum, fd[3].sum, fd[4].sum, fd[5].sum, fd[6].sum, fd[7].sum};
+                        stg_stream_4(codes + off / 2, pack_nibbles8(sums, neg[r][0], neg[r][1]));
+                    } else if constexpr (EPC == 8) {
                         stg_stream_8(codes + off, make_uint2(pack_codes(fd[0], fd[1], fd[2], fd[3], neg[r][0]), pack_codes(fd[4], fd[5], fd[6], fd[7], neg[r][1])));
                     } else {
                         stg_stream_4(codes + off, pack_codes(fd[0], fd[1], fd[2], fd[3], neg[r][0]));

@@ -254,3 +254,18 @@ def test_scale16_is_close_to_the_fp32_scale(bq):
     y = bq.bq4_dequantize_s16(p, s, x.numel(), block, cb, torch.float32)
     err = (x.float() - y).abs().view(-1, block) / sf.clamp_min(1e-30)[:, None]
     assert float(err.max()) <= 0.1125 * (1 + 1e-5)
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
+@pytest.mark.parametrize("block", [64, 128, 256, 512, 1024, 2048, 4096])
+def test_large_tensors_through_the_tiled_forward_kernel(bq, dtype, block):
+    """Above 8 Mi elements the whole tiles go through the persistent forward kernel of the 8-bit path in its 4-bit flavour, the
+    whole blocks left over through the 4-bit kernels, and a short last block through the general ones; packed bytes, absmax and
+    the dequantised tensor must be the oracle's."""
+    g = torch.Generator().manual_seed(block + 1)
+    n = (1 << 23) + 5 * 24576 + 3 * block + 37                    # whole tiles, then whole blocks, then a short block
+    x = (torch.randn(n, generator=g) * (1.0 + 30.0 * (torch.rand(n, generator=g) < 0.002))).to(dtype)
+    x[block:2 * block] = 0
+    x[7 * block] = -x[7 * block:8 * block].float().abs().max() * 2  # the absmax element is negative: xhat = -1 has no code of its own
+    x[9 * block + 1] = -0.0
+    check(bq, x, block, ydt=dtype)
