@@ -762,15 +762,14 @@ def run_mmd(bq, dev, args):
 
 DECODE_LAYER_COPIES = 4
 
-# DRAM bytes per full-size launch (dram__bytes_read.sum + dram__bytes_write.sum), from ncu
-# captures of the first 8192 rows scaled to 65536 rows: reads scale with the rows (they equal
-# the algorithmic bytes to 0.04 %); writes are the algorithmic bytes minus the 40-58 MB of
-# dirty lines that are still in L2 when the kernel ends, a size-independent residue measured
-# in the same capture.  Set an entry to None when its kernel changes until it is re-measured.
+# DRAM bytes per full-size launch (dram__bytes_read.sum + dram__bytes_write.sum): a one-pass ncu capture of the twelve full-size
+# launches of a step on the current binary (profiles/bench_sweep1g_dram_traffic_full_size.md).  Reads equal the algorithmic input
+# bytes to 0.03 %; writes fall short of the algorithmic output bytes by the dirty lines still in L2 when the kernel ends.  Set an
+# entry to None when its kernel changes until it is re-measured.
 TRAFFIC_BYTES = {
-    "quantize_b64": None, "quantize_b256": None, "quantize_b1024": None, "quantize_b4096": None,
-    "dequantize_b64": None, "dequantize_b256": None, "dequantize_b1024": None, "dequantize_b4096": None,
-    "roundtrip_b64": None, "roundtrip_b256": None, "roundtrip_b1024": None, "roundtrip_b4096": None,
+    "quantize_b64": 1587277568, "quantize_b256": 1562487040, "quantize_b1024": 1572259072, "quantize_b4096": 1574788608,
+    "dequantize_b64": 1582605568, "dequantize_b256": 1557005056, "dequantize_b1024": 1550627840, "dequantize_b4096": 1549636096,
+    "roundtrip_b64": 2094978560, "roundtrip_b256": 2095579904, "roundtrip_b1024": 2094396416, "roundtrip_b4096": 2094418944,
 }
 
 

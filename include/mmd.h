@@ -59,8 +59,13 @@ enum {
     MMD_PATH_TENSOR = 2,   /* a tcgen05 kernel; needs N % 8 == 0 and 16-byte aligned Y: the persistent CTA-pair
                               kernel for large products with at most 16 critical features, else one tile per CTA */
     MMD_PATH_TENSOR_TILE = 3, /* the one-tile-per-CTA tcgen05 kernel, whatever the size                */
-    MMD_PATH_TENSOR_SOLO = 4  /* the persistent kernel without CTA pairs (same limits as the pair kernel; MMD_ERR_PATH
+    MMD_PATH_TENSOR_SOLO = 4, /* the persistent kernel without CTA pairs (same limits as the pair kernel; MMD_ERR_PATH
                                  when the product is too small or has more than 16 critical features) */
+    MMD_PATH_TENSOR_STREAMK = 5 /* the decode-step kernel that deals the K steps of all tiles out over one CTA per SM: at most 64
+                                 rows, K a multiple of 128 and at least 2048, N >= 1024, fewer 128-column tiles than SMs
+                                 (MMD_ERR_PATH otherwise) and a workspace of mmd_workspace_bytes_streamk bytes
+                                 (MMD_ERR_WORKSPACE otherwise).  Only on request: measured slower than the cluster split that
+                                 AUTO uses for such calls (the partial sums cross global memory instead of shared memory). */
 };
 
 /* Opaque: the decomposed weights of one linear layer (int8 rows, row scales, 16-bit side
@@ -110,6 +115,14 @@ int mmd_weights_view(const mmd_weights* w, const int8_t** q, const float** scale
  * workspace, and its total size.  Host only.  offsets3 may be NULL.
  */
 int mmd_workspace_layout(const mmd_weights* w, int M, size_t* offsets3, size_t* total_bytes);
+
+/*
+ * mmd_workspace_bytes_streamk -- the size of a workspace that also lets mmd_linear take its decode-step kernel for
+ * M rows (MMD_PATH_TENSOR_STREAMK): mmd_workspace_layout's total plus, behind it, one counter per 128-column tile and the
+ * slots through which CTAs that share a tile hand over their partial sums (a few MB for an 8192 x 8192 layer).  Equal to
+ * mmd_workspace_layout's total for shapes that kernel does not take.  Host only.
+ */
+int mmd_workspace_bytes_streamk(const mmd_weights* w, int M, size_t* total_bytes);
 
 /*
  * mmd_linear -- Y = X W^T through the decomposition: one row kernel over X into the

@@ -69,7 +69,7 @@ bool make_map_kblocks(CUtensorMap* map, const void* base, uint64_t rows, uint64_
 
 template <int DT>
 cudaError_t launch_rowquant(const void* v, int R, int K, const int32_t* idx, int ko, int8_t* q, float* scale, void* side, int sm_count,
-                            cudaStream_t stream) {
+                            cudaStream_t stream, int* zero_words = nullptr, int n_zero_words = 0) {
     const size_t smem = round_up(size_t(K) / 8, 4);
     if (smem > 48 * 1024) return cudaErrorInvalidValue;          // K <= kMaxK keeps the mask within the default limit
     int grid = R;
@@ -88,13 +88,13 @@ cudaError_t launch_rowquant(const void* v, int R, int K, const int32_t* idx, int
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int side_cols = mmd_side_columns(ko);
-    return cudaLaunchKernelEx(&cfg, mmdk::rowquant<DT>, v, R, K, idx, ko, side_cols, q, scale, side);
+    return cudaLaunchKernelEx(&cfg, mmdk::rowquant<DT>, v, R, K, idx, ko, side_cols, q, scale, side, zero_words, n_zero_words);
 }
 
 cudaError_t rowquant_any(int dt, const void* v, int R, int K, const int32_t* idx, int ko, int8_t* q, float* scale, void* side, int sm_count,
-                         cudaStream_t stream) {
-    return dt == BQ_BF16 ? launch_rowquant<mmdk::kBF16>(v, R, K, idx, ko, q, scale, side, sm_count, stream)
-                         : launch_rowquant<mmdk::kF16>(v, R, K, idx, ko, q, scale, side, sm_count, stream);
+                         cudaStream_t stream, int* zero_words = nullptr, int n_zero_words = 0) {
+    return dt == BQ_BF16 ? launch_rowquant<mmdk::kBF16>(v, R, K, idx, ko, q, scale, side, sm_count, stream, zero_words, n_zero_words)
+                         : launch_rowquant<mmdk::kF16>(v, R, K, idx, ko, q, scale, side, sm_count, stream, zero_words, n_zero_words);
 }
 
 int check_features(const int32_t* idx_host, int ko, int K) {
@@ -285,6 +285,78 @@ cudaError_t launch_tc2(const mmd_weights* w, const CUtensorMap& mqx, const float
     return cudaGetLastError();
 }
 
+// One row of tiles (a decode step of at most 64 rows) with the K steps of all tiles dealt out over one CTA per SM: the
+// shape must have fewer 128-column tiles than SMs (so that a CTA's share touches at most two tiles) and the caller's
+// workspace must have room, behind the decomposed activations, for the tiles' counters and partial sums.
+struct SkPlan {
+    bool ok;
+    int n_tiles, grid, maxparts;
+    size_t counters, acc, side, total;                     // offsets behind the base workspace, and the extra bytes
+};
+
+SkPlan sk_plan(const mmd_weights* w, int M) {
+    SkPlan p = {};
+    if (!w->have_maps || !w->have_pair_map || M < 1 || M > 64 || w->N < 1024 || w->N % 8 != 0) return p;
+    p.n_tiles = (w->N + 127) / 128;
+    if (p.n_tiles >= w->sm_count) return p;
+    const long long ksteps = ((w->K + 127) / 128 + 1) / 2, upt = ksteps + (w->side_cols > 0 ? 1 : 0);
+    const long long total = (long long)p.n_tiles * upt;
+    if (ksteps < 8) return p;                              // too few steps per tile to be worth sharing
+    const long long G = total < w->sm_count ? total : w->sm_count;
+    p.grid = int(G);
+    for (int t = 0; t < p.n_tiles; ++t) {
+        const long long ta = (long long)t * upt, tb = ta + upt;
+        const int c_first = int(((ta + 1) * G + total - 1) / total) - 1, c_last = int((tb * G + total - 1) / total) - 1;
+        if (c_last - c_first + 1 > p.maxparts) p.maxparts = c_last - c_first + 1;
+    }
+    const size_t tile_values = size_t(64) * 128;
+    p.counters = 0;
+    p.acc = round_up(size_t(p.n_tiles) * 4, kWsAlign);
+    p.side = p.acc + round_up(size_t(p.n_tiles) * p.maxparts * tile_values * 4, kWsAlign);
+    p.total = p.side + (w->side_cols > 0 ? round_up(size_t(p.n_tiles) * tile_values * 4, kWsAlign) : 0);
+    p.ok = true;
+    return p;
+}
+
+template <int XDT, int YDT>
+cudaError_t launch_sk(const mmd_weights* w, const SkPlan& p, const int8_t* qx, const void* sidex, const float* sx, void* y, int M, char* extra,
+                      cudaStream_t stream) {
+    using Cfg = mmdk::TcCfg<mmdk::kSkBN, mmdk::kSkBM, mmdk::kSkKPB>;
+    static bool opted[kMaxDevices] = {};
+    if (w->device < 0 || w->device >= kMaxDevices) return cudaErrorInvalidDevice;
+    {
+        std::lock_guard<std::mutex> guard(g_cache_lock);
+        if (!opted[w->device]) {
+            const cudaError_t e = cudaFuncSetAttribute(mmdk::gemm_sk<XDT, YDT>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::kSmemBytes));
+            if (e != cudaSuccess) return e;
+            opted[w->device] = true;
+        }
+    }
+    CUtensorMap mqx, mqw, msx;
+    if (!make_map_kblocks(&mqx, qx, uint64_t(M), uint64_t(w->K), 64, mmdk::kSkKPB)) return cudaErrorInvalidValue;
+    if (!make_map_kblocks(&mqw, w->q, uint64_t(w->N), uint64_t(w->K), mmdk::kSkBN, mmdk::kSkKPB)) return cudaErrorInvalidValue;
+    if (w->side_cols > 0) {
+        if (!make_map(&msx, sidex, 2, uint64_t(M), uint64_t(w->side_cols), 64)) return cudaErrorInvalidValue;
+    } else {
+        msx = mqx;
+    }
+    const int slot = bn_slot(mmdk::kSkBN);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(unsigned(p.grid), 1, 1);
+    cfg.blockDim = dim3(mmdk::kTcThreads, 1, 1);
+    cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // starts under the row kernel; waits for it before reading its results
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, mmdk::gemm_sk<XDT, YDT>, mqx, mqw, msx, w->side_cols > 0 ? w->map_side[slot] : w->map_q[slot], sx,
+                              static_cast<const float*>(w->scale), y, M, w->N, (w->K + 127) / 128, w->side_cols / 64, p.n_tiles, p.maxparts,
+                              reinterpret_cast<int*>(extra + p.counters), reinterpret_cast<int*>(extra + p.acc),
+                              reinterpret_cast<float*>(extra + p.side), w->status);
+}
+
 // Large products with few critical features take the persistent kernels.
 bool wants_persistent(const mmd_weights* w, int M) {
     // from about half a wave of 128 x 256 tiles on: below that the one-tile-per-CTA kernel's narrower tiles fill the SMs better.
@@ -459,12 +531,20 @@ int mmd_workspace_layout(const mmd_weights* w, int M, size_t* offsets3, size_t* 
     return BQ_OK;
 }
 
+int mmd_workspace_bytes_streamk(const mmd_weights* w, int M, size_t* total_bytes) {
+    if (!w || !total_bytes) return BQ_ERR_NULL;
+    if (M < 0) return BQ_ERR_SIZE;
+    const SkPlan p = sk_plan(w, M);
+    *total_bytes = ws_layout(w, M).total + (p.ok ? p.total : 0);
+    return BQ_OK;
+}
+
 int mmd_linear(const mmd_weights* w, const void* X, int M, void* Y, bq_dtype ydt, void* workspace, size_t workspace_bytes, int path,
                void* cuda_stream) {
     if (!w) return BQ_ERR_NULL;
     if (ydt != BQ_F32 && int(ydt) != w->dtype) return BQ_ERR_DTYPE;
     if (M < 0) return BQ_ERR_SIZE;
-    if (path < MMD_PATH_AUTO || path > MMD_PATH_TENSOR_SOLO) return MMD_ERR_PATH;
+    if (path < MMD_PATH_AUTO || path > MMD_PATH_TENSOR_STREAMK) return MMD_ERR_PATH;
     if (M == 0) return BQ_OK;
     if (!X || !Y) return BQ_ERR_NULL;
     if (!aligned(X, 16)) return BQ_ERR_SIZE;
@@ -477,17 +557,27 @@ int mmd_linear(const mmd_weights* w, const void* X, int M, void* Y, bq_dtype ydt
     const bool use_tc = (path >= MMD_PATH_TENSOR) || (path == MMD_PATH_AUTO && tc_ok);
     const bool persistent = use_tc && path != MMD_PATH_TENSOR_TILE && wants_persistent(w, M);
     const bool pairs = persistent && path != MMD_PATH_TENSOR_SOLO && w->have_pair_map;      // the pair kernel's loads need K % 128 == 0
+    // a decode step over a layer with fewer tiles than SMs, on request: all tiles' K steps over one CTA per SM.  Not taken by
+    // AUTO: as measured, handing partial sums over through global memory costs more than the even shares save.
+    const SkPlan sk = (use_tc && !persistent && path == MMD_PATH_TENSOR_STREAMK) ? sk_plan(w, M) : SkPlan{};
+    const bool stream_k = sk.ok && workspace_bytes >= L.total + sk.total;
+    if (path == MMD_PATH_TENSOR_STREAMK && !stream_k) return sk.ok ? MMD_ERR_WORKSPACE : MMD_ERR_PATH;
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     char* ws = static_cast<char*>(workspace);
     int8_t* qx = reinterpret_cast<int8_t*>(ws + L.q);
     float* sx = reinterpret_cast<float*>(ws + L.scale);
     void* sidex = ws + L.side;
-    cudaError_t e = rowquant_any(w->dtype, X, M, w->K, w->idx, w->ko, qx, sx, sidex, w->sm_count, stream);
+    cudaError_t e = rowquant_any(w->dtype, X, M, w->K, w->idx, w->ko, qx, sx, sidex, w->sm_count, stream,
+                                 stream_k ? reinterpret_cast<int*>(ws + L.total + sk.counters) : nullptr, stream_k ? sk.n_tiles : 0);
     if (e != cudaSuccess) return cuda_fail(e);
 
     const bool bf = (w->dtype == BQ_BF16), f32out = (ydt == BQ_F32);
-    if (pairs) {
+    if (stream_k) {
+        char* extra = ws + L.total;
+        if (bf) e = f32out ? launch_sk<mmdk::kBF16, mmdk::kF32>(w, sk, qx, sidex, sx, Y, M, extra, stream) : launch_sk<mmdk::kBF16, mmdk::kBF16>(w, sk, qx, sidex, sx, Y, M, extra, stream);
+        else e = f32out ? launch_sk<mmdk::kF16, mmdk::kF32>(w, sk, qx, sidex, sx, Y, M, extra, stream) : launch_sk<mmdk::kF16, mmdk::kF16>(w, sk, qx, sidex, sx, Y, M, extra, stream);
+    } else if (pairs) {
         CUtensorMap mqx;
         if (!make_map_kblocks(&mqx, qx, uint64_t(M), uint64_t(w->K), 128, mmdk::kPairStepBlocks)) return MMD_ERR_PATH;
         if (bf) e = f32out ? launch_tc2<mmdk::kBF16, mmdk::kF32>(w, mqx, sx, sidex, Y, M, stream) : launch_tc2<mmdk::kBF16, mmdk::kBF16>(w, mqx, sx, sidex, Y, M, stream);

@@ -101,7 +101,8 @@ __device__ __forceinline__ uint32_t rq_keep_bytes(uint32_t mk, int h) {
 template <int DT>
 __global__ void __launch_bounds__(256, 6)                        // six CTAs per SM: the row's second read then mostly hits L1 / L2 while others load
 rowquant(const void* __restrict__ v, int R, int K, const int32_t* __restrict__ idx, int ko, int side_cols,
-         int8_t* __restrict__ q_out, float* __restrict__ scale_out, void* __restrict__ side_out) {
+         int8_t* __restrict__ q_out, float* __restrict__ scale_out, void* __restrict__ side_out,
+         int* __restrict__ zero_words, int n_zero_words /* counters of the product kernel that follows; may be none */) {
     extern __shared__ __align__(16) unsigned char mask[];       // K / 8 bytes
     __shared__ uint32_t red[8];
     // A product kernel launched behind this one with programmatic stream serialization may start its set-up and its
@@ -115,6 +116,8 @@ rowquant(const void* __restrict__ v, int R, int K, const int32_t* __restrict__ i
     // call may still be reading the buffers written below).
     asm volatile("griddepcontrol.wait;" ::: "memory");
     __syncthreads();
+    if (blockIdx.x == 0)
+        for (int j = threadIdx.x; j < n_zero_words; j += 256) zero_words[j] = 0;
     for (int j = threadIdx.x; j < ko; j += 256) {
         const int k = idx[j];
         atomicOr(reinterpret_cast<uint32_t*>(mask) + (k >> 5), 1u << (k & 31));
@@ -675,6 +678,313 @@ gemm_tc(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUte
     }
 }
 
+
+// ------------------------------------------------------------------------------------------
+// gemm_sk: one row of tiles (a decode step, at most 64 activation rows) with the K steps of ALL
+// tiles dealt out evenly over the CTAs of one launch ("stream K").
+//
+// gemm_tc gives every 128-column tile to one CTA, or to a cluster of 2-4 CTAs that share its K
+// steps; with 64 tiles on 148 SMs either 84 SMs stream weights or 128 do.  Here the units of
+// work (per tile: its int8 steps of two K blocks, then one unit for all of its side steps) are
+// numbered across the tiles and CTA c takes units [c T / G, (c + 1) T / G): every SM streams the
+// same number of bytes, whatever the number of tiles.  A CTA's range touches at most two tiles
+// (the host launches at least as many CTAs as tiles); the part of a tile that a CTA computes is a
+// "segment", accumulated in its own half of tensor memory, so the epilogue of the first segment
+// runs under the loads and MMAs of the second.
+//
+// Tiles that several CTAs share are put together without anybody waiting: a CTA writes its
+// segment's int32 sums (and, if it holds the tile's side unit, the fp32 side sums) to a slot of
+// global scratch, fences, and takes a ticket from the tile's counter; the CTA whose ticket is
+// the last one adds the other slots to its own sums, which are still in its tensor memory, and
+// runs the epilogue.  Integer sums do not depend on the order and the side sums come from one
+// CTA, so the result is the same bits as gemm_tc's.  The counters are zeroed by the row kernel
+// that runs before every product.  Waits are bounded as in gemm_tc.
+constexpr int kSkBN = 128, kSkBM = 64, kSkKPB = 2;
+
+template <int XDT, int YDT>
+__global__ void __launch_bounds__(kTcThreads, 1)
+gemm_sk(const __grid_constant__ CUtensorMap map_qx, const __grid_constant__ CUtensorMap map_qw,
+        const __grid_constant__ CUtensorMap map_sidex, const __grid_constant__ CUtensorMap map_sidew,
+        const float* __restrict__ sx, const float* __restrict__ sw, void* __restrict__ y,
+        int M, int N, int kblocks_all, int sblocks_all, int n_tiles, int maxparts,
+        int* __restrict__ counters, int* __restrict__ part_acc, float* __restrict__ part_side, int* status) {
+    using Cfg = TcCfg<kSkBN, kSkBM, kSkKPB>;
+    constexpr int BN = kSkBN, BM = kSkBM, KPB = kSkKPB, S = Cfg::kStages;
+    constexpr uint32_t kTxMain = Cfg::kStageBytes;
+    constexpr uint32_t kTxSide = Cfg::kASlabBytes + Cfg::kBSlabBytes;
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* ctrl = smem_raw + (tiles - smem_u32(smem_raw)) + S * Cfg::kStageBytes;
+    const uint32_t full0 = smem_u32(ctrl);                                      // S barriers: tile landed
+    const uint32_t empty0 = full0 + 8u * S;                                     // S barriers: tile consumed
+    const uint32_t accbar0 = empty0 + 8u * S;                                   // 2 barriers: a segment's accumulators complete
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl + 8 * (2 * S + 2));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 8 * (2 * S + 2) + 8);
+    volatile int* ticket = reinterpret_cast<volatile int*>(ctrl + 8 * (2 * S + 2) + 12);
+    static_assert(8 * (2 * S + 2) + 16 <= 256, "control words end before the column scales");
+    float* sw_s = reinterpret_cast<float*>(ctrl + 256);                         // 2 x BN scales: one set per segment
+
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ksteps = (kblocks_all + KPB - 1) / KPB;
+    const int upt = ksteps + (sblocks_all > 0 ? 1 : 0);                         // units per tile
+    const long long total = (long long)n_tiles * upt;
+    const long long G = gridDim.x, c = blockIdx.x;
+    const long long lo = total * c / G, hi = total * (c + 1) / G;               // this CTA's units
+    const int t_first = int(lo / upt), t_last = int((hi - 1) / upt);
+    const int nseg = (hi > lo) ? t_last - t_first + 1 : 0;                      // 0, 1 or 2
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, 1); }
+        mbar_init(accbar0, 1);
+        mbar_init(accbar0 + 8u, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = *tmem_slot;
+
+    // ring steps of a unit: an int8 unit is one step, the side unit is sblocks_all steps
+    auto steps_of = [&](long long g) -> int { return (int(g % upt) < ksteps) ? 1 : sblocks_all; };
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // The loads of one ring step: `side` < 0 is int8 step `kstep` of tile `t`, otherwise side step `side`.
+            auto issue_b = [&](int s, int t, int kstep, int side) {
+                const uint32_t b_dst = tiles + uint32_t(s) * Cfg::kStageBytes + Cfg::kABytes;
+                if (side < 0) tma_load_3d(b_dst, &map_qw, t * BN, kstep * KPB, full0 + 8u * s);
+                else tma_load_2d(b_dst, &map_sidew, side * 64, t * BN, full0 + 8u * s);
+            };
+            auto issue_a = [&](int s, int kstep, int side) {
+                const uint32_t a_dst = tiles + uint32_t(s) * Cfg::kStageBytes;
+                if (side < 0) tma_load_3d(a_dst, &map_qx, 0, kstep * KPB, full0 + 8u * s);
+                else tma_load_2d(a_dst, &map_sidex, side * 64, 0, full0 + 8u * s);
+            };
+            // The first ring-full of weight tiles does not depend on the row kernel before this one.
+            int it = 0;
+            bool waited = false, ok = true;
+            int pre_t[S], pre_k[S], pre_side[S], npre = 0;
+            for (long long g = lo; g < hi && ok; ++g) {
+                const int t = int(g / upt), u = int(g % upt);
+                const int nst = steps_of(g);
+                for (int j = 0; j < nst && ok; ++j, ++it) {
+                    const int s = it % S;
+                    const int kstep = (u < ksteps) ? u : 0, side = (u < ksteps) ? -1 : j;
+                    if (it < S) {                                                    // ring not yet wrapped: weights now, activations after the wait
+                        mbar_expect_tx(full0 + 8u * s, side < 0 ? kTxMain : kTxSide);
+                        issue_b(s, t, kstep, side);
+                        pre_t[npre] = t; pre_k[npre] = kstep; pre_side[npre] = side; ++npre;
+                        continue;
+                    }
+                    if (!waited) {
+                        asm volatile("griddepcontrol.wait;" ::: "memory");
+                        for (int q = 0; q < npre; ++q) issue_a(q, pre_k[q], pre_side[q]);
+                        waited = true;
+                    }
+                    ok = mbar_wait(empty0 + 8u * s, ((uint32_t(it / S) & 1u) ^ 1u), abort_flag, status, 1);
+                    if (!ok) break;
+                    mbar_expect_tx(full0 + 8u * s, side < 0 ? kTxMain : kTxSide);
+                    issue_a(s, kstep, side);
+                    issue_b(s, t, kstep, side);
+                }
+            }
+            if (!waited) {
+                asm volatile("griddepcontrol.wait;" ::: "memory");
+                for (int q = 0; q < npre; ++q) issue_a(q, pre_k[q], pre_side[q]);
+            }
+            (void)pre_t;
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc_i8 = umma_idesc(2, 1, BM, BN);
+            constexpr uint32_t idesc_16 = umma_idesc(1, XDT == kBF16 ? 1u : 0u, BM, BN);
+            int it = 0;
+            bool ok = true;
+            for (int seg = 0; seg < nseg && ok; ++seg) {
+                const int t = t_first + seg;
+                const long long a = (lo > (long long)t * upt) ? lo : (long long)t * upt;
+                const long long b = (hi < (long long)(t + 1) * upt) ? hi : (long long)(t + 1) * upt;
+                const uint32_t tm = tmem + uint32_t(seg & 1) * 256u;
+                bool first_i8 = true, first_side = true;
+                for (long long g = a; g < b && ok; ++g) {
+                    const int u = int(g % upt);
+                    const int nst = steps_of(g);
+                    for (int j = 0; j < nst && ok; ++j, ++it) {
+                        const int s = it % S;
+                        ok = mbar_wait(full0 + 8u * s, uint32_t(it / S) & 1u, abort_flag, status, 2);
+                        if (!ok) break;
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                        const uint32_t a_src = tiles + uint32_t(s) * Cfg::kStageBytes, b_src = a_src + Cfg::kABytes;
+                        if (u < ksteps) {
+#pragma unroll
+                            for (int jj = 0; jj < KPB; ++jj) {
+                                const uint64_t aj = umma_smem_desc(a_src + uint32_t(jj) * Cfg::kASlabBytes), bj = umma_smem_desc(b_src + uint32_t(jj) * Cfg::kBSlabBytes);
+#pragma unroll
+                                for (int k = 0; k < 4; ++k)
+                                    umma_i8(tm, aj + uint64_t(2 * k), bj + uint64_t(2 * k), idesc_i8, (first_i8 && jj == 0 && k == 0) ? 0u : 1u);
+                            }
+                            first_i8 = false;
+                        } else {
+                            const uint64_t adesc = umma_smem_desc(a_src), bdesc = umma_smem_desc(b_src);
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)
+                                umma_f16(tm + uint32_t(BN), adesc + uint64_t(2 * k), bdesc + uint64_t(2 * k), idesc_16, (first_side && k == 0) ? 0u : 1u);
+                            first_side = false;
+                        }
+                        umma_commit(empty0 + 8u * s);
+                    }
+                }
+                if (ok) umma_commit(accbar0 + 8u * uint32_t(seg & 1));
+            }
+        }
+        __syncwarp();
+    } else {
+        // epilogue: 128 threads; a 64-row accumulator keeps rows 16 q .. 16 q + 15 in the first 16 lanes of quarter q
+        const int et = threadIdx.x - 64;
+        const int quarter = warp & 3;
+        const bool row_lane = lane < 16;
+        const int m = row_lane ? quarter * 16 + lane : M;
+        asm volatile("griddepcontrol.wait;" ::: "memory");       // row scales and the zeroed counters come from the kernel before this one
+        const float sxm = (m < M) ? sx[m] : 0.0f;
+        const uint32_t row_in_tile = uint32_t(quarter * 16 + lane);
+        constexpr size_t kPart = size_t(BM) * BN;                                // values of one partial tile, stored [row][column]
+        for (int seg = 0; seg < nseg; ++seg) {
+            const int t = t_first + seg;
+            const int n0 = t * BN;
+            const long long ta = (long long)t * upt, tb = (long long)(t + 1) * upt;
+            const long long a = lo > ta ? lo : ta, b = hi < tb ? hi : tb;
+            const bool has_side = sblocks_all > 0 && b == tb;                    // the side unit is the tile's last
+            const bool has_i8 = a < ta + ksteps;                                 // a segment of the side unit alone has no integer sums
+            const int c_first = int(((ta + 1) * G + total - 1) / total) - 1, c_last = int((tb * G + total - 1) / total) - 1;
+            const int parts = c_last - c_first + 1, mypart = int(c) - c_first;
+            float* sws = sw_s + (seg & 1) * BN;
+            for (int cc = et; cc < BN; cc += 128) sws[cc] = (n0 + cc < N) ? sw[n0 + cc] : 0.0f;
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            bool ok = true;
+            if (lane == 0) ok = mbar_wait(accbar0 + 8u * uint32_t(seg & 1), 0, abort_flag, status, 3);
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t lane_base = tmem + uint32_t(seg & 1) * 256u + (uint32_t(quarter * 32) << 16);
+            bool last = true;
+            if (parts > 1) {
+                // this segment's sums into its slot, then a ticket: the last one to arrive finishes the tile
+                if (ok) {
+#pragma unroll 1
+                    for (int c0 = 0; c0 < BN; c0 += 32) {
+                        uint32_t ai[32], af[32];
+                        tmem_ld32(lane_base + uint32_t(c0), ai);
+                        if (has_side) tmem_ld32(lane_base + uint32_t(BN + c0), af);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                        if (!has_i8) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) ai[j] = 0u;
+                        }
+                        if (row_lane) {
+                            int* dst = part_acc + (size_t(t) * maxparts + mypart) * kPart + size_t(row_in_tile) * BN + c0;
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4) *reinterpret_cast<uint4*>(dst + j) = make_uint4(ai[j], ai[j + 1], ai[j + 2], ai[j + 3]);
+                            if (has_side) {
+                                float* ds = part_side + size_t(t) * kPart + size_t(row_in_tile) * BN + c0;
+#pragma unroll
+                                for (int j = 0; j < 32; j += 4) *reinterpret_cast<uint4*>(ds + j) = make_uint4(af[j], af[j + 1], af[j + 2], af[j + 3]);
+                            }
+                        }
+                    }
+                    __threadfence();
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (et == 0) *ticket = ok ? atomicAdd(counters + t, 1) : -1;      // a segment that gave up takes no ticket: the tile is then never finished
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                last = (*ticket == parts - 1);
+                __threadfence();
+            }
+            if (ok && last) {
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    uint32_t ai[32], af[32];
+                    tmem_ld32(lane_base + uint32_t(c0), ai);
+                    if (has_side) tmem_ld32(lane_base + uint32_t(BN + c0), af);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (!has_i8) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) ai[j] = 0u;
+                    }
+                    if (parts > 1 && row_lane) {
+                        for (int pp = 0; pp < parts; ++pp) {
+                            if (pp == mypart) continue;
+                            const int* src = part_acc + (size_t(t) * maxparts + pp) * kPart + size_t(row_in_tile) * BN + c0;
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4) {
+                                const uint4 v = __ldcg(reinterpret_cast<const uint4*>(src + j));
+                                ai[j] += v.x; ai[j + 1] += v.y; ai[j + 2] += v.z; ai[j + 3] += v.w;
+                            }
+                        }
+                        if (sblocks_all > 0 && !has_side) {
+                            const float* ss = part_side + size_t(t) * kPart + size_t(row_in_tile) * BN + c0;
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4) {
+                                const uint4 v = __ldcg(reinterpret_cast<const uint4*>(ss + j));
+                                af[j] = v.x; af[j + 1] = v.y; af[j + 2] = v.z; af[j + 3] = v.w;
+                            }
+                        }
+                    }
+                    float out[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const float sc = __fmul_rn(sxm, sws[c0 + j]);
+                        const float pside = (sblocks_all > 0) ? __uint_as_float(af[j]) : 0.0f;
+                        out[j] = __fmaf_rn(float(int(ai[j])), sc, pside);
+                    }
+                    if (m < M) {
+                        const int n = n0 + c0;
+                        if constexpr (YDT == kF32) {
+                            float* dst = static_cast<float*>(y) + size_t(m) * N + n;
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4)
+                                if (n + j < N) *reinterpret_cast<float4*>(dst + j) = make_float4(out[j], out[j + 1], out[j + 2], out[j + 3]);
+                        } else {
+                            uint16_t* dst = static_cast<uint16_t*>(y) + size_t(m) * N + n;
+#pragma unroll
+                            for (int j = 0; j < 32; j += 8) {
+                                uint32_t pk[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    if constexpr (YDT == kBF16) {
+                                        const __nv_bfloat162 h = __floats2bfloat162_rn(out[j + 2 * e], out[j + 2 * e + 1]);
+                                        pk[e] = *reinterpret_cast<const uint32_t*>(&h);
+                                    } else {
+                                        const __half2 h = __floats2half2_rn(out[j + 2 * e], out[j + 2 * e + 1]);
+                                        pk[e] = *reinterpret_cast<const uint32_t*>(&h);
+                                    }
+                                }
+                                if (n + j < N) *reinterpret_cast<uint4*>(dst + j) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                            }
+                        }
+                    }
+                }
+            }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    }
+
+    __syncthreads();
+    if (*abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(2000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+    }
+}
 
 // ------------------------------------------------------------------------------------------
 // gemm_tcp: persistent tensor-core kernel for large products with at most kTcpSide critical

@@ -10,11 +10,11 @@ import torch
 
 from .binding import _DT, BqError, _check, _dev, _stream, lib
 
-PATH_AUTO, PATH_GENERAL, PATH_TENSOR, PATH_TENSOR_TILE, PATH_TENSOR_SOLO = 0, 1, 2, 3, 4
+PATH_AUTO, PATH_GENERAL, PATH_TENSOR, PATH_TENSOR_TILE, PATH_TENSOR_SOLO, PATH_TENSOR_STREAMK = 0, 1, 2, 3, 4, 5
 _TORCH_OF = {0: torch.float32, 1: torch.float16, 2: torch.bfloat16}
 
 SYMBOLS = ("mmd_side_columns", "mmd_select_features", "mmd_rowquant", "mmd_decompose", "mmd_free", "mmd_weights_view",
-           "mmd_workspace_layout", "mmd_linear", "mmd_linear_static", "mmd_kernel_status", "mmd_selftest_bounded_wait")
+           "mmd_workspace_layout", "mmd_linear", "mmd_linear_static", "mmd_kernel_status", "mmd_selftest_bounded_wait", "mmd_workspace_bytes_streamk")
 SELFTEST_CODE = 77
 STATIC_SCRATCH_BYTES = 4 << 20
 _typed = False
@@ -32,6 +32,7 @@ def _lib() -> ctypes.CDLL:
         L.mmd_free.argtypes = [vp]
         L.mmd_weights_view.argtypes = [vp] + [ctypes.POINTER(vp)] * 4 + [ctypes.POINTER(i32)] * 4
         L.mmd_workspace_layout.argtypes = [vp, i32, ctypes.POINTER(sz), ctypes.POINTER(sz)]
+        L.mmd_workspace_bytes_streamk.argtypes = [vp, i32, ctypes.POINTER(sz)]
         L.mmd_linear.argtypes = [vp, vp, i32, vp, i32, vp, sz, i32, vp]
         L.mmd_linear_static.argtypes = [vp, vp, i32, vp, i32, i32, vp]
         L.mmd_kernel_status.argtypes = [vp, ctypes.POINTER(i32)]
@@ -125,8 +126,15 @@ class DecomposedLinear:
         _check(_lib().mmd_workspace_layout(self._h, M, offs, ctypes.byref(total)), "mmd_workspace_layout")
         return tuple(int(o) for o in offs), int(total.value)
 
-    def workspace(self, M: int) -> torch.Tensor:
-        _, total = self.workspace_layout(M)
+    def workspace_bytes(self, M: int) -> int:
+        """``mmd_workspace_bytes_streamk``: the workspace size that lets decode-size calls take the stream-K kernel."""
+        total = ctypes.c_size_t()
+        _check(_lib().mmd_workspace_bytes_streamk(self._h, M, ctypes.byref(total)), "mmd_workspace_bytes_streamk")
+        return int(total.value)
+
+    def workspace(self, M: int, streamk: bool = False) -> torch.Tensor:
+        """A workspace for M rows (cached); with ``streamk`` also the room the stream-K kernel's slots need."""
+        total = self.workspace_bytes(M) if streamk else self.workspace_layout(M)[1]
         if self._ws is None or self._ws.numel() < total:
             self._ws = torch.empty(total + 256, dtype=torch.uint8, device=self.device)
         off = (-self._ws.data_ptr()) % 256
@@ -139,7 +147,7 @@ class DecomposedLinear:
         if X.dtype != self.dtype or X.dim() != 2 or X.shape[1] != self.K:
             raise BqError("X must be [M, K] of the weights' element type")
         M = X.shape[0]
-        ws = self.workspace(M) if workspace is None else workspace
+        ws = self.workspace(M, streamk=(path == PATH_TENSOR_STREAMK)) if workspace is None else workspace
         if y_out is None:
             y_out = torch.empty((M, self.N), dtype=out_dtype or X.dtype, device=X.device)
         with torch.cuda.device(X.device):

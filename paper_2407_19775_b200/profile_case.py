@@ -18,7 +18,7 @@ from . import Codebook, Codebook4, bq4_dequantize, bq4_quantize, bq_dequantize, 
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="sweep1g")
-    ap.add_argument("--op", default="roundtrip", choices=["quantize", "dequantize", "roundtrip", "roundtrip_side", "quantize4", "dequantize4", "block_errors"])
+    ap.add_argument("--op", default="roundtrip", choices=["quantize", "dequantize", "roundtrip", "roundtrip_side", "quantize4", "dequantize4", "block_errors", "sweep"])
     ap.add_argument("--block", type=int, default=4096)
     ap.add_argument("--rows", type=int, default=8192)
     ap.add_argument("--launches", type=int, default=3)
@@ -31,7 +31,7 @@ def main() -> None:
     n = x.numel()
     cb = Codebook(device=dev)
     codes = torch.empty(n, dtype=torch.uint8, device=dev)
-    absmax = torch.empty((n + args.block - 1) // args.block, dtype=torch.float32, device=dev)
+    absmax = torch.empty((n + min(args.block, 64) - 1) // min(args.block, 64), dtype=torch.float32, device=dev)
     y = torch.empty_like(x)
     cb4 = Codebook4()
     packed = codes[: (n + 1) // 2]
@@ -42,6 +42,24 @@ def main() -> None:
     if args.op == "block_errors":                                # one candidate: the roundtrip, then the two kernels of the sums
         tune_ws = torch.empty(tune.workspace_bytes(x.dtype, n), dtype=torch.uint8, device=dev)
         tune_sums = torch.empty(2, dtype=torch.float64, device=dev)
+    if args.op == "sweep":
+        # the benchmark's step, launch by launch: for each block size quantize, dequantize, fused roundtrip (12 launches per pass)
+        for i in range(args.launches):
+            for block in (64, 256, 1024, 4096):
+                am = absmax[: n // block]
+                for op in ("quantize", "dequantize", "roundtrip"):
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    if op == "quantize":
+                        bq_quantize(x, block, cb, codes, am)
+                    elif op == "dequantize":
+                        bq_dequantize(codes, am, block, cb, x.dtype, y)
+                    else:
+                        bq_roundtrip(x, block, cb, y_out=y)
+                    e1.record()
+                    torch.cuda.synchronize()
+                    print(f"{op} {str(x.dtype)[6:]} block={block} n={n} pass {i}: {e0.elapsed_time(e1):.4f} ms")
+        return
     torch.cuda.synchronize()
     for i in range(args.launches):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

@@ -342,3 +342,48 @@ def test_a_bounded_wait_that_runs_out_leaves_a_status_and_a_usable_handle(bq):
     with pytest.raises(bq.BqError):
         lin.selftest_bounded_wait(0)
     lin.close()
+
+
+@pytest.mark.parametrize("M,K,N,ko", [(64, 8192, 8192, 8), (64, 4096, 4736, 2), (33, 2048, 6272, 0), (64, 8192, 1024, 70), (1, 4096, 18816, 3),
+                                       (64, 2048, 18944 - 128, 0)])
+def test_decode_step_with_the_k_steps_of_all_tiles_dealt_out(bq, M, K, N, ko):
+    """The stream-K kernel of decode-size calls: every CTA takes the same number of K steps across the tiles, tiles shared by
+    several CTAs are finished by the last one to arrive.  Its integer sums are exact and its side sums are accumulated by one
+    CTA in the order of the one-tile-per-CTA kernel, so the two must agree bit for bit; the oracle decides the rest.  Calls
+    alternate with the other kernel through the same workspace; a workspace without the extra room is refused."""
+    g = torch.Generator().manual_seed(M * 7 + N + ko)
+    X = (torch.randn(M, K, generator=g) * 0.6).to(torch.float16)
+    W = (torch.randn(N, K, generator=g) * 0.03).to(torch.float16)
+    idx = np.sort(torch.randperm(K, generator=g)[:ko].numpy()).astype(np.int32)
+    X[:, idx.tolist()] *= 25
+    lin = bq.DecomposedLinear(W.cuda(), idx)
+    Xd = X.cuda()
+    assert lin.workspace_bytes(M) > lin.workspace_layout(M)[1]
+    for out in (torch.float32, None):
+        y_tile = lin.linear(Xd, out, path=bq.mmd.PATH_TENSOR_TILE)
+        for _ in range(3):                                        # the counters are zeroed by every call's row kernel
+            y_sk = lin.linear(Xd, out, path=bq.mmd.PATH_TENSOR_STREAMK)
+            assert lin.kernel_status() == 0
+            assert torch.equal(y_sk, y_tile)
+        check_output(y_sk, X, W, idx, F16, exact_expected=(ko == 0))
+    small = lin.workspace(M)
+    with pytest.raises(bq.BqError):
+        lin.linear(Xd, torch.float32, path=bq.mmd.PATH_TENSOR_STREAMK, workspace=small)
+    lin.close()
+
+
+def test_stream_k_is_refused_for_shapes_it_does_not_take(bq):
+    g = torch.Generator().manual_seed(3)
+    W = (torch.randn(512, 2048, generator=g) * 0.03).to(torch.float16)                # N below 1024
+    lin = bq.DecomposedLinear(W.cuda(), np.zeros(0, np.int32))
+    X = torch.randn(16, 2048, generator=g).to(torch.float16).cuda()
+    assert lin.workspace_bytes(16) == lin.workspace_layout(16)[1]
+    with pytest.raises(bq.BqError):
+        lin.linear(X, torch.float32, path=bq.mmd.PATH_TENSOR_STREAMK)
+    lin.close()
+    W = (torch.randn(2048, 2048, generator=g) * 0.03).to(torch.float16)
+    lin = bq.DecomposedLinear(W.cuda(), np.zeros(0, np.int32))
+    X = torch.randn(100, 2048, generator=g).to(torch.float16).cuda()                   # more than 64 rows
+    with pytest.raises(bq.BqError):
+        lin.linear(X, torch.float32, path=bq.mmd.PATH_TENSOR_STREAMK)
+    lin.close()
