@@ -142,9 +142,12 @@ int bq_host_pipe_destroy(bq_host_pipe* pipe);
  * The three data calls, host to host.  Same results, bit for bit, as the device-pointer calls
  * on the whole tensor (pieces are whole numbers of blocks, and blocks are independent).
  *   x_host, y_host: n elements; codes_host: n bytes; absmax_host: ceil(n / block) floats.
- * Each call ENQUEUES its copies and kernels and returns; calls on one pipe run in the order
- * they were made (a later call may read what an earlier one wrote).  The host buffers belong
- * to the pipe until bq_host_pipe_wait returns.  Errors as for the device calls, plus
+ * Each call ENQUEUES its copies and kernels and returns; calls on one pipe take effect in the
+ * order they were made, and a later call may read host memory that an earlier one writes (the
+ * pipe sees the overlap and holds the later call's uploads back until the earlier call has
+ * finished; calls without such an overlap run into each other: the uploads of one under the
+ * downloads of the one before).  The host buffers belong to the pipe until bq_host_pipe_wait
+ * returns.  Errors as for the device calls, plus
  * BQ_ERR_BLOCK for block < min_block or block > chunk_elems and BQ_ERR_DTYPE for a type wider
  * than `widest`.  y_host may be x_host in bq_roundtrip_host when the types agree.
  */

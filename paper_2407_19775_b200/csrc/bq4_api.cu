@@ -147,13 +147,13 @@ cudaError_t quantize_t(const void* x, size_t n, size_t B, const bq4k::Tables4& t
     constexpr size_t EB = (DT == bq4k::kF32) ? 4 : 2;
     if (l2 >= 3 && l2 <= 16 && aligned(x, 16) && aligned(packed, 4) && n >= B) {
         const size_t nblocks = n / B, n_full = nblocks * B;
-        if (!S16 && DT != bq4k::kF32 && tab.folded && l2 >= 6 && l2 <= 12 && n_full > kFwd4MinElems && aligned(absmax, 4)) {
+        if (DT != bq4k::kF32 && tab.folded && l2 >= 6 && l2 <= 12 && n_full > kFwd4MinElems && aligned(absmax, S16 ? 2 : 4)) {
             bqk::Tables4Fast fast;
             std::memcpy(fast.entry, tab.entry, sizeof fast.entry);
             fast.neg_limit = tab.neg_limit;
             int dev = 0;
             cudaError_t e = cudaGetDevice(&dev);
-            if (e == cudaSuccess) e = bql::launch_fwd4_fast(DT == bq4k::kF16 ? BQ_F16 : BQ_BF16, int(B), x, packed, absmax, n_full, fast, sms, dev, s, &done);
+            if (e == cudaSuccess) e = bql::launch_fwd4_fast(DT == bq4k::kF16 ? BQ_F16 : BQ_BF16, int(B), S16, x, packed, absmax, n_full, fast, sms, dev, s, &done);
             if (e != cudaSuccess) return e;
         }
         if (done < n_full) {                                      // the whole blocks the tiles did not cover (all of them for small tensors)

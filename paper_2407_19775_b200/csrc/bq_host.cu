@@ -6,9 +6,14 @@
 //     up stream:    wait free[s] (the slot's previous download)   copy in   record in[s]
 //     run stream:   wait in[s]                                    kernel    record ran[s]
 //     down stream:  wait ran[s]                                   copy out  record free[s]
-// A call begins by making all three streams wait for the end of the call before it (`done`), so
-// calls on one pipe take effect in order; it ends by recording `done` on the down stream, which
-// has by then waited for everything else of the call.
+// Calls on one pipe take effect in order without waiting for each other more than they must.  The
+// three streams are each in order, the slots are guarded by their events, and a call ends by
+// recording `done` on the down stream (which has by then waited for everything else of the
+// call).  What the streams' own order does not give is a later call READING host memory that an
+// earlier, still unfinished call WRITES (the receiver expanding what the sender just produced):
+// the pipe remembers the host ranges its unfinished calls write, and a call whose inputs overlap
+// one of them first makes its uploads wait for `done`.  Otherwise the uploads of a call run under
+// the downloads of the call before it.
 #include "../../include/bq.h"
 #include "bq_error.h"
 
@@ -32,6 +37,10 @@ struct bq_host_pipe {
     cudaEvent_t in[8], ran[8], free_[8], done;
     bool used[8];            // the slot has a download in flight or behind it (free_[s] has been recorded)
     bool any;                // `done` has been recorded
+    // host ranges written by calls enqueued since the last wait on `done`
+    const char* out_lo[24];
+    const char* out_hi[24];
+    int n_out;
 };
 
 namespace {
@@ -69,15 +78,38 @@ struct Call {
         if (e_ != cudaSuccess) return cuda_fail(e_);   \
     } while (0)
 
+bool overlaps(const bq_host_pipe* p, const void* lo, size_t bytes) {
+    const char* a = static_cast<const char*>(lo);
+    for (int i = 0; i < p->n_out; ++i)
+        if (a < p->out_hi[i] && p->out_lo[i] < a + bytes) return true;
+    return false;
+}
+
+void remember_output(bq_host_pipe* p, void* lo, size_t bytes) {
+    p->out_lo[p->n_out] = static_cast<const char*>(lo);
+    p->out_hi[p->n_out] = static_cast<const char*>(lo) + bytes;
+    ++p->n_out;
+}
+
 int run_call(bq_host_pipe* p, const Call& c, size_t n, int block) {
     const size_t B = size_t(block);
     const size_t piece = (p->chunk / B) * B;          // whole blocks per piece
-    if (p->any) {
-        BQ_TRY(cudaStreamWaitEvent(p->up, p->done, 0));
-        BQ_TRY(cudaStreamWaitEvent(p->run, p->done, 0));
-        BQ_TRY(cudaStreamWaitEvent(p->down, p->done, 0));
-    }
     const int xs = bytes_of(c.xdt), ys = bytes_of(c.ydt);
+    const size_t nblocks = (n + B - 1) / B;
+    // does this call read what an unfinished call writes?  (or is the list of remembered ranges full?)
+    bool must_wait = p->n_out + 2 > 24;
+    if (c.op == kDequantize) must_wait = must_wait || overlaps(p, c.codes_in, n) || overlaps(p, c.absmax_in, nblocks * 4);
+    else must_wait = must_wait || overlaps(p, c.x, n * size_t(xs));
+    if (p->any && must_wait) {
+        BQ_TRY(cudaStreamWaitEvent(p->up, p->done, 0));          // everything enqueued so far has finished before the first upload
+        p->n_out = 0;
+    }
+    if (c.op == kQuantize) {
+        remember_output(p, c.codes_out, n);
+        remember_output(p, c.absmax_out, nblocks * 4);
+    } else {
+        remember_output(p, c.y, n * size_t(ys));
+    }
     size_t i = 0;
     for (size_t lo = 0; lo < n; lo += piece, ++i) {
         const int s = int(i % size_t(p->slots));
@@ -225,6 +257,7 @@ int bq_host_pipe_wait(bq_host_pipe* p) {
     if (!p) return BQ_ERR_NULL;
     if (!p->any) return BQ_OK;
     const cudaError_t e = cudaEventSynchronize(p->done);
+    p->n_out = 0;                                         // nothing is unfinished any more
     return e == cudaSuccess ? BQ_OK : cuda_fail(e);
 }
 

@@ -374,15 +374,27 @@ __device__ __forceinline__ float rcp_approx(float d) {
 //   BITS         8: the 256-entry codebook, one code per byte.  4: the 16-entry codebook of the 4-bit variant, two
 //                codes per byte (quantize only, 16-bit inputs, the shared-memory flavour); everything up to
 //                the search is the same code.
-template <int XDT, int B, int R, int TW, bool WRITE_Y, bool WRITE_Q, int NT, bool LITE, int BITS = 8>
+//   S16          (4-bit flavour only) the block's scale is its absmax rounded toward +infinity to a bf16, never above the
+//                largest finite bf16; x is divided by that scale and its two bytes are what absmax_out receives.
+template <int XDT, int B, int R, int TW, bool WRITE_Y, bool WRITE_Q, int NT, bool LITE, int BITS = 8, bool S16 = false>
 __global__ void __launch_bounds__(NT, 1)
 fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__ codes, float* __restrict__ absmax_out,
          size_t ntiles, const __grid_constant__ typename TabArg<BITS>::type tab) {
     static_assert(BITS == 8 || (BITS == 4 && !WRITE_Y && WRITE_Q && !LITE && Elem<XDT>::kPerChunk == 8), "the 4-bit flavour: quantize, 16-bit inputs, tables in shared memory");
+    static_assert(!S16 || BITS == 4, "the 16-bit scale belongs to the 4-bit flavour");
+    // the scale a block is divided by, from its absmax
+    auto scale_of = [](float a) -> float {
+        if constexpr (S16) return __uint_as_float(min((__float_as_uint(a) + 0xFFFFu) & 0xFFFF0000u, 0x7F7F0000u));
+        else return a;
+    };
+    auto store_scale = [&](size_t i, float s) {
+        if constexpr (S16) reinterpret_cast<uint16_t*>(absmax_out)[i] = uint16_t(__float_as_uint(s) >> 16);
+        else absmax_out[i] = s;
+    };
     constexpr int EPC = Elem<XDT>::kPerChunk;
     constexpr int EB = Elem<XDT>::kBytes;
     constexpr int ROW = 32 * EPC;
-    constexpr bool IN_ROW = (B <= ROW);
+    constexpr bool IN_ROW = (B < ROW);                         // a block of exactly one row is a whole-warp reduction: the paths below
     constexpr int LPB = IN_ROW ? B / EPC : 32;                 // lanes per block inside a row
     constexpr int RPB = IN_ROW ? 1 : (B / ROW) / TW;           // rows of one warp that belong to one block
     constexpr int NBLK = R / RPB;                              // blocks per tile when blocks span rows
@@ -480,6 +492,7 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
             float m = v[0];
 #pragma unroll
             for (int s = R; s < LPB; s <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, s));
+            m = scale_of(m);
             // this lane's block: row rho = sum_s bit_s(lane) * (R >> (s+1)), group lane / LPB
             const float dm = (m != 0.0f) ? m : 1.0f;
             const float rm = QUICK_OK ? rcp_approx(dm) : 0.0f;
@@ -489,7 +502,7 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
                 int rho = 0;
 #pragma unroll
                 for (int s = 0; s < LOGR; ++s) rho += ((lane >> s) & 1) * (R >> (s + 1));
-                if ((lane % LPB) < R) absmax_out[(base + size_t(rho) * ROW) / B] = m;
+                if ((lane % LPB) < R) store_scale((base + size_t(rho) * ROW) / B, m);
             }
             const int group_base = lane & ~(LPB - 1);
 #pragma unroll
@@ -508,7 +521,7 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
                 float a = amax[k * RPB];
 #pragma unroll
                 for (int r = 1; r < RPB; ++r) a = fmaxf(a, amax[k * RPB + r]);
-                a = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(a)));
+                a = scale_of(__uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(a))));
 #pragma unroll
                 for (int r = 0; r < RPB; ++r) amax[k * RPB + r] = a;
             }
@@ -529,6 +542,7 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
                 a = fmaxf(a, __uint_as_float(v));
             }
             parity ^= 1;
+            a = scale_of(a);
 #pragma unroll
             for (int r = 0; r < R; ++r) amax[r] = a;
         }
@@ -592,7 +606,7 @@ fwd_fast(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict__
         if constexpr (WRITE_Q && !IN_ROW) {
             if (lane == 0 && wt == 0) {
 #pragma unroll
-                for (int k = 0; k < NBLK; ++k) absmax_out[t * NBLK + k] = amax[k * RPB];
+                for (int k = 0; k < NBLK; ++k) store_scale(t * NBLK + k, amax[k * RPB]);
             }
         }
     }

@@ -38,9 +38,10 @@ cudaError_t launch_fwd_staged(int xdt, int block, bool write_y, bool write_q, co
                               bool* taken);
 
 // The forward kernel's 4-bit flavour on the leading whole tiles of n_full elements (whole blocks; 16-bit inputs, blocks of
-// 64 .. 4096): packed receives two codes per byte, absmax one float per block; *done = elements covered (0: not taken).
-cudaError_t launch_fwd4_fast(int xdt, int block, const void* x, uint8_t* packed, float* absmax, size_t n_full, const bqk::Tables4Fast& tab,
-                             int sm_count, int device, cudaStream_t stream, size_t* done);
+// 64 .. 4096): packed receives two codes per byte, absmax one float per block (with scale16: one bf16, the absmax rounded
+// up, in 16-bit words); *done = elements covered (0: not taken).
+cudaError_t launch_fwd4_fast(int xdt, int block, bool scale16, const void* x, uint8_t* packed, float* absmax, size_t n_full,
+                             const bqk::Tables4Fast& tab, int sm_count, int device, cudaStream_t stream, size_t* done);
 
 cudaError_t launch_fwd_general(int xdt, int ydt, bool write_y, bool write_q, const void* x, void* y, uint8_t* codes, float* absmax,
                                size_t n, size_t block, size_t first_block, const bqk::DeviceTables& tab, int sm_count,

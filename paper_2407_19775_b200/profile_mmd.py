@@ -13,7 +13,7 @@ import argparse
 import torch
 
 from . import DecomposedLinear, workloads
-from .mmd import PATH_AUTO, PATH_GENERAL, PATH_TENSOR, PATH_TENSOR_SOLO, PATH_TENSOR_TILE
+from .mmd import PATH_AUTO, PATH_GENERAL, PATH_TENSOR, PATH_TENSOR_SOLO, PATH_TENSOR_STREAMK, PATH_TENSOR_TILE
 
 
 def main() -> None:
@@ -22,7 +22,7 @@ def main() -> None:
     ap.add_argument("--tokens", type=int, default=None)
     ap.add_argument("--out-features", type=int, default=None)
     ap.add_argument("--launches", type=int, default=3)
-    ap.add_argument("--path", default="auto", choices=["auto", "general", "tensor", "tile", "solo"])
+    ap.add_argument("--path", default="auto", choices=["auto", "general", "tensor", "tile", "solo", "streamk"])
     ap.add_argument("--no-features", action="store_true", help="decompose without critical features")
     ap.add_argument("--graph", action="store_true", help="also time a CUDA-graph replay of the call")
     args = ap.parse_args()
@@ -34,8 +34,8 @@ def main() -> None:
     lin = DecomposedLinear(W, idx)
     M, N, K = X.shape[0], W.shape[0], W.shape[1]
     y = torch.empty((M, N), dtype=X.dtype, device=dev)
-    ws = lin.workspace(M)
-    path = {"auto": PATH_AUTO, "general": PATH_GENERAL, "tensor": PATH_TENSOR, "tile": PATH_TENSOR_TILE, "solo": PATH_TENSOR_SOLO}[args.path]
+    ws = lin.workspace(M, streamk=(args.path == "streamk"))
+    path = {"auto": PATH_AUTO, "general": PATH_GENERAL, "tensor": PATH_TENSOR, "tile": PATH_TENSOR_TILE, "solo": PATH_TENSOR_SOLO, "streamk": PATH_TENSOR_STREAMK}[args.path]
     torch.cuda.synchronize()
     for i in range(args.launches):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

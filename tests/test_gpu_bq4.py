@@ -269,3 +269,21 @@ def test_large_tensors_through_the_tiled_forward_kernel(bq, dtype, block):
     x[7 * block] = -x[7 * block:8 * block].float().abs().max() * 2  # the absmax element is negative: xhat = -1 has no code of its own
     x[9 * block + 1] = -0.0
     check(bq, x, block, ydt=dtype)
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
+@pytest.mark.parametrize("block", [64, 256, 512, 4096])
+def test_large_tensors_with_the_bf16_scale_through_the_tiled_forward_kernel(bq, dtype, block):
+    """The same split (tiles, left-over blocks, a short block) with the block scale stored as a bf16: absmax values on, just
+    above and far from the bf16 grid, a zero block, and the top of the fp16 range."""
+    g = torch.Generator().manual_seed(block + 5)
+    n = (1 << 23) + 3 * 24576 + 2 * block + 11
+    x = (torch.randn(n, generator=g) * (1.0 + 30.0 * (torch.rand(n, generator=g) < 0.002))).to(dtype)
+    x[block:2 * block] = 0
+    x[2 * block:3 * block] = x[2 * block:3 * block].clamp(-1, 1)
+    x[2 * block] = 1.0                                              # an absmax that is itself a bf16
+    x[3 * block:4 * block] = x[3 * block:4 * block].clamp(-1, 1)
+    x[3 * block + 1] = 1.00390625 if dtype == torch.bfloat16 else 1.0009765625      # just above one: rounds up
+    if dtype == torch.float16:
+        x[5 * block] = 65504.0
+    check_s16(bq, x, block)

@@ -318,6 +318,43 @@ def test_host_to_host_calls(bq, gcb, cb, dtype, block, chunk):
     hb.close()
 
 
+def test_host_to_host_calls_overlap_unless_one_reads_what_another_writes(bq, gcb, cb):
+    """Calls on one pipe that do not depend on each other run into each other (three roundtrips of different tensors into
+    different buffers, then all waited for at once); a call that reads a host range an unfinished call writes (the codes of a
+    quantize, a tensor rounded twice in place) is held back.  Many calls in a row overflow the pipe's list of unfinished
+    outputs, which must only cost a wait."""
+    g = torch.Generator().manual_seed(77)
+    n, block = 64 * 5000 + 19, 64
+    hb = bq.HostBoundary(gcb, torch.bfloat16, chunk=64 * 700, slots=3, min_block=64)
+    xs = [(torch.randn(n, generator=g) * (i + 1)).to(torch.bfloat16).pin_memory() for i in range(3)]
+    ys = [torch.empty(n, dtype=torch.bfloat16).pin_memory() for _ in xs]
+    for x, y in zip(xs, ys):
+        hb.roundtrip(x, block, y)
+    hb.wait()
+    refs = [oracle.roundtrip(_bits(x), oracle.BF16, block, cb, oracle.BF16) for x in xs]
+    for y, r in zip(ys, refs):
+        assert np.array_equal(_bits(y), r)
+    # a chain through host memory: quantize -> dequantize of the same buffers, then the result rounded again in place, twice
+    c = torch.empty(n, dtype=torch.uint8).pin_memory()
+    a = torch.empty((n + block - 1) // block, dtype=torch.float32).pin_memory()
+    z = torch.empty(n, dtype=torch.bfloat16).pin_memory()
+    hb.quantize(xs[1], block, c, a)
+    hb.dequantize(c, a, block, z)
+    hb.roundtrip(z, block, z)
+    hb.roundtrip(z, block, z)
+    hb.wait()
+    twice = oracle.roundtrip(refs[1], oracle.BF16, block, cb, oracle.BF16)
+    assert np.array_equal(_bits(z), oracle.roundtrip(twice, oracle.BF16, block, cb, oracle.BF16))
+    # more unfinished calls than the pipe remembers outputs for
+    outs = [torch.empty(n, dtype=torch.bfloat16).pin_memory() for _ in range(30)]
+    for i, y in enumerate(outs):
+        hb.roundtrip(xs[i % 3], block, y)
+    hb.wait()
+    for i, y in enumerate(outs):
+        assert np.array_equal(_bits(y), refs[i % 3])
+    hb.close()
+
+
 def test_host_to_host_calls_from_pageable_memory(bq, gcb, cb):
     x = workloads.make("prefill7b", rows=40).view(-1)
     n, block = x.numel(), 256

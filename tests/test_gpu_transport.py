@@ -113,3 +113,48 @@ def test_transport_refuses_what_the_mailbox_was_not_made_for(bq):
         transport.Sender(gcb, bytes(bad))
     tx.close()
     rx.close()
+
+
+def _shard_process(rank, world, port, tmp):
+    """One process per shard, both on device 0: rank 0 sends through the mailbox that rank 1 owns and exported (CUDA IPC
+    handles of the memory and of the events); the FILLED / DRAINED messages travel over a gloo group."""
+    import torch.distributed as dist
+    import paper_2407_19775_b200 as bq
+    dist.init_process_group("gloo", rank=rank, world_size=world, init_method=f"tcp://127.0.0.1:{port}")
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    gcb = bq.Codebook(device=dev)
+    n, block, chunk, slots = 256 * 64 * 9 + 256 * 2 + 5, 256, 256 * 64, 3
+    end = transport.ChainEndpoint(rank, world, transport.DistMessenger(),
+                                  lambda c, b, s: transport.Receiver(gcb, c, b, s), lambda d: transport.Sender(gcb, d, transport.STORE),
+                                  chunk, block, slots)
+    ok = True
+    for i in range(3):                                                   # tensors follow each other through the same slots
+        x = workloads.make("prefill7b", rows=40).view(-1)[: n].contiguous().roll(i * 1000)
+        if rank == 0:
+            end.send(x.to(dev), block)
+        else:
+            y = torch.empty(n, dtype=torch.bfloat16, device=dev)
+            end.recv(y, block)
+            torch.cuda.synchronize()
+            ok = ok and np.array_equal(_bits(y.cpu()), oracle.roundtrip(_bits(x), oracle.BF16, block, oracle.make_codebook(), oracle.BF16))
+    end.close()
+    torch.cuda.synchronize()
+    with open(f"{tmp}/ok{rank}", "w") as f:
+        f.write("ok" if ok else "mismatch")
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_processes_share_the_mailbox_through_ipc_handles(bq, tmp_path):
+    """The form a deployment uses (one process per GPU), with both processes on the one GPU there is: the sender opens the
+    receiver's mailbox and events through their IPC handles.  Nothing here waits on the device for the other process: the
+    order of the two processes' event calls is kept by host messages, the data dependencies by the events."""
+    import socket
+    import torch.multiprocessing as mp
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    mp.spawn(_shard_process, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    assert open(tmp_path / "ok0").read() == "ok" and open(tmp_path / "ok1").read() == "ok"
