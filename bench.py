@@ -524,7 +524,7 @@ def run_mtpp(bq, dev, args, name="mtpp_unet"):
 
 # ------------------------------------------------------------------------------------------ the boundary transport (loop-back)
 
-NVLINK_PEER_GBS = 770.0          # measured peer copy rate per direction on this pool's machines (context for the projection only)
+NVLINK_PEER_GBS = 770.0          # a measured NVLink 5 peer copy rate per direction between two B200s (context for the projection only)
 
 
 def run_transport(bq, dev, args, block=256):
