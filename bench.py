@@ -378,18 +378,23 @@ def run_ours(args):
                   bq4, tune, small, mmd, transport, mtpp)
 
 
+def workload_label(w) -> str:
+    """The line's `config.workload`, the same text for both arms."""
+    blocks = "/".join(str(b) for b in w.blocks)
+    return (f"{w.name}: {list(w.shape)} {str(w.dtype)[6:]}, {w.recipe}, seed {w.seed}; blocks {blocks}; "
+            "quantize+dequantize+roundtrip per block")
+
+
 def finish(rank, world, args, value, max_s, n, w, e2e, events, clocks, roofline, kernels, quality, cpu, input_sha, bq4, tune, small, mmd,
            transport=None, mtpp=None):
     if rank == 0:
-        blocks = "/".join(str(b) for b in BLOCKS)
         es = torch.empty(0, dtype=w.dtype).element_size()
         fits_l2 = 2 * n * es < (120 << 20)
         line = {
             "metric": METRIC, "value": round(value, 1), "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": round(max_s * 1e3 / args.steps, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
-            "config": {"workload": f"{WORKLOAD}: {list(w.shape)} {str(w.dtype)[6:]}, {w.recipe}, seed {w.seed}; blocks {blocks}; "
-                                   "quantize+dequantize+roundtrip per block", "elements": n,
+            "config": {"workload": workload_label(w), "elements": n,
                        "l2": ("tensor fits in L2: a 256 MiB buffer is written before every launch and the value counts the launches' own "
                               "event times" if fits_l2 else f"input ({n * es >> 20} MiB) larger than L2, no flush needed"),
                        "parallelism": f"replicated x{world}, no collective", "input_sha256": input_sha},
@@ -846,32 +851,40 @@ def cpu_baseline(x_pin, w, rank, elems=1 << 24):
 
 
 def run_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on all host cores, on a bounded sample (a prefix of whole rows) of the
+    same workload per step, sized so that the run ends within about two minutes."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     import oracle
+    global WORKLOAD, BLOCKS
+    WORKLOAD = args.config
+    w = workloads.WORKLOADS[WORKLOAD]
+    BLOCKS = tuple(w.blocks)
+    odt = {torch.float32: oracle.F32, torch.float16: oracle.F16, torch.bfloat16: oracle.BF16}[w.dtype]
     threads = os.cpu_count() or 1
-    # size the sample so that the whole run stays within about two minutes
-    per_elem_s = 3.3e-6 / max(1, threads) * 1.5
-    rows = int(120.0 / ((args.steps + args.warmup) * per_elem_s) // 8192)
-    rows = max(8, min(rows, 4096))
-    x = workloads.make(WORKLOAD, rows=rows).view(-1)
-    xb = workloads.as_numpy_bits(x)
+    hidden = w.shape[-1]
+    total_rows = w.n // hidden
+    # one element through one (block size x 3 operations) costs about 0.8 us of one core
+    per_elem_s = 0.83e-6 * len(BLOCKS) / max(1, threads) * 1.5
+    rows = int(120.0 / ((args.steps + args.warmup) * per_elem_s) // hidden)
+    rows = max(1, min(rows, 4096, total_rows))
+    x = workloads.make(WORKLOAD, rows=rows).reshape(-1)
+    xb = workloads.as_numpy_bits(x) if w.dtype != torch.float32 else x.numpy()
     cb = oracle.make_codebook()
     for _ in range(args.warmup):
-        oracle_step(oracle, xb, oracle.BF16, cb, threads)
+        oracle_step(oracle, xb, odt, cb, threads)
     t = time.perf_counter()
     for _ in range(args.steps):
-        oracle_step(oracle, xb, oracle.BF16, cb, threads)
+        oracle_step(oracle, xb, odt, cb, threads)
     sec = time.perf_counter() - t
-    value = xb.size * 2 * len(BLOCKS) * len(OPS) * args.steps / sec / 1e9
-    sample = f"first {rows} rows ({xb.size} elements) of sweep1g per step, all 4 block sizes x 3 ops, {threads} threads over whole blocks"
+    value = xb.size * x.element_size() * len(BLOCKS) * len(OPS) * args.steps / sec / 1e9
+    sample = (f"first {rows} rows ({xb.size} elements) of {w.name} per step, {len(BLOCKS)} block size(s) x 3 ops, {threads} threads over whole blocks")
     line = {
         "impl": "reference", "metric": METRIC, "value": round(value, 5), "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(sec * 1e3 / args.steps, 3), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "sweep1g: [16,4096,8192] bf16, Laplace(0,0.5), 8 outlier channels x60, seed 4; blocks 64/256/1024/4096; "
-                               "quantize+dequantize+roundtrip per block", "sample": sample},
+        "config": {"workload": workload_label(w), "sample": sample},
         "cpu_baseline": {"value": round(value, 5), "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": round(value, 5), "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
