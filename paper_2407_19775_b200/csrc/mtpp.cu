@@ -26,6 +26,7 @@ namespace {
 constexpr int kSliceThreads = 256;
 constexpr int kDecodeWarps = 4;
 constexpr long long kInf = 0x7fffffffffffffffLL;
+constexpr size_t kSliceSmemLimit = 227 * 1024;         // what one CTA may take
 
 int cuda_fail(cudaError_t e) {
     bql::set_last_cuda_error(cudaGetErrorString(e));
@@ -47,29 +48,36 @@ __host__ __device__ inline size_t round_up(size_t v, size_t a) { return (v + a -
 
 // Shared memory of slice_orders for (n, kmax): 64-bit arrays first, then 32-bit, then 16-bit.
 struct SliceLayout {
-    size_t col, f, dp, pos, last, prev, arg, total;
+    size_t col, f, dp, attr, pos, last, prev, pptr, pred, order, arg, total;
 };
-__host__ __device__ inline SliceLayout slice_layout(int n, int kmax) {
+// `edges` > 0: the graph itself (attributes, producer lists) and the order are staged in shared memory too, so that the n
+// dependent steps of the programme never wait for global memory; 0: they are read from global memory (graphs too large
+// to fit beside the programme's own arrays).
+__host__ __device__ inline SliceLayout slice_layout(int n, int kmax, int edges) {
     SliceLayout L;
     size_t o = 0;
     L.col = o;  o += size_t(5) * n * 8;                 // work | param | peak | in | out, indexed by l - 1
     L.f = o;    o += size_t(n) * 8;                     // F(l, r) of the current r
     L.dp = o;   o += size_t(kmax) * (n + 1) * 8;        // dp[kk - 1][r]
+    L.attr = o; o += edges > 0 ? size_t(3) * n * 8 : 0; // work | sizeparam | sizeout of the nodes
     L.pos = o;  o += size_t(n) * 4;                     // 1-based position of each node (0: not seen)
     L.last = o; o += size_t(n) * 4;                     // position of each node's last consumer (0: none)
     L.prev = o; o += size_t(n) * 4;                     // position of each node's latest consumer so far (0: none)
+    L.pptr = o; o += edges > 0 ? size_t(n + 1) * 4 : 0; // producer lists: offsets ...
+    L.pred = o; o += edges > 0 ? size_t(edges) * 4 : 0; // ... and entries
+    L.order = o; o += edges > 0 ? size_t(n) * 4 : 0;    // the order itself
     L.arg = o;  o += size_t(kmax) * (n + 1) * 2;        // the cut that gave dp[kk - 1][r]
     L.total = (o + 15) / 16 * 16;
     return L;
 }
 
 __global__ void __launch_bounds__(kSliceThreads)
-slice_orders(DeviceGraph g, const int* __restrict__ orders, int k, long long B, long long M, long long* __restrict__ cost_out,
+slice_orders(DeviceGraph g, int staged_edges, const int* __restrict__ orders, int k, long long B, long long M, long long* __restrict__ cost_out,
              int* __restrict__ blocks_out, int* __restrict__ cuts_out, int* __restrict__ status_out) {
     extern __shared__ __align__(16) unsigned char smem[];
     const int n = g.n;
     const int kmax = k < n ? k : n;
-    const SliceLayout L = slice_layout(n, kmax);
+    const SliceLayout L = slice_layout(n, kmax, staged_edges);
     long long* c_work = reinterpret_cast<long long*>(smem + L.col);
     long long* c_param = c_work + n;
     long long* c_peak = c_param + n;
@@ -84,9 +92,24 @@ slice_orders(DeviceGraph g, const int* __restrict__ orders, int k, long long B, 
     __shared__ int bad;
 
     const int p = blockIdx.x;
-    const int* pi = orders + size_t(p) * n;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int kWarps = kSliceThreads / 32;
+    const int* pi = orders + size_t(p) * n;
+    const long long* a_work = g.work;
+    const long long* a_param = g.sizeparam;
+    const long long* a_out = g.sizeout;
+    const int* pred_ptr = g.pred_ptr;
+    const int* pred = g.pred;
+    if (staged_edges > 0) {
+        long long* sa = reinterpret_cast<long long*>(smem + L.attr);
+        int* sp = reinterpret_cast<int*>(smem + L.pptr);
+        int* sl = reinterpret_cast<int*>(smem + L.pred);
+        int* so = reinterpret_cast<int*>(smem + L.order);
+        for (int i = tid; i < n; i += kSliceThreads) { sa[i] = g.work[i]; sa[n + i] = g.sizeparam[i]; sa[2 * n + i] = g.sizeout[i]; so[i] = pi[i]; }
+        for (int i = tid; i <= n; i += kSliceThreads) sp[i] = g.pred_ptr[i];
+        for (int i = tid; i < staged_edges; i += kSliceThreads) sl[i] = g.pred[i];
+        a_work = sa; a_param = sa + n; a_out = sa + 2 * n; pred_ptr = sp; pred = sl; pi = so;
+    }
 
     // positions, and the check that the row is a topological order of this graph
     if (tid == 0) bad = 0;
@@ -118,9 +141,9 @@ slice_orders(DeviceGraph g, const int* __restrict__ orders, int k, long long B, 
 
     for (int r = 1; r <= n; ++r) {
         const int v = pi[r - 1];
-        const int pb = g.pred_ptr[v], pe = g.pred_ptr[v + 1];
-        const long long so_v = g.sizeout[v], w_v = g.work[v], pa_v = g.sizeparam[v];
-        const long long gain_out = (g.cons_ptr[v + 1] > g.cons_ptr[v]) ? so_v : 0;
+        const int pb = pred_ptr[v], pe = pred_ptr[v + 1];
+        const long long so_v = a_out[v], w_v = a_work[v], pa_v = a_param[v];
+        const long long gain_out = (last[v] != 0) ? so_v : 0;            // v has consumers (they all come later)
         // the column of r: one thread per first position l
         for (int l = tid + 1; l <= r; l += kSliceThreads) {
             long long cw, cp, ck, ci, co;
@@ -131,9 +154,9 @@ slice_orders(DeviceGraph g, const int* __restrict__ orders, int k, long long B, 
             ck = so_v > ck ? so_v : ck;
             co += gain_out;
             for (int e = pb; e < pe; ++e) {
-                const int u = g.pred[e];
+                const int u = pred[e];
                 const int pu = pos[u], pc = prev[u];
-                const long long so_u = g.sizeout[u];
+                const long long so_u = a_out[u];
                 if (l > (pu > pc ? pu : pc)) ci += so_u;             // u lies before l and nothing in l..r-1 read it
                 if (last[u] == r && pu >= l) co -= so_u;              // u is inside and v was its last consumer
             }
@@ -168,7 +191,7 @@ slice_orders(DeviceGraph g, const int* __restrict__ orders, int k, long long B, 
             }
         }
         if (tid == kSliceThreads - 1) {                              // v has now been seen as a consumer of its producers
-            for (int e = pb; e < pe; ++e) prev[g.pred[e]] = r;
+            for (int e = pb; e < pe; ++e) prev[pred[e]] = r;
         }
         __syncthreads();
     }
@@ -250,8 +273,7 @@ cudaError_t allow_slice_smem(int device) {
     std::lock_guard<std::mutex> guard(g_attr_lock);
     const bool tracked = device >= 0 && device < 64;
     if (tracked && g_attr_done[device]) return cudaSuccess;
-    const SliceLayout L = slice_layout(MTPP_MAX_NODES, MTPP_MAX_BLOCKS);
-    const cudaError_t e = cudaFuncSetAttribute(slice_orders, cudaFuncAttributeMaxDynamicSharedMemorySize, int(L.total));
+    const cudaError_t e = cudaFuncSetAttribute(slice_orders, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSliceSmemLimit));
     if (e == cudaSuccess && tracked) g_attr_done[device] = true;
     return e;
 }
@@ -369,12 +391,18 @@ int mtpp_slice_orders(const mtpp_graph* g, const int32_t* orders, int P, int k, 
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev != g->device) return BQ_ERR_CUDA;
     const int kmax = k < g->d.n ? k : g->d.n;
-    const SliceLayout L = slice_layout(g->d.n, kmax);
+    // the graph rides in shared memory when it fits beside the programme's arrays
+    int staged_edges = g->m > 0 ? g->m : 1;
+    SliceLayout L = slice_layout(g->d.n, kmax, staged_edges);
+    if (L.total > kSliceSmemLimit) {
+        staged_edges = 0;
+        L = slice_layout(g->d.n, kmax, 0);
+    }
     cudaError_t e = cudaSuccess;
     if (L.total > 48 * 1024) e = allow_slice_smem(g->device);
     if (e != cudaSuccess) return cuda_fail(e);
     slice_orders<<<unsigned(P), kSliceThreads, L.total, static_cast<cudaStream_t>(cuda_stream)>>>(
-        g->d, orders, k, static_cast<long long>(B), static_cast<long long>(M), reinterpret_cast<long long*>(cost_out), blocks_out, cuts_out, status_out);
+        g->d, staged_edges, orders, k, static_cast<long long>(B), static_cast<long long>(M), reinterpret_cast<long long*>(cost_out), blocks_out, cuts_out, status_out);
     e = cudaGetLastError();
     return e == cudaSuccess ? BQ_OK : cuda_fail(e);
 }
