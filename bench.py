@@ -271,7 +271,7 @@ def run_ours(args):
                              "kernels": kernels, "input_sha256": input_sha})
 
     # end to end: host buffers in, host buffers out, copies inside the timed region
-    e2e = run_e2e(bq, cb, x_pin, dev, w.dtype, n, args, world)
+    e2e = guarded("e2e", lambda: run_e2e(bq, cb, x_pin, dev, w.dtype, n, args, world))
     if rank == 0:
         progress("e2e", e2e)
     full = WORKLOAD == "sweep1g"                     # the variants and the other configurations ride on the headline run only
@@ -290,88 +290,32 @@ def run_ours(args):
     if rank == 0:
         progress("quality", quality)
 
-    # the 4-bit variant of the same path (16-entry codebook, two codes per byte) on the same tensor
-    cb4 = bq.Codebook4()
-    bq4 = {}
-    for b, s16 in (((64, False), (1024, False), (64, True)) if full else ()):       # s16: the block scale stored as a bf16 (2 bytes instead of 4)
-        packed = codes[: n // 2]
-        scale16 = absmax[b].view(torch.bfloat16)[: n // b]
-        times = {}
-        if s16:
-            ops = (("quantize4", lambda: bq.bq4_quantize_s16(x, b, cb4, packed, scale16)),
-                   ("dequantize4", lambda: bq.bq4_dequantize_s16(packed, scale16, n, b, cb4, w.dtype, y)))
-        else:
-            ops = (("quantize4", lambda: bq.bq4_quantize(x, b, cb4, packed, absmax[b])),
-                   ("dequantize4", lambda: bq.bq4_dequantize(packed, absmax[b], n, b, cb4, w.dtype, y)))
-        for op, fn in ops:
-            for _ in range(3):
-                fn()
-            ev = []
-            for _ in range(10):
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record(); fn(); e1.record()
-                ev.append((e0, e1))
-            torch.cuda.synchronize()
-            times[op] = float(np.mean([a.elapsed_time(b_) for a, b_ in ev]))
-        scale_bytes = 2 if s16 else 4
-        ab = n * 2 + n // 2 + scale_bytes * (n // b)
-        num = torch.zeros((), dtype=torch.float64, device=dev)
-        den = torch.zeros((), dtype=torch.float64, device=dev)
-        for s in range(0, n, 1 << 27):
-            xs, ys = x[s:s + (1 << 27)].float(), y[s:s + (1 << 27)].float()
-            num += ((xs - ys) ** 2).sum(dtype=torch.float64)
-            den += (xs ** 2).sum(dtype=torch.float64)
-        bq4[f"b{b}" + ("_scale16" if s16 else "")] = {
-            "quantize_ms": round(times["quantize4"], 4), "dequantize_ms": round(times["dequantize4"], 4), "algorithmic_bytes": int(ab),
-            "quantize_frac_of_measured": round(ab / times["quantize4"] / 1e6 / peak, 4),
-            "dequantize_frac_of_measured": round(ab / times["dequantize4"] / 1e6 / peak, 4),
-            "compression_ratio": round(2.0 * n / (n / 2 + scale_bytes * (n // b)), 3),
-            "rel_rms_error": round(float((num / den).sqrt().item()), 5), "gpu_launches": 26}
-
+    bq4 = guarded("bq4", lambda: run_bq4(bq, dev, x, y, codes, absmax, n, w, peak)) if full else {}
     if rank == 0 and full:
         progress("bq4", bq4)
-    cpu = cpu_baseline(x_pin, w, rank) if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
+    cpu = guarded("cpu_baseline", lambda: cpu_baseline(x_pin, w, rank)) if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
     if cpu is not None:
         progress("cpu_baseline", cpu)
     if not full:
         return finish(rank, world, args, value, max_s, n, w, e2e, events, clocks, roofline, kernels, quality, cpu, input_sha,
                       None, None, None, None)
 
-    # block-size selection on the same tensor: the roundtrip and the error sums of four candidates in one call
-    tune_blocks = [64, 256, 1024, 4096]
-    tune_ws = torch.empty(bq.tune.workspace_bytes(w.dtype, n), dtype=torch.uint8, device=dev)
-    tune_sums = torch.empty(len(tune_blocks) + 1, dtype=torch.float64, device=dev)
-    for _ in range(2):
-        bq.tune.block_errors(x, tune_blocks, cb, tune_ws, tune_sums)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(5):
-        bq.tune.block_errors(x, tune_blocks, cb, tune_ws, tune_sums)
-    e1.record()
-    torch.cuda.synchronize()
-    tune_ms = e0.elapsed_time(e1) / 5
-    tune_bytes = len(tune_blocks) * 4 * n * 2                     # per candidate: roundtrip reads x and writes y, the sums read both
-    sums_host = tune_sums.cpu().numpy()
-    tune = {"blocks": tune_blocks, "ms_per_call": round(tune_ms, 4), "algorithmic_bytes": int(tune_bytes),
-            "frac_of_measured": round(tune_bytes / tune_ms / 1e6 / peak, 4),
-            "rel_rms_error": [round(float(v), 5) for v in np.sqrt(sums_host[:-1] / sums_host[-1])],
-            "picked_for_rel_rms_0.01": bq.tune.pick_block(tune_blocks, sums_host, 0.01), "gpu_launches": 7 * 3 * len(tune_blocks)}
-    del tune_ws
+    tune = guarded("autotune", lambda: run_autotune(bq, dev, x, cb, n, w, peak))
     if rank == 0:
         progress("autotune", tune)
 
     del x, y, codes, absmax
     torch.cuda.empty_cache()
-    small = run_small(bq, dev) if rank == 0 else None
+    small = guarded("small_configs", lambda: run_small(bq, dev)) if rank == 0 else None
     if rank == 0:
         progress("small_configs", small)
-    mmd = run_mmd(bq, dev, args) if (rank == 0 and not args.no_mmd) else None
+    mmd = guarded("mmd", lambda: run_mmd(bq, dev, args)) if (rank == 0 and not args.no_mmd) else None
     if mmd is not None:
         progress("mmd", mmd)
-    transport = run_transport(bq, dev, args) if (rank == 0 and not args.no_transport) else None
+    transport = guarded("transport", lambda: run_transport(bq, dev, args)) if (rank == 0 and not args.no_transport) else None
     if transport is not None:
         progress("transport", transport)
-    mtpp = run_mtpp(bq, dev, args) if (rank == 0 and not args.no_mtpp) else None
+    mtpp = guarded("mtpp", lambda: run_mtpp(bq, dev, args)) if (rank == 0 and not args.no_mtpp) else None
     if mtpp is not None:
         progress("mtpp", mtpp)
     return finish(rank, world, args, value, max_s, n, w, e2e, events, clocks, roofline, kernels, quality, cpu, input_sha,
@@ -407,6 +351,80 @@ def finish(rank, world, args, value, max_s, n, w, e2e, events, clocks, roofline,
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
+
+
+def guarded(name: str, fn):
+    """The sections beside the headline measurement must not take the line down with them: an exception in one of them is
+    recorded under its key (and on stderr) and the run goes on."""
+    try:
+        return fn()
+    except Exception as exc:                                   # noqa: BLE001 - whatever it is, the headline numbers are kept
+        sys.stderr.write(f"bench.py: section {name} failed: {exc!r}\n")
+        return {"error": repr(exc)}
+
+
+def run_bq4(bq, dev, x, y, codes, absmax, n, w, peak):
+    """The 4-bit variant of the same path (16-entry codebook, two codes per byte) on the same tensor."""
+    cb4 = bq.Codebook4()
+    bq4 = {}
+    for b, s16 in ((64, False), (1024, False), (64, True)):       # s16: the block scale stored as a bf16 (2 bytes instead of 4)
+        packed = codes[: n // 2]
+        scale16 = absmax[b].view(torch.bfloat16)[: n // b]
+        times = {}
+        if s16:
+            ops = (("quantize4", lambda: bq.bq4_quantize_s16(x, b, cb4, packed, scale16)),
+                   ("dequantize4", lambda: bq.bq4_dequantize_s16(packed, scale16, n, b, cb4, w.dtype, y)))
+        else:
+            ops = (("quantize4", lambda: bq.bq4_quantize(x, b, cb4, packed, absmax[b])),
+                   ("dequantize4", lambda: bq.bq4_dequantize(packed, absmax[b], n, b, cb4, w.dtype, y)))
+        for op, fn in ops:
+            for _ in range(3):
+                fn()
+            ev = []
+            for _ in range(10):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); fn(); e1.record()
+                ev.append((e0, e1))
+            torch.cuda.synchronize()
+            times[op] = float(np.mean([a.elapsed_time(b_) for a, b_ in ev]))
+        scale_bytes = 2 if s16 else 4
+        ab = n * 2 + n // 2 + scale_bytes * (n // b)
+        num = torch.zeros((), dtype=torch.float64, device=dev)
+        den = torch.zeros((), dtype=torch.float64, device=dev)
+        for s in range(0, n, 1 << 27):
+            xs, ys = x[s:s + (1 << 27)].float(), y[s:s + (1 << 27)].float()
+            num += ((xs - ys) ** 2).sum(dtype=torch.float64)
+            den += (xs ** 2).sum(dtype=torch.float64)
+        bq4[f"b{b}" + ("_scale16" if s16 else "")] = {
+            "quantize_ms": round(times["quantize4"], 4), "dequantize_ms": round(times["dequantize4"], 4), "algorithmic_bytes": int(ab),
+            "quantize_frac_of_measured": round(ab / times["quantize4"] / 1e6 / peak, 4),
+            "dequantize_frac_of_measured": round(ab / times["dequantize4"] / 1e6 / peak, 4),
+            "compression_ratio": round(2.0 * n / (n / 2 + scale_bytes * (n // b)), 3),
+            "rel_rms_error": round(float((num / den).sqrt().item()), 5), "gpu_launches": 26}
+    return bq4
+
+
+def run_autotune(bq, dev, x, cb, n, w, peak):
+    """Block-size selection on the same tensor: the roundtrip and the error sums of four candidates in one call."""
+    tune_blocks = [64, 256, 1024, 4096]
+    tune_ws = torch.empty(bq.tune.workspace_bytes(w.dtype, n), dtype=torch.uint8, device=dev)
+    tune_sums = torch.empty(len(tune_blocks) + 1, dtype=torch.float64, device=dev)
+    for _ in range(2):
+        bq.tune.block_errors(x, tune_blocks, cb, tune_ws, tune_sums)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(5):
+        bq.tune.block_errors(x, tune_blocks, cb, tune_ws, tune_sums)
+    e1.record()
+    torch.cuda.synchronize()
+    tune_ms = e0.elapsed_time(e1) / 5
+    tune_bytes = len(tune_blocks) * 4 * n * 2                     # per candidate: roundtrip reads x and writes y, the sums read both
+    sums_host = tune_sums.cpu().numpy()
+    tune = {"blocks": tune_blocks, "ms_per_call": round(tune_ms, 4), "algorithmic_bytes": int(tune_bytes),
+            "frac_of_measured": round(tune_bytes / tune_ms / 1e6 / peak, 4),
+            "rel_rms_error": [round(float(v), 5) for v in np.sqrt(sums_host[:-1] / sums_host[-1])],
+            "picked_for_rel_rms_0.01": bq.tune.pick_block(tune_blocks, sums_host, 0.01), "gpu_launches": 7 * 3 * len(tune_blocks)}
+    return tune
 
 
 # ------------------------------------------------------------------------------------------ the small configurations
