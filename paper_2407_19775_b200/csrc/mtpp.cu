@@ -8,9 +8,9 @@
 //               in l..r-1 yet, i.e. for l > max(pos(u), position of u's previous consumer);
 //     out(l, r) gains sizeout(v) if v has consumers (they all come later), and loses sizeout(u)
 //               for each producer u of v inside l..r whose last consumer is v.
-// So a CTA keeps five running values per l (one thread per l), the dp rows of every block count,
-// and the positions of each node, its last consumer and its latest consumer so far: a few tens
-// of kilobytes of shared memory, no global scratch.  Per step one barrier separates the column
+// So a CTA keeps five running values per l (in the registers of the thread that owns l), the dp rows
+// of every block count, and the positions of each node, its last consumer and its latest
+// consumer so far: a few tens of kilobytes of shared memory, no global scratch.  Per step one barrier separates the column
 // update from the minimisations, which warp kk does for block count kk.
 #include "../../include/mtpp.h"
 #include "bq_error.h"
@@ -26,7 +26,7 @@ namespace {
 constexpr int kSliceThreads = 256;
 constexpr int kDecodeWarps = 4;
 constexpr long long kInf = 0x7fffffffffffffffLL;
-constexpr size_t kSliceSmemLimit = 227 * 1024;         // what one CTA may take
+constexpr size_t kSliceSmemLimit = 226 * 1024;         // dynamic part of the 227 KB one CTA may take; the kernel's static words fit in the rest
 
 int cuda_fail(cudaError_t e) {
     bql::set_last_cuda_error(cudaGetErrorString(e));
@@ -48,7 +48,7 @@ __host__ __device__ inline size_t round_up(size_t v, size_t a) { return (v + a -
 
 // Shared memory of slice_orders for (n, kmax): 64-bit arrays first, then 32-bit, then 16-bit.
 struct SliceLayout {
-    size_t col, f, dp, attr, pos, last, prev, pptr, pred, order, arg, total;
+    size_t f, dp, attr, pos, last, prev, pptr, pred, order, arg, total;
 };
 // `edges` > 0: the graph itself (attributes, producer lists) and the order are staged in shared memory too, so that the n
 // dependent steps of the programme never wait for global memory; 0: they are read from global memory (graphs too large
@@ -56,7 +56,6 @@ struct SliceLayout {
 __host__ __device__ inline SliceLayout slice_layout(int n, int kmax, int edges) {
     SliceLayout L;
     size_t o = 0;
-    L.col = o;  o += size_t(5) * n * 8;                 // work | param | peak | in | out, indexed by l - 1
     L.f = o;    o += size_t(n) * 8;                     // F(l, r) of the current r
     L.dp = o;   o += size_t(kmax) * (n + 1) * 8;        // dp[kk - 1][r]
     L.attr = o; o += edges > 0 ? size_t(3) * n * 8 : 0; // work | sizeparam | sizeout of the nodes
@@ -71,6 +70,7 @@ __host__ __device__ inline SliceLayout slice_layout(int n, int kmax, int edges) 
     return L;
 }
 
+template <int kOwned>                                               // first positions per thread: n <= kOwned * kSliceThreads
 __global__ void __launch_bounds__(kSliceThreads)
 slice_orders(DeviceGraph g, int staged_edges, const int* __restrict__ orders, int k, long long B, long long M, long long* __restrict__ cost_out,
              int* __restrict__ blocks_out, int* __restrict__ cuts_out, int* __restrict__ status_out) {
@@ -78,11 +78,6 @@ slice_orders(DeviceGraph g, int staged_edges, const int* __restrict__ orders, in
     const int n = g.n;
     const int kmax = k < n ? k : n;
     const SliceLayout L = slice_layout(n, kmax, staged_edges);
-    long long* c_work = reinterpret_cast<long long*>(smem + L.col);
-    long long* c_param = c_work + n;
-    long long* c_peak = c_param + n;
-    long long* c_in = c_peak + n;
-    long long* c_out = c_in + n;
     long long* F = reinterpret_cast<long long*>(smem + L.f);
     long long* dp = reinterpret_cast<long long*>(smem + L.dp);
     int* pos = reinterpret_cast<int*>(smem + L.pos);
@@ -139,30 +134,33 @@ slice_orders(DeviceGraph g, int staged_edges, const int* __restrict__ orders, in
         return;
     }
 
+    long long cw[kOwned], cp[kOwned], ck[kOwned], ci[kOwned], co[kOwned];
+#pragma unroll
+    for (int j = 0; j < kOwned; ++j) { cw[j] = 0; cp[j] = 0; ck[j] = 0; ci[j] = 0; co[j] = 0; }
     for (int r = 1; r <= n; ++r) {
         const int v = pi[r - 1];
         const int pb = pred_ptr[v], pe = pred_ptr[v + 1];
         const long long so_v = a_out[v], w_v = a_work[v], pa_v = a_param[v];
         const long long gain_out = (last[v] != 0) ? so_v : 0;            // v has consumers (they all come later)
-        // the column of r: one thread per first position l
-        for (int l = tid + 1; l <= r; l += kSliceThreads) {
-            long long cw, cp, ck, ci, co;
-            if (l == r) { cw = 0; cp = 0; ck = 0; ci = 0; co = 0; }
-            else { cw = c_work[l - 1]; cp = c_param[l - 1]; ck = c_peak[l - 1]; ci = c_in[l - 1]; co = c_out[l - 1]; }
-            cw += w_v;
-            cp += pa_v;
-            ck = so_v > ck ? so_v : ck;
-            co += gain_out;
+        // the column of r: thread t owns the first positions l = t + 1, t + 257, ... and keeps their five running values in registers
+#pragma unroll
+        for (int j = 0; j < kOwned; ++j) {
+            const int l = tid + 1 + j * kSliceThreads;
+            if (l > r) continue;
+            if (l == r) { cw[j] = 0; cp[j] = 0; ck[j] = 0; ci[j] = 0; co[j] = 0; }
+            cw[j] += w_v;
+            cp[j] += pa_v;
+            ck[j] = so_v > ck[j] ? so_v : ck[j];
+            co[j] += gain_out;
             for (int e = pb; e < pe; ++e) {
                 const int u = pred[e];
                 const int pu = pos[u], pc = prev[u];
                 const long long so_u = a_out[u];
-                if (l > (pu > pc ? pu : pc)) ci += so_u;             // u lies before l and nothing in l..r-1 read it
-                if (last[u] == r && pu >= l) co -= so_u;              // u is inside and v was its last consumer
+                if (l > (pu > pc ? pu : pc)) ci[j] += so_u;          // u lies before l and nothing in l..r-1 read it
+                if (last[u] == r && pu >= l) co[j] -= so_u;           // u is inside and v was its last consumer
             }
-            c_work[l - 1] = cw; c_param[l - 1] = cp; c_peak[l - 1] = ck; c_in[l - 1] = ci; c_out[l - 1] = co;
-            const long long excess = cp + ck - M;
-            F[l - 1] = ci + B * cw + (excess > 0 ? excess : 0) + ck + co;
+            const long long excess = cp[j] + ck[j] - M;
+            F[l - 1] = ci[j] + B * cw[j] + (excess > 0 ? excess : 0) + ck[j] + co[j];
         }
         __syncthreads();
         // dp[kk][r] = min over l of max(dp[kk - 1][l], F(l + 1, r)); the earlier l on equal values
@@ -178,12 +176,14 @@ slice_orders(DeviceGraph g, int staged_edges, const int* __restrict__ orders, in
                     const long long cand = a > b ? a : b;
                     if (cand < best) { best = cand; where = l; }     // l ascends within a lane: strict < keeps the earlier one
                 }
-#pragma unroll
-                for (int s = 16; s >= 1; s >>= 1) {
-                    const long long ob = __shfl_xor_sync(0xffffffffu, best, s);
-                    const int ow = __shfl_xor_sync(0xffffffffu, where, s);
-                    if (ob < best || (ob == best && ob != kInf && ow < where)) { best = ob; where = ow; }
-                }
+                // the warp's smallest (value, position) pair by three 32-bit reductions: the high words, then the low words
+                // among the lanes that hold the smallest high word, then the positions among the lanes that hold the smallest value
+                const unsigned hi = unsigned(static_cast<unsigned long long>(best) >> 32), lo = unsigned(static_cast<unsigned long long>(best));
+                const unsigned mh = __reduce_min_sync(0xffffffffu, hi);
+                const unsigned ml = __reduce_min_sync(0xffffffffu, hi == mh ? lo : 0xffffffffu);
+                const unsigned mi = __reduce_min_sync(0xffffffffu, (hi == mh && lo == ml) ? unsigned(where) : 0x7fffffffu);
+                best = static_cast<long long>((static_cast<unsigned long long>(mh) << 32) | ml);
+                where = int(mi);
             }
             if (lane == 0) {
                 dp[size_t(kk - 1) * (n + 1) + r] = best;
@@ -273,7 +273,9 @@ cudaError_t allow_slice_smem(int device) {
     std::lock_guard<std::mutex> guard(g_attr_lock);
     const bool tracked = device >= 0 && device < 64;
     if (tracked && g_attr_done[device]) return cudaSuccess;
-    const cudaError_t e = cudaFuncSetAttribute(slice_orders, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSliceSmemLimit));
+    cudaError_t e = cudaFuncSetAttribute(slice_orders<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSliceSmemLimit));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(slice_orders<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSliceSmemLimit));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(slice_orders<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSliceSmemLimit));
     if (e == cudaSuccess && tracked) g_attr_done[device] = true;
     return e;
 }
@@ -401,7 +403,9 @@ int mtpp_slice_orders(const mtpp_graph* g, const int32_t* orders, int P, int k, 
     cudaError_t e = cudaSuccess;
     if (L.total > 48 * 1024) e = allow_slice_smem(g->device);
     if (e != cudaSuccess) return cuda_fail(e);
-    slice_orders<<<unsigned(P), kSliceThreads, L.total, static_cast<cudaStream_t>(cuda_stream)>>>(
+    static_assert(MTPP_MAX_NODES <= 4 * kSliceThreads, "the widest instance owns four first positions per thread");
+    auto* kernel = g->d.n <= kSliceThreads ? slice_orders<1> : g->d.n <= 2 * kSliceThreads ? slice_orders<2> : slice_orders<4>;
+    kernel<<<unsigned(P), kSliceThreads, L.total, static_cast<cudaStream_t>(cuda_stream)>>>(
         g->d, staged_edges, orders, k, static_cast<long long>(B), static_cast<long long>(M), reinterpret_cast<long long*>(cost_out), blocks_out, cuts_out, status_out);
     e = cudaGetLastError();
     return e == cudaSuccess ? BQ_OK : cuda_fail(e);

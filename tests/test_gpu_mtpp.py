@@ -88,6 +88,78 @@ def test_random_graphs_fuzz(bq):
         dg.close()
 
 
+def banded_graph(n, seed):
+    rng = random.Random(seed)
+    edges = np.asarray([(u, v) for u in range(n) for v in range(u + 1, min(n, u + 40)) if rng.random() < 0.08], np.int32).reshape(-1, 2)
+    work = np.asarray([rng.randrange(0, 50) for _ in range(n)], np.int64)
+    sizeparam = np.asarray([rng.randrange(0, 500) for _ in range(n)], np.int64)
+    sizeout = np.asarray([rng.randrange(0, 80) for _ in range(n)], np.int64)
+    return edges, work, sizeparam, sizeout
+
+
+@pytest.mark.parametrize("n,k", [(257, 16), (300, 5), (520, 3)])
+def test_graphs_wider_than_one_position_per_thread(bq, n, k):
+    """Above 256 and above 512 nodes a thread of the slicing kernel owns two and four first positions: one order of each in
+    full against the oracle."""
+    edges, work, sizeparam, sizeout = banded_graph(n, n)
+    g = oracle_graph(n, edges, work, sizeparam, sizeout)
+    dg = bq.mtpp.SliceGraph(n, edges, work, sizeparam, sizeout, device="cuda:0")
+    keys = torch.rand((3, n), generator=torch.Generator().manual_seed(n))
+    orders = dg.decode_orders(keys.cuda())
+    cost, blocks, cuts, status = dg.slice_orders(orders, k, 3, 20000)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [0, 0, 0]
+    pi = orders[1].cpu().tolist()
+    assert pi == mo.decode_order(g, keys[1].tolist())
+    assert (int(cost[1]), int(blocks[1]), cuts[1][:int(blocks[1])].cpu().tolist()) == mo.slice_order(g, pi, k, 3, 20000)
+    dg.close()
+
+
+def test_largest_graph(bq):
+    """1024 nodes, 16 blocks, the limits of the call.  A chain of equal nodes has a closed form: every block's cost grows with
+    its length, so the best slicing is the balanced one and its bottleneck is the cost of an inner block of ceil(n / k) nodes.
+    On a banded random graph the oracle re-costs the returned cuts (16 blocks an order) and no perturbed cut set does better."""
+    n, k, B, M = 1024, 16, 3, 20000
+    chain = np.asarray([(i, i + 1) for i in range(n - 1)], np.int32)
+    ones = np.ones(n, np.int64)
+    g = oracle_graph(n, chain, 7 * ones, 300 * ones, 11 * ones)
+    dg = bq.mtpp.SliceGraph(n, chain, 7 * ones, 300 * ones, 11 * ones, device="cuda:0")
+    orders = dg.decode_orders(torch.rand((2, n), generator=torch.Generator().manual_seed(1)).cuda())
+    assert orders.cpu().tolist() == [list(range(n))] * 2                   # a chain has one topological order
+    cost, blocks, cuts, status = dg.slice_orders(orders, k, B, M)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [0, 0]
+    assert cost.cpu().tolist() == [mo.segment_cost(g, list(range(n)), 65, 128, B, M)] * 2
+    ends = cuts[0][:int(blocks[0])].cpu().tolist()
+    assert max(e - s for s, e in zip([0] + ends[:-1], ends)) == 64 and ends[-1] == n
+    dg.close()
+
+    edges, work, sizeparam, sizeout = banded_graph(n, 5)
+    g = oracle_graph(n, edges, work, sizeparam, sizeout)
+    dg = bq.mtpp.SliceGraph(n, edges, work, sizeparam, sizeout, device="cuda:0")
+    keys = torch.rand((4, n), generator=torch.Generator().manual_seed(2))
+    orders = dg.decode_orders(keys.cuda())
+    cost, blocks, cuts, status = dg.slice_orders(orders, k, B, M)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [0] * 4
+    rng = random.Random(9)
+
+    def bottleneck(pi, ends):
+        return max(mo.segment_cost(g, pi, s, e, B, M) for s, e in zip([1] + [e + 1 for e in ends[:-1]], ends))
+
+    for p in range(4):
+        pi = orders[p].cpu().tolist()
+        assert pi == mo.decode_order(g, keys[p].tolist())
+        ends = cuts[p][:int(blocks[p])].cpu().tolist()
+        assert ends == sorted(set(ends)) and ends[-1] == n and 1 <= len(ends) <= k
+        assert bottleneck(pi, ends) == int(cost[p])
+        for _ in range(6):                                                # other cut sets: a nudge of every cut, and a fresh draw
+            nudged = sorted({min(n - 1, max(1, e + rng.randrange(-2, 3))) for e in ends[:-1]}) + [n]
+            drawn = sorted(rng.sample(range(1, n), k - 1)) + [n]
+            assert bottleneck(pi, nudged) >= int(cost[p]) and bottleneck(pi, drawn) >= int(cost[p])
+    dg.close()
+
+
 def test_rows_that_are_not_topological_orders_are_flagged(bq):
     n, edges, work, sizeparam, sizeout = workloads.make_graph("mtpp_tiny")
     g = oracle_graph(n, edges, work, sizeparam, sizeout)
