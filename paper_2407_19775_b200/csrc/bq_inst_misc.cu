@@ -41,9 +41,9 @@ constexpr int kDeqU = BQ_DEQ_U;
 template <int YDT, bool WIDE>
 cudaError_t deq_fast_go(const uint8_t* codes, const float* absmax, void* y, size_t n16, int log2_block, const bqk::DeviceTables& tab,
                         int sm_count, cudaStream_t stream) {
-    if (n16 <= (size_t(1) << (BQ_LITE_MAX_LOG2 + 2 - 4))) {      // up to 8 Mi elements: no shared-memory table, one chunk per thread
+    if (n16 <= (size_t(1) << (BQ_LITE_MAX_LOG2 + 2 - 4))) {      // up to 8 Mi elements: one plain copy of the values, one chunk per thread
         const size_t grid = (n16 + 255) / 256;
-        bqk::deq_fast<YDT, 256, 1, true, WIDE><<<unsigned(grid), 256, 0, stream>>>(codes, absmax, y, n16, log2_block, tab);
+        bqk::deq_fast<YDT, 256, 1, true, WIDE><<<unsigned(grid), 256, bqk::kDeqLiteSmemBytes, stream>>>(codes, absmax, y, n16, log2_block, tab);
         return cudaGetLastError();
     }
     const size_t tile = size_t(kDeqNT) * kDeqU;

@@ -8,7 +8,8 @@
 //                  per lane in shared memory (large tensors), and LITE, which reads the
 //                  tables through L1 and has no set-up (small tensors).
 //   deq_fast     : dequantize, 16 codes per 128-bit load, one 256-bit store per 16 outputs;
-//                  the same two flavours.
+//                  the same two flavours (its LITE one keeps one plain 1 KB copy of the
+//                  values in shared memory: a word per thread to fill).
 //   *_general    : any block size, any alignment, any codebook; one warp per block.
 //
 // Arithmetic contract shared by all of them (it is what makes the results bit-identical
@@ -41,6 +42,7 @@ constexpr uint32_t kFwdSmemBytes = kRedOff + 2u * 32u * 4u + 128u;    // + slack
 constexpr uint32_t kFwdLiteSmemBytes = 2u * 32u * 4u + 128u;
 
 constexpr uint32_t kDeqSmemBytes = 256u * 128u;         // signed code values, replicated per lane
+constexpr uint32_t kDeqLiteSmemBytes = 256u * 4u;       // LITE: one plain copy
 
 struct DeviceTables {
     const float* values;        // [256]
@@ -637,11 +639,16 @@ deq_fast(const uint8_t* __restrict__ codes, const float* __restrict__ absmax, vo
             for (int k = 0; k < 32; ++k) sts_u32(sm_lane + uint32_t(row0 + k) * 128u, __shfl_sync(0xffffffffu, mine, k));
         }
         __syncthreads();
+    } else {
+        // one plain copy of the 256 values (kDeqLiteSmemBytes)
+        for (int i = threadIdx.x; i < 256; i += NT) sts_u32(sm_base + uint32_t(i) * 4u, __float_as_uint(__ldg(tab.values + i)));
+        __syncthreads();
     }
     // value of one code byte sitting at bit `shift` of a packed word
     auto value = [&](uint32_t word, int shift) -> float {
         if constexpr (LITE) {
-            return __ldg(tab.values + ((word >> shift) & 0xffu));
+            const uint32_t off = (shift >= 2 ? (word >> (shift - 2)) : (word << (2 - shift))) & 0x3fcu;
+            return __uint_as_float(lds_u32(sm_base + off));
         } else {
             const uint32_t row = (shift >= 7 ? (word >> (shift - 7)) : (word << (7 - shift))) & 0x7f80u;
             return __uint_as_float(lds_u32(sm_lane + row));
