@@ -95,7 +95,7 @@ fwd_staged(const void* __restrict__ x, void* __restrict__ y, uint8_t* __restrict
     const uint32_t ctrl = sm_base + kRedOff + 128u + uint32_t(team) * (STAGES * 8u + 48u);
     const uint32_t full0 = ctrl;                                            // STAGES mbarriers
     const uint32_t part0 = ctrl + STAGES * 8u;                              // 8 partial maxima
-    const uint32_t flag = part0 + 32u;                                      // the elected thread's verdict on the wait
+    const uint32_t flag = part0 + 32u;                                      // what the elected thread's wait came to
     const uint32_t ring = sm_base + kStagedRingOff + uint32_t(team) * STAGES * Cfg::kBlockBytes;
 
     fill_fwd_tables<NT>(tab, sm_base);

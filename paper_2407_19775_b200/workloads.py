@@ -247,7 +247,7 @@ GRAPH_WORKLOADS = {
     "mtpp_heads": GraphWorkload("mtpp_heads", "heads", 96, 4, 24, 125, 6 << 20, 21,
                                 "a trunk of 40 operations and 4 heads of 8..20 operations reading different trunk depths; 1 Gbit/s link"),
     "mtpp_unet": GraphWorkload("mtpp_unet", "unet", 256, 8, 2048, 125, 48 << 20, 22,
-                               "U-shaped denoiser: 8 stages down, 8 up, skip connections, one conditioning node feeding every stage; 1 Gbit/s link"),
+                               "U-shaped denoiser: 7 stages down, one across, 7 up, each an entry, three parallel branches, a merge and a closing operation; skip connections; one conditioning node feeding every stage; 1 Gbit/s link"),
 }
 
 
@@ -272,15 +272,30 @@ def make_graph(name: str):
             at += depth
         assert at == n
     else:
-        stages, per = 8, (n - 1) // 16                        # node 0 is the conditioning node
-        body = list(range(1, 1 + 16 * per))
-        extra = list(range(1 + 16 * per, n))                  # left-over nodes extend the last stage
-        chain = body + extra
-        edges += [(a, b) for a, b in zip(chain, chain[1:])]
-        for s in range(16):
-            edges.append((0, chain[s * per]))                 # conditioning enters every stage
+        # node 0 is the conditioning node; then stages of 17 operations: an entry, three parallel branches of 7, 5 and 2
+        # operations (so that a stage has many topological orders), a merge and a closing operation
+        per, branches = 17, (7, 5, 2)
+        stages = (n - 1) // per
+        assert 1 + stages * per == n and stages % 2 == 1
+        closing = []
+        merges = []
         for s in range(stages):
-            edges.append((chain[s * per + per - 1], chain[(15 - s) * per]))      # skip: end of down-stage s -> start of up-stage 15 - s
+            entry = 1 + s * per
+            edges.append((0, entry))                          # conditioning enters every stage
+            if s:
+                edges.append((closing[-1], entry))
+            at = entry + 1
+            merge = entry + 1 + sum(branches)
+            for depth in branches:
+                edges.append((entry, at))
+                edges += [(at + i, at + i + 1) for i in range(depth - 1)]
+                edges.append((at + depth - 1, merge))
+                at += depth
+            edges.append((merge, merge + 1))
+            merges.append(merge)
+            closing.append(merge + 1)
+        for s in range(stages // 2):
+            edges.append((closing[s], merges[stages - 1 - s]))                   # skip: end of down-stage s -> merge of its up-stage
     work = rng.integers(20, 2000, n)
     sizeparam = rng.integers(0, 8 << 20, n) * (rng.random(n) < 0.6)
     sizeout = rng.integers(64 << 10, 4 << 20, n)
