@@ -19,13 +19,13 @@
 
 #include <mutex>
 #include <new>
+#include <type_traits>
 #include <vector>
 
 namespace {
 
 constexpr int kSliceThreads = 256;
 constexpr int kDecodeWarps = 4;
-constexpr long long kInf = 0x7fffffffffffffffLL;
 constexpr size_t kSliceSmemLimit = 226 * 1024;         // dynamic part of the 227 KB one CTA may take; the kernel's static words fit in the rest
 
 int cuda_fail(cudaError_t e) {
@@ -35,6 +35,7 @@ int cuda_fail(cudaError_t e) {
 
 struct DeviceGraph {
     int n;
+    int edges;                 // distinct (producer, consumer) pairs
     const int* pred_ptr;       // [n + 1]
     const int* pred;           // producers of each node
     const int* cons_ptr;       // [n + 1]
@@ -46,43 +47,82 @@ struct DeviceGraph {
 
 __host__ __device__ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// Shared memory of slice_orders for (n, kmax): 64-bit arrays first, then 32-bit, then 16-bit.
+// Shared memory of slice_orders for (n, kmax) and costs of `cs` bytes (8, or 4 when every segment cost of the call fits a
+// signed 32-bit word): 16-byte records first, then the cost arrays, then 32-bit, then 16-bit.
 struct SliceLayout {
-    size_t f, dp, attr, pos, last, prev, pptr, pred, order, arg, total;
+    size_t attr, f, dp, eso, pos, last, epos, order, ethr, epu, arg, total;
 };
-// `edges` > 0: the graph itself (attributes, producer lists) and the order are staged in shared memory too, so that the n
-// dependent steps of the programme never wait for global memory; 0: they are read from global memory (graphs too large
-// to fit beside the programme's own arrays).
-__host__ __device__ inline SliceLayout slice_layout(int n, int kmax, int edges) {
+// `edges` > 0: the producer edges of the order, re-laid in the order's own sequence (see the kernel), sit in shared memory
+// too; 0: graphs with too many edges to fit beside the programme's arrays look them up in global memory at every step.
+__host__ __device__ inline SliceLayout slice_layout(int n, int kmax, int edges, int cs) {
     SliceLayout L;
     size_t o = 0;
-    L.f = o;    o += size_t(n) * 8;                     // F(l, r) of the current r
-    L.dp = o;   o += size_t(kmax) * (n + 1) * 8;        // dp[kk - 1][r]
-    L.attr = o; o += edges > 0 ? size_t(3) * n * 8 : 0; // work | sizeparam | sizeout of the nodes
-    L.pos = o;  o += size_t(n) * 4;                     // 1-based position of each node (0: not seen)
-    L.last = o; o += size_t(n) * 4;                     // position of each node's last consumer (0: none)
-    L.prev = o; o += size_t(n) * 4;                     // position of each node's latest consumer so far (0: none)
-    L.pptr = o; o += edges > 0 ? size_t(n + 1) * 4 : 0; // producer lists: offsets ...
-    L.pred = o; o += edges > 0 ? size_t(edges) * 4 : 0; // ... and entries
-    L.order = o; o += edges > 0 ? size_t(n) * 4 : 0;    // the order itself
-    L.arg = o;  o += size_t(kmax) * (n + 1) * 2;        // the cut that gave dp[kk - 1][r]
+    L.attr = o; o += size_t(4) * n * cs;                               // by position: work, sizeparam, sizeout, sizeout if it has consumers
+    L.f = o;    o += round_up(size_t(2) * n * cs, 8);                  // F(l, r) of the current r and of the next one
+    L.dp = o;   o += round_up(size_t(kmax) * (n + 1) * cs, 8);         // dp[kk - 1][r]
+    L.eso = o;  o += round_up(size_t(edges) * cs, 8);                  // per edge: the producer's sizeout
+    L.pos = o;  o += size_t(n) * 4;                                    // 1-based position of each node (0: not seen)
+    L.last = o; o += size_t(n) * 4;                                    // position of each node's last consumer (0: none)
+    L.epos = o; o += size_t(n + 1) * 4;                                // edges of position r: [epos[r - 1], epos[r])
+    L.order = o; o += size_t(n) * 4;                                   // the order itself
+    L.ethr = o; o += round_up(size_t(edges) * 2, 4);                   // per edge: max(producer's position, its latest consumer before r)
+    L.epu = o;  o += round_up(size_t(edges) * 2, 4);                   // per edge: producer's position if r is its last consumer, else 0
+    L.arg = o;  o += size_t(kmax) * (n + 1) * 2;                       // the cut that gave dp[kk - 1][r]
     L.total = (o + 15) / 16 * 16;
     return L;
 }
 
-template <int kOwned>                                               // first positions per thread: n <= kOwned * kSliceThreads
+// The smallest (value, position) pair of a warp.  64-bit values: three 32-bit reductions (the high words, the low words among
+// the lanes that hold the smallest high word, the positions among the lanes that hold the smallest value); 32-bit values: two.
+__device__ __forceinline__ void warp_min_pair(long long& best, int& where) {
+    const unsigned hi = unsigned(static_cast<unsigned long long>(best) >> 32), lo = unsigned(static_cast<unsigned long long>(best));
+    const unsigned mh = __reduce_min_sync(0xffffffffu, hi);
+    const unsigned ml = __reduce_min_sync(0xffffffffu, hi == mh ? lo : 0xffffffffu);
+    const unsigned mi = __reduce_min_sync(0xffffffffu, (hi == mh && lo == ml) ? unsigned(where) : 0x7fffffffu);
+    best = static_cast<long long>((static_cast<unsigned long long>(mh) << 32) | ml);
+    where = int(mi);
+}
+__device__ __forceinline__ void warp_min_pair(int& best, int& where) {              // values are non-negative
+    const int m = __reduce_min_sync(0xffffffffu, best);
+    where = int(__reduce_min_sync(0xffffffffu, best == m ? unsigned(where) : 0x7fffffffu));
+    best = m;
+}
+
+template <class C> struct alignas(4 * sizeof(C)) NodeRecord { C work, param, out, gain; };
+
+// One CTA per order.  The n^2 segment costs are never tabulated: for a fixed right end r the costs F(l, r) of all first positions
+// l form a column that follows from the column of r - 1 by adding the node at position r.  Per step of r: the owners of the
+// first positions update their five running values and write the column, and warp kk - 1 takes
+// dp[kk][r] = min over l of max(dp[kk - 1][l], F(l + 1, r)).  The column of r + 1 is written (into the other of two buffers)
+// in the same pass that reads the column of r, so a step costs one barrier.
+//
+// What a step needs of the graph is prepared once per order, in the order's own sequence: a record of the node at position r
+// (work, parameters, output, and the output again if it has consumers: they all come later), and for each producer u of that
+// node the three things the update asks of an edge: u's output size; max(position of u, position of u's latest consumer before
+// r), below which a first position l does not count u as an input any more; and u's position if r is u's last consumer (else 0),
+// from which on l holds u inside and stops counting it as an output.
+//
+// C: the word costs are kept in.  int when the host has bounded every segment cost of the call below 2^31, long long otherwise.
+template <int kOwned, class C, bool kEdgesInSmem>                   // first positions per thread: n <= kOwned * kSliceThreads
 __global__ void __launch_bounds__(kSliceThreads)
-slice_orders(DeviceGraph g, int staged_edges, const int* __restrict__ orders, int k, long long B, long long M, long long* __restrict__ cost_out,
+slice_orders(DeviceGraph g, const int* __restrict__ orders, int k, C B, C M, long long* __restrict__ cost_out,
              int* __restrict__ blocks_out, int* __restrict__ cuts_out, int* __restrict__ status_out) {
+    constexpr bool kNarrow = sizeof(C) == 4;
+    constexpr C kInf = kNarrow ? C(0x7fffffff) : C(0x7fffffffffffffffLL);
     extern __shared__ __align__(16) unsigned char smem[];
     const int n = g.n;
     const int kmax = k < n ? k : n;
-    const SliceLayout L = slice_layout(n, kmax, staged_edges);
-    long long* F = reinterpret_cast<long long*>(smem + L.f);
-    long long* dp = reinterpret_cast<long long*>(smem + L.dp);
+    const SliceLayout L = slice_layout(n, kmax, kEdgesInSmem ? g.edges : 0, int(sizeof(C)));
+    NodeRecord<C>* attr = reinterpret_cast<NodeRecord<C>*>(smem + L.attr);
+    C* F = reinterpret_cast<C*>(smem + L.f);
+    C* dp = reinterpret_cast<C*>(smem + L.dp);
+    C* eso = reinterpret_cast<C*>(smem + L.eso);
     int* pos = reinterpret_cast<int*>(smem + L.pos);
     int* last = reinterpret_cast<int*>(smem + L.last);
-    int* prev = reinterpret_cast<int*>(smem + L.prev);
+    int* epos = reinterpret_cast<int*>(smem + L.epos);
+    int* ord = reinterpret_cast<int*>(smem + L.order);
+    unsigned short* ethr = reinterpret_cast<unsigned short*>(smem + L.ethr);
+    unsigned short* epu = reinterpret_cast<unsigned short*>(smem + L.epu);
     unsigned short* arg = reinterpret_cast<unsigned short*>(smem + L.arg);
     __shared__ int bad;
 
@@ -90,28 +130,13 @@ slice_orders(DeviceGraph g, int staged_edges, const int* __restrict__ orders, in
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int kWarps = kSliceThreads / 32;
     const int* pi = orders + size_t(p) * n;
-    const long long* a_work = g.work;
-    const long long* a_param = g.sizeparam;
-    const long long* a_out = g.sizeout;
-    const int* pred_ptr = g.pred_ptr;
-    const int* pred = g.pred;
-    if (staged_edges > 0) {
-        long long* sa = reinterpret_cast<long long*>(smem + L.attr);
-        int* sp = reinterpret_cast<int*>(smem + L.pptr);
-        int* sl = reinterpret_cast<int*>(smem + L.pred);
-        int* so = reinterpret_cast<int*>(smem + L.order);
-        for (int i = tid; i < n; i += kSliceThreads) { sa[i] = g.work[i]; sa[n + i] = g.sizeparam[i]; sa[2 * n + i] = g.sizeout[i]; so[i] = pi[i]; }
-        for (int i = tid; i <= n; i += kSliceThreads) sp[i] = g.pred_ptr[i];
-        for (int i = tid; i < staged_edges; i += kSliceThreads) sl[i] = g.pred[i];
-        a_work = sa; a_param = sa + n; a_out = sa + 2 * n; pred_ptr = sp; pred = sl; pi = so;
-    }
 
     // positions, and the check that the row is a topological order of this graph
     if (tid == 0) bad = 0;
-    for (int i = tid; i < n; i += kSliceThreads) { pos[i] = 0; last[i] = 0; prev[i] = 0; }
+    for (int i = tid; i < n; i += kSliceThreads) { pos[i] = 0; ord[i] = pi[i]; }
     __syncthreads();
     for (int i = tid; i < n; i += kSliceThreads) {
-        const int v = pi[i];
+        const int v = ord[i];
         if (v < 0 || v >= n) bad = 1;
         else if (atomicExch(&pos[v], i + 1) != 0) bad = 1;          // a node listed twice (so another one is missing)
     }
@@ -134,65 +159,112 @@ slice_orders(DeviceGraph g, int staged_edges, const int* __restrict__ orders, in
         return;
     }
 
-    long long cw[kOwned], cp[kOwned], ck[kOwned], ci[kOwned], co[kOwned];
+    // the node records by position, and how many producer edges each position has
+    if (tid == 0) epos[0] = 0;
+    for (int i = tid; i < n; i += kSliceThreads) {
+        const int v = ord[i];
+        const C so = C(g.sizeout[v]);
+        attr[i] = NodeRecord<C>{C(g.work[v]), C(g.sizeparam[v]), so, last[v] != 0 ? so : C(0)};
+        epos[i + 1] = g.pred_ptr[v + 1] - g.pred_ptr[v];
+    }
+    __syncthreads();
+    if (warp == 0) {                                                 // running sum of the counts: a chunk per lane, then across the lanes
+        const int chunk = (n + 31) / 32, lo = 1 + lane * chunk, hi = (lo + chunk <= n + 1) ? lo + chunk : n + 1;
+        int sum = 0;
+        for (int i = lo; i < hi; ++i) sum += epos[i];
+        int incl = sum;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int o = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += o;
+        }
+        int run = incl - sum;
+        for (int i = lo; i < hi; ++i) { run += epos[i]; epos[i] = run; }
+    }
+    __syncthreads();
+    // what the update asks of the edge u -> (node at position r)
+    struct EdgeInfo { int thr, pu; C so; };
+    auto edge_info = [&](int u, int r) -> EdgeInfo {
+        const int pu = pos[u];
+        int pc = 0;                                                  // u's latest consumer before r
+        for (int e = g.cons_ptr[u]; e < g.cons_ptr[u + 1]; ++e) {
+            const int q = pos[g.cons[e]];
+            if (q < r && q > pc) pc = q;
+        }
+        return EdgeInfo{pu > pc ? pu : pc, last[u] == r ? pu : 0, C(g.sizeout[u])};
+    };
+    if constexpr (kEdgesInSmem) {
+        for (int i = tid; i < n; i += kSliceThreads) {
+            const int v = ord[i];
+            const int from = g.pred_ptr[v], at = epos[i], deg = epos[i + 1] - at;
+            for (int j = 0; j < deg; ++j) {
+                const EdgeInfo ei = edge_info(g.pred[from + j], i + 1);
+                ethr[at + j] = static_cast<unsigned short>(ei.thr);
+                epu[at + j] = static_cast<unsigned short>(ei.pu);
+                eso[at + j] = ei.so;
+            }
+        }
+        __syncthreads();
+    }
+
+    C cw[kOwned], cp[kOwned], ck[kOwned], ci[kOwned], co[kOwned];
 #pragma unroll
     for (int j = 0; j < kOwned; ++j) { cw[j] = 0; cp[j] = 0; ck[j] = 0; ci[j] = 0; co[j] = 0; }
-    for (int r = 1; r <= n; ++r) {
-        const int v = pi[r - 1];
-        const int pb = pred_ptr[v], pe = pred_ptr[v + 1];
-        const long long so_v = a_out[v], w_v = a_work[v], pa_v = a_param[v];
-        const long long gain_out = (last[v] != 0) ? so_v : 0;            // v has consumers (they all come later)
-        // the column of r: thread t owns the first positions l = t + 1, t + 257, ... and keeps their five running values in registers
+    // the column of r into Fw: thread t owns the first positions l = t + 1, t + 257, ... and keeps their five running values in registers
+    auto column = [&](int r, C* __restrict__ Fw) {
+        const NodeRecord<C> node = attr[r - 1];
+        const int pb = epos[r - 1], pe = epos[r];
+        const int from = kEdgesInSmem ? 0 : g.pred_ptr[ord[r - 1]];
 #pragma unroll
         for (int j = 0; j < kOwned; ++j) {
             const int l = tid + 1 + j * kSliceThreads;
             if (l > r) continue;
             if (l == r) { cw[j] = 0; cp[j] = 0; ck[j] = 0; ci[j] = 0; co[j] = 0; }
-            cw[j] += w_v;
-            cp[j] += pa_v;
-            ck[j] = so_v > ck[j] ? so_v : ck[j];
-            co[j] += gain_out;
+            cw[j] += node.work;
+            cp[j] += node.param;
+            ck[j] = node.out > ck[j] ? node.out : ck[j];
+            co[j] += node.gain;
             for (int e = pb; e < pe; ++e) {
-                const int u = pred[e];
-                const int pu = pos[u], pc = prev[u];
-                const long long so_u = a_out[u];
-                if (l > (pu > pc ? pu : pc)) ci[j] += so_u;          // u lies before l and nothing in l..r-1 read it
-                if (last[u] == r && pu >= l) co[j] -= so_u;           // u is inside and v was its last consumer
+                int thr, pu;
+                C so_u;
+                if constexpr (kEdgesInSmem) {
+                    thr = ethr[e]; pu = epu[e]; so_u = eso[e];
+                } else {
+                    const EdgeInfo ei = edge_info(g.pred[from + e - pb], r);
+                    thr = ei.thr; pu = ei.pu; so_u = ei.so;
+                }
+                if (l > thr) ci[j] += so_u;                          // u lies before l and nothing in l..r-1 read it
+                if (pu >= l) co[j] -= so_u;                          // u is inside and this was its last consumer
             }
-            const long long excess = cp[j] + ck[j] - M;
-            F[l - 1] = ci[j] + B * cw[j] + (excess > 0 ? excess : 0) + ck[j] + co[j];
+            const C excess = cp[j] + ck[j] - M;
+            Fw[l - 1] = ci[j] + B * cw[j] + (excess > 0 ? excess : C(0)) + ck[j] + co[j];
         }
-        __syncthreads();
+    };
+    column(1, F + n);                                                // the column of r sits in F + (r & 1) * n
+    __syncthreads();
+    for (int r = 1; r <= n; ++r) {
+        const C* __restrict__ Fr = F + (r & 1) * n;
         // dp[kk][r] = min over l of max(dp[kk - 1][l], F(l + 1, r)); the earlier l on equal values
         for (int kk = warp + 1; kk <= kmax; kk += kWarps) {
-            long long best = kInf;
+            C best = kInf;
             int where = 0;
             if (kk == 1) {
-                best = F[0];
+                best = Fr[0];
             } else if (r >= kk) {
-                const long long* below = dp + size_t(kk - 2) * (n + 1);
+                const C* below = dp + size_t(kk - 2) * (n + 1);
                 for (int l = kk - 1 + lane; l < r; l += 32) {
-                    const long long a = below[l], b = F[l];
-                    const long long cand = a > b ? a : b;
+                    const C a = below[l], b = Fr[l];
+                    const C cand = a > b ? a : b;
                     if (cand < best) { best = cand; where = l; }     // l ascends within a lane: strict < keeps the earlier one
                 }
-                // the warp's smallest (value, position) pair by three 32-bit reductions: the high words, then the low words
-                // among the lanes that hold the smallest high word, then the positions among the lanes that hold the smallest value
-                const unsigned hi = unsigned(static_cast<unsigned long long>(best) >> 32), lo = unsigned(static_cast<unsigned long long>(best));
-                const unsigned mh = __reduce_min_sync(0xffffffffu, hi);
-                const unsigned ml = __reduce_min_sync(0xffffffffu, hi == mh ? lo : 0xffffffffu);
-                const unsigned mi = __reduce_min_sync(0xffffffffu, (hi == mh && lo == ml) ? unsigned(where) : 0x7fffffffu);
-                best = static_cast<long long>((static_cast<unsigned long long>(mh) << 32) | ml);
-                where = int(mi);
+                warp_min_pair(best, where);
             }
             if (lane == 0) {
                 dp[size_t(kk - 1) * (n + 1) + r] = best;
                 arg[size_t(kk - 1) * (n + 1) + r] = static_cast<unsigned short>(where);
             }
         }
-        if (tid == kSliceThreads - 1) {                              // v has now been seen as a consumer of its producers
-            for (int e = pb; e < pe; ++e) prev[pred[e]] = r;
-        }
+        if (r < n) column(r + 1, F + ((r + 1) & 1) * n);             // the other buffer: nobody reads it before the barrier
         __syncthreads();
     }
 
@@ -200,7 +272,7 @@ slice_orders(DeviceGraph g, int staged_edges, const int* __restrict__ orders, in
         int best_k = 1;
         for (int kk = 2; kk <= kmax; ++kk)
             if (dp[size_t(kk - 1) * (n + 1) + n] < dp[size_t(best_k - 1) * (n + 1) + n]) best_k = kk;
-        cost_out[p] = dp[size_t(best_k - 1) * (n + 1) + n];
+        cost_out[p] = static_cast<long long>(dp[size_t(best_k - 1) * (n + 1) + n]);
         blocks_out[p] = best_k;
         status_out[p] = 0;
         int r = n;
@@ -260,7 +332,7 @@ struct mtpp_graph {
     DeviceGraph d;
     int device;
     int m;
-    long long total_work;
+    long long total_work, total_param, total_out, max_out;
     void* blob;
 };
 
@@ -269,13 +341,30 @@ namespace {
 std::mutex g_attr_lock;
 bool g_attr_done[64] = {};
 
+// the instances of slice_orders: first positions per thread x cost word x where the edges are kept
+template <int kOwned, class C, bool kEdgesInSmem>
+const void* slice_kernel() { return reinterpret_cast<const void*>(&slice_orders<kOwned, C, kEdgesInSmem>); }
+const void* slice_kernel(int owned, bool narrow, bool edges_in_smem) {
+#define MTPP_PICK(O) (narrow ? (edges_in_smem ? slice_kernel<O, int, true>() : slice_kernel<O, int, false>()) \
+                             : (edges_in_smem ? slice_kernel<O, long long, true>() : slice_kernel<O, long long, false>()))
+    return owned == 1 ? MTPP_PICK(1) : owned == 2 ? MTPP_PICK(2) : MTPP_PICK(4);
+#undef MTPP_PICK
+}
+std::vector<const void*> slice_kernels() {
+    std::vector<const void*> all;
+    for (int owned : {1, 2, 4})
+        for (bool narrow : {false, true})
+            for (bool in_smem : {false, true}) all.push_back(slice_kernel(owned, narrow, in_smem));
+    return all;
+}
+
 cudaError_t allow_slice_smem(int device) {
     std::lock_guard<std::mutex> guard(g_attr_lock);
     const bool tracked = device >= 0 && device < 64;
     if (tracked && g_attr_done[device]) return cudaSuccess;
-    cudaError_t e = cudaFuncSetAttribute(slice_orders<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSliceSmemLimit));
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(slice_orders<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSliceSmemLimit));
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(slice_orders<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSliceSmemLimit));
+    cudaError_t e = cudaSuccess;
+    for (const void* kernel : slice_kernels())
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSliceSmemLimit));
     if (e == cudaSuccess && tracked) g_attr_done[device] = true;
     return e;
 }
@@ -291,11 +380,12 @@ int mtpp_graph_create(int n, int m, const int32_t* edges_host, const int64_t* wo
     if (n < 1 || n > MTPP_MAX_NODES || m < 0 || m > (1 << 22)) return BQ_ERR_SIZE;
     if ((m > 0 && !edges_host) || !work_host || !sizeparam_host || !sizeout_host) return BQ_ERR_NULL;
     constexpr long long kCap = 1LL << 40;
-    long long tw = 0, tp = 0, ts = 0;
+    long long tw = 0, tp = 0, ts = 0, mo = 0;
     for (int v = 0; v < n; ++v) {
         if (work_host[v] < 0 || sizeparam_host[v] < 0 || sizeout_host[v] < 0) return BQ_ERR_SIZE;
         if (work_host[v] >= kCap || sizeparam_host[v] >= kCap || sizeout_host[v] >= kCap) return BQ_ERR_SIZE;
         tw += work_host[v]; tp += sizeparam_host[v]; ts += sizeout_host[v];
+        mo = sizeout_host[v] > mo ? sizeout_host[v] : mo;
         if (tw >= kCap || tp >= kCap || ts >= kCap) return BQ_ERR_SIZE;
     }
     // consumer lists without duplicates
@@ -348,6 +438,7 @@ int mtpp_graph_create(int n, int m, const int32_t* edges_host, const int64_t* wo
     }
     const char* base = static_cast<const char*>(g->blob);
     g->d.n = n;
+    g->d.edges = int(edges);
     g->d.work = reinterpret_cast<const long long*>(base);
     g->d.sizeparam = g->d.work + n;
     g->d.sizeout = g->d.sizeparam + n;
@@ -357,6 +448,9 @@ int mtpp_graph_create(int n, int m, const int32_t* edges_host, const int64_t* wo
     g->d.cons = reinterpret_cast<const int*>(base + o_cons);
     g->m = int(edges);
     g->total_work = tw;
+    g->total_param = tp;
+    g->total_out = ts;
+    g->max_out = mo;
     *out = g;
     return BQ_OK;
 }
@@ -393,20 +487,34 @@ int mtpp_slice_orders(const mtpp_graph* g, const int32_t* orders, int P, int k, 
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev != g->device) return BQ_ERR_CUDA;
     const int kmax = k < g->d.n ? k : g->d.n;
-    // the graph rides in shared memory when it fits beside the programme's arrays
-    int staged_edges = g->m > 0 ? g->m : 1;
-    SliceLayout L = slice_layout(g->d.n, kmax, staged_edges);
+    // Every segment cost is at most in + out (disjoint sets of nodes: at most the sum of all outputs) + B * work + excess (at most
+    // all parameters and one output) + peak (one output).  Below 2^31 the whole programme runs in 32-bit words.
+    const long long cost_bound = g->total_out + 2 * g->max_out + g->total_param + B * g->total_work;     // no overflow: checked above
+    const bool narrow = cost_bound < 0x7fffffffLL;
+    const int cs = narrow ? 4 : 8;
+    // the order's edges ride in shared memory when they fit beside the programme's arrays
+    bool edges_in_smem = true;
+    SliceLayout L = slice_layout(g->d.n, kmax, g->d.edges, cs);
     if (L.total > kSliceSmemLimit) {
-        staged_edges = 0;
-        L = slice_layout(g->d.n, kmax, 0);
+        edges_in_smem = false;
+        L = slice_layout(g->d.n, kmax, 0, cs);
     }
+    if (L.total > kSliceSmemLimit) return BQ_ERR_SIZE;                // cannot happen within MTPP_MAX_NODES and MTPP_MAX_BLOCKS
     cudaError_t e = cudaSuccess;
     if (L.total > 48 * 1024) e = allow_slice_smem(g->device);
     if (e != cudaSuccess) return cuda_fail(e);
     static_assert(MTPP_MAX_NODES <= 4 * kSliceThreads, "the widest instance owns four first positions per thread");
-    auto* kernel = g->d.n <= kSliceThreads ? slice_orders<1> : g->d.n <= 2 * kSliceThreads ? slice_orders<2> : slice_orders<4>;
-    kernel<<<unsigned(P), kSliceThreads, L.total, static_cast<cudaStream_t>(cuda_stream)>>>(
-        g->d, staged_edges, orders, k, static_cast<long long>(B), static_cast<long long>(M), reinterpret_cast<long long*>(cost_out), blocks_out, cuts_out, status_out);
+    const int owned = g->d.n <= kSliceThreads ? 1 : g->d.n <= 2 * kSliceThreads ? 2 : 4;
+    const void* kernel = slice_kernel(owned, narrow, edges_in_smem);
+    long long* cost = reinterpret_cast<long long*>(cost_out);
+    DeviceGraph d = g->d;
+    long long B64 = B, M64 = M;
+    int B32 = g->total_work > 0 ? int(B) : 0;                         // B * total_work < 2^31; without work the factor multiplies zeros
+    int M32 = M < 0x7fffffffLL ? int(M) : 0x7fffffff;                 // parameters + peak stay below the bound: a larger M never shows
+    void* args[] = {&d, &orders, &k, narrow ? static_cast<void*>(&B32) : static_cast<void*>(&B64),
+                    narrow ? static_cast<void*>(&M32) : static_cast<void*>(&M64), &cost, &blocks_out, &cuts_out, &status_out};
+    e = cudaLaunchKernel(kernel, dim3(unsigned(P)), dim3(kSliceThreads), args, L.total, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(e);
     e = cudaGetLastError();
     return e == cudaSuccess ? BQ_OK : cuda_fail(e);
 }

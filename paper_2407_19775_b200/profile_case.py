@@ -5,6 +5,10 @@
 `--rows 8192` of `sweep1g` is 64 Mi bf16 elements (128 MiB in, larger than L2) and keeps the
 device footprint well under 1 GB, which is what a counter-collecting profiler wants.  Prints
 the CUDA-event time of each launch.
+
+    python -m paper_2407_19775_b200.profile_case --op mtpp --workload mtpp_unet --launches 3
+
+decodes and slices the workload's population of topological orders (two kernels per launch).
 """
 from __future__ import annotations
 
@@ -12,19 +16,36 @@ import argparse
 
 import torch
 
-from . import Codebook, Codebook4, bq4_dequantize, bq4_quantize, bq_dequantize, bq_quantize, bq_roundtrip, tune, workloads
+from . import Codebook, Codebook4, bq4_dequantize, bq4_quantize, bq_dequantize, bq_quantize, bq_roundtrip, mtpp, tune, workloads
 
 
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="sweep1g")
-    ap.add_argument("--op", default="roundtrip", choices=["quantize", "dequantize", "roundtrip", "roundtrip_side", "quantize4", "dequantize4", "block_errors", "sweep"])
+    ap.add_argument("--op", default="roundtrip", choices=["quantize", "dequantize", "roundtrip", "roundtrip_side", "quantize4", "dequantize4", "block_errors", "sweep", "mtpp"])
     ap.add_argument("--block", type=int, default=4096)
     ap.add_argument("--rows", type=int, default=8192)
     ap.add_argument("--launches", type=int, default=3)
     ap.add_argument("--dtype", default=None, choices=[None, "bf16", "fp16", "fp32"], help="cast the workload to this type first")
     args = ap.parse_args()
     dev = torch.device("cuda:0")
+    if args.op == "mtpp":
+        name = args.workload if args.workload in workloads.GRAPH_WORKLOADS else "mtpp_unet"
+        w = workloads.GRAPH_WORKLOADS[name]
+        graph = mtpp.SliceGraph(*workloads.make_graph(name), device=dev)
+        keys = workloads.make_keys(name, w.population).to(dev)
+        orders = out = None
+        for i in range(args.launches):
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            ev[0].record()
+            orders = graph.decode_orders(keys, orders)
+            ev[1].record()
+            out = graph.slice_orders(orders, w.k, w.B, w.M, out)
+            ev[2].record()
+            torch.cuda.synchronize()
+            print(f"{name} population {w.population} launch {i}: decode {ev[0].elapsed_time(ev[1]):.4f} ms, slice {ev[1].elapsed_time(ev[2]):.4f} ms, "
+                  f"flagged {int(out[3].sum())}")
+        return
     x = workloads.make(args.workload, rows=args.rows).view(-1).to(dev)
     if args.dtype is not None:
         x = x.to({"bf16": torch.bfloat16, "fp16": torch.float16, "fp32": torch.float32}[args.dtype])

@@ -68,9 +68,10 @@ def test_random_graphs_fuzz(bq):
     for case in range(12):
         n = rng.choice([1, 2, 3, 17, 33, 64, 100])
         edges = np.asarray([(u, v) for u in range(n) for v in range(u + 1, n) if rng.random() < rng.choice([0.0, 0.05, 0.3])], np.int32).reshape(-1, 2)
+        scale = 1 << 21 if case % 2 else 1                                   # odd cases: costs beyond 32 bits, the wide instances
         work = np.asarray([rng.randrange(0, 50) for _ in range(n)], np.int64)
-        sizeparam = np.asarray([rng.randrange(0, 500) for _ in range(n)], np.int64)
-        sizeout = np.asarray([rng.randrange(0, 80) for _ in range(n)], np.int64)
+        sizeparam = np.asarray([rng.randrange(0, 500) for _ in range(n)], np.int64) * scale
+        sizeout = np.asarray([rng.randrange(0, 80) for _ in range(n)], np.int64) * scale
         g = oracle_graph(n, edges, work, sizeparam, sizeout)
         dg = bq.mtpp.SliceGraph(n, edges, work, sizeparam, sizeout, device="cuda:0")
         P = 5
@@ -78,7 +79,7 @@ def test_random_graphs_fuzz(bq):
         if case % 3 == 0:
             keys = (keys * 3).floor() / 3                                    # many equal keys: the node index decides
         orders = dg.decode_orders(keys.cuda())
-        B, M, k = rng.randrange(1, 9), rng.randrange(0, 2000), rng.choice([1, 2, 5, 16])
+        B, M, k = rng.randrange(1, 9) * scale, rng.randrange(0, 2000) * scale, rng.choice([1, 2, 5, 16])
         cost, blocks, cuts, status = dg.slice_orders(orders, k, B, M)
         torch.cuda.synchronize()
         for p in range(P):
@@ -88,42 +89,45 @@ def test_random_graphs_fuzz(bq):
         dg.close()
 
 
-def banded_graph(n, seed):
+def banded_graph(n, seed, scale=1, density=0.08):
     rng = random.Random(seed)
-    edges = np.asarray([(u, v) for u in range(n) for v in range(u + 1, min(n, u + 40)) if rng.random() < 0.08], np.int32).reshape(-1, 2)
+    edges = np.asarray([(u, v) for u in range(n) for v in range(u + 1, min(n, u + 40)) if rng.random() < density], np.int32).reshape(-1, 2)
     work = np.asarray([rng.randrange(0, 50) for _ in range(n)], np.int64)
-    sizeparam = np.asarray([rng.randrange(0, 500) for _ in range(n)], np.int64)
-    sizeout = np.asarray([rng.randrange(0, 80) for _ in range(n)], np.int64)
+    sizeparam = np.asarray([rng.randrange(0, 500) for _ in range(n)], np.int64) * scale
+    sizeout = np.asarray([rng.randrange(0, 80) for _ in range(n)], np.int64) * scale
     return edges, work, sizeparam, sizeout
 
 
-@pytest.mark.parametrize("n,k", [(257, 16), (300, 5), (520, 3)])
-def test_graphs_wider_than_one_position_per_thread(bq, n, k):
+@pytest.mark.parametrize("n,k,scale", [(257, 16, 1), (300, 5, 1 << 21), (520, 3, 1), (513, 2, 1 << 21)])
+def test_graphs_wider_than_one_position_per_thread(bq, n, k, scale):
     """Above 256 and above 512 nodes a thread of the slicing kernel owns two and four first positions: one order of each in
-    full against the oracle."""
-    edges, work, sizeparam, sizeout = banded_graph(n, n)
+    full against the oracle, with costs inside 32 bits and beyond them."""
+    edges, work, sizeparam, sizeout = banded_graph(n, n, scale)
     g = oracle_graph(n, edges, work, sizeparam, sizeout)
     dg = bq.mtpp.SliceGraph(n, edges, work, sizeparam, sizeout, device="cuda:0")
     keys = torch.rand((3, n), generator=torch.Generator().manual_seed(n))
     orders = dg.decode_orders(keys.cuda())
-    cost, blocks, cuts, status = dg.slice_orders(orders, k, 3, 20000)
+    cost, blocks, cuts, status = dg.slice_orders(orders, k, 3 * scale, 20000 * scale)
     torch.cuda.synchronize()
     assert status.cpu().tolist() == [0, 0, 0]
     pi = orders[1].cpu().tolist()
     assert pi == mo.decode_order(g, keys[1].tolist())
-    assert (int(cost[1]), int(blocks[1]), cuts[1][:int(blocks[1])].cpu().tolist()) == mo.slice_order(g, pi, k, 3, 20000)
+    assert (int(cost[1]), int(blocks[1]), cuts[1][:int(blocks[1])].cpu().tolist()) == mo.slice_order(g, pi, k, 3 * scale, 20000 * scale)
     dg.close()
 
 
-def test_largest_graph(bq):
+@pytest.mark.parametrize("scale,density", [(1, 0.08), (1 << 21, 0.08), (1, 0.4)])
+def test_largest_graph(bq, scale, density):
     """1024 nodes, 16 blocks, the limits of the call.  A chain of equal nodes has a closed form: every block's cost grows with
     its length, so the best slicing is the balanced one and its bottleneck is the cost of an inner block of ceil(n / k) nodes.
-    On a banded random graph the oracle re-costs the returned cuts (16 blocks an order) and no perturbed cut set does better."""
-    n, k, B, M = 1024, 16, 3, 20000
+    On a banded random graph the oracle re-costs the returned cuts (16 blocks an order) and no perturbed cut set does better.
+    With costs beyond 32 bits, or with some 15,000 edges, the order's edges no longer fit in shared memory beside the programme's
+    arrays and are looked up in global memory."""
+    n, k, B, M = 1024, 16, 3 * scale, 20000 * scale
     chain = np.asarray([(i, i + 1) for i in range(n - 1)], np.int32)
-    ones = np.ones(n, np.int64)
-    g = oracle_graph(n, chain, 7 * ones, 300 * ones, 11 * ones)
-    dg = bq.mtpp.SliceGraph(n, chain, 7 * ones, 300 * ones, 11 * ones, device="cuda:0")
+    ones = np.ones(n, np.int64) * scale
+    g = oracle_graph(n, chain, 7 * ones // scale, 300 * ones, 11 * ones)
+    dg = bq.mtpp.SliceGraph(n, chain, 7 * ones // scale, 300 * ones, 11 * ones, device="cuda:0")
     orders = dg.decode_orders(torch.rand((2, n), generator=torch.Generator().manual_seed(1)).cuda())
     assert orders.cpu().tolist() == [list(range(n))] * 2                   # a chain has one topological order
     cost, blocks, cuts, status = dg.slice_orders(orders, k, B, M)
@@ -134,7 +138,7 @@ def test_largest_graph(bq):
     assert max(e - s for s, e in zip([0] + ends[:-1], ends)) == 64 and ends[-1] == n
     dg.close()
 
-    edges, work, sizeparam, sizeout = banded_graph(n, 5)
+    edges, work, sizeparam, sizeout = banded_graph(n, 5, scale, density)
     g = oracle_graph(n, edges, work, sizeparam, sizeout)
     dg = bq.mtpp.SliceGraph(n, edges, work, sizeparam, sizeout, device="cuda:0")
     keys = torch.rand((4, n), generator=torch.Generator().manual_seed(2))
@@ -157,6 +161,34 @@ def test_largest_graph(bq):
             nudged = sorted({min(n - 1, max(1, e + rng.randrange(-2, 3))) for e in ends[:-1]}) + [n]
             drawn = sorted(rng.sample(range(1, n), k - 1)) + [n]
             assert bottleneck(pi, nudged) >= int(cost[p]) and bottleneck(pi, drawn) >= int(cost[p])
+    dg.close()
+
+
+@pytest.mark.parametrize("pad", [-3, -2, -1, 0, 1, 2])
+@pytest.mark.parametrize("M", [0, 10 ** 9, (1 << 62) - 1])
+def test_costs_on_either_side_of_the_32_bit_bound(bq, pad, M):
+    """The library runs the programme in 32-bit words when its bound on any segment cost, sum of outputs + 2 largest output
+    + sum of parameters + B * sum of work, is below 2^31 - 1, and in 64-bit words otherwise: graphs whose bound sits at
+    2^31 - 1 + pad, and whose whole-order cost comes close to it, against the oracle."""
+    n, B, k = 40, 3, 4
+    rng = random.Random(pad * 7 + 100)
+    edges = np.asarray([(i, i + 1) for i in range(n - 1)] + [(i, i + 5) for i in range(0, n - 5, 3)], np.int32)
+    work = np.asarray([rng.randrange(1, 10 ** 6) for _ in range(n)], np.int64)
+    sizeout = np.asarray([rng.randrange(1, 10 ** 6) for _ in range(n)], np.int64)
+    sizeparam = np.asarray([rng.randrange(0, 10 ** 7) for _ in range(n)], np.int64)
+    bound = int(sizeout.sum() + 2 * sizeout.max() + sizeparam.sum() + B * work.sum())
+    sizeparam[7] += (1 << 31) - 1 + pad - bound                              # parameters take up the slack
+    assert int(sizeout.sum() + 2 * sizeout.max() + sizeparam.sum() + B * work.sum()) == (1 << 31) - 1 + pad
+    g = oracle_graph(n, edges, work, sizeparam, sizeout)
+    dg = bq.mtpp.SliceGraph(n, edges, work, sizeparam, sizeout, device="cuda:0")
+    orders = dg.decode_orders(torch.rand((2, n), generator=torch.Generator().manual_seed(3)).cuda())
+    for kk in (1, k):
+        cost, blocks, cuts, status = dg.slice_orders(orders, kk, B, M)
+        torch.cuda.synchronize()
+        assert status.cpu().tolist() == [0, 0]
+        for p in range(2):
+            pi = orders[p].cpu().tolist()
+            assert (int(cost[p]), int(blocks[p]), cuts[p][:int(blocks[p])].cpu().tolist()) == mo.slice_order(g, pi, kk, B, M), (kk, p)
     dg.close()
 
 
