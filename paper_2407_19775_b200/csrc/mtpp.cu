@@ -54,13 +54,16 @@ struct SliceLayout {
 };
 // `edges` > 0: the producer edges of the order, re-laid in the order's own sequence (see the kernel), sit in shared memory
 // too; 0: graphs with too many edges to fit beside the programme's arrays look them up in global memory at every step.
+// rows of F and of dp start on 16-byte boundaries and are read four (two) words at a time
+__host__ __device__ inline size_t slice_fstride(int n) { return round_up(size_t(n) + 4, 4); }
+__host__ __device__ inline size_t slice_dstride(int n) { return round_up(size_t(n) + 1, 4); }
 __host__ __device__ inline SliceLayout slice_layout(int n, int kmax, int edges, int cs) {
     SliceLayout L;
     size_t o = 0;
     L.attr = o; o += size_t(4) * n * cs;                               // by position: work, sizeparam, sizeout, sizeout if it has consumers
-    L.f = o;    o += round_up(size_t(2) * n * cs, 8);                  // F(l, r) of the current r and of the next one
-    L.dp = o;   o += round_up(size_t(kmax) * (n + 1) * cs, 8);         // dp[kk - 1][r]
-    L.eso = o;  o += round_up(size_t(edges) * cs, 8);                  // per edge: the producer's sizeout
+    L.f = o;    o += size_t(2) * slice_fstride(n) * cs;                // F(l, r) of the current r and of the next one
+    L.dp = o;   o += size_t(kmax) * slice_dstride(n) * cs;             // dp[kk - 1][r]
+    L.eso = o;  o += round_up(size_t(edges) * cs, 16);                 // per edge: the producer's sizeout
     L.pos = o;  o += size_t(n) * 4;                                    // 1-based position of each node (0: not seen)
     L.last = o; o += size_t(n) * 4;                                    // position of each node's last consumer (0: none)
     L.epos = o; o += size_t(n + 1) * 4;                                // edges of position r: [epos[r - 1], epos[r])
@@ -89,6 +92,9 @@ __device__ __forceinline__ void warp_min_pair(int& best, int& where) {          
 }
 
 template <class C> struct alignas(4 * sizeof(C)) NodeRecord { C work, param, out, gain; };
+template <class C> struct CostVec;                                   // 16 bytes of cost words
+template <> struct CostVec<int> { using T = int4; static constexpr int N = 4; };
+template <> struct CostVec<long long> { using T = longlong2; static constexpr int N = 2; };
 
 // One CTA per order.  The n^2 segment costs are never tabulated: for a fixed right end r the costs F(l, r) of all first positions
 // l form a column that follows from the column of r - 1 by adding the node at position r.  Per step of r: the owners of the
@@ -129,6 +135,9 @@ slice_orders(DeviceGraph g, const int* __restrict__ orders, int k, C B, C M, lon
     const int p = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int kWarps = kSliceThreads / 32;
+    constexpr int V = CostVec<C>::N;
+    using VecT = typename CostVec<C>::T;
+    const int fs = int(slice_fstride(n)), ds = int(slice_dstride(n));
     const int* pi = orders + size_t(p) * n;
 
     // positions, and the check that the row is a topological order of this graph
@@ -161,6 +170,7 @@ slice_orders(DeviceGraph g, const int* __restrict__ orders, int k, C B, C M, lon
 
     // the node records by position, and how many producer edges each position has
     if (tid == 0) epos[0] = 0;
+    if (tid < kmax) dp[size_t(tid) * ds] = kInf;                     // no block holds the first 0 nodes: the vector reads below may start there
     for (int i = tid; i < n; i += kSliceThreads) {
         const int v = ord[i];
         const C so = C(g.sizeout[v]);
@@ -218,7 +228,10 @@ slice_orders(DeviceGraph g, const int* __restrict__ orders, int k, C B, C M, lon
 #pragma unroll
         for (int j = 0; j < kOwned; ++j) {
             const int l = tid + 1 + j * kSliceThreads;
-            if (l > r) continue;
+            if (l > r) {
+                if (l < r + V) Fw[l - 1] = kInf;                     // what a vector read of the column's end takes in beside it
+                continue;
+            }
             if (l == r) { cw[j] = 0; cp[j] = 0; ck[j] = 0; ci[j] = 0; co[j] = 0; }
             cw[j] += node.work;
             cp[j] += node.param;
@@ -240,10 +253,10 @@ slice_orders(DeviceGraph g, const int* __restrict__ orders, int k, C B, C M, lon
             Fw[l - 1] = ci[j] + B * cw[j] + (excess > 0 ? excess : C(0)) + ck[j] + co[j];
         }
     };
-    column(1, F + n);                                                // the column of r sits in F + (r & 1) * n
+    column(1, F + fs);                                               // the column of r sits in F + (r & 1) * fs
     __syncthreads();
     for (int r = 1; r <= n; ++r) {
-        const C* __restrict__ Fr = F + (r & 1) * n;
+        const C* __restrict__ Fr = F + (r & 1) * fs;
         // dp[kk][r] = min over l of max(dp[kk - 1][l], F(l + 1, r)); the earlier l on equal values
         for (int kk = warp + 1; kk <= kmax; kk += kWarps) {
             C best = kInf;
@@ -251,28 +264,35 @@ slice_orders(DeviceGraph g, const int* __restrict__ orders, int k, C B, C M, lon
             if (kk == 1) {
                 best = Fr[0];
             } else if (r >= kk) {
-                const C* below = dp + size_t(kk - 2) * (n + 1);
-                for (int l = kk - 1 + lane; l < r; l += 32) {
-                    const C a = below[l], b = Fr[l];
-                    const C cand = a > b ? a : b;
-                    if (cand < best) { best = cand; where = l; }     // l ascends within a lane: strict < keeps the earlier one
+                // 16 bytes of each row per lane and trip.  Entries before l = kk - 1 hold "no such slicing" in the row below, entries
+                // from l = r on hold it in the column: they never win.
+                const C* below = dp + size_t(kk - 2) * ds;
+                for (int base = ((kk - 1) & ~(V - 1)) + lane * V; base < r; base += 32 * V) {
+                    C a[V], b[V];
+                    *reinterpret_cast<VecT*>(a) = *reinterpret_cast<const VecT*>(below + base);
+                    *reinterpret_cast<VecT*>(b) = *reinterpret_cast<const VecT*>(Fr + base);
+#pragma unroll
+                    for (int i = 0; i < V; ++i) {
+                        const C cand = a[i] > b[i] ? a[i] : b[i];
+                        if (cand < best) { best = cand; where = base + i; }     // l ascends within a lane: strict < keeps the earlier one
+                    }
                 }
                 warp_min_pair(best, where);
             }
             if (lane == 0) {
-                dp[size_t(kk - 1) * (n + 1) + r] = best;
+                dp[size_t(kk - 1) * ds + r] = best;
                 arg[size_t(kk - 1) * (n + 1) + r] = static_cast<unsigned short>(where);
             }
         }
-        if (r < n) column(r + 1, F + ((r + 1) & 1) * n);             // the other buffer: nobody reads it before the barrier
+        if (r < n) column(r + 1, F + ((r + 1) & 1) * fs);            // the other buffer: nobody reads it before the barrier
         __syncthreads();
     }
 
     if (tid == 0) {
         int best_k = 1;
         for (int kk = 2; kk <= kmax; ++kk)
-            if (dp[size_t(kk - 1) * (n + 1) + n] < dp[size_t(best_k - 1) * (n + 1) + n]) best_k = kk;
-        cost_out[p] = static_cast<long long>(dp[size_t(best_k - 1) * (n + 1) + n]);
+            if (dp[size_t(kk - 1) * ds + n] < dp[size_t(best_k - 1) * ds + n]) best_k = kk;
+        cost_out[p] = static_cast<long long>(dp[size_t(best_k - 1) * ds + n]);
         blocks_out[p] = best_k;
         status_out[p] = 0;
         int r = n;
