@@ -538,7 +538,21 @@ def run_mtpp(bq, dev, args, name="mtpp_unet"):
         mo.slice_order(g, mo.decode_order(g, keys_host[p].tolist()), w.k, w.B, w.M)
     cpu_s = (time.perf_counter() - t) / sample
     dg.close()
+    # What bounds the slicing kernel is integer arithmetic.  Algorithmic operations of one order: every candidate cut of the
+    # dynamic programme is one max and one compare (rows 2..k, right ends r, cuts l = row - 1 .. r - 1); every column entry
+    # (l, r) takes 4 running updates, 7 operations to put the cost together and 2 compares + 2 conditional adds per producer
+    # edge of the node at r.  Peak: one 16-lane integer pipe per scheduler, 4 schedulers per SM, at the top SM clock.
+    rr = np.arange(1, n + 1, dtype=np.int64)
+    kmax = min(w.k, n)
+    dp_ops = 2 * sum(int(np.maximum(rr - kk + 1, 0).sum()) for kk in range(2, kmax + 1))
+    col_ops = 11 * int(rr.sum()) + 4 * edges.shape[0] * (n + 1) // 2          # an edge's consumer sits at position (n + 1) / 2 on average
+    sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
+    alu_peak = sm_count * 4 * 16 * 1.965e9
+    alu_achieved = P * (dp_ops + col_ops) / (ms_slice * 1e-3)
     return {"workload": f"{name}: {w.recipe}; n = {n} nodes, {edges.shape[0]} edges, at most k = {w.k} blocks, population {P}",
+            "roofline": {"bound": "alu", "kernel": "slice_orders", "achieved": round(alu_achieved / 1e12, 3), "peak": round(alu_peak / 1e12, 2),
+                         "peak_kind": "derived: SMs x 4 schedulers x 16 integer lanes x 1965 MHz", "unit": "Tint-op/s", "frac": round(alu_achieved / alu_peak, 4),
+                         "algorithmic_ops_per_order": dp_ops + col_ops, "traffic": None},
             "decode_ms": round(ms_decode, 4), "slice_ms": round(ms_slice, 4), "orders_per_s": round(P / (ms_decode + ms_slice) * 1e3, 1),
             "us_per_order": round((ms_decode + ms_slice) * 1e3 / P, 3), "best_bottleneck": int(cost.min()), "worst_bottleneck": int(cost.max()),
             "cpu_baseline": {"value": round(1.0 / cpu_s, 3), "unit": "orders/s", "cores": 1, "kind": "oracle", "sample": f"{sample} orders of the population, decode + slice"},

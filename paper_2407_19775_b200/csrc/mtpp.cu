@@ -304,44 +304,90 @@ slice_orders(DeviceGraph g, const int* __restrict__ orders, int k, C B, C M, lon
     }
 }
 
-// One warp per key vector.  Per step the lanes look through the nodes for the ready one with the
-// highest key (equal keys: the smaller node), the winner is appended and its consumers' counts of
-// missing producers drop.
+// Shared memory of decode_orders: per warp the counts of missing producers, the keys as ordered integers and the ready mask
+// (a bit per node, word w owned by lane w); per CTA the consumer lists when `staged_edges` > 0.
+struct DecodeLayout {
+    size_t ukey, ready, missing, cptr, cons, total;
+};
+__host__ __device__ inline DecodeLayout decode_layout(int n, int staged_edges) {
+    DecodeLayout L;
+    size_t o = 0;
+    L.ukey = o;    o += size_t(kDecodeWarps) * n * 4;
+    L.ready = o;   o += size_t(kDecodeWarps) * 32 * 4;
+    L.cptr = o;    o += staged_edges > 0 ? size_t(n + 1) * 4 : 0;
+    L.cons = o;    o += staged_edges > 0 ? size_t(staged_edges) * 4 : 0;
+    L.missing = o; o += size_t(kDecodeWarps) * n * 2;
+    L.total = round_up(o, 16);
+    return L;
+}
+constexpr int kDecodeStagedEdgesMax = 4096;                         // keeps the CTA within 48 KB at n = 1024
+
+// One warp per key vector.  Ready nodes are a bit mask (at most 32 words: one per lane), so a step looks only at the nodes
+// that are ready, not at all n: each lane walks the set bits of its word for its best key (equal keys: the smaller node),
+// two warp reductions pick the winner (the largest key, then the smallest node that has it), the winner is appended, its bit
+// cleared, and its consumers' counts of missing producers drop; a count that reaches zero sets the consumer's bit.
+// Keys are compared as integers: k + 0.0f (which turns -0.0 into +0.0) mapped so that the order of finite floats is the
+// order of unsigned words; no finite key maps to 0, which stands for "no ready node here".
 __global__ void __launch_bounds__(kDecodeWarps * 32)
-decode_orders(DeviceGraph g, const float* __restrict__ keys, int P, int* __restrict__ orders_out) {
+decode_orders(DeviceGraph g, int staged_edges, const float* __restrict__ keys, int P, int* __restrict__ orders_out) {
     extern __shared__ __align__(16) unsigned char smem[];
     const int n = g.n;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int p = blockIdx.x * kDecodeWarps + warp;
-    if (p >= P) return;
-    short* missing = reinterpret_cast<short*>(smem) + size_t(warp) * n;      // producers not yet placed; -1 once the node is placed
-    float* key = reinterpret_cast<float*>(smem + round_up(size_t(kDecodeWarps) * n * 2, 16)) + size_t(warp) * n;
-    for (int v = lane; v < n; v += 32) {
-        missing[v] = short(g.pred_ptr[v + 1] - g.pred_ptr[v]);
-        key[v] = keys[size_t(p) * n + v];
+    const DecodeLayout L = decode_layout(n, staged_edges);
+    unsigned* ukey = reinterpret_cast<unsigned*>(smem + L.ukey) + size_t(warp) * n;
+    unsigned* ready = reinterpret_cast<unsigned*>(smem + L.ready) + warp * 32;
+    short* missing = reinterpret_cast<short*>(smem + L.missing) + size_t(warp) * n;
+    const int* cons_ptr = g.cons_ptr;
+    const int* cons = g.cons;
+    if (staged_edges > 0) {
+        int* sp = reinterpret_cast<int*>(smem + L.cptr);
+        int* sc = reinterpret_cast<int*>(smem + L.cons);
+        for (int i = threadIdx.x; i <= n; i += kDecodeWarps * 32) sp[i] = g.cons_ptr[i];
+        for (int i = threadIdx.x; i < staged_edges; i += kDecodeWarps * 32) sc[i] = g.cons[i];
+        cons_ptr = sp;
+        cons = sc;
+        __syncthreads();
     }
+    if (p >= P) return;
+    const int words = (n + 31) / 32;
+    for (int w = 0; w < words; ++w) {                                        // word w: nodes 32w .. 32w + 31, kept by lane w
+        const int v = w * 32 + lane;
+        int deg = 1;
+        if (v < n) {
+            deg = g.pred_ptr[v + 1] - g.pred_ptr[v];
+            missing[v] = short(deg);
+            const unsigned bits = __float_as_uint(keys[size_t(p) * n + v] + 0.0f);
+            ukey[v] = (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+        }
+        const unsigned mask = __ballot_sync(0xffffffffu, deg == 0);
+        if (lane == w) ready[lane] = mask;
+    }
+    if (lane >= words) ready[lane] = 0;
     __syncwarp();
     for (int step = 0; step < n; ++step) {
-        float bk = 0.0f;
-        int bv = n;                                                          // n: no ready node seen
-        for (int v = lane; v < n; v += 32) {
-            if (missing[v] == 0) {
-                const float kv = key[v];
-                if (bv == n || kv > bk) { bk = kv; bv = v; }                 // v ascends within a lane: strict > keeps the smaller node
-            }
+        unsigned w = ready[lane];
+        unsigned bk = 0;
+        int bv = 0x7fffffff;
+        while (w) {
+            const int v = lane * 32 + __ffs(int(w)) - 1;
+            w &= w - 1;
+            const unsigned kv = ukey[v];
+            if (kv > bk) { bk = kv; bv = v; }                                // v ascends within a lane: strict > keeps the smaller node
         }
-#pragma unroll
-        for (int s = 16; s >= 1; s >>= 1) {
-            const float ok = __shfl_xor_sync(0xffffffffu, bk, s);
-            const int ov = __shfl_xor_sync(0xffffffffu, bv, s);
-            if (ov != n && (bv == n || ok > bk || (ok == bk && ov < bv))) { bk = ok; bv = ov; }
-        }
-        if (bv == n) break;                                                  // cannot happen for an acyclic graph (checked at upload)
+        const unsigned top = __reduce_max_sync(0xffffffffu, bk);
+        if (top == 0) break;                                                 // no ready node: cannot happen for an acyclic graph (checked at upload)
+        const int win = int(__reduce_min_sync(0xffffffffu, bk == top ? unsigned(bv) : 0x7fffffffu));
         if (lane == 0) {
-            orders_out[size_t(p) * n + step] = bv;
-            missing[bv] = -1;
+            orders_out[size_t(p) * n + step] = win;
+            atomicAnd(&ready[win >> 5], ~(1u << (win & 31)));
         }
-        for (int e = g.cons_ptr[bv] + lane; e < g.cons_ptr[bv + 1]; e += 32) missing[g.cons[e]] -= 1;    // consumers are distinct nodes
+        for (int e = cons_ptr[win] + lane; e < cons_ptr[win + 1]; e += 32) {  // consumers are distinct nodes
+            const int c = cons[e];
+            const short left = short(missing[c] - 1);
+            missing[c] = left;
+            if (left == 0) atomicOr(&ready[c >> 5], 1u << (c & 31));
+        }
         __syncwarp();
     }
 }
@@ -489,9 +535,10 @@ int mtpp_decode_orders(const mtpp_graph* g, const float* keys, int P, int32_t* o
     if (!keys || !orders_out) return BQ_ERR_NULL;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev != g->device) return BQ_ERR_CUDA;
-    const size_t smem = round_up(size_t(kDecodeWarps) * g->d.n * 2, 16) + size_t(kDecodeWarps) * g->d.n * 4;
+    const int staged_edges = (g->d.edges > 0 && g->d.edges <= kDecodeStagedEdgesMax) ? g->d.edges : 0;     // larger lists stay in global memory
+    const size_t smem = decode_layout(g->d.n, staged_edges).total;                                         // at most 45 KB
     const unsigned grid = unsigned((P + kDecodeWarps - 1) / kDecodeWarps);
-    decode_orders<<<grid, kDecodeWarps * 32, smem, static_cast<cudaStream_t>(cuda_stream)>>>(g->d, keys, P, orders_out);
+    decode_orders<<<grid, kDecodeWarps * 32, smem, static_cast<cudaStream_t>(cuda_stream)>>>(g->d, staged_edges, keys, P, orders_out);
     const cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? BQ_OK : cuda_fail(e);
 }

@@ -192,6 +192,27 @@ def test_costs_on_either_side_of_the_32_bit_bound(bq, pad, M):
     dg.close()
 
 
+def test_decoding_with_keys_of_either_sign_zeros_and_repeats(bq):
+    """Keys are compared as floats: negative keys, -0.0 beside +0.0 (equal: the smaller node goes first), repeated values,
+    huge and tiny magnitudes, infinities; on graphs with one word of ready bits, several, and the most (1024 nodes), with the
+    consumer lists in shared memory and, for the dense one, in global memory."""
+    rng = random.Random(11)
+    pool = [0.0, -0.0, 1.0, -1.0, 0.5, -0.5, 1e-38, -1e-38, 3e38, -3e38, float("inf"), float("-inf"), 0.25, 0.25, 2.0 ** -149, -(2.0 ** -149)]
+    for n, density in ((20, 0.2), (100, 0.05), (333, 0.08), (1024, 0.08), (1024, 0.3)):
+        edges = np.asarray([(u, v) for u in range(n) for v in range(u + 1, min(n, u + 40)) if rng.random() < density], np.int32).reshape(-1, 2)
+        ones = np.ones(n, np.int64)
+        g = oracle_graph(n, edges, ones, ones, ones)
+        dg = bq.mtpp.SliceGraph(n, edges, ones, ones, ones, device="cuda:0")
+        P = 6
+        keys = torch.tensor([[rng.choice(pool) if p % 2 else rng.uniform(-1, 1) for _ in range(n)] for p in range(P)], dtype=torch.float32)
+        keys[2] = -0.0
+        keys[2, ::3] = 0.0
+        orders = dg.decode_orders(keys.cuda()).cpu()
+        for p in range(P if n <= 333 else 3):
+            assert orders[p].tolist() == mo.decode_order(g, keys[p].tolist()), (n, density, p)
+        dg.close()
+
+
 def test_rows_that_are_not_topological_orders_are_flagged(bq):
     n, edges, work, sizeparam, sizeout = workloads.make_graph("mtpp_tiny")
     g = oracle_graph(n, edges, work, sizeparam, sizeout)
