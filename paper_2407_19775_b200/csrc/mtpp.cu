@@ -24,7 +24,6 @@
 
 namespace {
 
-constexpr int kSliceThreads = 256;
 constexpr int kDecodeWarps = 4;
 constexpr size_t kSliceSmemLimit = 226 * 1024;         // dynamic part of the 227 KB one CTA may take; the kernel's static words fit in the rest
 
@@ -109,8 +108,8 @@ template <> struct CostVec<long long> { using T = longlong2; static constexpr in
 // from which on l holds u inside and stops counting it as an output.
 //
 // C: the word costs are kept in.  int when the host has bounded every segment cost of the call below 2^31, long long otherwise.
-template <int kOwned, class C, bool kEdgesInSmem>                   // first positions per thread: n <= kOwned * kSliceThreads
-__global__ void __launch_bounds__(kSliceThreads)
+template <int NT, int kOwned, class C, bool kEdgesInSmem>           // NT threads, kOwned first positions per thread: n <= kOwned * NT
+__global__ void __launch_bounds__(NT)
 slice_orders(DeviceGraph g, const int* __restrict__ orders, int k, C B, C M, long long* __restrict__ cost_out,
              int* __restrict__ blocks_out, int* __restrict__ cuts_out, int* __restrict__ status_out) {
     constexpr bool kNarrow = sizeof(C) == 4;
@@ -134,7 +133,7 @@ slice_orders(DeviceGraph g, const int* __restrict__ orders, int k, C B, C M, lon
 
     const int p = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    constexpr int kWarps = kSliceThreads / 32;
+    constexpr int kWarps = NT / 32;
     constexpr int V = CostVec<C>::N;
     using VecT = typename CostVec<C>::T;
     const int fs = int(slice_fstride(n)), ds = int(slice_dstride(n));
@@ -142,16 +141,16 @@ slice_orders(DeviceGraph g, const int* __restrict__ orders, int k, C B, C M, lon
 
     // positions, and the check that the row is a topological order of this graph
     if (tid == 0) bad = 0;
-    for (int i = tid; i < n; i += kSliceThreads) { pos[i] = 0; ord[i] = pi[i]; }
+    for (int i = tid; i < n; i += NT) { pos[i] = 0; ord[i] = pi[i]; }
     __syncthreads();
-    for (int i = tid; i < n; i += kSliceThreads) {
+    for (int i = tid; i < n; i += NT) {
         const int v = ord[i];
         if (v < 0 || v >= n) bad = 1;
         else if (atomicExch(&pos[v], i + 1) != 0) bad = 1;          // a node listed twice (so another one is missing)
     }
     __syncthreads();
     if (!bad) {
-        for (int v = tid; v < n; v += kSliceThreads) {
+        for (int v = tid; v < n; v += NT) {
             int lc = 0;
             for (int e = g.cons_ptr[v]; e < g.cons_ptr[v + 1]; ++e) {
                 const int pc = pos[g.cons[e]];
@@ -164,14 +163,14 @@ slice_orders(DeviceGraph g, const int* __restrict__ orders, int k, C B, C M, lon
     __syncthreads();
     if (bad) {
         if (tid == 0) { cost_out[p] = -1; blocks_out[p] = 0; status_out[p] = 1; }
-        for (int j = tid; j < k; j += kSliceThreads) cuts_out[size_t(p) * k + j] = 0;
+        for (int j = tid; j < k; j += NT) cuts_out[size_t(p) * k + j] = 0;
         return;
     }
 
     // the node records by position, and how many producer edges each position has
     if (tid == 0) epos[0] = 0;
     if (tid < kmax) dp[size_t(tid) * ds] = kInf;                     // no block holds the first 0 nodes: the vector reads below may start there
-    for (int i = tid; i < n; i += kSliceThreads) {
+    for (int i = tid; i < n; i += NT) {
         const int v = ord[i];
         const C so = C(g.sizeout[v]);
         attr[i] = NodeRecord<C>{C(g.work[v]), C(g.sizeparam[v]), so, last[v] != 0 ? so : C(0)};
@@ -204,7 +203,7 @@ slice_orders(DeviceGraph g, const int* __restrict__ orders, int k, C B, C M, lon
         return EdgeInfo{pu > pc ? pu : pc, last[u] == r ? pu : 0, C(g.sizeout[u])};
     };
     if constexpr (kEdgesInSmem) {
-        for (int i = tid; i < n; i += kSliceThreads) {
+        for (int i = tid; i < n; i += NT) {
             const int v = ord[i];
             const int from = g.pred_ptr[v], at = epos[i], deg = epos[i + 1] - at;
             for (int j = 0; j < deg; ++j) {
@@ -220,14 +219,14 @@ slice_orders(DeviceGraph g, const int* __restrict__ orders, int k, C B, C M, lon
     C cw[kOwned], cp[kOwned], ck[kOwned], ci[kOwned], co[kOwned];
 #pragma unroll
     for (int j = 0; j < kOwned; ++j) { cw[j] = 0; cp[j] = 0; ck[j] = 0; ci[j] = 0; co[j] = 0; }
-    // the column of r into Fw: thread t owns the first positions l = t + 1, t + 257, ... and keeps their five running values in registers
+    // the column of r into Fw: thread t owns the first positions l = t + 1, t + 1 + NT, ... and keeps their five running values in registers
     auto column = [&](int r, C* __restrict__ Fw) {
         const NodeRecord<C> node = attr[r - 1];
         const int pb = epos[r - 1], pe = epos[r];
         const int from = kEdgesInSmem ? 0 : g.pred_ptr[ord[r - 1]];
 #pragma unroll
         for (int j = 0; j < kOwned; ++j) {
-            const int l = tid + 1 + j * kSliceThreads;
+            const int l = tid + 1 + j * NT;
             if (l > r) {
                 if (l < r + V) Fw[l - 1] = kInf;                     // what a vector read of the column's end takes in beside it
                 continue;
@@ -266,7 +265,7 @@ slice_orders(DeviceGraph g, const int* __restrict__ orders, int k, C B, C M, lon
             } else if (r >= kk) {
                 // 16 bytes of each row per lane and trip.  Entries before l = kk - 1 hold "no such slicing" in the row below, entries
                 // from l = r on hold it in the column: they never win.
-                const C* below = dp + size_t(kk - 2) * ds;
+                const C* below = dp + (kk - 2) * ds;
                 for (int base = ((kk - 1) & ~(V - 1)) + lane * V; base < r; base += 32 * V) {
                     C a[V], b[V];
                     *reinterpret_cast<VecT*>(a) = *reinterpret_cast<const VecT*>(below + base);
@@ -280,8 +279,8 @@ slice_orders(DeviceGraph g, const int* __restrict__ orders, int k, C B, C M, lon
                 warp_min_pair(best, where);
             }
             if (lane == 0) {
-                dp[size_t(kk - 1) * ds + r] = best;
-                arg[size_t(kk - 1) * (n + 1) + r] = static_cast<unsigned short>(where);
+                dp[(kk - 1) * ds + r] = best;
+                arg[(kk - 1) * (n + 1) + r] = static_cast<unsigned short>(where);
             }
         }
         if (r < n) column(r + 1, F + ((r + 1) & 1) * fs);            // the other buffer: nobody reads it before the barrier
@@ -407,20 +406,31 @@ namespace {
 std::mutex g_attr_lock;
 bool g_attr_done[64] = {};
 
-// the instances of slice_orders: first positions per thread x cost word x where the edges are kept
-template <int kOwned, class C, bool kEdgesInSmem>
-const void* slice_kernel() { return reinterpret_cast<const void*>(&slice_orders<kOwned, C, kEdgesInSmem>); }
-const void* slice_kernel(int owned, bool narrow, bool edges_in_smem) {
-#define MTPP_PICK(O) (narrow ? (edges_in_smem ? slice_kernel<O, int, true>() : slice_kernel<O, int, false>()) \
-                             : (edges_in_smem ? slice_kernel<O, long long, true>() : slice_kernel<O, long long, false>()))
-    return owned == 1 ? MTPP_PICK(1) : owned == 2 ? MTPP_PICK(2) : MTPP_PICK(4);
-#undef MTPP_PICK
+// The instances of slice_orders: (threads, first positions per thread) x cost word x where the edges are kept.  Small graphs take
+// CTAs of four warps: what a step costs beside its arithmetic (the barrier, a warp's share of loop control) grows with the warps.
+struct SliceShape { int threads, owned; };
+inline SliceShape slice_shape(int n) {
+    if (n <= 128) return {128, 1};
+    if (n <= 256) return {128, 2};
+    if (n <= 512) return {256, 2};
+    return {256, 4};
+}
+template <int NT, int kOwned>
+const void* slice_kernel_of(bool narrow, bool edges_in_smem) {
+    if (narrow) return edges_in_smem ? reinterpret_cast<const void*>(&slice_orders<NT, kOwned, int, true>)
+                                     : reinterpret_cast<const void*>(&slice_orders<NT, kOwned, int, false>);
+    return edges_in_smem ? reinterpret_cast<const void*>(&slice_orders<NT, kOwned, long long, true>)
+                         : reinterpret_cast<const void*>(&slice_orders<NT, kOwned, long long, false>);
+}
+const void* slice_kernel(SliceShape shape, bool narrow, bool edges_in_smem) {
+    if (shape.threads == 128) return shape.owned == 1 ? slice_kernel_of<128, 1>(narrow, edges_in_smem) : slice_kernel_of<128, 2>(narrow, edges_in_smem);
+    return shape.owned == 2 ? slice_kernel_of<256, 2>(narrow, edges_in_smem) : slice_kernel_of<256, 4>(narrow, edges_in_smem);
 }
 std::vector<const void*> slice_kernels() {
     std::vector<const void*> all;
-    for (int owned : {1, 2, 4})
+    for (SliceShape shape : {SliceShape{128, 1}, SliceShape{128, 2}, SliceShape{256, 2}, SliceShape{256, 4}})
         for (bool narrow : {false, true})
-            for (bool in_smem : {false, true}) all.push_back(slice_kernel(owned, narrow, in_smem));
+            for (bool in_smem : {false, true}) all.push_back(slice_kernel(shape, narrow, in_smem));
     return all;
 }
 
@@ -570,9 +580,9 @@ int mtpp_slice_orders(const mtpp_graph* g, const int32_t* orders, int P, int k, 
     cudaError_t e = cudaSuccess;
     if (L.total > 48 * 1024) e = allow_slice_smem(g->device);
     if (e != cudaSuccess) return cuda_fail(e);
-    static_assert(MTPP_MAX_NODES <= 4 * kSliceThreads, "the widest instance owns four first positions per thread");
-    const int owned = g->d.n <= kSliceThreads ? 1 : g->d.n <= 2 * kSliceThreads ? 2 : 4;
-    const void* kernel = slice_kernel(owned, narrow, edges_in_smem);
+    static_assert(MTPP_MAX_NODES <= 4 * 256, "the widest instance owns four first positions per thread");
+    const SliceShape shape = slice_shape(g->d.n);
+    const void* kernel = slice_kernel(shape, narrow, edges_in_smem);
     long long* cost = reinterpret_cast<long long*>(cost_out);
     DeviceGraph d = g->d;
     long long B64 = B, M64 = M;
@@ -580,7 +590,7 @@ int mtpp_slice_orders(const mtpp_graph* g, const int32_t* orders, int P, int k, 
     int M32 = M < 0x7fffffffLL ? int(M) : 0x7fffffff;                 // parameters + peak stay below the bound: a larger M never shows
     void* args[] = {&d, &orders, &k, narrow ? static_cast<void*>(&B32) : static_cast<void*>(&B64),
                     narrow ? static_cast<void*>(&M32) : static_cast<void*>(&M64), &cost, &blocks_out, &cuts_out, &status_out};
-    e = cudaLaunchKernel(kernel, dim3(unsigned(P)), dim3(kSliceThreads), args, L.total, static_cast<cudaStream_t>(cuda_stream));
+    e = cudaLaunchKernel(kernel, dim3(unsigned(P)), dim3(unsigned(shape.threads)), args, L.total, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return cuda_fail(e);
     e = cudaGetLastError();
     return e == cudaSuccess ? BQ_OK : cuda_fail(e);

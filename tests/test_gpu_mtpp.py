@@ -98,10 +98,10 @@ def banded_graph(n, seed, scale=1, density=0.08):
     return edges, work, sizeparam, sizeout
 
 
-@pytest.mark.parametrize("n,k,scale", [(257, 16, 1), (300, 5, 1 << 21), (520, 3, 1), (513, 2, 1 << 21)])
+@pytest.mark.parametrize("n,k,scale", [(130, 3, 1), (200, 4, 1 << 21), (257, 16, 1), (300, 5, 1 << 21), (520, 3, 1), (513, 2, 1 << 21)])
 def test_graphs_wider_than_one_position_per_thread(bq, n, k, scale):
-    """Above 256 and above 512 nodes a thread of the slicing kernel owns two and four first positions: one order of each in
-    full against the oracle, with costs inside 32 bits and beyond them."""
+    """Above 128 nodes a thread of the slicing kernel owns two first positions, above 256 the CTA has eight warps, above 512 a
+    thread owns four: one order of each in full against the oracle, with costs inside 32 bits and beyond them."""
     edges, work, sizeparam, sizeout = banded_graph(n, n, scale)
     g = oracle_graph(n, edges, work, sizeparam, sizeout)
     dg = bq.mtpp.SliceGraph(n, edges, work, sizeparam, sizeout, device="cuda:0")
@@ -211,6 +211,27 @@ def test_decoding_with_keys_of_either_sign_zeros_and_repeats(bq):
         for p in range(P if n <= 333 else 3):
             assert orders[p].tolist() == mo.decode_order(g, keys[p].tolist()), (n, density, p)
         dg.close()
+
+
+@pytest.mark.parametrize("scale", [1, 1 << 21])
+def test_complete_graph_whose_edges_stay_in_global_memory(bq, scale):
+    """Every pair (u, v), u < v, is an edge: 232 nodes have 26,796 edges, more than fit in shared memory beside the
+    programme's arrays, so the four-warp instance looks them up in global memory.  One topological order; in full against the oracle."""
+    n, k = 232, 4
+    edges = np.asarray([(u, v) for u in range(n) for v in range(u + 1, n)], np.int32)
+    work = np.full(n, 3, np.int64)
+    sizeparam = np.full(n, 5, np.int64) * scale
+    sizeout = np.asarray([7 + i % 5 for i in range(n)], np.int64) * scale
+    g = oracle_graph(n, edges, work, sizeparam, sizeout)
+    dg = bq.mtpp.SliceGraph(n, edges, work, sizeparam, sizeout, device="cuda:0")
+    orders = dg.decode_orders(torch.rand((2, n), generator=torch.Generator().manual_seed(4)).cuda())
+    assert orders.cpu().tolist() == [list(range(n))] * 2
+    cost, blocks, cuts, status = dg.slice_orders(orders, k, 2 * scale, 100 * scale)
+    torch.cuda.synchronize()
+    want = mo.slice_order(g, list(range(n)), k, 2 * scale, 100 * scale)
+    for p in range(2):
+        assert int(status[p]) == 0 and (int(cost[p]), int(blocks[p]), cuts[p][:int(blocks[p])].cpu().tolist()) == want
+    dg.close()
 
 
 def test_rows_that_are_not_topological_orders_are_flagged(bq):
