@@ -45,7 +45,8 @@ typedef enum {
     BQ_ERR_BLOCK = 3,     /* block < 1                                          */
     BQ_ERR_SIZE = 4,      /* n does not fit the launch limits (n >= 2^40)       */
     BQ_ERR_CODEBOOK = 5,  /* unknown kind, bad user values, NULL handle or wrong device */
-    BQ_ERR_CUDA = 6       /* a CUDA runtime call or a launch failed             */
+    BQ_ERR_CUDA = 6,      /* a CUDA runtime call or a launch failed             */
+    BQ_ERR_ASSERT = 11    /* a debug build's assertion failed (bq_debug_build); the condition is the last error text */
 } bq_status;
 
 enum { BQ_CODEBOOK_DYNAMIC_TREE = 0, BQ_CODEBOOK_USER = 1 };
@@ -70,6 +71,10 @@ typedef struct bq_codebook bq_codebook;
  *          current device and synchronises that device once.  Free with bq_free_codebook.
  */
 int bq_make_codebook(int kind, const float* user_values256, float* host_values_out256, bq_codebook** out);
+
+/* 1 if this library was built with its host-side assertions (overlapping buffers, the split of
+ * a tensor between kernels; they return BQ_ERR_ASSERT before anything is launched), else 0. */
+int bq_debug_build(void);
 
 /* Frees the handle and its device memory.  NULL is allowed. */
 int bq_free_codebook(bq_codebook* cb);

@@ -18,7 +18,7 @@ LIB_PATH = os.environ.get("BQ_LIB", os.path.join(_HERE, "libbq.so"))    # BQ_LIB
 _lib = None
 
 SYMBOLS = ("bq_make_codebook", "bq_free_codebook", "bq_quantize", "bq_dequantize", "bq_roundtrip",
-           "bq_status_string", "bq_last_cuda_error", "bq_codebook_is_folded",
+           "bq_status_string", "bq_last_cuda_error", "bq_codebook_is_folded", "bq_debug_build",
            "bq_host_pipe_create", "bq_host_pipe_destroy", "bq_quantize_host", "bq_dequantize_host", "bq_roundtrip_host",
            "bq_host_pipe_wait", "bq_host_pipe_wait_on_stream", "bq_set_staging", "bq_kernel_status")
 
@@ -60,7 +60,7 @@ def _check(rc: int, what: str) -> None:
     if rc != 0:
         L = lib()
         msg = L.bq_status_string(rc).decode()
-        if rc == 6:
+        if rc in (6, 10, 11):                                     # CUDA errors, the static limit and debug assertions leave a text
             msg += ": " + L.bq_last_cuda_error().decode()
         raise BqError(f"{what} failed with status {rc} ({msg})")
 
@@ -119,6 +119,11 @@ class Codebook:
 def set_staging(on: bool) -> bool:
     """``bq_set_staging``: blocks of 2048 / 4096 through the shared-memory-staged kernel; returns the previous setting."""
     return bool(lib().bq_set_staging(int(bool(on))))
+
+
+def debug_build() -> bool:
+    """``bq_debug_build``: whether the loaded library carries its host-side assertions."""
+    return bool(lib().bq_debug_build())
 
 
 def kernel_status(cb: "Codebook") -> int:

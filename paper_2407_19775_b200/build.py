@@ -1,9 +1,13 @@
 """Builds ``libbq.so`` (the CUDA library) in-tree with nvcc for sm_100a.
 
-    python -m paper_2407_19775_b200.build [--force] [--verbose]
+    python -m paper_2407_19775_b200.build [--force] [--verbose] [--debug]
 
 Each translation unit is compiled on its own (in parallel) and the objects are linked into
 ``paper_2407_19775_b200/libbq.so``.  nvcc cross-compiles, so no GPU is needed to build.
+
+``--debug`` also links ``libbq_debug.so``: the units that use the host-side assertions of
+``csrc/bq_debug.h`` compiled with ``-DBQ_DEBUG``, the kernels as in the release build.  Load it
+with ``BQ_LIB=.../libbq_debug.so``.
 """
 from __future__ import annotations
 
@@ -16,6 +20,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libbq.so")
+OBJ_DEBUG = os.path.join(HERE, "_build_debug")
+LIB_DEBUG = os.path.join(HERE, "libbq_debug.so")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 
 NVCC_FLAGS = [
@@ -70,5 +76,36 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+def build_debug(force: bool = False) -> str:
+    """libbq_debug.so: the release objects, except that the units with assertions are compiled with -DBQ_DEBUG."""
+    build(force=force)
+    os.makedirs(OBJ_DEBUG, exist_ok=True)
+    hdr = _newest_header()
+    objs = []
+    for src in _sources():
+        s = os.path.join(CSRC, src)
+        with open(s) as f:
+            asserting = "bq_debug.h" in f.read()
+        if not asserting:
+            objs.append(os.path.join(OBJ, src[:-3] + ".o"))
+            continue
+        o = os.path.join(OBJ_DEBUG, src[:-3] + ".o")
+        if force or not os.path.exists(o) or os.path.getmtime(o) < max(os.path.getmtime(s), hdr):
+            r = subprocess.run(["nvcc", *NVCC_FLAGS, "-DBQ_DEBUG", "-c", s, "-o", o], capture_output=True, text=True)
+            if r.returncode != 0:
+                raise RuntimeError(f"nvcc failed on {s}:\n{r.stdout}\n{r.stderr}")
+        objs.append(o)
+    if force or not os.path.exists(LIB_DEBUG) or any(os.path.getmtime(o) > os.path.getmtime(LIB_DEBUG) for o in objs):
+        tmp = LIB_DEBUG + f".tmp{os.getpid()}"
+        r = subprocess.run(["nvcc", "-shared", "-o", tmp, *objs, "-gencode", "arch=compute_100a,code=sm_100a"], capture_output=True, text=True)
+        if r.returncode != 0:
+            raise RuntimeError(f"link failed:\n{r.stdout}\n{r.stderr}")
+        os.replace(tmp, LIB_DEBUG)
+    return LIB_DEBUG
+
+
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    if "--debug" in sys.argv:
+        print(build_debug(force="--force" in sys.argv))
+    else:
+        print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))

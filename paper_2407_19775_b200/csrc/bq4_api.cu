@@ -3,6 +3,7 @@
 // of kernel.
 #include "../../include/bq4.h"
 #include "bq4_kernels.cuh"
+#include "bq_debug.h"
 #include "bq_launch.h"
 #include "bq_error.h"
 
@@ -245,6 +246,10 @@ int bq4_quantize(const void* x, bq_dtype xdt, size_t n, int block, const bq4_cod
     if (!cb) return BQ_ERR_CODEBOOK;
     if (n == 0) return BQ_OK;
     if (!x || !packed_out || !absmax_out) return BQ_ERR_NULL;
+    {
+        const size_t xs = n * (xdt == BQ_F32 ? 4 : 2), ps = (n + 1) / 2, as = ((n + size_t(block) - 1) / size_t(block)) * sizeof(float);
+        BQ_ASSERT(bqd::disjoint(x, xs, packed_out, ps) && bqd::disjoint(x, xs, absmax_out, as) && bqd::disjoint(packed_out, ps, absmax_out, as));
+    }
     int sms = 0;
     const int rc = sm_count_of_current(&sms);
     if (rc != BQ_OK) return rc;
@@ -266,6 +271,10 @@ int bq4_dequantize(const uint8_t* packed, const float* absmax, size_t n, int blo
     if (!cb) return BQ_ERR_CODEBOOK;
     if (n == 0) return BQ_OK;
     if (!packed || !absmax || !y_out) return BQ_ERR_NULL;
+    {
+        const size_t ys = n * (ydt == BQ_F32 ? 4 : 2), ps = (n + 1) / 2, as = ((n + size_t(block) - 1) / size_t(block)) * sizeof(float);
+        BQ_ASSERT(bqd::disjoint(y_out, ys, packed, ps) && bqd::disjoint(y_out, ys, absmax, as));
+    }
     int sms = 0;
     const int rc = sm_count_of_current(&sms);
     if (rc != BQ_OK) return rc;
@@ -287,6 +296,10 @@ int bq4_quantize_s16(const void* x, bq_dtype xdt, size_t n, int block, const bq4
     if (!cb) return BQ_ERR_CODEBOOK;
     if (n == 0) return BQ_OK;
     if (!x || !packed_out || !scale_out) return BQ_ERR_NULL;
+    {
+        const size_t xs = n * (xdt == BQ_F32 ? 4 : 2), ps = (n + 1) / 2, ss = ((n + size_t(block) - 1) / size_t(block)) * sizeof(uint16_t);
+        BQ_ASSERT(bqd::disjoint(x, xs, packed_out, ps) && bqd::disjoint(x, xs, scale_out, ss) && bqd::disjoint(packed_out, ps, scale_out, ss));
+    }
     int sms = 0;
     const int rc = sm_count_of_current(&sms);
     if (rc != BQ_OK) return rc;
@@ -309,6 +322,10 @@ int bq4_dequantize_s16(const uint8_t* packed, const uint16_t* scale, size_t n, i
     if (!cb) return BQ_ERR_CODEBOOK;
     if (n == 0) return BQ_OK;
     if (!packed || !scale || !y_out) return BQ_ERR_NULL;
+    {
+        const size_t ys = n * (ydt == BQ_F32 ? 4 : 2), ps = (n + 1) / 2, ss = ((n + size_t(block) - 1) / size_t(block)) * sizeof(uint16_t);
+        BQ_ASSERT(bqd::disjoint(y_out, ys, packed, ps) && bqd::disjoint(y_out, ys, scale, ss));
+    }
     int sms = 0;
     const int rc = sm_count_of_current(&sms);
     if (rc != BQ_OK) return rc;

@@ -2,6 +2,7 @@
 // the choice of kernel.  Kernel instantiations live in bq_inst_*.cu so that they compile in
 // parallel; this file only calls their launchers.
 #include "../../include/mmd.h"
+#include "bq_debug.h"
 #include "bq_error.h"
 #include "bq_launch.h"
 
@@ -19,6 +20,7 @@ int cuda_fail(cudaError_t e) {
 }
 
 bool known_dtype(int dt) { return dt == BQ_F32 || dt == BQ_F16 || dt == BQ_BF16; }
+size_t elem_bytes(int dt) { return dt == BQ_F32 ? 4 : 2; }
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
@@ -65,6 +67,7 @@ const char* bq_status_string(int status) {
         case BQ_ERR_SIZE: return "element count out of range";
         case BQ_ERR_CODEBOOK: return "invalid codebook kind, values or handle";
         case BQ_ERR_CUDA: return "CUDA runtime error (see bq_last_cuda_error)";
+        case BQ_ERR_ASSERT: return "an assertion of the debug build failed (see bq_last_cuda_error)";
         case MMD_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case MMD_ERR_FEATURES: return "feature list not ascending, out of range or too long";
         case MMD_ERR_PATH: return "the requested kernel path cannot take this shape";
@@ -132,6 +135,8 @@ int bq_free_codebook(bq_codebook* cb) {
 
 int bq_codebook_is_folded(const bq_codebook* cb) { return (cb && cb->host.folded) ? 1 : 0; }
 
+int bq_debug_build(void) { return bqd::kOn ? 1 : 0; }
+
 int bq_set_staging(int on) { return g_staging.exchange(on ? 1 : 0); }
 
 int bq_kernel_status(const bq_codebook* cb, int* status_out) {
@@ -161,6 +166,14 @@ int forward(const void* x, int xdt, size_t n, int block, const bq_codebook* cb, 
             uint8_t* codes, float* absmax, bool write_q, cudaStream_t stream) {
     const size_t B = size_t(block);
     size_t done = 0;        // elements covered by the tuned kernel
+    {
+        const size_t xs = n * elem_bytes(xdt), ys = write_y ? n * elem_bytes(ydt) : 0, cs = write_q ? n : 0;
+        const size_t as = write_q ? ((n + B - 1) / B) * sizeof(float) : 0;
+        BQ_ASSERT(!write_y || y == x || bqd::disjoint(x, xs, y, ys));          // in place, or apart
+        BQ_ASSERT(!write_y || y != x || xdt == ydt);
+        BQ_ASSERT(bqd::disjoint(x, xs, codes, cs) && bqd::disjoint(x, xs, absmax, as));
+        BQ_ASSERT(bqd::disjoint(y, ys, codes, cs) && bqd::disjoint(y, ys, absmax, as) && bqd::disjoint(codes, cs, absmax, as));
+    }
     const bool can_tune = cb->host.folded && tuned_block(block) && aligned(x, 16) && (!write_y || (aligned(y, 16) && ydt == xdt)) &&
                           (!write_q || (aligned(codes, 8) && aligned(absmax, 4)));
     if (can_tune && n >= B && g_staging.load() && (block == 2048 || block == 4096)) {
@@ -177,6 +190,7 @@ int forward(const void* x, int xdt, size_t n, int block, const bq_codebook* cb, 
                                              &done);
         if (e != cudaSuccess) return cuda_fail(e);
     }
+    BQ_ASSERT(done % B == 0 && done <= n);                                   // the general kernel starts on a block border
     if (done < n) {
         cudaError_t e = bql::launch_fwd_general(xdt, ydt, write_y, write_q, x, y, codes, absmax, n, B, done / B, cb->dev, cb->sm_count, stream);
         if (e != cudaSuccess) return cuda_fail(e);
@@ -226,6 +240,10 @@ int bq_dequantize(const uint8_t* codes, const float* absmax, size_t n, int block
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const size_t B = size_t(block);
     size_t done = 0;
+    {
+        const size_t ys = n * elem_bytes(ydt), as = ((n + B - 1) / B) * sizeof(float);
+        BQ_ASSERT(bqd::disjoint(y_out, ys, codes, n) && bqd::disjoint(y_out, ys, absmax, as));
+    }
     const int l2 = log2_exact(B);
     if (l2 >= 4 && aligned(codes, 16) && aligned(y_out, 16) && n >= 16) {
         const size_t n16 = n / 16;
@@ -233,6 +251,7 @@ int bq_dequantize(const uint8_t* codes, const float* absmax, size_t n, int block
         if (e != cudaSuccess) return cuda_fail(e);
         done = n16 * 16;
     }
+    BQ_ASSERT(done % 16 == 0 && done <= n);
     if (done < n) {
         cudaError_t e = bql::launch_deq_general(ydt, codes, absmax, y_out, n, B, done, cb->dev, cb->sm_count, stream);
         if (e != cudaSuccess) return cuda_fail(e);

@@ -146,9 +146,20 @@ def test_mmd_argument_errors_need_no_device(bq):
 def test_status_strings(bq):
     from paper_2407_19775_b200 import binding
     L = binding.lib()
-    seen = {L.bq_status_string(i).decode() for i in range(7)}
-    assert len(seen) == 7 and L.bq_status_string(0) == b"ok"
+    seen = {L.bq_status_string(i).decode() for i in range(12)}
+    assert len(seen) == 12 and L.bq_status_string(0) == b"ok" and "unknown status" not in seen
     assert L.bq_status_string(99) == b"unknown status"
+
+
+def test_release_and_debug_builds_say_which_they_are(bq):
+    """The library the package loads is the release build; the debug build links the same kernels behind API units compiled
+    with their assertions and says so.  (Its behaviour on a GPU: tests/test_gpu_debug_build.py.)"""
+    from paper_2407_19775_b200 import binding, build
+    assert binding.lib().bq_debug_build() == 0 and bq.debug_build() is False
+    dbg = ctypes.CDLL(build.build_debug())
+    assert dbg.bq_debug_build() == 1
+    for name in binding.SYMBOLS:
+        assert hasattr(dbg, name), name
 
 
 def test_argument_errors_need_no_device(bq):
