@@ -8,10 +8,11 @@
 //               in l..r-1 yet, i.e. for l > max(pos(u), position of u's previous consumer);
 //     out(l, r) gains sizeout(v) if v has consumers (they all come later), and loses sizeout(u)
 //               for each producer u of v inside l..r whose last consumer is v.
-// So a CTA keeps five running values per l (in the registers of the thread that owns l), the dp rows
-// of every block count, and the positions of each node, its last consumer and its latest
-// consumer so far: a few tens of kilobytes of shared memory, no global scratch.  Per step one barrier separates the column
-// update from the minimisations, which warp kk does for block count kk.
+// So a CTA keeps five running values per l (in the registers of the thread that owns l), two columns,
+// the dp rows of every block count, and per order a record of each position's node and three
+// numbers per producer edge: a few tens of kilobytes of shared memory, no global scratch.  The
+// column of r + 1 is written in the pass that takes the minima over the column of r (warp kk - 1
+// for block count kk), so a step costs one barrier.
 #include "../../include/mtpp.h"
 #include "bq_error.h"
 
