@@ -387,3 +387,30 @@ def test_stream_k_is_refused_for_shapes_it_does_not_take(bq):
     with pytest.raises(bq.BqError):
         lin.linear(X, torch.float32, path=bq.mmd.PATH_TENSOR_STREAMK)
     lin.close()
+
+
+def test_output_of_more_than_2_32_elements(bq):
+    """32768 tokens through a 256 -> 131080 layer: the output has 2^32 + 262144 elements, so the rows from 32766 on lie past
+    element 2^32 (and every row past 16383 past byte 2^32).  No critical features, so every kernel's result is the oracle's
+    bit for bit: the kernels are compared with each other on the whole output and with the oracle on the first, the last and
+    64 drawn rows."""
+    M, K, N = 32768, 256, 131080
+    g = torch.Generator().manual_seed(77)
+    X = (torch.randn((M, K), generator=g) * 0.5).to(torch.bfloat16)
+    W = (torch.randn((N, K), generator=g) * 0.02).to(torch.bfloat16)
+    idx = np.zeros(0, np.int32)
+    lin = bq.DecomposedLinear(W.cuda(), idx)
+    Xd = X.cuda()
+    assert M * N > 1 << 32
+    y_auto = lin.linear(Xd, None)
+    assert lin.kernel_status() == 0
+    rows = sorted(set(range(64)) | set(range(M - 64, M)) | set(np.random.default_rng(5).choice(M, 64, replace=False).tolist()))
+    qw, sw, wo = mo.rowquant(bits(W), BF16, idx)
+    y_ref = mo.linear(bits(X[rows]), BF16, qw, sw, wo, idx, BF16)
+    assert np.array_equal(bits(y_auto[rows]), y_ref)
+    for path in (1, 3, 4):
+        y = lin.linear(Xd, None, path=path)
+        assert lin.kernel_status() == 0
+        assert torch.equal(y.view(torch.int16), y_auto.view(torch.int16)), path
+        del y
+    lin.close()
