@@ -141,3 +141,45 @@ def test_four_bit_codes_of_more_than_2_32_elements(bq):
     assert np.array_equal(packed[t0 // 2:].cpu().numpy(), wp)
     assert np.array_equal(absmax[nb - 1:].cpu().numpy().view(np.uint32), wa.view(np.uint32))
     assert np.array_equal(_bits(y[t0:].cpu()), bq4_oracle.dequantize(wp, wa, n - t0, BLOCK, ref4, bq4_oracle.BF16))
+
+
+def test_boundary_transfer_of_more_than_2_32_elements(bq):
+    """The same tensor handed across a (loop-back) shard boundary in 133 pieces of 32 Mi elements through three mailbox
+    slots: what arrives is the oracle's roundtrip of every repetition, piece offsets past 2^32 included."""
+    from paper_2407_19775_b200 import transport
+    dev = torch.device("cuda:0")
+    cb = bq.Codebook(device=dev)
+    ref = oracle.make_codebook()
+    pat = workloads.make("sweep1g", rows=8192).view(-1)
+    L = pat.numel()
+    n = (1 << 32) + (1 << 27) + 100
+    reps = (n + L - 1) // L
+    want = []
+    for s in SCALES:
+        xs = (pat.float() * s).to(torch.bfloat16)
+        y, _, _ = oracle.roundtrip_sharded(_bits(xs), oracle.BF16, BLOCK, ref, oracle.BF16, THREADS)
+        want.append(workloads.from_numpy_bits(y, torch.bfloat16).to(dev))
+    pd = pat.to(dev)
+    x = torch.empty(n, dtype=torch.bfloat16, device=dev)
+    for r in range(reps):
+        m = min(L, n - r * L)
+        x[r * L: r * L + m] = (pd[:m].float() * SCALES[r % 5]).to(torch.bfloat16)
+    y = torch.zeros(n, dtype=torch.bfloat16, device=dev)
+    chunk, slots = 1 << 25, 3
+    rx = transport.Receiver(cb, chunk, min_block=BLOCK, slots=slots)
+    tx = transport.Sender(cb, rx.export(), transport.STORE)
+    s_send, s_recv = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    torch.cuda.synchronize()
+    transport.transfer(tx, rx, x, BLOCK, y, s_send, s_recv)
+    s_recv.synchronize()
+    s_send.synchronize()
+    assert len(transport.plan(n, BLOCK, chunk, slots)) == 133
+    for r in range(reps):
+        m = min(L, n - r * L)
+        whole = (m // BLOCK) * BLOCK
+        assert torch.equal(y[r * L: r * L + whole].view(torch.int16), want[r % 5][:whole].view(torch.int16)), r
+    t0 = (n // BLOCK) * BLOCK
+    ty = oracle.roundtrip(_bits(x[t0:].cpu()), oracle.BF16, BLOCK, ref, oracle.BF16)
+    assert np.array_equal(_bits(y[t0:].cpu()), ty)
+    tx.close()
+    rx.close()
